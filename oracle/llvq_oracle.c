@@ -1,0 +1,639 @@
+/*
+ * CPU oracle for the multi-shell Leech-lattice (Lambda24(12)) index decode, the unfolded
+ * records and the f64 dequantize-plus-matvec.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain reference the CUDA library is
+ * checked against.  It shares no code, table or header with the CUDA path, and nothing in
+ * the product may call it: only the tests, the smoke check and the benchmark's CPU-baseline
+ * leg do.
+ *
+ * What it follows (paper sections):
+ *   Sec. 2.1  "What a Lambda24 index is": the ball Lambda24(12) in sqrt(8)*Lambda24 < Z^24,
+ *             its three membership conditions, the 301 classes, the 47-bit index that lists
+ *             classes first and arrangements and signs inside a class, the gain bit.
+ *   Sec. 2.2  "Unfolding at load time": the decoded-field record (class id, gain bit,
+ *             sign mask, per-coordinate magnitude level as bit planes or one-hot masks).
+ *   Sec. 2.3  "The kernel": y[row] = r_row * sum over blocks of the decoded unit
+ *             direction times the gain centroid, dotted with x (here in f64).
+ *
+ * Readings taken where the paper is silent (each is listed in the design notes):
+ *   - Golay code: extended cyclic code, generator polynomial 0xC75 on coordinates 0..22,
+ *     coordinate 23 is the overall parity bit; bit i of a word is coordinate i.
+ *   - Class order: shell ascending; even type before odd type; Golay weight ascending;
+ *     then the sorted magnitude tuples compared lexicographically (support part first).
+ *   - Order inside a class: mixed radix, codeword rank most significant, then the
+ *     arrangement rank on the support, the arrangement rank off the support, signs least
+ *     significant (even type); arrangement rank times 4096 plus the 12 message bits of the
+ *     codeword (odd type).
+ *   - Bit-plane level of a coordinate = |x_i| >> 1 (the class fixes the parity of every
+ *     magnitude, so |x_i| = 2*level + parity).  One-hot level = rank of |x_i| among the
+ *     distinct magnitudes of the class, ascending; masks exist for ranks 1..4.
+ *
+ * Parity pins (tests/test_oracle_pins.py): Golay weight enumerator and self-duality, 301
+ * classes, the total N = 111 043 117 458 000, the count through shell 13, per-shell counts
+ * against the Leech theta series, membership of every decoded point by a test written
+ * separately in Python, exhaustive injectivity on shell 2, encode/decode round trips, worked
+ * index -> point examples, unit norm of every block direction, and textbook special cases
+ * of the matvec.  Literal equality with the paper's own on-disk numbering: parity unpinned
+ * (the paper prints neither its order nor its fingerprint).
+ */
+#include <math.h>
+#include <pthread.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define NCOORD 24
+#define MAX_CLASSES 1024
+#define MAX_SHELL_LIMIT 13
+
+/* ------------------------------------------------------------------------------------ */
+/* Extended binary Golay code (Sec. 2.1 cites it through the lattice's definition).       */
+/* ------------------------------------------------------------------------------------ */
+
+static uint32_t g_row[12];        /* generator rows                                      */
+static uint32_t g_word[4096];     /* word for message k = XOR of rows selected by k's bits */
+static uint32_t g_sorted[4096];   /* all words, ascending as integers                      */
+static int g_nw[25];              /* number of words of each weight                        */
+static uint32_t *g_byw[25];       /* words of one weight, ascending as integers            */
+
+static int popcount32(uint32_t v) { int n = 0; while (v) { v &= v - 1; n++; } return n; }
+
+static int cmp_u32(const void *a, const void *b) {
+    uint32_t x = *(const uint32_t *)a, y = *(const uint32_t *)b;
+    return (x > y) - (x < y);
+}
+
+static void golay_build(void) {
+    const uint32_t poly = 0xC75u; /* x^11+x^10+x^6+x^5+x^4+x^2+1 */
+    for (int i = 0; i < 12; i++) {
+        uint32_t w = poly << i;                       /* cyclic shift stays inside 23 bits */
+        if (popcount32(w) & 1) w |= 1u << 23;         /* overall parity on coordinate 23   */
+        g_row[i] = w;
+    }
+    memset(g_nw, 0, sizeof g_nw);
+    for (int k = 0; k < 4096; k++) {
+        uint32_t w = 0;
+        for (int i = 0; i < 12; i++) if ((k >> i) & 1) w ^= g_row[i];
+        g_word[k] = w;
+        g_sorted[k] = w;
+        g_nw[popcount32(w)]++;
+    }
+    qsort(g_sorted, 4096, sizeof(uint32_t), cmp_u32);
+    for (int w = 0; w <= 24; w++) {
+        free(g_byw[w]);
+        g_byw[w] = NULL;
+        if (!g_nw[w]) continue;
+        g_byw[w] = (uint32_t *)malloc(sizeof(uint32_t) * (size_t)g_nw[w]);
+        int n = 0;
+        for (int k = 0; k < 4096; k++) if (popcount32(g_sorted[k]) == w) g_byw[w][n++] = g_sorted[k];
+    }
+}
+
+static int golay_contains(uint32_t w) {
+    return bsearch(&w, g_sorted, 4096, sizeof(uint32_t), cmp_u32) != NULL;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Classes (Sec. 2.1: orbits fixed by a codeword weight, a magnitude multiset, a coset).  */
+/* ------------------------------------------------------------------------------------ */
+
+typedef struct {
+    int shell;            /* m: sum of squares = 16 m                                     */
+    int odd;              /* 0: all coordinates even, 1: all odd                          */
+    int w;                /* Golay weight of the support (even type); 0 for odd type      */
+    int mags[NCOORD];     /* even: sorted support magnitudes (w of them) then sorted
+                             off-support magnitudes; odd: the 24 sorted magnitudes        */
+    uint64_t permA, permB;/* distinct arrangements of each part (odd: permA, permB = 1)   */
+    int nzB;              /* non-zero off-support entries (even type)                     */
+    uint64_t size, base;  /* points in the class, index of its first point               */
+    int ndist;            /* number of distinct magnitudes                                */
+    int dist[8];          /* the distinct magnitudes, ascending                           */
+} cls_t;
+
+static cls_t g_cls[MAX_CLASSES];
+static int g_ncls = 0;
+static uint64_t g_total = 0;
+static int g_maxshell = 0;
+static uint64_t g_shell_count[MAX_SHELL_LIMIT + 1];
+
+/* number of distinct orderings of a sorted multiset a[0..n) */
+static uint64_t multiset_perms(const int *a, int n) {
+    /* product of binomials: choose the places of each run among what is left */
+    uint64_t r = 1;
+    int left = n, i = 0;
+    while (i < n) {
+        int j = i;
+        while (j < n && a[j] == a[i]) j++;
+        int k = j - i;
+        /* r *= C(left, k), exact at every step */
+        uint64_t c = 1;
+        for (int t = 1; t <= k; t++) c = c * (uint64_t)(left - k + t) / (uint64_t)t;
+        r *= c;
+        left -= k;
+        i = j;
+    }
+    return r;
+}
+
+static int cls_cmp(const void *pa, const void *pb) {
+    const cls_t *a = (const cls_t *)pa, *b = (const cls_t *)pb;
+    if (a->shell != b->shell) return a->shell - b->shell;
+    if (a->odd != b->odd) return a->odd - b->odd;
+    if (a->w != b->w) return a->w - b->w;
+    for (int i = 0; i < NCOORD; i++) if (a->mags[i] != b->mags[i]) return a->mags[i] - b->mags[i];
+    return 0;
+}
+
+static void cls_finish(cls_t *c) {
+    if (c->odd) {
+        c->permA = multiset_perms(c->mags, NCOORD);
+        c->permB = 1;
+        c->nzB = 0;
+        c->size = c->permA * 4096u;
+    } else {
+        c->permA = multiset_perms(c->mags, c->w);
+        c->permB = multiset_perms(c->mags + c->w, NCOORD - c->w);
+        c->nzB = 0;
+        for (int i = c->w; i < NCOORD; i++) if (c->mags[i]) c->nzB++;
+        uint64_t signs = (uint64_t)1 << c->nzB;
+        if (c->w > 0) signs <<= (c->w - 1);
+        c->size = (uint64_t)g_nw[c->w] * c->permA * c->permB * signs;
+    }
+    int tmp[NCOORD];
+    memcpy(tmp, c->mags, sizeof tmp);
+    for (int i = 1; i < NCOORD; i++) { /* insertion sort of the whole multiset */
+        int v = tmp[i], j = i - 1;
+        while (j >= 0 && tmp[j] > v) { tmp[j + 1] = tmp[j]; j--; }
+        tmp[j + 1] = v;
+    }
+    c->ndist = 0;
+    for (int i = 0; i < NCOORD; i++)
+        if (i == 0 || tmp[i] != tmp[i - 1]) c->dist[c->ndist++] = tmp[i];
+}
+
+/* recursive listing of sorted multisets: n entries from vals[vi..nv) with given sum of squares */
+typedef void (*emit_fn)(const int *a, int n, void *ctx);
+
+static void multisets_rec(const int *vals, int nv, int vi, int n, int pos, int sq, int *a, emit_fn emit, void *ctx) {
+    if (pos == n) { if (sq == 0) emit(a, n, ctx); return; }
+    for (int i = vi; i < nv; i++) {
+        int v = vals[i], rem = n - pos;
+        if (v * v * rem > sq) break;              /* values ascend: all later are too large */
+        a[pos] = v;
+        multisets_rec(vals, nv, i, n, pos + 1, sq - v * v, a, emit, ctx);
+    }
+}
+
+typedef struct { int shell, w, sqA; const int *valsB; int nvB; int a[NCOORD]; } even_ctx;
+
+static void emit_even_B(const int *b, int n, void *vctx) {
+    even_ctx *e = (even_ctx *)vctx;
+    if (e->w == 0) { /* no support: the sum condition falls on the multiset itself */
+        int s = 0;
+        for (int i = 0; i < n; i++) s += b[i];
+        if (s % 8) return;
+    }
+    cls_t *c = &g_cls[g_ncls++];
+    memset(c, 0, sizeof *c);
+    c->shell = e->shell; c->odd = 0; c->w = e->w;
+    memcpy(c->mags, e->a, sizeof(int) * (size_t)e->w);
+    memcpy(c->mags + e->w, b, sizeof(int) * (size_t)n);
+}
+
+static void emit_even_A(const int *a, int n, void *vctx) {
+    even_ctx *e = (even_ctx *)vctx;
+    memcpy(e->a, a, sizeof(int) * (size_t)n);
+    int sqA = 0;
+    for (int i = 0; i < n; i++) sqA += a[i] * a[i];
+    int b[NCOORD] = {0};
+    multisets_rec(e->valsB, e->nvB, 0, NCOORD - e->w, 0, 16 * e->shell - sqA, b, emit_even_B, e);
+}
+
+typedef struct { int shell; } odd_ctx;
+
+static void emit_odd(const int *a, int n, void *vctx) {
+    odd_ctx *o = (odd_ctx *)vctx;
+    /* with the zero codeword every coordinate is congruent to 1 mod 4: +a if a = 1 mod 4, else -a */
+    int s = 0;
+    for (int i = 0; i < n; i++) s += (a[i] % 4 == 1) ? a[i] : -a[i];
+    if (((s % 8) + 8) % 8 != 4) return;
+    cls_t *c = &g_cls[g_ncls++];
+    memset(c, 0, sizeof *c);
+    c->shell = o->shell; c->odd = 1; c->w = 0;
+    memcpy(c->mags, a, sizeof(int) * (size_t)n);
+}
+
+/* Build the class list for shells 2..max_shell. Returns the number of classes. */
+int llvqo_init_shells(int max_shell) {
+    if (max_shell < 2 || max_shell > MAX_SHELL_LIMIT) return -1;
+    golay_build();
+    g_ncls = 0;
+    static const int valsA[] = {2, 6, 10, 14};       /* support: congruent to 2 mod 4 */
+    static const int valsB[] = {0, 4, 8, 12};        /* off support: multiples of 4    */
+    static const int valsM[] = {1, 3, 5, 7, 9, 11, 13};
+    static const int weights[] = {0, 8, 12, 16, 24};
+    for (int m = 2; m <= max_shell; m++) {
+        for (int wi = 0; wi < 5; wi++) {
+            even_ctx e;
+            e.shell = m; e.w = weights[wi]; e.valsB = valsB; e.nvB = 4;
+            int a[NCOORD];
+            /* every split of 16 m between the support and the rest */
+            for (int sqA = 0; sqA <= 16 * m; sqA += 4) {
+                if (e.w == 0 && sqA) break;
+                multisets_rec(valsA, 4, 0, e.w, 0, sqA, a, emit_even_A, &e);
+            }
+        }
+        odd_ctx o; o.shell = m;
+        int a[NCOORD];
+        multisets_rec(valsM, 7, 0, NCOORD, 0, 16 * m, a, emit_odd, &o);
+    }
+    qsort(g_cls, (size_t)g_ncls, sizeof(cls_t), cls_cmp);
+    g_total = 0;
+    memset(g_shell_count, 0, sizeof g_shell_count);
+    for (int c = 0; c < g_ncls; c++) {
+        cls_finish(&g_cls[c]);
+        g_cls[c].base = g_total;
+        g_total += g_cls[c].size;
+        g_shell_count[g_cls[c].shell] += g_cls[c].size;
+    }
+    g_maxshell = max_shell;
+    return g_ncls;
+}
+
+int llvqo_init(void) { return llvqo_init_shells(12); }
+
+int llvqo_num_classes(void) { return g_ncls; }
+uint64_t llvqo_total_points(void) { return g_total; }
+uint64_t llvqo_shell_count(int m) { return (m >= 0 && m <= MAX_SHELL_LIMIT) ? g_shell_count[m] : 0; }
+
+/* out[0..5] = shell, odd, w, ndist, nzB, (unused); mags[24]; size, base */
+int llvqo_class_info(int c, int *out, int *mags, uint64_t *size, uint64_t *base) {
+    if (c < 0 || c >= g_ncls) return -1;
+    const cls_t *k = &g_cls[c];
+    out[0] = k->shell; out[1] = k->odd; out[2] = k->w; out[3] = k->ndist; out[4] = k->nzB; out[5] = 0;
+    for (int i = 0; i < NCOORD; i++) mags[i] = k->mags[i];
+    *size = k->size; *base = k->base;
+    return 0;
+}
+
+uint32_t llvqo_golay_word(int k) { return g_word[k & 4095]; }
+uint32_t llvqo_golay_sorted(int k) { return g_sorted[k & 4095]; }
+
+/* ------------------------------------------------------------------------------------ */
+/* Arrangement ranks: lexicographic over the distinct orderings, smaller magnitude first. */
+/* ------------------------------------------------------------------------------------ */
+
+/* rank -> sequence. cnt[v] = copies of magnitude v still to place. */
+static void unrank_arrangement(uint64_t rank, const int *sorted, int n, int *seq) {
+    int cnt[16] = {0};
+    for (int i = 0; i < n; i++) cnt[sorted[i]]++;
+    uint64_t total = multiset_perms(sorted, n);
+    int left = n;
+    for (int pos = 0; pos < n; pos++) {
+        for (int v = 0; v < 16; v++) {
+            if (!cnt[v]) continue;
+            /* orderings that put v here: total * cnt[v] / left */
+            uint64_t sub = total * (uint64_t)cnt[v] / (uint64_t)left;
+            if (rank < sub) { seq[pos] = v; cnt[v]--; total = sub; left--; break; }
+            rank -= sub;
+        }
+    }
+}
+
+static uint64_t rank_arrangement(const int *seq, int n) {
+    int cnt[16] = {0}, sorted[NCOORD];
+    for (int i = 0; i < n; i++) cnt[seq[i]]++;
+    int k = 0;
+    for (int v = 0; v < 16; v++) for (int j = 0; j < cnt[v]; j++) sorted[k++] = v;
+    uint64_t total = multiset_perms(sorted, n), rank = 0;
+    int left = n;
+    for (int pos = 0; pos < n; pos++) {
+        for (int v = 0; v < seq[pos]; v++) {
+            if (!cnt[v]) continue;
+            rank += total * (uint64_t)cnt[v] / (uint64_t)left;
+        }
+        int v = seq[pos];
+        total = total * (uint64_t)cnt[v] / (uint64_t)left;
+        cnt[v]--; left--;
+    }
+    return rank;
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Index -> point (Sec. 2.1: classes first, then arrangements and signs in a fixed order). */
+/* ------------------------------------------------------------------------------------ */
+
+static int find_class(uint64_t idx) {
+    for (int c = 0; c < g_ncls; c++) if (idx < g_cls[c].base + g_cls[c].size) return c;
+    return -1;
+}
+
+/* Returns the class id, or -1 when idx is not below the number of points. */
+int llvqo_decode(uint64_t idx, int8_t *x) {
+    int c = (idx < g_total) ? find_class(idx) : -1;
+    if (c < 0) { memset(x, 0, NCOORD); return -1; }
+    const cls_t *k = &g_cls[c];
+    uint64_t r = idx - k->base;
+    if (k->odd) {
+        uint64_t msg = r % 4096u, rho = r / 4096u;
+        uint32_t cw = g_word[msg];
+        int seq[NCOORD];
+        unrank_arrangement(rho, k->mags, NCOORD, seq);
+        for (int i = 0; i < NCOORD; i++) {
+            int a = seq[i];
+            int want = 1 + 2 * (int)((cw >> i) & 1);           /* x_i mod 4 */
+            x[i] = (int8_t)((a % 4 == want) ? a : -a);
+        }
+        return c;
+    }
+    int w = k->w;
+    uint64_t nsign = (uint64_t)1 << (k->nzB + (w > 0 ? w - 1 : 0));
+    uint64_t sigma = r % nsign; r /= nsign;
+    uint64_t rhoB = r % k->permB; r /= k->permB;
+    uint64_t rhoA = r % k->permA; r /= k->permA;
+    uint32_t cw = g_byw[w][r];                                 /* r-th word of that weight */
+    int seqA[NCOORD], seqB[NCOORD];
+    unrank_arrangement(rhoA, k->mags, w, seqA);
+    unrank_arrangement(rhoB, k->mags + w, NCOORD - w, seqB);
+    int ia = 0, ib = 0, v[NCOORD];
+    for (int i = 0; i < NCOORD; i++) v[i] = ((cw >> i) & 1) ? seqA[ia++] : seqB[ib++];
+    /* signs: first the non-zero off-support coordinates, ascending, one bit each */
+    int bit = 0;
+    for (int i = 0; i < NCOORD; i++)
+        if (!((cw >> i) & 1) && v[i]) { if ((sigma >> bit) & 1) v[i] = -v[i]; bit++; }
+    /* then the support coordinates except the last one */
+    int last = -1, seen = 0;
+    for (int i = 0; i < NCOORD; i++)
+        if ((cw >> i) & 1) {
+            seen++;
+            if (seen == w) { last = i; break; }
+            if ((sigma >> bit) & 1) v[i] = -v[i];
+            bit++;
+        }
+    /* the last support sign repairs the sum condition: sum = 0 mod 8 */
+    if (last >= 0) {
+        int s = 0;
+        for (int i = 0; i < NCOORD; i++) s += v[i];
+        if (((s % 8) + 8) % 8 != 0) v[last] = -v[last];
+    }
+    for (int i = 0; i < NCOORD; i++) x[i] = (int8_t)v[i];
+    return c;
+}
+
+/* Point -> index; -1 when the point is not in the ball or not in the lattice. */
+int64_t llvqo_encode(const int8_t *x) {
+    int par = ((x[0] % 2) + 2) % 2, sq = 0, sum = 0;
+    for (int i = 0; i < NCOORD; i++) {
+        if ((((x[i] % 2) + 2) % 2) != par) return -1;
+        sq += x[i] * x[i]; sum += x[i];
+    }
+    if (sq % 16 || sq / 16 < 2 || sq / 16 > g_maxshell) return -1;
+    if ((((sum - 4 * par) % 8) + 8) % 8) return -1;
+    uint32_t cw = 0;
+    for (int i = 0; i < NCOORD; i++) {
+        int res = ((x[i] % 4) + 4) % 4;                        /* even: 0 or 2; odd: 1 or 3 */
+        if (res >= 2) cw |= 1u << i;
+    }
+    if (!golay_contains(cw)) return -1;
+    cls_t key;
+    memset(&key, 0, sizeof key);
+    key.shell = sq / 16; key.odd = par;
+    int seqA[NCOORD], seqB[NCOORD], na = 0, nb = 0;
+    if (par) {
+        for (int i = 0; i < NCOORD; i++) seqA[na++] = abs(x[i]);
+    } else {
+        key.w = popcount32(cw);
+        for (int i = 0; i < NCOORD; i++) { if ((cw >> i) & 1) seqA[na++] = abs(x[i]); else seqB[nb++] = abs(x[i]); }
+    }
+    /* sorted copies make the class key */
+    int sa[NCOORD], sb[NCOORD];
+    memcpy(sa, seqA, sizeof(int) * (size_t)na); memcpy(sb, seqB, sizeof(int) * (size_t)nb);
+    for (int i = 1; i < na; i++) { int v = sa[i], j = i - 1; while (j >= 0 && sa[j] > v) { sa[j + 1] = sa[j]; j--; } sa[j + 1] = v; }
+    for (int i = 1; i < nb; i++) { int v = sb[i], j = i - 1; while (j >= 0 && sb[j] > v) { sb[j + 1] = sb[j]; j--; } sb[j + 1] = v; }
+    memcpy(key.mags, sa, sizeof(int) * (size_t)na); memcpy(key.mags + na, sb, sizeof(int) * (size_t)nb);
+    int c = -1;
+    for (int i = 0; i < g_ncls; i++) if (cls_cmp(&key, &g_cls[i]) == 0) { c = i; break; }
+    if (c < 0) return -1;
+    const cls_t *k = &g_cls[c];
+    if (par) {
+        /* message bits: solve cw = XOR of rows; the code is small enough to search */
+        int msg = -1;
+        for (int m = 0; m < 4096; m++) if (g_word[m] == cw) { msg = m; break; }
+        return (int64_t)(k->base + rank_arrangement(seqA, NCOORD) * 4096u + (uint64_t)msg);
+    }
+    uint64_t kw = 0;
+    for (int i = 0; i < g_nw[key.w]; i++) if (g_byw[key.w][i] == cw) { kw = (uint64_t)i; break; }
+    uint64_t sigma = 0; int bit = 0;
+    for (int i = 0; i < NCOORD; i++)
+        if (!((cw >> i) & 1) && x[i]) { if (x[i] < 0) sigma |= (uint64_t)1 << bit; bit++; }
+    int seen = 0;
+    for (int i = 0; i < NCOORD; i++)
+        if ((cw >> i) & 1) { seen++; if (seen == key.w) break; if (x[i] < 0) sigma |= (uint64_t)1 << bit; bit++; }
+    uint64_t nsign = (uint64_t)1 << (k->nzB + (key.w > 0 ? key.w - 1 : 0));
+    uint64_t r = kw;
+    r = r * k->permA + rank_arrangement(seqA, na);
+    r = r * k->permB + rank_arrangement(seqB, nb);
+    r = r * nsign + sigma;
+    return (int64_t)(k->base + r);
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Records (Sec. 2.2) and the two in-memory layouts.                                       */
+/* ------------------------------------------------------------------------------------ */
+
+#define SENTINEL_CLASS 511   /* class id of a code that names no point: all fields zero */
+
+typedef struct {
+    int cls, gain;
+    uint32_t smask;            /* bit i: x_i < 0                                          */
+    uint32_t plane[3];         /* bit i of plane t: bit t of (|x_i| >> 1)                 */
+    uint32_t onehot[4];        /* bit i of mask l-1: rank level of x_i equals l, l = 1..4 */
+    int8_t x[NCOORD];
+} record_t;
+
+/* code word = index | gain << 47 */
+static void make_record(uint64_t code, record_t *rec) {
+    memset(rec, 0, sizeof *rec);
+    rec->gain = (int)((code >> 47) & 1);
+    uint64_t idx = code & (((uint64_t)1 << 47) - 1);
+    int c = (code >> 48) ? -1 : llvqo_decode(idx, rec->x);
+    if (c < 0) { rec->cls = SENTINEL_CLASS; rec->gain = 0; memset(rec->x, 0, NCOORD); return; }
+    rec->cls = c;
+    const cls_t *k = &g_cls[c];
+    for (int i = 0; i < NCOORD; i++) {
+        int a = abs(rec->x[i]);
+        if (rec->x[i] < 0) rec->smask |= 1u << i;
+        for (int t = 0; t < 3; t++) if (((a >> 1) >> t) & 1) rec->plane[t] |= 1u << i;
+        int lvl = 0;
+        while (k->dist[lvl] != a) lvl++;
+        if (lvl > 0) rec->onehot[lvl - 1] |= 1u << i;
+    }
+}
+
+/* fields[0]=class, [1]=gain, [2]=smask, [3..5]=planes, [6..9]=one-hot masks */
+int llvqo_record(uint64_t code, uint32_t *fields, int8_t *x) {
+    record_t r;
+    make_record(code, &r);
+    fields[0] = (uint32_t)r.cls; fields[1] = (uint32_t)r.gain; fields[2] = r.smask;
+    for (int t = 0; t < 3; t++) fields[3 + t] = r.plane[t];
+    for (int t = 0; t < 4; t++) fields[6 + t] = r.onehot[t];
+    memcpy(x, r.x, NCOORD);
+    return r.cls;
+}
+
+size_t llvqo_planes_bytes(int64_t rows, int64_t nb) { return (size_t)((rows + 31) / 32) * (size_t)nb * 448u; }
+size_t llvqo_onehot_bytes(int64_t rows, int64_t nb) { return (size_t)((rows + 31) / 32) * (size_t)nb * 640u; }
+
+/*
+ * Bit-plane layout, 14 bytes a block.  Rows are taken 32 at a time (a row group); rows past the
+ * end are filled with the sentinel record.  The cell of (row group, block column b) holds, for
+ * each of its 32 rows, three payload words and a 16-bit header:
+ *   header  = class | gain << 9
+ *   word j (j = 0,1,2) carries coordinates 8j .. 8j+7.  Coordinate 8j + 2k + e (pair k = 0..3,
+ *   e = 0 low / 1 high) has its level bit t at bit (4 + t + 16 e + 4 k) mod 32 and its sign
+ *   at bit (15 + 16 e + 4 k) mod 32.
+ * Four consecutive cells of a row group form a 1792-byte tile: for row l, bytes 512 j + 16 l
+ * hold word j of the four cells in order, bytes 1536 + 8 l their four headers.  The nb mod 4
+ * cells left at the end of a row group are stored alone, 448 bytes each: word j of row l at
+ * 128 j + 4 l, header at 384 + 2 l.  A row group occupies 448 nb bytes.
+ */
+void llvqo_pack_planes(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t *out) {
+    int64_t ngroups = (rows + 31) / 32, nfull = nb / 4;
+    for (int64_t rg = 0; rg < ngroups; rg++) {
+        uint8_t *grp = out + (size_t)rg * (size_t)nb * 448u;
+        for (int l = 0; l < 32; l++) {
+            int64_t row = rg * 32 + l;
+            for (int64_t b = 0; b < nb; b++) {
+                record_t r;
+                if (row < rows) make_record(codes[row * nb + b], &r);
+                else { memset(&r, 0, sizeof r); r.cls = SENTINEL_CLASS; }
+                uint32_t word[3] = {0, 0, 0};
+                for (int i = 0; i < NCOORD; i++) {
+                    int j = i / 8, k = (i % 8) / 2, e = i % 2;
+                    for (int t = 0; t < 3; t++)
+                        if ((r.plane[t] >> i) & 1) word[j] |= 1u << ((4 + t + 16 * e + 4 * k) % 32);
+                    if ((r.smask >> i) & 1) word[j] |= 1u << ((15 + 16 * e + 4 * k) % 32);
+                }
+                uint16_t hdr = (uint16_t)(r.cls | (r.gain << 9));
+                if (b < nfull * 4) {
+                    uint8_t *tile = grp + (size_t)(b / 4) * 1792u;
+                    int q = (int)(b % 4);
+                    for (int j = 0; j < 3; j++) memcpy(tile + 512 * j + 16 * l + 4 * q, &word[j], 4);
+                    memcpy(tile + 1536 + 8 * l + 2 * q, &hdr, 2);
+                } else {
+                    uint8_t *cell = grp + (size_t)nfull * 1792u + (size_t)(b - nfull * 4) * 448u;
+                    for (int j = 0; j < 3; j++) memcpy(cell + 128 * j + 4 * l, &word[j], 4);
+                    memcpy(cell + 384 + 2 * l, &hdr, 2);
+                }
+            }
+        }
+    }
+}
+
+/*
+ * One-hot layout, 20 bytes a block: the cell of (row group, block column) is five arrays of 32
+ * words, one entry a row: V0 = smask | class[7:0] << 24, V1 = mask1 | class[8] << 24 | gain << 25,
+ * V2 = mask2, V3 = mask3, V4 = mask4.  Word t of row l sits at 128 t + 4 l; a row group occupies
+ * 640 nb bytes.
+ */
+void llvqo_pack_onehot(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t *out) {
+    int64_t ngroups = (rows + 31) / 32;
+    for (int64_t rg = 0; rg < ngroups; rg++)
+        for (int l = 0; l < 32; l++) {
+            int64_t row = rg * 32 + l;
+            for (int64_t b = 0; b < nb; b++) {
+                record_t r;
+                if (row < rows) make_record(codes[row * nb + b], &r);
+                else { memset(&r, 0, sizeof r); r.cls = SENTINEL_CLASS; }
+                uint32_t v[5];
+                v[0] = r.smask | ((uint32_t)(r.cls & 255) << 24);
+                v[1] = r.onehot[0] | ((uint32_t)(r.cls >> 8) << 24) | ((uint32_t)r.gain << 25);
+                v[2] = r.onehot[1]; v[3] = r.onehot[2]; v[4] = r.onehot[3];
+                uint8_t *cell = out + ((size_t)rg * (size_t)nb + (size_t)b) * 640u;
+                for (int t = 0; t < 5; t++) memcpy(cell + 128 * t + 4 * l, &v[t], 4);
+            }
+        }
+}
+
+/* ------------------------------------------------------------------------------------ */
+/* Dequantised weights and the f64 matvec (Sec. 2.3).                                      */
+/* ------------------------------------------------------------------------------------ */
+
+static double half_to_double(uint16_t h) {
+    int s = h >> 15, e = (h >> 10) & 31, f = h & 1023;
+    double v;
+    if (e == 0) v = ldexp((double)f, -24);
+    else if (e == 31) v = f ? NAN : INFINITY;
+    else v = ldexp((double)(f + 1024), e - 25);
+    return s ? -v : v;
+}
+
+/* W[row, 24 b + i] = r_row * gain[g] * x_i / (4 sqrt(m)); one block written to w[24] */
+static void block_weights(uint64_t code, double rscale, const double *gain, double *w) {
+    record_t r;
+    make_record(code, &r);
+    if (r.cls == SENTINEL_CLASS) { for (int i = 0; i < NCOORD; i++) w[i] = 0.0; return; }
+    double unit = 1.0 / (4.0 * sqrt((double)g_cls[r.cls].shell));
+    for (int i = 0; i < NCOORD; i++) w[i] = rscale * gain[r.gain] * (double)r.x[i] * unit;
+}
+
+void llvqo_dequant(const uint64_t *codes, int64_t rows, int64_t nb, const uint16_t *row_scale,
+                   const double *gain, double *W) {
+    for (int64_t row = 0; row < rows; row++)
+        for (int64_t b = 0; b < nb; b++)
+            block_weights(codes[row * nb + b], half_to_double(row_scale[row]), gain, W + (row * nb + b) * NCOORD);
+}
+
+typedef struct {
+    const uint64_t *codes; int64_t rows, nb, row0, row1;
+    const uint16_t *row_scale, *x; const double *gain;
+    double *y, *wnorm, *abssum;
+} mv_job;
+
+static void *mv_worker(void *arg) {
+    mv_job *j = (mv_job *)arg;
+    for (int64_t row = j->row0; row < j->row1; row++) {
+        double acc = 0.0, n2 = 0.0, as = 0.0, w[NCOORD];
+        double rs = half_to_double(j->row_scale[row]);
+        for (int64_t b = 0; b < j->nb; b++) {
+            block_weights(j->codes[row * j->nb + b], rs, j->gain, w);
+            for (int i = 0; i < NCOORD; i++) {
+                double xv = half_to_double(j->x[b * NCOORD + i]);
+                acc += w[i] * xv; n2 += w[i] * w[i]; as += fabs(w[i] * xv);
+            }
+        }
+        j->y[row] = acc;
+        if (j->wnorm) j->wnorm[row] = sqrt(n2);
+        if (j->abssum) j->abssum[row] = as;
+    }
+    return NULL;
+}
+
+/* y = W x in f64; wnorm[row] = ||W[row,:]||_2, abssum[row] = sum |w x| (either may be NULL).
+ * Rows are split over nthreads threads; every row is summed in the same order whatever the split. */
+void llvqo_matvec(const uint64_t *codes, int64_t rows, int64_t nb, const uint16_t *row_scale,
+                  const double *gain, const uint16_t *x, double *y, double *wnorm, double *abssum, int nthreads) {
+    if (nthreads < 1) nthreads = 1;
+    if (nthreads > 256) nthreads = 256;
+    pthread_t th[256]; mv_job job[256];
+    int64_t per = (rows + nthreads - 1) / nthreads;
+    int started = 0;
+    for (int t = 0; t < nthreads; t++) {
+        int64_t r0 = t * per, r1 = r0 + per > rows ? rows : r0 + per;
+        if (r0 >= r1) break;
+        job[t] = (mv_job){codes, rows, nb, r0, r1, row_scale, x, gain, y, wnorm, abssum};
+        if (nthreads == 1) mv_worker(&job[t]); else pthread_create(&th[t], NULL, mv_worker, &job[t]);
+        started++;
+    }
+    if (nthreads > 1) for (int t = 0; t < started; t++) pthread_join(th[t], NULL);
+}
+
+/* decode a batch: x[n][24], cls[n] (sentinel -1 for codes that name no point) */
+void llvqo_decode_batch(const uint64_t *codes, int64_t n, int8_t *x, int32_t *cls) {
+    for (int64_t i = 0; i < n; i++) {
+        uint64_t idx = codes[i] & (((uint64_t)1 << 47) - 1);
+        cls[i] = (codes[i] >> 48) ? -1 : llvqo_decode(idx, x + i * NCOORD);
+        if (cls[i] < 0) memset(x + i * NCOORD, 0, NCOORD);
+    }
+}

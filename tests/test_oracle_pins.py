@@ -1,0 +1,352 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix (no GPU).
+
+Nothing here re-calls the oracle's own formulas: the Golay code, the lattice membership test,
+the theta series and the layout unpackers below are written separately in Python.
+"""
+import itertools
+import math
+
+import numpy as np
+import pytest
+
+N_PAPER = 111_043_117_458_000           # Sec. 2.1
+N13_PAPER = 280_974_212_784_720         # Sec. 2.4, "Invariant locks upstream"
+KISSING = 196_560                       # Sec. 2.4
+
+
+# ---------------------------------------------------------------- independent ingredients
+def golay_set():
+    """All multiples of g(x) = x^11+x^10+x^6+x^5+x^4+x^2+1 of degree < 23, plus a parity bit."""
+    g = (1 << 11) | (1 << 10) | (1 << 6) | (1 << 5) | (1 << 4) | (1 << 2) | 1
+    words = set()
+    for m in range(4096):
+        w = 0
+        for i in range(12):
+            if (m >> i) & 1:
+                w ^= g << i          # carry-less product m(x) g(x)
+        if bin(w).count("1") & 1:
+            w |= 1 << 23
+        words.add(w)
+    return words
+
+
+GOLAY = golay_set()
+
+
+def is_leech_point(x) -> bool:
+    """Sec. 2.1's three conditions in sqrt(8) Lambda24: parity, Golay word on a residue class mod 4, sum mod 8."""
+    x = [int(v) for v in x]
+    par = x[0] % 2
+    if any(v % 2 != par for v in x):
+        return False
+    word = 0
+    for i, v in enumerate(x):
+        if ((v - par) // 2) % 2:
+            word |= 1 << i
+    return word in GOLAY and sum(x) % 8 == (4 * par) % 8
+
+
+def tau(nmax):
+    poly = [1] + [0] * nmax
+    for n in range(1, nmax + 1):
+        for _ in range(24):
+            for k in range(nmax, n - 1, -1):
+                poly[k] -= poly[k - n]
+    return [0] + poly[:nmax]
+
+
+def theta(m, t):
+    s11 = sum(d**11 for d in range(1, m + 1) if m % d == 0)
+    v, r = divmod(65520 * (s11 - t[m]), 691)
+    assert r == 0
+    return v
+
+
+# ---------------------------------------------------------------- Golay code
+def test_golay_weight_enumerator_and_duality(oracle):
+    words = oracle.golay_words()
+    assert len(set(words.tolist())) == 4096
+    assert set(words.tolist()) == GOLAY
+    hist = np.bincount([bin(int(w)).count("1") for w in words], minlength=25)
+    assert {int(k): int(v) for k, v in enumerate(hist) if v} == {0: 1, 8: 759, 12: 2576, 16: 759, 24: 1}
+    rows = [int(words[1 << i]) for i in range(12)]
+    for a, b in itertools.product(rows, rows):
+        assert bin(a & b).count("1") % 2 == 0          # self-dual
+    # cyclic on the first 23 coordinates: g(x) divides x^23 - 1
+    for w in rows:
+        lo = w & ((1 << 23) - 1)
+        rot = ((lo << 1) | (lo >> 22)) & ((1 << 23) - 1)
+        assert (rot | (w & (1 << 23))) in GOLAY
+
+
+# ---------------------------------------------------------------- classes
+def test_class_count_and_totals(oracle):
+    assert oracle.num_classes() == 301                 # Sec. 2.1
+    assert oracle.total_points() == N_PAPER
+    assert math.ceil(math.log2(N_PAPER)) == 47
+    t = tau(13)
+    assert t[1:8] == [1, -24, 252, -1472, 4830, -6048, -16744]   # textbook values of Ramanujan's tau
+    assert theta(2, t) == KISSING
+    for m in range(2, 13):
+        assert oracle.shell_count(m) == theta(m, t), m
+    infos = [oracle.class_info(c) for c in range(301)]
+    assert sum(i["size"] for i in infos) == N_PAPER
+    assert all(1 <= i["ndist"] <= 5 for i in infos)    # Sec. 2.3: at most five values a class
+    assert sum(1 for i in infos if i["odd"]) == 121
+    base = 0
+    for i in infos:                                    # contiguous, in order
+        assert i["base"] == base
+        base += i["size"]
+    keys = [(i["shell"], i["odd"], i["w"], tuple(i["mags"])) for i in infos]
+    assert keys == sorted(keys) and len(set(keys)) == 301
+
+
+def test_count_through_shell_13(oracle):
+    try:
+        assert oracle.init_shells(13) == 383
+        assert oracle.total_points() == N13_PAPER      # Sec. 2.4
+        assert oracle.shell_count(13) == theta(13, tau(13))
+    finally:
+        oracle.init_shells(12)
+    assert oracle.num_classes() == 301
+
+
+def test_shell2_classes_by_hand(oracle):
+    # the 196 560 minimal vectors: (+-4^2, 0^22), (+-2^8, 0^16), (-+3, +-1^23)
+    sizes = [oracle.class_info(c)["size"] for c in range(3)]
+    assert sizes == [1104, 97152, 98304]
+
+
+# ---------------------------------------------------------------- decoder
+def _sample_indices(oracle, per_shell=300, seed=7):
+    rng = np.random.default_rng(seed)
+    out = []
+    for c in range(301):
+        i = oracle.class_info(c)
+        out += [i["base"], i["base"] + i["size"] - 1]
+        out += (i["base"] + rng.integers(0, i["size"], size=6)).tolist()
+    out += rng.integers(0, N_PAPER, size=per_shell * 11).tolist()
+    return np.array(out, dtype=np.uint64)
+
+
+def test_decoded_points_are_lattice_points_of_the_right_shell(oracle):
+    idx = _sample_indices(oracle)
+    xs, cls = oracle.decode_batch(idx)
+    assert (cls >= 0).all()
+    for i, x, c in zip(idx.tolist(), xs, cls.tolist()):
+        info = oracle.class_info(c)
+        assert info["base"] <= i < info["base"] + info["size"]
+        assert is_leech_point(x), (i, x)
+        assert int((x.astype(int) ** 2).sum()) == 16 * info["shell"]
+        mags = np.abs(x.astype(int))
+        if info["odd"]:
+            assert sorted(mags.tolist()) == info["mags"]
+        else:
+            assert sorted(mags.tolist()) == sorted(info["mags"])
+    # lattice closure and integrality of the scaled inner product
+    X = xs.astype(np.int64)
+    rng = np.random.default_rng(3)
+    for _ in range(2000):
+        a, b = X[rng.integers(len(X))], X[rng.integers(len(X))]
+        assert int(a @ b) % 8 == 0 and int(a @ a) % 16 == 0
+        assert is_leech_point(a + b) and is_leech_point(a - b)
+
+
+def test_round_trip_encode_decode(oracle):
+    idx = _sample_indices(oracle, per_shell=1000, seed=11)
+    xs, _ = oracle.decode_batch(idx)
+    for i, x in zip(idx.tolist(), xs):
+        assert oracle.encode(x) == i
+    assert oracle.decode(N_PAPER)[0] == -1
+    assert oracle.decode((1 << 47) - 1)[0] == -1
+    assert oracle.encode(np.zeros(24, np.int8)) == -1
+    bad = np.array([4, 4] + [0] * 22, np.int8)
+    bad[0] = 2
+    assert oracle.encode(bad) == -1
+
+
+def test_shell2_is_enumerated_exactly_once(oracle):
+    xs, cls = oracle.decode_batch(np.arange(KISSING, dtype=np.uint64))
+    assert set(cls.tolist()) == {0, 1, 2}
+    packed = np.ascontiguousarray(xs).view([("a", "u8"), ("b", "u8"), ("c", "u8")]).ravel()
+    assert np.unique(packed).size == KISSING           # injective, and 196 560 is the whole shell
+    assert ((xs.astype(int) ** 2).sum(1) == 32).all()
+    assert all(is_leech_point(x) for x in xs[::97])
+
+
+@pytest.mark.parametrize("lo,hi", [(196_560, 196_560 + 2_000_000), (16_969_680 - 1_500_000, 16_969_680)])
+def test_shell3_ranges_are_injective(oracle, lo, hi):
+    xs, _ = oracle.decode_batch(np.arange(lo, hi, dtype=np.uint64))
+    packed = np.ascontiguousarray(xs).view([("a", "u8"), ("b", "u8"), ("c", "u8")]).ravel()
+    assert np.unique(packed).size == hi - lo
+    assert ((xs.astype(int) ** 2).sum(1) == 48).all()
+
+
+def test_worked_examples_derived_by_hand(oracle):
+    """First and last points of the first classes, worked out from the stated order by hand."""
+    # class 0: off-support multiset {0^22, 4, 4}; rank 0 puts the zeros first; sign bit 0 is the
+    # first non-zero coordinate
+    assert oracle.decode(0)[1].tolist() == [0] * 22 + [4, 4]
+    assert oracle.decode(1)[1].tolist() == [0] * 22 + [-4, 4]
+    assert oracle.decode(1103)[1].tolist() == [-4, -4] + [0] * 22       # 276 * 4 - 1
+    # class 1 starts with the smallest weight-8 word; its support all +2 sums to 16 = 0 mod 8
+    c, x = oracle.decode(1104)
+    assert c == 1 and sorted(np.flatnonzero(x).tolist()) == [i for i in range(24) if (min(w for w in GOLAY if bin(w).count("1") == 8) >> i) & 1]
+    assert (x[np.flatnonzero(x)] == 2).all()
+    # next index flips the first support coordinate; the last one repairs the sum
+    x2 = oracle.decode(1105)[1]
+    sup = np.flatnonzero(x).tolist()
+    assert x2[sup[0]] == -2 and x2[sup[-1]] == -2 and (x2[sup[1:-1]] == 2).all()
+    # class 2, zero codeword: every coordinate is 1 mod 4, so the 3 comes out negative
+    assert oracle.decode(1104 + 97152)[1].tolist() == [1] * 23 + [-3]
+    # first point of shell 4 and of shell 12
+    assert oracle.decode(16_969_680)[1].tolist() == [0] * 23 + [8]
+    assert oracle.decode(40_556_880_458_640)[1].tolist() == [0] * 21 + [8, 8, 8]
+
+
+# ---------------------------------------------------------------- records and layouts
+def _unpack_planes_cell(buf, nb, row, b):
+    """Reader of the bit-plane layout written from its description (not from the packer)."""
+    rg, l = divmod(row, 32)
+    grp = rg * nb * 448
+    nfull = nb // 4
+    if b < nfull * 4:
+        t, q = divmod(b, 4)
+        base = grp + t * 1792
+        words = [int.from_bytes(buf[base + 512 * j + 16 * l + 4 * q: base + 512 * j + 16 * l + 4 * q + 4].tobytes(), "little") for j in range(3)]
+        hdr = int.from_bytes(buf[base + 1536 + 8 * l + 2 * q: base + 1536 + 8 * l + 2 * q + 2].tobytes(), "little")
+    else:
+        base = grp + nfull * 1792 + (b - nfull * 4) * 448
+        words = [int.from_bytes(buf[base + 128 * j + 4 * l: base + 128 * j + 4 * l + 4].tobytes(), "little") for j in range(3)]
+        hdr = int.from_bytes(buf[base + 384 + 2 * l: base + 384 + 2 * l + 2].tobytes(), "little")
+    cls, gain = hdr & 511, (hdr >> 9) & 1
+    assert hdr >> 10 == 0
+    level, sign = [0] * 24, [0] * 24
+    for j, w in enumerate(words):
+        for k in range(4):
+            r = ((w >> (4 * k)) | (w << (32 - 4 * k))) & 0xFFFFFFFF
+            for e in range(2):
+                i = 8 * j + 2 * k + e
+                level[i] = (r >> (4 + 16 * e)) & 7
+                sign[i] = (r >> (15 + 16 * e)) & 1
+    return cls, gain, level, sign
+
+
+def _codes(oracle, rows, nb, seed):
+    from paper_2609_02652_b200 import datagen
+
+    return datagen.make_codes(rows, nb, seed).numpy().astype(np.uint64)
+
+
+@pytest.mark.parametrize("rows,nb", [(32, 4), (40, 7), (3, 1), (64, 9)])
+def test_planes_layout_round_trip(oracle, rows, nb):
+    codes = _codes(oracle, rows, nb, seed=5)
+    codes[0] = N_PAPER                       # a code that names no point
+    buf = oracle.pack_planes(codes, rows, nb)
+    assert buf.size == ((rows + 31) // 32) * nb * 448
+    xs, cls = oracle.decode_batch(codes)
+    for row in range(((rows + 31) // 32) * 32):
+        for b in range(nb):
+            c, g, level, sign = _unpack_planes_cell(buf, nb, row, b)
+            if row >= rows or cls[row * nb + b] < 0:
+                assert c == 511 and g == 0 and not any(level) and not any(sign)
+                continue
+            code = int(codes[row * nb + b])
+            assert c == cls[row * nb + b] and g == code >> 47
+            par = oracle.class_info(c)["odd"]
+            x = [(-1 if s else 1) * (2 * lv + par) for lv, s in zip(level, sign)]
+            assert x == xs[row * nb + b].tolist()
+
+
+@pytest.mark.parametrize("rows,nb", [(32, 3), (37, 5)])
+def test_onehot_layout_round_trip_and_field_widths(oracle, rows, nb):
+    codes = _codes(oracle, rows, nb, seed=6)
+    buf = oracle.pack_onehot(codes, rows, nb).view(np.uint32)
+    assert buf.size * 4 == ((rows + 31) // 32) * nb * 640
+    xs, cls = oracle.decode_batch(codes)
+    for row in range(rows):
+        rg, l = divmod(row, 32)
+        for b in range(nb):
+            v = [int(buf[(rg * nb + b) * 160 + 32 * t + l]) for t in range(5)]
+            c = (v[0] >> 24) | (((v[1] >> 24) & 1) << 8)
+            g = (v[1] >> 25) & 1
+            smask = v[0] & 0xFFFFFF
+            masks = [v[1] & 0xFFFFFF, v[2], v[3], v[4]]
+            info = oracle.class_info(c)
+            dist = sorted(set(info["mags"]))
+            assert c == cls[row * nb + b] and g == int(codes[row * nb + b]) >> 47
+            assert all(m >> 24 == 0 for m in masks[1:])
+            assert all(masks[t] == 0 for t in range(len(dist) - 1, 4))        # 9 + 1 + 24 L bits used
+            x = []
+            for i in range(24):
+                lv = sum((t + 1) * ((masks[t] >> i) & 1) for t in range(4))
+                assert sum((masks[t] >> i) & 1 for t in range(4)) <= 1
+                x.append((-1 if (smask >> i) & 1 else 1) * dist[lv])
+            assert x == xs[row * nb + b].tolist()
+            # the same block through the logical record: planes and one-hot agree
+            rec = oracle.record(int(codes[row * nb + b]))
+            lv_planes = [sum(((rec["planes"][t] >> i) & 1) << t for t in range(3)) for i in range(24)]
+            assert [2 * p + info["odd"] for p in lv_planes] == [abs(a) for a in x]
+            assert rec["smask"] == smask and rec["cls"] == c
+
+
+def test_record_payload_is_106_bits():
+    assert 9 + 1 + 24 + 3 * 24 == 106 <= 14 * 8        # Sec. 2.3: 106 payload bits in a 112-bit record
+
+
+# ---------------------------------------------------------------- f64 matvec
+def test_matvec_against_numpy_and_special_cases(oracle):
+    from paper_2609_02652_b200 import datagen
+
+    rows, nb = 21, 13
+    codes = _codes(oracle, rows, nb, seed=8)
+    rs = datagen.make_row_scale(rows, 8).numpy()
+    x = datagen.make_x(nb * 24 - 5, nb * 24, 8).numpy()
+    gain = (0.75, 1.5)
+    xs, cls = oracle.decode_batch(codes)
+    # weights written out independently: r * gamma_g * x_i / (4 sqrt m)
+    W = np.zeros((rows, nb * 24))
+    for r in range(rows):
+        for b in range(nb):
+            m = oracle.class_info(int(cls[r * nb + b]))["shell"]
+            g = gain[int(codes[r * nb + b]) >> 47]
+            W[r, 24 * b:24 * b + 24] = float(rs[r]) * g * xs[r * nb + b].astype(float) / (4 * math.sqrt(m))
+    y, wn, ab = oracle.matvec(codes, rows, nb, rs, gain, x, nthreads=3)
+    ref = W @ x.astype(np.float64)
+    assert np.allclose(y, ref, rtol=0, atol=1e-13)
+    assert np.allclose(wn, np.linalg.norm(W, axis=1), rtol=1e-13)
+    assert np.allclose(ab, np.abs(W * x.astype(np.float64)).sum(1), rtol=1e-13)
+    assert np.allclose(oracle.dequant(codes, rows, nb, rs, gain), W, rtol=0, atol=1e-15)
+    y1, _, _ = oracle.matvec(codes, rows, nb, rs, gain, x, nthreads=1)
+    assert (y1 == y).all()                                   # thread split does not change a row
+    # unit directions: with r = 1 and gamma = 1 every block has norm 1
+    one = np.ones(rows, np.float16)
+    Wu = oracle.dequant(codes, rows, nb, one, (1.0, 1.0)).reshape(rows, nb, 24)
+    assert np.allclose((Wu**2).sum(-1), 1.0, atol=1e-14)
+    # x = e_j picks column j
+    for j in (0, 17, nb * 24 - 1):
+        e = np.zeros(nb * 24, np.float16)
+        e[j] = 1
+        yj, _, _ = oracle.matvec(codes, rows, nb, one, (1.0, 1.0), e)
+        assert np.allclose(yj, Wu.reshape(rows, -1)[:, j], atol=1e-15)
+    # a code that names no point contributes nothing
+    codes2 = codes.copy()
+    codes2[:] = N_PAPER
+    assert (oracle.matvec(codes2, rows, nb, rs, gain, x)[0] == 0).all()
+
+
+def test_generator_draws_valid_shell_uniform_indices(oracle):
+    from paper_2609_02652_b200 import datagen
+
+    sizes, bases = datagen.shell_sizes(), datagen.shell_bases()
+    assert [sizes[m] for m in range(2, 13)] == [oracle.shell_count(m) for m in range(2, 13)]
+    assert bases[13] == N_PAPER
+    codes = datagen.make_codes(64, 128, 0).numpy().astype(np.uint64)
+    idx = codes & np.uint64((1 << 47) - 1)
+    assert (idx < N_PAPER).all()
+    shell = np.searchsorted([bases[m] for m in range(2, 14)], idx, side="right") + 1
+    hist = np.bincount(shell, minlength=13)[2:13]
+    assert hist.min() > 0.7 * hist.mean() and hist.max() < 1.3 * hist.mean()
+    g = (codes >> np.uint64(47)).astype(int)
+    assert 0.45 < g.mean() < 0.55 and g.max() == 1
+    assert (datagen.make_codes(64, 128, 0, start=100, count=50).numpy() == datagen.make_codes(64, 128, 0).numpy()[100:150]).all()
