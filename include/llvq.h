@@ -1,0 +1,137 @@
+/*
+ * llvq.h - C ABI of the B200 (sm_100a) library for the batch-1 fused dequantize-plus-matvec over
+ * weights quantised to the multi-shell Leech-lattice codebook Lambda24(12).
+ *
+ * The path (paper sections in brackets):
+ *   llvq_expand      [Sec. 2.2 "Unfolding at load time"]  48-bit block codes -> in-memory records
+ *   llvq_gemv        [Sec. 2.3 "The kernel"]               records, row scales, x -> y
+ *   llvq_gemv_grouped[Sec. 3.4 "Attribution": row-concatenated q/k/v and gate/up launches]
+ *   llvq_gemv_fp16, llvq_gemv_noweights [Sec. 3.2, Table "layout scale": the FP16 control and the
+ *                    no-weights control that prices the launch geometry]
+ *   llvq_dequant_fp16, llvq_decode_i8: helpers that feed the FP16 arm and the bit-exact decode check.
+ *
+ * Conventions.
+ *   - A block is 24 consecutive weights of one row.  A matrix has `rows` rows and `nb` blocks a
+ *     row; k_padded = 24 * nb.  x has k_padded entries; the caller zero-fills the padding.
+ *   - A code word is a uint64: bits 0..46 the index into the ball (valid below
+ *     111 043 117 458 000), bit 47 the gain bit, bits 48..63 zero  [Sec. 2.1].
+ *   - Every pointer is a DEVICE pointer owned by the caller unless it says "host".  The library
+ *     allocates only what a context owns (its tables and its reduction scratch) at llvq_create.
+ *   - Every call takes the caller's CUDA stream (a cudaStream_t passed as void*), enqueues its
+ *     work there and returns without synchronising, unless stated otherwise.
+ *   - A context holds reduction scratch that its GEMV launches share: launches on one context
+ *     must be ordered on one stream (or otherwise serialised).  Use one context per stream.
+ *   - Return value: 0 on success, a negative LLVQ_E* code otherwise.  No call aborts, throws or
+ *     traps; a failed call enqueues nothing.
+ *
+ * Layouts (both written by llvq_expand, read by the GEMV; rows are taken 32 at a time, a "row
+ * group", rows past the end are filled with the empty record, class id 511):
+ *   LLVQ_PLANES  14 bytes a block [Sec. 3.2 "Planes14": class id 9 b, gain 1 b, sign mask 24 b,
+ *                three binary planes of the per-coordinate level 3 x 24 b = 106 bits in 112].
+ *                The level of a coordinate is |x_i| >> 1; the class fixes the parity of every
+ *                magnitude, so |x_i| = 2 level + parity.  Per (row group, block column) "cell"
+ *                and per row: a 16-bit header = class | gain << 9 and three 32-bit words; word j
+ *                carries coordinates 8j..8j+7; coordinate 8j+2k+e (k = 0..3, e = 0..1) has level
+ *                bit t at bit (4+t+16e+4k) mod 32 and its sign at bit (15+16e+4k) mod 32.  Four
+ *                consecutive cells form a 1792-byte tile (row l: bytes 512j+16l = word j of the
+ *                four cells, bytes 1536+8l = the four headers); the nb mod 4 last cells of a row
+ *                group are stored alone, 448 bytes each (word j of row l at 128j+4l, header at
+ *                384+2l).  A row group takes 448*nb bytes.
+ *   LLVQ_ONEHOT  20 bytes a block [Sec. 3.2 "Slot32": class id, gain, sign mask, one 24-bit
+ *                one-hot mask per non-zero level].  Level = rank of |x_i| among the class's
+ *                distinct magnitudes.  Per cell five arrays of 32 words (word t of row l at
+ *                128t+4l): V0 = smask | class[7:0]<<24, V1 = mask1 | class[8]<<24 | gain<<25,
+ *                V2..V4 = mask2..mask4.  A row group takes 640*nb bytes.
+ */
+#ifndef LLVQ_H
+#define LLVQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LLVQ_PLANES 0
+#define LLVQ_ONEHOT 1
+
+#define LLVQ_OK 0
+#define LLVQ_EINVAL (-1) /* null pointer, bad shape, unknown layout                         */
+#define LLVQ_EALIGN (-2) /* a device pointer is not aligned as documented                   */
+#define LLVQ_ESIZE (-3)  /* a buffer or the context's scratch is too small for the request  */
+#define LLVQ_ECUDA (-4)  /* a CUDA runtime call failed                                      */
+#define LLVQ_EINDEX (-5) /* at least one code word named no point (llvq_expand_check only)  */
+
+#define LLVQ_MAX_GROUP 8       /* matrices in one grouped launch                             */
+#define LLVQ_MAX_K 98304       /* largest k_padded the GEMV stages in shared memory          */
+
+typedef struct llvq_ctx llvq_ctx;
+
+/* One matrix of a grouped launch: its records, fp16 row scales, two gain centroids, output. */
+typedef struct {
+    const void *layout;     /* device, 128-byte aligned                                      */
+    const void *row_scale;  /* device, fp16[rows]                                            */
+    float *y;               /* device, f32[rows]                                             */
+    int64_t rows;
+    float gain[2];          /* centroid chosen by each block's gain bit [Sec. 2.1]           */
+} llvq_problem;
+
+/* Builds the class, index-base and Golay tables on the host, uploads them to `device`, and
+ * allocates the context's reduction scratch (scratch_bytes; 0 = default 32 MiB).  Synchronous. */
+int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes);
+void llvq_destroy(llvq_ctx *ctx);
+const char *llvq_strerror(int code);
+
+/* Host queries.  Number of classes (301), points in the ball, and first index of class c
+ * (c = 301 gives the number of points)  [Sec. 2.1]. */
+int llvq_num_classes(const llvq_ctx *ctx);
+uint64_t llvq_class_base(const llvq_ctx *ctx, int c);
+
+/* Bytes of a layout buffer for a rows x (k_padded/24) matrix. Host query. */
+int llvq_layout_bytes(int layout, int64_t rows, int64_t k_padded, size_t *bytes);
+
+/* [Sec. 2.2] Unfolds rows*nb code words (row-major, codes[row*nb + b]) into `layout_out`
+ * (128-byte aligned, at least llvq_layout_bytes).  A code that names no point (index not below
+ * the number of points, or bits above bit 47 set) becomes the empty record (class 511, all
+ * fields zero) and, if bad_count is not null, adds one to *bad_count (device uint32, which the
+ * caller zeroes).  Bit-exact by construction: integer arithmetic only. */
+int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, int64_t nb,
+                void *layout_out, size_t out_bytes, uint32_t *bad_count, void *stream);
+
+/* [Sec. 2.3] y[row] = row_scale[row] * sum_b gain[g_b] / (4 sqrt(m_b)) * sum_i x_b,i * x[24b+i],
+ * m_b the shell of block b's class, with f32 accumulation (the products of the small integer
+ * coordinates with fp16 x are exact in f32).  gain is a HOST pointer to two floats.  x is fp16,
+ * 16-byte aligned; y is f32.  The summation order of a row depends only on nb, never on the
+ * launch geometry, so a grouped launch returns bit-identical rows. */
+int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row_scale,
+              const float *gain, const void *x, float *y, int64_t rows, int64_t k_padded, void *stream);
+
+/* [Sec. 3.4] One launch over n <= LLVQ_MAX_GROUP row-concatenated matrices that share x and
+ * k_padded (q/k/v, gate/up).  `problems` is a HOST array, copied before the call returns. */
+int llvq_gemv_grouped(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n,
+                      const void *x, int64_t k_padded, void *stream);
+
+/* [Table "layout scale", FP16 control] y = W x, W fp16 row-major rows x k (k a multiple of 8,
+ * W and x 16-byte aligned), f32 accumulation, f32 y. */
+int llvq_gemv_fp16(const void *W, const void *x, float *y, int64_t rows, int64_t k, void *stream);
+
+/* [Table "layout scale", no-weights control] The launch llvq_gemv(LLVQ_PLANES) would make - same
+ * grid, shared memory, x staging, reduction and epilogue - with no record read; y = 0. */
+int llvq_gemv_noweights(llvq_ctx *ctx, const void *row_scale, const void *x, float *y,
+                        int64_t rows, int64_t k_padded, void *stream);
+
+/* Decoded weights as fp16, W[row*k_padded + 24b + i] = fp16(row_scale * gain[g] * x_i / (4 sqrt m))
+ * (product formed in f32, rounded once).  Feeds llvq_gemv_fp16. */
+int llvq_dequant_fp16(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row_scale,
+                      const float *gain, void *W, int64_t rows, int64_t k_padded, void *stream);
+
+/* Test hook: the integer coordinates (coords[(row*nb + b)*24 + i]) and class id
+ * (class_ids[row*nb + b]) a layout buffer decodes to, for the bit-exact check of Sec. 2.4. */
+int llvq_decode_i8(llvq_ctx *ctx, int layout, const void *layout_buf, int8_t *coords,
+                   uint16_t *class_ids, int64_t rows, int64_t nb, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LLVQ_H */

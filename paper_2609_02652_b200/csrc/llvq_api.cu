@@ -1,0 +1,236 @@
+// C ABI of the library: argument checks, context set-up, and the hand-off to the kernels.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "llvq_internal.cuh"
+
+using namespace llvq;
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+int layout_cell_bytes(int layout) { return layout == LLVQ_PLANES ? kCellBytes : kOneHotCellBytes; }
+
+}  // namespace
+
+extern "C" {
+
+const char *llvq_strerror(int code) {
+    switch (code) {
+        case LLVQ_OK: return "ok";
+        case LLVQ_EINVAL: return "invalid argument (null pointer, bad shape or unknown layout)";
+        case LLVQ_EALIGN: return "device pointer not aligned as documented";
+        case LLVQ_ESIZE: return "buffer or context scratch too small";
+        case LLVQ_ECUDA: return "CUDA runtime error";
+        case LLVQ_EINDEX: return "a code word names no lattice point";
+        default: return "unknown error";
+    }
+}
+
+int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
+    if (!out) return LLVQ_EINVAL;
+    *out = nullptr;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess) return LLVQ_ECUDA;
+    if (device < 0 || device >= ndev) return LLVQ_EINVAL;
+    DeviceGuard guard(device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    llvq_ctx *ctx = new (std::nothrow) llvq_ctx();
+    if (!ctx) return LLVQ_ECUDA;
+    ctx->device = device;
+    ctx->table_blob = nullptr; ctx->partial = nullptr; ctx->counter = nullptr;
+    if (!build_tables(ctx->host)) { delete ctx; return LLVQ_EINVAL; }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
+
+    const HostTables &h = ctx->host;
+    struct Part { const void *src; size_t bytes; size_t off; } parts[8] = {
+        {h.base.data(), h.base.size() * 8, 0},          {h.desc.data(), h.desc.size() * sizeof(ClassDesc), 0},
+        {h.golay_by_weight.data(), 4096 * 4, 0},        {h.golay_by_message.data(), 4096 * 4, 0},
+        {h.cls_scale.data(), kClassSlots * 4, 0},       {h.cls_parity.data(), kClassSlots * 4, 0},
+        {h.cls_value.data(), kClassSlots * 8 * 4, 0},   {h.cls_dist.data(), kClassSlots * 8, 0}};
+    size_t total = 0;
+    for (auto &p : parts) { p.off = total; total += round_up(p.bytes, 256); }
+    if (cudaMalloc(&ctx->table_blob, total) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
+    for (auto &p : parts)
+        if (cudaMemcpy((char *)ctx->table_blob + p.off, p.src, p.bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
+            llvq_destroy(ctx);
+            return LLVQ_ECUDA;
+        }
+    char *blob = (char *)ctx->table_blob;
+    DeviceTables &d = ctx->dev;
+    d.base = (const uint64_t *)(blob + parts[0].off);
+    d.desc = (const ClassDesc *)(blob + parts[1].off);
+    d.golay_by_weight = (const uint32_t *)(blob + parts[2].off);
+    d.golay_by_message = (const uint32_t *)(blob + parts[3].off);
+    d.cls_scale = (const float *)(blob + parts[4].off);
+    d.cls_parity = (const uint32_t *)(blob + parts[5].off);
+    d.cls_value = (const float *)(blob + parts[6].off);
+    d.cls_dist = (const uint8_t *)(blob + parts[7].off);
+    std::memcpy(d.weight_offset, h.weight_offset, sizeof d.weight_offset);
+    d.num_classes = h.num_classes;
+    d.num_points = h.num_points;
+
+    if (scratch_bytes == 0) scratch_bytes = (size_t)32 << 20;
+    ctx->partial_floats = scratch_bytes / 4;
+    ctx->counter_slots = ctx->partial_floats / 32 + 1;     // a row group has at least one item
+    if (cudaMalloc(&ctx->partial, ctx->partial_floats * 4) != cudaSuccess ||
+        cudaMalloc(&ctx->counter, ctx->counter_slots * 4) != cudaSuccess ||
+        cudaMemset(ctx->counter, 0, ctx->counter_slots * 4) != cudaSuccess) {
+        llvq_destroy(ctx);
+        return LLVQ_ECUDA;
+    }
+    if (gemv_configure(ctx) != 0 || cudaDeviceSynchronize() != cudaSuccess) { llvq_destroy(ctx); return LLVQ_ECUDA; }
+    *out = ctx;
+    return LLVQ_OK;
+}
+
+void llvq_destroy(llvq_ctx *ctx) {
+    if (!ctx) return;
+    DeviceGuard guard(ctx->device);
+    cudaFree(ctx->table_blob);
+    cudaFree(ctx->partial);
+    cudaFree(ctx->counter);
+    delete ctx;
+}
+
+int llvq_num_classes(const llvq_ctx *ctx) { return ctx ? ctx->host.num_classes : LLVQ_EINVAL; }
+
+uint64_t llvq_class_base(const llvq_ctx *ctx, int c) {
+    if (!ctx || c < 0 || c > ctx->host.num_classes) return ~0ull;
+    return ctx->host.base[(size_t)c];
+}
+
+int llvq_layout_bytes(int layout, int64_t rows, int64_t k_padded, size_t *bytes) {
+    if (!bytes || rows <= 0 || k_padded <= 0 || k_padded % 24 != 0) return LLVQ_EINVAL;
+    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT) return LLVQ_EINVAL;
+    const size_t groups = (size_t)((rows + kRowsPerGroup - 1) / kRowsPerGroup);
+    *bytes = groups * (size_t)(k_padded / 24) * (size_t)layout_cell_bytes(layout);
+    return LLVQ_OK;
+}
+
+int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, int64_t nb, void *layout_out,
+                size_t out_bytes, uint32_t *bad_count, void *stream) {
+    if (!ctx || !codes || !layout_out || rows <= 0 || nb <= 0) return LLVQ_EINVAL;
+    size_t need = 0;
+    if (llvq_layout_bytes(layout, rows, nb * 24, &need) != LLVQ_OK) return LLVQ_EINVAL;
+    if (out_bytes < need) return LLVQ_ESIZE;
+    if (!aligned(layout_out, 128) || !aligned(codes, 8) || (bad_count && !aligned(bad_count, 4))) return LLVQ_EALIGN;
+    if (rows * nb > ((int64_t)1 << 36)) return LLVQ_ESIZE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    return launch_expand(ctx, layout, codes, rows, nb, layout_out, bad_count, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+}
+
+static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n, const void *x, int64_t k_padded,
+                    bool no_weights, void *stream) {
+    if (!ctx || !problems || !x || n < 1 || n > LLVQ_MAX_GROUP) return LLVQ_EINVAL;
+    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT) return LLVQ_EINVAL;
+    if (k_padded <= 0 || k_padded % 24 != 0) return LLVQ_EINVAL;
+    if (k_padded > LLVQ_MAX_K) return LLVQ_ESIZE;
+    if (!aligned(x, 16)) return LLVQ_EALIGN;
+    GemvParams p;
+    std::memset(&p, 0, sizeof p);
+    p.nprob = n;
+    p.x = (const __half *)x;
+    p.nb = (int)(k_padded / 24);
+    p.tiles = p.nb / kTileCells;
+    p.tail_cells = p.nb % kTileCells;
+    p.nchunk = p.tiles ? (p.tiles + kChunkTiles - 1) / kChunkTiles : 1;
+    int64_t groups = 0;
+    for (int i = 0; i < n; i++) {
+        const llvq_problem &q = problems[i];
+        if ((!q.layout && !no_weights) || !q.row_scale || !q.y || q.rows <= 0) return LLVQ_EINVAL;
+        if (!aligned(q.layout, 128) || !aligned(q.row_scale, 2) || !aligned(q.y, 4)) return LLVQ_EALIGN;
+        p.prob[i].layout = (const uint8_t *)q.layout;
+        p.prob[i].row_scale = (const __half *)q.row_scale;
+        p.prob[i].y = q.y;
+        p.prob[i].rows = (int)q.rows;
+        p.prob[i].group_begin = (int)groups;
+        p.prob[i].gain0 = q.gain[0];
+        p.prob[i].gain1 = q.gain[1];
+        if (q.rows > ((int64_t)1 << 30)) return LLVQ_ESIZE;
+        groups += (q.rows + kRowsPerGroup - 1) / kRowsPerGroup;
+    }
+    const int64_t items = groups * p.nchunk;
+    if (items > ((int64_t)1 << 30)) return LLVQ_ESIZE;
+    if (p.nchunk > 1 && ((size_t)items * 32 > ctx->partial_floats || (size_t)groups > ctx->counter_slots)) return LLVQ_ESIZE;
+    p.total_groups = (int)groups;
+    p.total_items = (int)items;
+    p.partial = ctx->partial;
+    p.counter = ctx->counter;
+    p.cls_scale = ctx->dev.cls_scale;
+    p.cls_parity = ctx->dev.cls_parity;
+    p.cls_value = ctx->dev.cls_value;
+    if (gemv_smem_bytes(layout, p.nb, n) > (size_t)ctx->max_smem_optin) return LLVQ_ESIZE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    return launch_gemv(ctx, layout, p, no_weights, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+}
+
+int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row_scale, const float *gain, const void *x,
+              float *y, int64_t rows, int64_t k_padded, void *stream) {
+    if (!gain) return LLVQ_EINVAL;
+    llvq_problem q;
+    q.layout = layout_buf; q.row_scale = row_scale; q.y = y; q.rows = rows; q.gain[0] = gain[0]; q.gain[1] = gain[1];
+    return run_gemv(ctx, layout, &q, 1, x, k_padded, false, stream);
+}
+
+int llvq_gemv_grouped(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n, const void *x, int64_t k_padded,
+                      void *stream) {
+    return run_gemv(ctx, layout, problems, n, x, k_padded, false, stream);
+}
+
+int llvq_gemv_noweights(llvq_ctx *ctx, const void *row_scale, const void *x, float *y, int64_t rows, int64_t k_padded,
+                        void *stream) {
+    llvq_problem q;
+    q.layout = nullptr; q.row_scale = row_scale; q.y = y; q.rows = rows; q.gain[0] = 1.f; q.gain[1] = 1.f;
+    return run_gemv(ctx, LLVQ_PLANES, &q, 1, x, k_padded, true, stream);
+}
+
+int llvq_gemv_fp16(const void *W, const void *x, float *y, int64_t rows, int64_t k, void *stream) {
+    if (!W || !x || !y || rows <= 0 || k <= 0 || k % 8 != 0) return LLVQ_EINVAL;
+    if (!aligned(W, 16) || !aligned(x, 16) || !aligned(y, 4)) return LLVQ_EALIGN;
+    if ((rows + 7) / 8 > 0x7fffffffll) return LLVQ_ESIZE;
+    return launch_gemv_fp16((const __half *)W, (const __half *)x, y, rows, k, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+}
+
+int llvq_dequant_fp16(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row_scale, const float *gain, void *W,
+                      int64_t rows, int64_t k_padded, void *stream) {
+    if (!ctx || !layout_buf || !row_scale || !gain || !W || rows <= 0 || k_padded <= 0 || k_padded % 24 != 0) return LLVQ_EINVAL;
+    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT) return LLVQ_EINVAL;
+    if (!aligned(layout_buf, 128) || !aligned(W, 16) || !aligned(row_scale, 2)) return LLVQ_EALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    return launch_dequant(ctx, layout, (const uint8_t *)layout_buf, (const __half *)row_scale, gain[0], gain[1], (__half *)W, rows,
+                          k_padded / 24, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+}
+
+int llvq_decode_i8(llvq_ctx *ctx, int layout, const void *layout_buf, int8_t *coords, uint16_t *class_ids, int64_t rows,
+                   int64_t nb, void *stream) {
+    if (!ctx || !layout_buf || !coords || !class_ids || rows <= 0 || nb <= 0) return LLVQ_EINVAL;
+    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT) return LLVQ_EINVAL;
+    if (!aligned(layout_buf, 128) || !aligned(class_ids, 2)) return LLVQ_EALIGN;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    return launch_decode_i8(ctx, layout, (const uint8_t *)layout_buf, coords, class_ids, rows, nb, (cudaStream_t)stream) == cudaSuccess
+               ? LLVQ_OK : LLVQ_ECUDA;
+}
+
+}  // extern "C"

@@ -1,0 +1,226 @@
+// The expander (paper Sec. 2.2, "Unfolding at load time"): one pass that turns every 48-bit code
+// word into its decoded-field record - class id, gain bit, sign mask, per-coordinate level - in
+// the bit-plane or the one-hot layout.  Integer arithmetic only, so the output is bit-exact.
+//
+// The index splits as the paper states it (Sec. 2.1: classes first, then arrangements and signs
+// inside a class, as a mixed-radix number).  The digit order used here:
+//   even type:  ((codeword rank * perm_a + rank_a) * perm_b + rank_b) << sign_bits | signs
+//   odd type:   arrangement rank * 4096 + message bits of the codeword
+// Arrangement ranks are lexicographic over the distinct orderings, smaller magnitude first; sign
+// bits run over the non-zero off-support coordinates first, then the support coordinates but the
+// last, whose sign restores the sum condition mod 8.
+#include "llvq_internal.cuh"
+
+namespace llvq {
+namespace {
+
+struct Unranker {
+    uint64_t rank, total;
+    int left;
+    int cnt[7];
+};
+
+// Next value index (0..NV-1) of the lexicographically rank-th ordering.
+template <int NV>
+__device__ __forceinline__ int unrank_step(Unranker &u) {
+    int pick = 0;
+    bool done = false;
+#pragma unroll
+    for (int v = 0; v < NV; v++) {
+        if (!done && u.cnt[v] > 0) {
+            uint64_t sub = u.total * (uint64_t)u.cnt[v] / (uint64_t)u.left;   // orderings starting with v
+            if (u.rank < sub) {
+                pick = v; u.total = sub; u.cnt[v]--; done = true;
+            } else {
+                u.rank -= sub;
+            }
+        }
+    }
+    u.left--;
+    return pick;
+}
+
+struct Decoded {
+    int cls, gain;
+    uint32_t smask;
+    uint32_t mag[3];   // magnitude of coordinate i in nibble i%8 of word i/8
+};
+
+__device__ __forceinline__ void set_mag(Decoded &d, int i, int a) { d.mag[i >> 3] |= (uint32_t)a << (4 * (i & 7)); }
+
+__device__ bool decode_code(uint64_t code, const DeviceTables &T, Decoded &d) {
+    d.cls = kEmptyClass; d.gain = 0; d.smask = 0; d.mag[0] = d.mag[1] = d.mag[2] = 0;
+    const uint64_t idx = code & ((1ull << kIndexBits) - 1);
+    if ((code >> 48) != 0 || idx >= T.num_points) return false;
+    // class: last c with base[c] <= idx
+    int lo = 0, hi = T.num_classes;
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (__ldg(&T.base[mid]) <= idx) lo = mid; else hi = mid;
+    }
+    const ClassDesc c = T.desc[lo];
+    uint64_t r = idx - __ldg(&T.base[lo]);
+    d.cls = lo;
+    d.gain = (int)((code >> kIndexBits) & 1);
+
+    if (c.odd) {
+        const uint32_t cw = __ldg(&T.golay_by_message[(uint32_t)r & 4095u]);
+        Unranker u;
+        u.rank = r >> 12; u.total = c.perm_a; u.left = 24;
+#pragma unroll
+        for (int v = 0; v < 7; v++) u.cnt[v] = c.cnt[v];
+#pragma unroll
+        for (int i = 0; i < 24; i++) {
+            const int a = 1 + 2 * unrank_step<7>(u);
+            const int want = 1 + 2 * (int)((cw >> i) & 1);     // residue of x_i mod 4
+            if ((a & 3) != want) d.smask |= 1u << i;
+            set_mag(d, i, a);
+        }
+        return true;
+    }
+
+    const uint64_t sigma = r & ((1ull << c.sign_bits) - 1);
+    r >>= c.sign_bits;
+    const uint64_t rank_b = r % c.perm_b; r /= c.perm_b;
+    const uint64_t rank_a = r % c.perm_a; r /= c.perm_a;
+    const uint32_t cw = __ldg(&T.golay_by_weight[T.weight_offset[c.w] + (int)r]);
+    Unranker ua, ub;
+    ua.rank = rank_a; ua.total = c.perm_a; ua.left = c.w;
+    ub.rank = rank_b; ub.total = c.perm_b; ub.left = 24 - c.w;
+#pragma unroll
+    for (int v = 0; v < 4; v++) { ua.cnt[v] = c.cnt[v]; ub.cnt[v] = c.cnt[4 + v]; }
+    int off_bit = 0, sup_seen = 0, last = -1, sum = 0;
+#pragma unroll
+    for (int i = 0; i < 24; i++) {
+        int a; bool neg = false;
+        if ((cw >> i) & 1) {
+            a = 2 + 4 * unrank_step<4>(ua);
+            sup_seen++;
+            if (sup_seen < c.w) neg = (sigma >> (c.nz_b + sup_seen - 1)) & 1; else last = i;
+        } else {
+            a = 4 * unrank_step<4>(ub);
+            if (a) { neg = (sigma >> off_bit) & 1; off_bit++; }
+        }
+        set_mag(d, i, a);
+        if (neg) d.smask |= 1u << i;
+        sum += neg ? -a : a;
+    }
+    if (last >= 0 && (sum & 7) != 0) d.smask |= 1u << last;     // the repair sign
+    return true;
+}
+
+// word j of the bit-plane record: coordinate 8j+2k+e -> level at (4+16e+4k) mod 32, sign at (15+16e+4k) mod 32
+__device__ __forceinline__ uint32_t planes_word(const Decoded &d, int j) {
+    uint32_t w = 0;
+#pragma unroll
+    for (int n = 0; n < 8; n++) {
+        const int k = n >> 1, e = n & 1, i = 8 * j + n;
+        const uint32_t level = ((d.mag[j] >> (4 * n)) & 15u) >> 1;
+        w |= level << ((4 + 16 * e + 4 * k) & 31);
+        w |= ((d.smask >> i) & 1u) << ((15 + 16 * e + 4 * k) & 31);
+    }
+    return w;
+}
+
+__global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, const uint64_t *__restrict__ codes, int64_t rows, int64_t nb,
+                                                            uint8_t *__restrict__ out, uint32_t *bad_count) {
+    const int64_t tiles = nb / kTileCells, tail = nb % kTileCells, units = tiles + tail;
+    const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = (int)(gid & 31);
+    const int64_t unit_id = gid >> 5;
+    const int64_t groups = (rows + kRowsPerGroup - 1) / kRowsPerGroup;
+    if (unit_id >= groups * units) return;
+    const int64_t rg = unit_id / units, u = unit_id % units;
+    const int64_t row = rg * kRowsPerGroup + lane;
+    uint8_t *grp = out + (size_t)rg * (size_t)nb * kCellBytes;
+    const bool full = u < tiles;
+    const int ncell = full ? kTileCells : 1;
+    const int64_t b0 = full ? u * kTileCells : tiles * kTileCells + (u - tiles);
+    uint32_t w[3][4];
+    uint32_t hdr[4];
+    int bad = 0;
+#pragma unroll 1
+    for (int q = 0; q < ncell; q++) {
+        Decoded d;
+        if (row < rows) {
+            if (!decode_code(codes[row * nb + b0 + q], T, d)) bad++;
+        } else {
+            d.cls = kEmptyClass; d.gain = 0; d.smask = 0; d.mag[0] = d.mag[1] = d.mag[2] = 0;
+        }
+#pragma unroll
+        for (int qq = 0; qq < 4; qq++)
+            if (qq == q) {
+                w[0][qq] = planes_word(d, 0); w[1][qq] = planes_word(d, 1); w[2][qq] = planes_word(d, 2);
+                hdr[qq] = (uint32_t)d.cls | ((uint32_t)d.gain << 9);
+            }
+    }
+    if (full) {
+        uint8_t *tile = grp + (size_t)u * kTileBytes;
+#pragma unroll
+        for (int j = 0; j < 3; j++)
+            *reinterpret_cast<uint4 *>(tile + 512 * j + 16 * lane) = make_uint4(w[j][0], w[j][1], w[j][2], w[j][3]);
+        *reinterpret_cast<uint2 *>(tile + 1536 + 8 * lane) = make_uint2(hdr[0] | (hdr[1] << 16), hdr[2] | (hdr[3] << 16));
+    } else {
+        uint8_t *cell = grp + (size_t)tiles * kTileBytes + (size_t)(u - tiles) * kCellBytes;
+#pragma unroll
+        for (int j = 0; j < 3; j++) *reinterpret_cast<uint32_t *>(cell + 128 * j + 4 * lane) = w[j][0];
+        *reinterpret_cast<uint16_t *>(cell + 384 + 2 * lane) = (uint16_t)hdr[0];
+    }
+    if (bad && bad_count) atomicAdd(bad_count, (uint32_t)bad);
+}
+
+__global__ void __launch_bounds__(256) expand_onehot_kernel(DeviceTables T, const uint64_t *__restrict__ codes, int64_t rows, int64_t nb,
+                                                            uint8_t *__restrict__ out, uint32_t *bad_count) {
+    const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = (int)(gid & 31);
+    const int64_t cell_id = gid >> 5;
+    const int64_t groups = (rows + kRowsPerGroup - 1) / kRowsPerGroup;
+    if (cell_id >= groups * nb) return;
+    const int64_t rg = cell_id / nb, b = cell_id % nb;
+    const int64_t row = rg * kRowsPerGroup + lane;
+    Decoded d;
+    bool ok = true;
+    if (row < rows) ok = decode_code(codes[row * nb + b], T, d);
+    else { d.cls = kEmptyClass; d.gain = 0; d.smask = 0; d.mag[0] = d.mag[1] = d.mag[2] = 0; }
+    uint32_t mask[4] = {0, 0, 0, 0};
+    if (d.cls != kEmptyClass) {
+        const uint8_t *dist = T.cls_dist + d.cls * 8;
+        const int d1 = dist[1], d2 = dist[2], d3 = dist[3], d4 = dist[4];
+        const int nd = T.desc[d.cls].ndist;
+#pragma unroll
+        for (int i = 0; i < 24; i++) {
+            const int a = (int)((d.mag[i >> 3] >> (4 * (i & 7))) & 15u);
+            if (nd > 1 && a == d1) mask[0] |= 1u << i;
+            if (nd > 2 && a == d2) mask[1] |= 1u << i;
+            if (nd > 3 && a == d3) mask[2] |= 1u << i;
+            if (nd > 4 && a == d4) mask[3] |= 1u << i;
+        }
+    }
+    uint32_t *cell = reinterpret_cast<uint32_t *>(out + (size_t)cell_id * kOneHotCellBytes);
+    cell[0 * 32 + lane] = d.smask | ((uint32_t)(d.cls & 255) << 24);
+    cell[1 * 32 + lane] = mask[0] | ((uint32_t)(d.cls >> 8) << 24) | ((uint32_t)d.gain << 25);
+    cell[2 * 32 + lane] = mask[1];
+    cell[3 * 32 + lane] = mask[2];
+    cell[4 * 32 + lane] = mask[3];
+    if (!ok && bad_count) atomicAdd(bad_count, 1u);
+}
+
+}  // namespace
+
+cudaError_t launch_expand(const llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, int64_t nb,
+                          void *out, uint32_t *bad_count, cudaStream_t s) {
+    const int64_t groups = (rows + kRowsPerGroup - 1) / kRowsPerGroup;
+    if (layout == LLVQ_PLANES) {
+        const int64_t units = nb / kTileCells + nb % kTileCells;
+        const int64_t threads = groups * units * 32;
+        const int64_t blocks = (threads + 255) / 256;
+        expand_planes_kernel<<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count);
+    } else {
+        const int64_t threads = groups * nb * 32;
+        const int64_t blocks = (threads + 255) / 256;
+        expand_onehot_kernel<<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace llvq

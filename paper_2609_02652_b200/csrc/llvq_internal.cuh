@@ -1,0 +1,85 @@
+// Internal declarations shared by the translation units of the library (not part of the ABI).
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "../../include/llvq.h"
+#include "llvq_tables.h"
+
+namespace llvq {
+
+// Geometry of the bit-plane layout (see include/llvq.h).
+constexpr int kRowsPerGroup = 32;
+constexpr int kCellBytes = 448;        // 32 rows x 14 bytes
+constexpr int kTileCells = 4;
+constexpr int kTileBytes = 1792;
+constexpr int kOneHotCellBytes = 640;  // 32 rows x 20 bytes
+
+// A GEMV work item is one row group times one "chunk" of consecutive tiles.  The chunk length
+// depends on nb only, so the order in which a row is summed never depends on the launch.
+constexpr int kChunkTiles = 3;
+
+struct DeviceTables {
+    const uint64_t *base;            // num_classes + 1
+    const ClassDesc *desc;           // num_classes
+    const uint32_t *golay_by_weight; // 4096
+    const uint32_t *golay_by_message;// 4096
+    const float *cls_scale;          // 512
+    const uint32_t *cls_parity;      // 512
+    const float *cls_value;          // 512 x 8
+    const uint8_t *cls_dist;         // 512 x 8
+    int weight_offset[25];
+    int num_classes;
+    uint64_t num_points;
+};
+
+struct GemvProblemDev {
+    const uint8_t *layout;
+    const __half *row_scale;
+    float *y;
+    int rows;
+    int group_begin;   // index of this matrix's first row group in the concatenation
+    float gain0, gain1;
+};
+
+struct GemvParams {
+    GemvProblemDev prob[LLVQ_MAX_GROUP];
+    int nprob;
+    const __half *x;
+    int nb, tiles, tail_cells, nchunk;
+    int total_groups, total_items;
+    float *partial;        // total_items x 32 floats (context scratch)
+    unsigned *counter;     // total_groups (context scratch, zero between launches)
+    const float *cls_scale;
+    const uint32_t *cls_parity;
+    const float *cls_value;
+};
+
+}  // namespace llvq
+
+struct llvq_ctx {
+    int device;
+    llvq::HostTables host;
+    llvq::DeviceTables dev;
+    void *table_blob;        // one allocation holding every table
+    float *partial;
+    unsigned *counter;
+    size_t partial_floats, counter_slots;
+    int sm_count;
+    int max_smem_optin;
+};
+
+namespace llvq {
+cudaError_t launch_expand(const llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, int64_t nb,
+                          void *out, uint32_t *bad_count, cudaStream_t s);
+cudaError_t launch_gemv(const llvq_ctx *ctx, int layout, const GemvParams &p, bool no_weights, cudaStream_t s);
+cudaError_t launch_gemv_fp16(const __half *W, const __half *x, float *y, int64_t rows, int64_t k, cudaStream_t s);
+cudaError_t launch_dequant(const llvq_ctx *ctx, int layout, const uint8_t *buf, const __half *row_scale, float g0, float g1,
+                           __half *W, int64_t rows, int64_t nb, cudaStream_t s);
+cudaError_t launch_decode_i8(const llvq_ctx *ctx, int layout, const uint8_t *buf, int8_t *coords, uint16_t *class_ids,
+                             int64_t rows, int64_t nb, cudaStream_t s);
+size_t gemv_smem_bytes(int layout, int nb, int nprob);
+int gemv_configure(const llvq_ctx *ctx);   // sets the kernels' shared-memory attributes once
+}  // namespace llvq

@@ -1,0 +1,199 @@
+"""Parity of the CUDA path against the CPU oracle, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import GAIN, check_gemv, make_case
+
+pytestmark = pytest.mark.gpu
+
+N_POINTS = 111_043_117_458_000
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2609_02652_b200 import binding
+
+    binding.load()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def ctx(B):
+    c = B.create(0)
+    yield c
+    c.close()
+
+
+def _expected(oracle, layout, case):
+    return oracle.pack_planes(case.codes, case.rows, case.nb) if layout == 0 else oracle.pack_onehot(case.codes, case.rows, case.nb)
+
+
+SMALL = [(1, 24), (3, 48), (33, 24 * 33), (40, 24 * 7), (64, 24 * 9 - 5), (32, 96), (31, 24 * 13), (257, 24 * 21)]
+
+
+def test_tables_agree_with_oracle(B, ctx, oracle):
+    assert B.num_classes(ctx) == oracle.num_classes() == 301
+    for c in range(301):
+        assert B.class_base(ctx, c) == oracle.class_info(c)["base"]
+    assert B.class_base(ctx, 301) == N_POINTS
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("rows,k", SMALL)
+def test_expand_bit_exact_small(B, ctx, oracle, layout, rows, k):
+    case = make_case(rows, k, seed=20 + rows)
+    out = B.expand(ctx, layout, case.d_codes, rows, case.nb)
+    torch.cuda.synchronize()
+    assert out.numel() == B.layout_bytes(layout, rows, case.nb * 24)
+    assert np.array_equal(out.cpu().numpy(), _expected(oracle, layout, case))
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_expand_bit_exact_config0_and_extra_indices(B, ctx, oracle, layout):
+    from paper_2609_02652_b200 import datagen
+
+    case = make_case(3072, 3072, seed=0)
+    out = B.expand(ctx, layout, case.d_codes, case.rows, case.nb)
+    assert np.array_equal(out.cpu().numpy(), _expected(oracle, layout, case))
+    # 10 000 more indices, no gain bit, as a 100 x 100 matrix
+    extra = datagen.make_indices(10_000, seed=0)
+    case.rows, case.nb, case.codes = 100, 100, extra.numpy().astype(np.uint64)
+    out = B.expand(ctx, layout, extra.cuda(), 100, 100)
+    assert np.array_equal(out.cpu().numpy(), _expected(oracle, layout, case))
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_expand_whole_first_shell_class_edges_and_bad_codes(B, ctx, oracle, layout):
+    # all 196 560 indices of shell 2 as a 4095 x 48 matrix
+    codes = np.arange(196_560, dtype=np.uint64)
+    case = make_case(1, 24, 0, device=None)
+    case.rows, case.nb, case.codes = 4095, 48, codes
+    out = B.expand(ctx, layout, torch.from_numpy(codes.astype(np.int64)).cuda(), 4095, 48)
+    assert np.array_equal(out.cpu().numpy(), _expected(oracle, layout, case))
+    # first and last index of every class, with and without the gain bit; then codes naming no point
+    edges = []
+    for c in range(301):
+        i = oracle.class_info(c)
+        edges += [i["base"], i["base"] + i["size"] - 1, (i["base"] + i["size"] // 2) | (1 << 47)]
+    bad = [N_POINTS, N_POINTS + 12345, (1 << 47) - 1, N_POINTS | (1 << 47), 1 << 48, (1 << 63) | 5]
+    codes = np.array(edges + bad + [0] * (7 * 131 - len(edges) - len(bad)), dtype=np.uint64)
+    case.rows, case.nb, case.codes = 131, 7, codes
+    cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = B.expand(ctx, layout, torch.from_numpy(codes.view(np.int64)).cuda(), 131, 7, bad_count=cnt)
+    assert np.array_equal(out.cpu().numpy(), _expected(oracle, layout, case))
+    assert int(cnt.item()) == len(bad)
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("rows,k", [(40, 24 * 7), (257, 24 * 21), (3072, 3072)])
+def test_decode_bit_exact(B, ctx, oracle, layout, rows, k):
+    case = make_case(rows, k, seed=3)
+    buf = B.expand(ctx, layout, case.d_codes, rows, case.nb)
+    coords, cls = B.decode_i8(ctx, layout, buf, rows, case.nb)
+    xs, ref_cls = oracle.decode_batch(case.codes)
+    assert np.array_equal(coords.cpu().numpy().reshape(-1, 24), xs)
+    assert np.array_equal(cls.cpu().numpy().ravel().astype(np.int32), ref_cls)
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("rows,k", SMALL + [(3072, 3072), (1024, 2560), (96, 24 * 406)])
+def test_gemv_every_row(B, ctx, oracle, layout, rows, k):
+    case = make_case(rows, k, seed=rows + k)
+    buf = B.expand(ctx, layout, case.d_codes, rows, case.nb)
+    y = B.gemv(ctx, layout, buf, case.d_scale, GAIN, case.d_x, rows, case.nb * 24)
+    check_gemv(oracle, case, y)
+    # a second launch on the same context finds the scratch clean
+    y2 = B.gemv(ctx, layout, buf, case.d_scale, GAIN, case.d_x, rows, case.nb * 24)
+    assert torch.equal(y, y2)
+
+
+def test_gemv_special_cases(B, ctx, oracle):
+    case = make_case(70, 24 * 30, seed=9)
+    case.row_scale[5] = 0.0            # a scale that rounds to zero: y must be exactly zero
+    case.codes[17] = N_POINTS          # a code naming no point contributes nothing
+    case.d_scale = torch.from_numpy(case.row_scale).cuda()
+    case.d_codes = torch.from_numpy(case.codes.view(np.int64)).cuda()
+    buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    y = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
+    check_gemv(oracle, case, y)
+    assert y[5].item() == 0.0
+    # gain (1, 1) is the gain-free result
+    y1 = B.gemv(ctx, 0, buf, case.d_scale, (1.0, 1.0), case.d_x, case.rows, case.nb * 24)
+    check_gemv(oracle, case, y1, gain=(1.0, 1.0))
+    # x = e_j returns column j of the dequantised matrix
+    W = oracle.dequant(case.codes, case.rows, case.nb, case.row_scale, GAIN)
+    for j in (0, 23, 24 * 30 - 1, 333):
+        e = torch.zeros(case.nb * 24, dtype=torch.float16, device="cuda")
+        e[j] = 1
+        yj = B.gemv(ctx, 0, buf, case.d_scale, GAIN, e, case.rows, case.nb * 24).cpu().numpy()
+        assert np.allclose(yj, W[:, j], rtol=2e-7, atol=0)
+
+
+def test_planes_and_onehot_agree(B, ctx):
+    case = make_case(520, 24 * 45, seed=4)
+    bp = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    bo = B.expand(ctx, 1, case.d_codes, case.rows, case.nb)
+    cp, kp = B.decode_i8(ctx, 0, bp, case.rows, case.nb)
+    co, ko = B.decode_i8(ctx, 1, bo, case.rows, case.nb)
+    assert torch.equal(cp, co) and torch.equal(kp, ko)
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_grouped_launch_is_bit_identical(B, ctx, oracle, layout):
+    k = 2560
+    shapes = [(4096, 0), (1024, 1), (1000, 2)]
+    cases = [make_case(r, k, seed=1, tensor_id=t) for r, t in shapes]
+    for c in cases[1:]:
+        c.x, c.d_x = cases[0].x, cases[0].d_x          # a fused group shares x
+    bufs = [B.expand(ctx, layout, c.d_codes, c.rows, c.nb) for c in cases]
+    gains = [(0.75, 1.5), (1.0, 0.5), (1.25, 2.0)]
+    single = [B.gemv(ctx, layout, b, c.d_scale, g, c.d_x, c.rows, c.nb * 24) for b, c, g in zip(bufs, cases, gains)]
+    ys = [torch.full((c.rows,), float("nan"), dtype=torch.float32, device="cuda") for c in cases]
+    B.gemv_grouped(ctx, layout, [(b, c.d_scale, g, y, c.rows) for b, c, g, y in zip(bufs, cases, gains, ys)], cases[0].d_x, cases[0].nb * 24)
+    for s, y, c, g in zip(single, ys, cases, gains):
+        assert torch.equal(s, y)
+        check_gemv(oracle, c, y, gain=g)
+
+
+def test_fp16_arm_and_dequant(B, ctx, oracle):
+    case = make_case(300, 24 * 50, seed=12)
+    for layout in (0, 1):
+        buf = B.expand(ctx, layout, case.d_codes, case.rows, case.nb)
+        W = B.dequant_fp16(ctx, layout, buf, case.d_scale, GAIN, case.rows, case.nb * 24)
+        ref = oracle.dequant(case.codes, case.rows, case.nb, case.row_scale, GAIN)
+        got = W.cpu().numpy().astype(np.float64)
+        # one rounding to fp16 of an f32 product: within one fp16 ulp of the exactly rounded value
+        ulp = np.maximum(np.abs(ref) * 2.0**-10, 2.0**-24)
+        assert (np.abs(got - ref) <= ulp).all()
+    y = B.gemv_fp16(W, case.d_x, case.rows, case.nb * 24)
+    ref_y = W.cpu().numpy().astype(np.float64) @ case.x.astype(np.float64)
+    scale = np.linalg.norm(W.cpu().numpy().astype(np.float64), axis=1) * np.linalg.norm(case.x.astype(np.float64))
+    assert (np.abs(y.cpu().numpy() - ref_y) <= 1e-5 * np.maximum(scale, 1e-30)).all()
+
+
+def test_noweights_control_returns_zero(B, ctx):
+    case = make_case(4096, 4096, seed=2)
+    y = torch.full((case.rows,), float("nan"), dtype=torch.float32, device="cuda")
+    B.gemv_noweights(ctx, case.d_scale, case.d_x, case.rows, case.nb * 24, y=y)
+    assert (y == 0).all()
+
+
+def test_error_codes(B, ctx):
+    case = make_case(64, 96, seed=1)
+    buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    with pytest.raises(B.LlvqError) as e:
+        B.gemv(ctx, 7, buf, case.d_scale, GAIN, case.d_x, case.rows, 96)
+    assert e.value.code == -1
+    with pytest.raises(B.LlvqError) as e:
+        B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, 95)
+    assert e.value.code == -1
+    with pytest.raises(B.LlvqError) as e:
+        B.gemv(ctx, 0, buf[16:], case.d_scale, GAIN, case.d_x, case.rows, 96)      # misaligned layout
+    assert e.value.code == -2
+    with pytest.raises(B.LlvqError) as e:
+        B.expand(ctx, 0, case.d_codes, case.rows, case.nb, out=torch.empty(100, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == -3
+    # the context is still usable
+    y = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, 96)
+    assert torch.isfinite(y).all()
