@@ -253,9 +253,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-arms", action="store_true", help="skip the one-hot / FP16 / no-weights comparison arms")
     ap.add_argument("--no-verify", action="store_true", help="skip the oracle check (profiling runs only)")
+    ap.add_argument("--lean", action="store_true", help="profiling runs: no clock ramp, no end-to-end leg, no arms, no oracle check")
     ap.add_argument("--ungrouped", action="store_true", help="one launch a matrix instead of row-concatenated groups")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    if args.lean:
+        args.no_arms = args.no_verify = True
     wl = datagen.workload(args.config, args.layers)
 
     if args.impl == "reference":
@@ -316,8 +319,8 @@ def main():
                             "blocks_per_s": oblocks / osecs}
 
     # warm-up: ramp the clocks, then W untimed steps, then exactly K timed steps
-    ramp = capture_graphs(B, ctx, B.PLANES, copies, min(512, max(64, ncopies * 8)))
-    t_end = time.perf_counter() + 0.4
+    ramp = capture_graphs(B, ctx, B.PLANES, copies, 1 if args.lean else min(512, max(64, ncopies * 8)))
+    t_end = time.perf_counter() + (0.0 if args.lean else 0.4)
     while time.perf_counter() < t_end:
         time_graphs(ramp)
     warm = capture_graphs(B, ctx, B.PLANES, copies, args.warmup)
@@ -360,8 +363,8 @@ def main():
                 py.copy_(y, non_blocking=True)
         torch.cuda.current_stream().synchronize()
 
-    e2e_steps = min(args.steps, 300)
-    for i in range(10):
+    e2e_steps = 1 if args.lean else min(args.steps, 300)
+    for i in range(0 if args.lean else 10):
         e2e_step(i)
     t1 = time.perf_counter()
     for i in range(e2e_steps):

@@ -61,7 +61,7 @@ extern "C" {
 #define LLVQ_EALIGN (-2) /* a device pointer is not aligned as documented                   */
 #define LLVQ_ESIZE (-3)  /* a buffer or the context's scratch is too small for the request  */
 #define LLVQ_ECUDA (-4)  /* a CUDA runtime call failed                                      */
-#define LLVQ_EINDEX (-5) /* at least one code word named no point (llvq_expand_check only)  */
+#define LLVQ_ETIMEOUT (-5) /* a bounded wait inside a kernel ran out (llvq_status only)         */
 
 #define LLVQ_MAX_GROUP 8       /* matrices in one grouped launch                             */
 #define LLVQ_MAX_K 98304       /* largest k_padded the GEMV stages in shared memory          */
@@ -78,10 +78,22 @@ typedef struct {
 } llvq_problem;
 
 /* Builds the class, index-base and Golay tables on the host, uploads them to `device`, and
- * allocates the context's reduction scratch (scratch_bytes; 0 = default 32 MiB).  Synchronous. */
+ * allocates the context's reduction scratch (scratch_bytes; 0 = default 8 MiB, eight bytes a row
+ * of the largest launch, rows rounded up to 32 per matrix).  Synchronous. */
 int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes);
 void llvq_destroy(llvq_ctx *ctx);
 const char *llvq_strerror(int code);
+
+/* Synchronises `stream` and reports whether any GEMV launched on this context since the last
+ * call gave up on one of its bounded waits (LLVQ_ETIMEOUT; the flag and the scratch are then
+ * reset).  Every wait inside the kernels - on an asynchronous copy or on the previous kernel -
+ * has an iteration limit; none can spin forever. */
+int llvq_status(llvq_ctx *ctx, void *stream);
+
+/* The GEMV is launched with programmatic dependent launch (on by default): its record prefetch
+ * starts while the previous kernel of the stream drains, and it waits for that kernel before it
+ * touches x, y or the scratch.  enabled = 0 launches it as an ordinary kernel. */
+int llvq_set_pdl(llvq_ctx *ctx, int enabled);
 
 /* Host queries.  Number of classes (301), points in the ball, and first index of class c
  * (c = 301 gives the number of points)  [Sec. 2.1]. */
@@ -102,8 +114,10 @@ int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, 
 /* [Sec. 2.3] y[row] = row_scale[row] * sum_b gain[g_b] / (4 sqrt(m_b)) * sum_i x_b,i * x[24b+i],
  * m_b the shell of block b's class, with f32 accumulation (the products of the small integer
  * coordinates with fp16 x are exact in f32).  gain is a HOST pointer to two floats.  x is fp16,
- * 16-byte aligned; y is f32.  The summation order of a row depends only on nb, never on the
- * launch geometry, so a grouped launch returns bit-identical rows. */
+ * 16-byte aligned; y is f32; x must be finite.  A row is summed in chunks of blocks whose bounds
+ * depend on nb alone; the chunk sums meet in a fixed-point accumulator (integer addition, exact
+ * and order-free, finer than f32), so the result never depends on the launch geometry and a
+ * grouped launch returns bit-identical rows. */
 int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row_scale,
               const float *gain, const void *x, float *y, int64_t rows, int64_t k_padded, void *stream);
 

@@ -1,4 +1,5 @@
 // C ABI of the library: argument checks, context set-up, and the hand-off to the kernels.
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -36,7 +37,7 @@ const char *llvq_strerror(int code) {
         case LLVQ_EALIGN: return "device pointer not aligned as documented";
         case LLVQ_ESIZE: return "buffer or context scratch too small";
         case LLVQ_ECUDA: return "CUDA runtime error";
-        case LLVQ_EINDEX: return "a code word names no lattice point";
+        case LLVQ_ETIMEOUT: return "a bounded wait inside a kernel ran out; the affected outputs are incomplete";
         default: return "unknown error";
     }
 }
@@ -52,7 +53,7 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
     llvq_ctx *ctx = new (std::nothrow) llvq_ctx();
     if (!ctx) return LLVQ_ECUDA;
     ctx->device = device;
-    ctx->table_blob = nullptr; ctx->partial = nullptr; ctx->counter = nullptr;
+    ctx->table_blob = nullptr; ctx->accum = nullptr; ctx->error = nullptr; ctx->use_pdl = 1;
     if (!build_tables(ctx->host)) { delete ctx; return LLVQ_EINVAL; }
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
@@ -60,11 +61,12 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
     ctx->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
 
     const HostTables &h = ctx->host;
-    struct Part { const void *src; size_t bytes; size_t off; } parts[8] = {
+    struct Part { const void *src; size_t bytes; size_t off; } parts[9] = {
         {h.base.data(), h.base.size() * 8, 0},          {h.desc.data(), h.desc.size() * sizeof(ClassDesc), 0},
         {h.golay_by_weight.data(), 4096 * 4, 0},        {h.golay_by_message.data(), 4096 * 4, 0},
         {h.cls_scale.data(), kClassSlots * 4, 0},       {h.cls_parity.data(), kClassSlots * 4, 0},
-        {h.cls_value.data(), kClassSlots * 8 * 4, 0},   {h.cls_dist.data(), kClassSlots * 8, 0}};
+        {h.cls_value.data(), kClassSlots * 8 * 4, 0},   {h.cls_dist.data(), kClassSlots * 8, 0},
+        {h.cls_pack.data(), kClassSlots * 8, 0}};
     size_t total = 0;
     for (auto &p : parts) { p.off = total; total += round_up(p.bytes, 256); }
     if (cudaMalloc(&ctx->table_blob, total) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
@@ -83,16 +85,16 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
     d.cls_parity = (const uint32_t *)(blob + parts[5].off);
     d.cls_value = (const float *)(blob + parts[6].off);
     d.cls_dist = (const uint8_t *)(blob + parts[7].off);
+    d.cls_pack = (const float2 *)(blob + parts[8].off);
     std::memcpy(d.weight_offset, h.weight_offset, sizeof d.weight_offset);
     d.num_classes = h.num_classes;
     d.num_points = h.num_points;
 
-    if (scratch_bytes == 0) scratch_bytes = (size_t)32 << 20;
-    ctx->partial_floats = scratch_bytes / 4;
-    ctx->counter_slots = ctx->partial_floats / 32 + 1;     // a row group has at least one item
-    if (cudaMalloc(&ctx->partial, ctx->partial_floats * 4) != cudaSuccess ||
-        cudaMalloc(&ctx->counter, ctx->counter_slots * 4) != cudaSuccess ||
-        cudaMemset(ctx->counter, 0, ctx->counter_slots * 4) != cudaSuccess) {
+    if (scratch_bytes == 0) scratch_bytes = (size_t)8 << 20;
+    ctx->accum_slots = scratch_bytes / 8;
+    if (cudaMalloc(&ctx->accum, ctx->accum_slots * 8) != cudaSuccess ||
+        cudaMemset(ctx->accum, 0, ctx->accum_slots * 8) != cudaSuccess ||
+        cudaMalloc(&ctx->error, 4) != cudaSuccess || cudaMemset(ctx->error, 0, 4) != cudaSuccess) {
         llvq_destroy(ctx);
         return LLVQ_ECUDA;
     }
@@ -105,9 +107,30 @@ void llvq_destroy(llvq_ctx *ctx) {
     if (!ctx) return;
     DeviceGuard guard(ctx->device);
     cudaFree(ctx->table_blob);
-    cudaFree(ctx->partial);
-    cudaFree(ctx->counter);
+    cudaFree(ctx->accum);
+    cudaFree(ctx->error);
     delete ctx;
+}
+
+int llvq_status(llvq_ctx *ctx, void *stream) {
+    if (!ctx) return LLVQ_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    int flag = 0;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaMemcpy(&flag, ctx->error, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return LLVQ_ECUDA;
+    if (flag) {
+        cudaMemset(ctx->error, 0, 4);
+        cudaMemset(ctx->accum, 0, ctx->accum_slots * 8);   // an abandoned reduction leaves sums behind
+        return LLVQ_ETIMEOUT;
+    }
+    return LLVQ_OK;
+}
+
+int llvq_set_pdl(llvq_ctx *ctx, int enabled) {
+    if (!ctx) return LLVQ_EINVAL;
+    ctx->use_pdl = enabled ? 1 : 0;
+    return LLVQ_OK;
 }
 
 int llvq_num_classes(const llvq_ctx *ctx) { return ctx ? ctx->host.num_classes : LLVQ_EINVAL; }
@@ -152,8 +175,9 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
     p.nb = (int)(k_padded / 24);
     p.tiles = p.nb / kTileCells;
     p.tail_cells = p.nb % kTileCells;
-    p.nchunk = p.tiles ? (p.tiles + kChunkTiles - 1) / kChunkTiles : 1;
+    p.units = p.tiles + (p.tail_cells ? 1 : 0);
     int64_t groups = 0;
+    float gain_max = 0.f;
     for (int i = 0; i < n; i++) {
         const llvq_problem &q = problems[i];
         if ((!q.layout && !no_weights) || !q.row_scale || !q.y || q.rows <= 0) return LLVQ_EINVAL;
@@ -165,20 +189,31 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
         p.prob[i].group_begin = (int)groups;
         p.prob[i].gain0 = q.gain[0];
         p.prob[i].gain1 = q.gain[1];
+        gain_max = std::fmax(gain_max, std::fmax(std::fabs(q.gain[0]), std::fabs(q.gain[1])));
         if (q.rows > ((int64_t)1 << 30)) return LLVQ_ESIZE;
         groups += (q.rows + kRowsPerGroup - 1) / kRowsPerGroup;
     }
-    const int64_t items = groups * p.nchunk;
-    if (items > ((int64_t)1 << 30)) return LLVQ_ESIZE;
-    if (p.nchunk > 1 && ((size_t)items * 32 > ctx->partial_floats || (size_t)groups > ctx->counter_slots)) return LLVQ_ESIZE;
+    if (groups > ((int64_t)1 << 26) || p.units > 2047) return LLVQ_ESIZE;
+    if ((size_t)groups * 32 > ctx->accum_slots) return LLVQ_ESIZE;
+    if (!(gain_max < 3.0e38f)) return LLVQ_EINVAL;
+    // quantum of the fixed-point row accumulators, per matrix so that grouping does not change it:
+    // a unit sums at most four blocks, each bounded by max|gain| * sqrt(24) * max|x| < 2^ge * 5 * 2^xe;
+    // 4 * 5 < 2^5, and the unit value is kept under 2^39 quanta (see deliver() in llvq_gemv.cu)
+    for (int i = 0; i < n; i++) {
+        const float gm = std::fmax(std::fabs(problems[i].gain[0]), std::fabs(problems[i].gain[1]));
+        int ge = 0;
+        std::frexp(gm > 0.f ? gm : 1.f, &ge);                              // gm < 2^ge
+        p.prob[i].qexp_base = ge + 5 - 39;
+    }
     p.total_groups = (int)groups;
-    p.total_items = (int)items;
-    p.partial = ctx->partial;
-    p.counter = ctx->counter;
+    p.total_units = groups * p.units;
+    p.accum = ctx->accum;
     p.cls_scale = ctx->dev.cls_scale;
     p.cls_parity = ctx->dev.cls_parity;
     p.cls_value = ctx->dev.cls_value;
-    if (gemv_smem_bytes(layout, p.nb, n) > (size_t)ctx->max_smem_optin) return LLVQ_ESIZE;
+    p.cls_pack = ctx->dev.cls_pack;
+    p.error = ctx->error;
+    if (gemv_smem_bytes(layout, p.nb, n) + 1024 > (size_t)ctx->max_smem_optin) return LLVQ_ESIZE;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
     return launch_gemv(ctx, layout, p, no_weights, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;

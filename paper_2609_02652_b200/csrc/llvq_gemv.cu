@@ -2,18 +2,32 @@
 //
 // Geometry.  A lane owns a row: the 32 lanes of a warp work on the 32 rows of one row group and
 // walk the same block columns together, so every read of x is a shared-memory broadcast and no
-// shuffle reduction is needed.  A work item is (row group, chunk of kChunkTiles tiles); items
-// are dealt round-robin to the warps of a grid sized to the machine.  Each item leaves a
-// 32-float partial in the context's scratch; the warp that delivers the last partial of a row
-// group adds them in chunk order, applies the row scale and writes y.  The order of additions
-// for a row therefore depends on nb alone.
+// shuffle reduction is needed.  The records of a launch form one sequence of units - a unit is a
+// tile of four block columns of a row group, or the row group's last nb mod 4 columns - and the
+// sequence is cut into equal contiguous ranges, one per warp of a grid of one CTA a
+// multiprocessor, so every warp streams the same number of bytes (give or take one unit).
+//
+// Reduction.  The float sum of a unit (at most four blocks, fixed order) is converted to fixed
+// point and from there on everything is integer: a warp adds its units of a row group in a
+// 64-bit register and hands the sum, with the number of units it covers, to the row's 64-bit
+// accumulator in the context's scratch by one atomic add.  Integer addition is exact and
+// order-free, so a row's result does not depend on how the units were dealt or on which warp
+// arrives last; the arrival that completes the unit count converts the total back to float,
+// applies the row scale, writes y and clears the accumulator.  The quantum is 2^-39 of a bound on
+// a unit's sum derived from max |x| and the gain, i.e. far below f32 resolution.
 //
 // Decode.  One rotate and one three-input logic op turn a payload word into a pair of fp16 bit
 // patterns whose value is (+-)|x_i| * 2^-21 (a subnormal built in place: level bits at [6:4],
 // the class parity or-ed in at bit 3, the sign at bit 15).  A mixed-precision fused multiply-add
-// (fp16 x fp16 + f32) accumulates the exact product with the fp16 activation.  Per block one
-// multiply applies gain[g] * 2^21 / (4 sqrt m), looked up by the 10-bit header.  Every lane runs
-// the same instructions whatever its class.
+// (fp16 x fp16 + f32, one instruction) accumulates the exact product with the fp16 activation.
+// Per block one multiply applies gain[g] * 2^21 / (4 sqrt m), looked up by the class id.  Every
+// lane runs the same instructions whatever its class.
+//
+// Memory.  Each warp streams its units through a private ring of 1792-byte shared-memory slots
+// filled by bulk asynchronous copies (cp.async.bulk, completion on an mbarrier) that lane 0 issues
+// kSlots units ahead.  The first copies go out before the kernel waits for its predecessor in the
+// stream (records never depend on it), so under programmatic dependent launch the ring fills
+// while the previous kernel drains.  Every wait is bounded.
 #include "llvq_internal.cuh"
 
 namespace llvq {
@@ -21,9 +35,13 @@ namespace {
 
 constexpr int kWarps = 16;                 // warps per CTA
 constexpr int kThreads = kWarps * 32;
+constexpr int kSlots = 4;                  // ring slots per warp
 constexpr uint32_t kPairMask = 0x80708070u;
 
-struct BlockConst { float scale; uint32_t parity; };   // indexed by class | gain << 9
+// fixed-point accumulator word: bits 53..63 count units, bits 0..52 sum the biased unit values
+constexpr int kCountShift = 53;
+constexpr unsigned long long kSumMask = (1ull << kCountShift) - 1;
+constexpr long long kUnitBias = 1ll << 41;     // a unit's value is below 2^40 quanta in magnitude
 
 __device__ __forceinline__ void fma_pair(float &lo, float &hi, uint32_t w, uint32_t x) {
     asm("{\n\t.reg .f16 wl, wh, xl, xh;\n\t"
@@ -79,121 +97,287 @@ __device__ __forceinline__ int find_problem(const GemvParams &p, int group) {
     return q;
 }
 
-// Delivers one item's partial; the last arrival of a row group finishes the rows.
-__device__ __forceinline__ void deliver(const GemvParams &p, const GemvProblemDev &pr, int group, int chunk, int lane, float acc) {
+// exact power of two as a float, |e| < 126
+__device__ __forceinline__ float pow2f(int e) { return __int_as_float((127 + e) << 23); }
+
+// The contiguous range of units [u0, u1) of this warp; warps are numbered with the CTA index
+// fastest, so the ranges that are one unit longer spread over all multiprocessors.
+__device__ __forceinline__ void warp_range(const GemvParams &p, int warp, long long &u0, long long &u1) {
+    const long long warps = (long long)gridDim.x * kWarps, gw = (long long)warp * gridDim.x + blockIdx.x;
+    const long long base = p.total_units / warps, rem = p.total_units % warps;
+    u0 = gw * base + (gw < rem ? gw : rem);
+    u1 = u0 + base + (gw < rem ? 1 : 0);
+}
+
+// Hands the warp's sum over `count` units of row group `group` to the row accumulators.
+__device__ __forceinline__ void deliver(const GemvParams &p, const GemvProblemDev &pr, int group, int lane,
+                                        long long sum, int count, int qexp) {
     const int row = (group - pr.group_begin) * kRowsPerGroup + lane;
-    if (p.nchunk == 1) {
-        if (row < pr.rows) pr.y[row] = acc * __half2float(pr.row_scale[row]);
-        return;
+    if (row >= pr.rows) return;                      // padding rows of the last row group
+    const unsigned long long addend = (unsigned long long)sum + ((unsigned long long)count << kCountShift);
+    unsigned long long *slot = p.accum + (size_t)group * 32 + lane;
+    const unsigned long long old = atomicAdd(slot, addend);
+    if ((int)(old >> kCountShift) + count == p.units) {
+        const long long total = (long long)((old + addend) & kSumMask) - (long long)p.units * kUnitBias;
+        pr.y[row] = ((float)total * pow2f(qexp)) * __half2float(pr.row_scale[row]);
+        *slot = 0ull;                                // ready for the next launch on this context
     }
-    float *slot = p.partial + ((size_t)group * p.nchunk) * 32;
-    __stcg(slot + chunk * 32 + lane, acc);
-    __threadfence();
-    unsigned old = 0;
-    if (lane == 0) old = atomicAdd(p.counter + group, 1u);
-    old = __shfl_sync(0xffffffffu, old, 0);
-    if (old == (unsigned)p.nchunk - 1) {
-        __threadfence();
-        float sum = 0.f;
-        for (int c = 0; c < p.nchunk; c++) sum += __ldcg(slot + c * 32 + lane);
-        if (row < pr.rows) pr.y[row] = sum * __half2float(pr.row_scale[row]);
-        if (lane == 0) p.counter[group] = 0;      // leave the scratch ready for the next launch
+}
+
+// ---- asynchronous copies: global -> shared, completion counted on an mbarrier in shared memory
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Every wait is bounded: after kSpinLimit failed polls the caller records an error and winds down.
+constexpr int kSpinLimit = 1 << 22;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    for (int i = 0; i < kSpinLimit; i++)
+        if (mbar_try(bar, parity)) return true;
+    return false;
+}
+
+// Position in the unit sequence: row group, unit inside it, the matrix it belongs to.
+struct Pos {
+    int group, k, q;
+    const uint8_t *grp;     // first byte of the row group's records
+};
+
+__device__ __forceinline__ void pos_set_group(const GemvParams &p, Pos &c, int cell_bytes) {
+    c.q = find_problem(p, c.group);
+    c.grp = p.prob[c.q].layout + (size_t)(c.group - p.prob[c.q].group_begin) * (size_t)p.nb * cell_bytes;
+}
+__device__ __forceinline__ void pos_init(const GemvParams &p, Pos &c, long long u, int cell_bytes) {
+    c.group = (int)(u / p.units);
+    c.k = (int)(u - (long long)c.group * p.units);
+    if (c.group < p.total_groups) pos_set_group(p, c, cell_bytes);
+}
+__device__ __forceinline__ void pos_next(const GemvParams &p, Pos &c, int cell_bytes) {
+    if (++c.k == p.units) {
+        c.k = 0;
+        c.group++;
+        if (c.group < p.total_groups) pos_set_group(p, c, cell_bytes);
     }
 }
 
 template <bool NO_WEIGHTS>
-__global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
-    extern __shared__ __align__(16) unsigned char smem[];
-    BlockConst *bc = reinterpret_cast<BlockConst *>(smem);                 // 1024 entries a matrix of the group
-    uint4 *xs = reinterpret_cast<uint4 *>(smem + (size_t)p.nprob * 1024 * sizeof(BlockConst));
+__global__ void __launch_bounds__(kThreads, 2) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char *ring = smem;
+    const float2 *cls = reinterpret_cast<const float2 *>(smem + kWarps * kSlots * kTileBytes);
+    const uint4 *xs = reinterpret_cast<const uint4 *>(smem + kWarps * kSlots * kTileBytes + kClassSlots * 8);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kWarps * kSlots * kTileBytes + kClassSlots * 8 + ((p.nb * 48 + 127) / 128) * 128);
+    uint32_t *xor_word = reinterpret_cast<uint32_t *>(bars + kWarps * kSlots + 1);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t my_ring = smem_addr(ring + warp * kSlots * kTileBytes);
+    const uint32_t my_bar = smem_addr(bars + warp * kSlots);
+    const uint32_t pro_bar = smem_addr(bars + kWarps * kSlots);
 
-    // block constants per problem: gain[g] * 2^21 / (4 sqrt m) and the parity pattern
-    for (int e = tid; e < p.nprob * 1024; e += kThreads) {
-        const int q = e >> 10, c = e & 511, g = (e >> 9) & 1;
-        BlockConst v;
-        v.scale = p.cls_scale[c] * (g ? p.prob[q].gain1 : p.prob[q].gain0);
-        v.parity = p.cls_parity[c];
-        bc[e] = v;
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kSlots; s++) mbar_init(my_bar + 8 * s, 1);
+        if (warp == 0) { mbar_init(pro_bar, 1); *xor_word = 0; }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // x, once per CTA: 3 nb 16-byte words
-    const uint4 *xg = reinterpret_cast<const uint4 *>(p.x);
-    for (int e = tid; e < 3 * p.nb; e += kThreads) xs[e] = __ldg(xg + e);
     __syncthreads();
 
-    const int warps_total = gridDim.x * kWarps;
-    for (int item = warp * gridDim.x + blockIdx.x; item < p.total_items; item += warps_total) {
-        const int group = item / p.nchunk, chunk = item - group * p.nchunk;
-        const int q = find_problem(p, group);
-        const GemvProblemDev &pr = p.prob[q];
-        const uint8_t *grp = pr.layout + (size_t)(group - pr.group_begin) * (size_t)p.nb * kCellBytes;
-        const BlockConst *bcq = bc + q * 1024;
-        const int t0 = chunk * kChunkTiles, t1 = min(t0 + kChunkTiles, p.tiles);
-        float acc = 0.f;
+    long long u0, u1;
+    warp_range(p, warp, u0, u1);
+    Pos pi, pc;                            // issue side, consume side
+    pos_init(p, pi, u0, kCellBytes);
+    pc = pi;
+    long long ui = u0;
+    const uint32_t tail_bytes = (uint32_t)p.tail_cells * kCellBytes;
+
+    auto issue = [&](int s) {
+        if (lane == 0) {
+            const bool tile = pi.k < p.tiles;
+            const uint32_t bytes = tile ? (uint32_t)kTileBytes : tail_bytes;
+            mbar_expect(my_bar + 8 * s, bytes);
+            bulk_g2s(my_ring + s * kTileBytes, pi.grp + (size_t)(tile ? pi.k : p.tiles) * kTileBytes, bytes, my_bar + 8 * s);
+        }
+        pos_next(p, pi, kCellBytes);
+        ui++;
+    };
+
+    if (!NO_WEIGHTS) {
+#pragma unroll
+        for (int s = 0; s < kSlots; s++)
+            if (ui < u1) issue(s);
+    }
+    if (tid == 0) {
+        mbar_expect(pro_bar, kClassSlots * 8 + p.nb * 48);
+        bulk_g2s(smem_addr(cls), p.cls_pack, kClassSlots * 8, pro_bar);
+    }
+    // let the next kernel in the stream start its own prefetch, then wait for the previous one:
+    // x, y and the reduction scratch may still be in use by it
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (tid == 0) bulk_g2s(smem_addr(xs), p.x, p.nb * 48, pro_bar);
+
+    bool failed = !mbar_wait(pro_bar, 0);
+    // every |x| is below 2^(e-14), e the biased exponent of the OR of all magnitudes
+    int xexp;
+    {
+        uint32_t m = 0;
+        const uint32_t *xw = reinterpret_cast<const uint32_t *>(xs);
+        for (int e = tid; e < p.nb * 12; e += kThreads) m |= xw[e];
+        m = __reduce_or_sync(0xffffffffu, (m | (m >> 16)) & 0x7fffu);
+        if (lane == 0 && m) atomicOr(xor_word, m);
+        __syncthreads();
+        xexp = max((int)(*xor_word >> 10), 1) - 14;
+    }
+
+    uint32_t phases = 0;
+    int slot = 0, count = 0;
+    long long sum = 0;
+    int qexp = xexp + p.prob[pc.q].qexp_base;
+    float inv_q = pow2f(-qexp);
+
+    for (long long u = u0; u < u1 && !failed; u++) {
+        const GemvProblemDev &pr = p.prob[pc.q];
+        float s = 0.f;
         if (!NO_WEIGHTS) {
-            for (int t = t0; t < t1; t++) {
-                const uint8_t *tile = grp + (size_t)t * kTileBytes;
-                const uint4 a0 = __ldcs(reinterpret_cast<const uint4 *>(tile + 16 * lane));
-                const uint4 a1 = __ldcs(reinterpret_cast<const uint4 *>(tile + 512 + 16 * lane));
-                const uint4 a2 = __ldcs(reinterpret_cast<const uint4 *>(tile + 1024 + 16 * lane));
-                const uint2 hh = __ldcs(reinterpret_cast<const uint2 *>(tile + 1536 + 8 * lane));
+            const uint32_t bar = my_bar + 8 * slot;
+            if (!mbar_wait(bar, (phases >> slot) & 1u)) { failed = true; break; }
+            phases ^= 1u << slot;
+            const unsigned char *buf = ring + (warp * kSlots + slot) * kTileBytes;
+            if (pc.k < p.tiles) {
+                const uint4 a0 = *reinterpret_cast<const uint4 *>(buf + 16 * lane);
+                const uint4 a1 = *reinterpret_cast<const uint4 *>(buf + 512 + 16 * lane);
+                const uint4 a2 = *reinterpret_cast<const uint4 *>(buf + 1024 + 16 * lane);
+                const uint2 hh = *reinterpret_cast<const uint2 *>(buf + 1536 + 8 * lane);
                 const uint32_t w0[4] = {a0.x, a0.y, a0.z, a0.w}, w1[4] = {a1.x, a1.y, a1.z, a1.w}, w2[4] = {a2.x, a2.y, a2.z, a2.w};
                 const uint32_t hd[4] = {hh.x & 0xffffu, hh.x >> 16, hh.y & 0xffffu, hh.y >> 16};
 #pragma unroll
                 for (int c = 0; c < 4; c++) {
-                    const BlockConst k = bcq[hd[c] & 1023u];
-                    const float dot = block_dot(w0[c], w1[c], w2[c], k.parity, xs + 3 * (4 * t + c));
-                    acc = fmaf(k.scale, dot, acc);
+                    const float2 k = cls[hd[c] & 511u];
+                    const float g = (hd[c] & 512u) ? pr.gain1 : pr.gain0;
+                    const float dot = block_dot(w0[c], w1[c], w2[c], __float_as_uint(k.y), xs + 3 * (4 * pc.k + c));
+                    s = fmaf(k.x * g, dot, s);
+                    if (c == 1) {
+                        // the slot's words are in registers: refill it with the unit kSlots ahead
+                        __syncwarp();
+                        if (ui < u1) issue(slot);
+                    }
                 }
+            } else {
+                uint32_t tw[3][3], th[3];
+#pragma unroll
+                for (int c = 0; c < 3; c++)
+                    if (c < p.tail_cells) {
+                        const unsigned char *cell = buf + c * kCellBytes;
+                        tw[c][0] = *reinterpret_cast<const uint32_t *>(cell + 4 * lane);
+                        tw[c][1] = *reinterpret_cast<const uint32_t *>(cell + 128 + 4 * lane);
+                        tw[c][2] = *reinterpret_cast<const uint32_t *>(cell + 256 + 4 * lane);
+                        th[c] = *reinterpret_cast<const uint16_t *>(cell + 384 + 2 * lane);
+                    }
+#pragma unroll
+                for (int c = 0; c < 3; c++)
+                    if (c < p.tail_cells) {
+                        const float2 k = cls[th[c] & 511u];
+                        const float g = (th[c] & 512u) ? pr.gain1 : pr.gain0;
+                        const float dot = block_dot(tw[c][0], tw[c][1], tw[c][2], __float_as_uint(k.y), xs + 3 * (4 * p.tiles + c));
+                        s = fmaf(k.x * g, dot, s);
+                    }
+                __syncwarp();
+                if (ui < u1) issue(slot);
             }
-            if (chunk == p.nchunk - 1) {
-                for (int c = 0; c < p.tail_cells; c++) {
-                    const uint8_t *cell = grp + (size_t)p.tiles * kTileBytes + (size_t)c * kCellBytes;
-                    const uint32_t w0 = __ldcs(reinterpret_cast<const uint32_t *>(cell + 4 * lane));
-                    const uint32_t w1 = __ldcs(reinterpret_cast<const uint32_t *>(cell + 128 + 4 * lane));
-                    const uint32_t w2 = __ldcs(reinterpret_cast<const uint32_t *>(cell + 256 + 4 * lane));
-                    const uint32_t hd = *reinterpret_cast<const uint16_t *>(cell + 384 + 2 * lane);
-                    const BlockConst k = bcq[hd & 1023u];
-                    const float dot = block_dot(w0, w1, w2, k.parity, xs + 3 * (4 * p.tiles + c));
-                    acc = fmaf(k.scale, dot, acc);
-                }
+            slot = (slot + 1 == kSlots) ? 0 : slot + 1;
+        }
+        sum += __float2ll_rn(s * inv_q) + kUnitBias;
+        count++;
+        const int group = pc.group;
+        pos_next(p, pc, kCellBytes);
+        if (pc.k == 0 || u + 1 == u1) {
+            deliver(p, pr, group, lane, sum, count, qexp);
+            sum = 0;
+            count = 0;
+            if (pc.group < p.total_groups) {
+                qexp = xexp + p.prob[pc.q].qexp_base;
+                inv_q = pow2f(-qexp);
             }
         }
-        deliver(p, pr, group, chunk, lane, acc);
+    }
+
+    if (failed) {
+        // a wait ran out: report it, then give the copies still in flight a bounded chance to land
+        if (lane == 0) atomicExch(p.error, 1);
+        const int pending = (int)min((long long)kSlots, ui - u0);     // generous: wait on every slot once
+        for (int s = 0; s < pending; s++) {
+            mbar_wait(my_bar + 8 * slot, (phases >> slot) & 1u);
+            slot = (slot + 1 == kSlots) ? 0 : slot + 1;
+        }
     }
 }
 
+// One-hot comparison arm: same unit sequence, same reduction, records read with plain loads.
 __global__ void __launch_bounds__(kThreads, 1) gemv_onehot_kernel(const __grid_constant__ GemvParams p) {
-    extern __shared__ __align__(16) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem[];
     uint4 *xs4 = reinterpret_cast<uint4 *>(smem);
     const __half *xs = reinterpret_cast<const __half *>(smem);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ uint32_t xor_word;
+    if (tid == 0) xor_word = 0;
     const uint4 *xg = reinterpret_cast<const uint4 *>(p.x);
-    for (int e = tid; e < 3 * p.nb; e += kThreads) xs4[e] = __ldg(xg + e);
+    uint32_t m = 0;
+    for (int e = tid; e < 3 * p.nb; e += kThreads) {
+        const uint4 v = __ldg(xg + e);
+        xs4[e] = v;
+        m |= v.x | v.y | v.z | v.w;
+    }
     __syncthreads();
-    const int warps_total = gridDim.x * kWarps;
-    for (int item = warp * gridDim.x + blockIdx.x; item < p.total_items; item += warps_total) {
-        const int group = item / p.nchunk, chunk = item - group * p.nchunk;
-        const int q = find_problem(p, group);
-        const GemvProblemDev &pr = p.prob[q];
-        const uint8_t *grp = pr.layout + (size_t)(group - pr.group_begin) * (size_t)p.nb * kOneHotCellBytes;
-        // same chunking as the bit-plane kernel: tiles of four cells, the tail cells in the last chunk
-        const int c0 = chunk * kChunkTiles * kTileCells;
-        const int c1 = (chunk == p.nchunk - 1) ? p.nb : min(c0 + kChunkTiles * kTileCells, p.tiles * kTileCells);
-        float acc = 0.f;
+    m = __reduce_or_sync(0xffffffffu, (m | (m >> 16)) & 0x7fffu);
+    if (lane == 0 && m) atomicOr(&xor_word, m);
+    __syncthreads();
+    const int xexp = max((int)(xor_word >> 10), 1) - 14;
+
+    long long u0, u1;
+    warp_range(p, warp, u0, u1);
+    Pos pc;
+    pos_init(p, pc, u0, kOneHotCellBytes);
+    long long sum = 0;
+    int count = 0;
+    for (long long u = u0; u < u1; u++) {
+        const GemvProblemDev &pr = p.prob[pc.q];
+        const int qexp = xexp + pr.qexp_base;
+        const int c0 = pc.k * kTileCells, c1 = pc.k < p.tiles ? c0 + kTileCells : p.nb;
+        float s = 0.f;
         for (int c = c0; c < c1; c++) {
-            const uint32_t *cell = reinterpret_cast<const uint32_t *>(grp + (size_t)c * kOneHotCellBytes);
+            const uint32_t *cell = reinterpret_cast<const uint32_t *>(pc.grp + (size_t)c * kOneHotCellBytes);
             uint32_t v[5];
 #pragma unroll
             for (int t = 0; t < 5; t++) v[t] = __ldcs(cell + 32 * t + lane);
-            const int cls = (int)(v[0] >> 24) | (int)(((v[1] >> 24) & 1u) << 8);
+            const int cid = (int)(v[0] >> 24) | (int)(((v[1] >> 24) & 1u) << 8);
             const float g = ((v[1] >> 25) & 1u) ? pr.gain1 : pr.gain0;
-            const float4 lv = __ldg(reinterpret_cast<const float4 *>(p.cls_value + cls * 8));
-            const float l4 = __ldg(p.cls_value + cls * 8 + 4);
+            const float4 lv = __ldg(reinterpret_cast<const float4 *>(p.cls_value + cid * 8));
+            const float l4 = __ldg(p.cls_value + cid * 8 + 4);
             const float val[5] = {lv.x, lv.y, lv.z, lv.w, l4};
-            acc = fmaf(g, onehot_dot(v, val, xs + 24 * c), acc);
+            s = fmaf(g, onehot_dot(v, val, xs + 24 * c), s);
         }
-        deliver(p, pr, group, chunk, lane, acc);
+        sum += __float2ll_rn(s * pow2f(-qexp)) + kUnitBias;
+        count++;
+        const int group = pc.group;
+        pos_next(p, pc, kOneHotCellBytes);
+        if (pc.k == 0 || u + 1 == u1) {
+            deliver(p, pr, group, lane, sum, count, qexp);
+            sum = 0;
+            count = 0;
+        }
     }
 }
 
@@ -304,31 +488,48 @@ __global__ void __launch_bounds__(256) dequant_kernel(int layout, const uint8_t 
 }  // namespace
 
 size_t gemv_smem_bytes(int layout, int nb, int nprob) {
-    const size_t xbytes = (size_t)nb * 48;
-    return layout == LLVQ_PLANES ? (size_t)nprob * 1024 * sizeof(BlockConst) + xbytes : xbytes;
+    (void)nprob;
+    const size_t xbytes = ((size_t)nb * 48 + 127) / 128 * 128;
+    if (layout != LLVQ_PLANES) return xbytes;
+    return (size_t)kWarps * kSlots * kTileBytes + kClassSlots * 8 + xbytes + (kWarps * kSlots + 2) * 8;
+}
+
+template <typename K>
+static int allow_max_smem(K kernel, int optin) {
+    cudaFuncAttributes a;
+    if (cudaFuncGetAttributes(&a, kernel) != cudaSuccess) return -1;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - (int)a.sharedSizeBytes) == cudaSuccess ? 0 : -1;
 }
 
 int gemv_configure(const llvq_ctx *ctx) {
     const int bytes = ctx->max_smem_optin;
-    if (cudaFuncSetAttribute(gemv_planes_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return -1;
-    if (cudaFuncSetAttribute(gemv_planes_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return -1;
-    if (cudaFuncSetAttribute(gemv_onehot_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return -1;
+    if (allow_max_smem(gemv_planes_kernel<false>, bytes)) return -1;
+    if (allow_max_smem(gemv_planes_kernel<true>, bytes)) return -1;
+    if (allow_max_smem(gemv_onehot_kernel, bytes)) return -1;
     return 0;
 }
 
 cudaError_t launch_gemv(const llvq_ctx *ctx, int layout, const GemvParams &p, bool no_weights, cudaStream_t s) {
     const size_t smem = gemv_smem_bytes(layout, p.nb, p.nprob);
-    int grid = ctx->sm_count;
-    const int needed = (p.total_items + kWarps - 1) / kWarps;
-    if (grid > needed) grid = needed;
-    if (grid < 1) grid = 1;
+    // one CTA a multiprocessor; fewer only when there are fewer units than warps
+    long long grid = (p.total_units + kWarps - 1) / kWarps;
+    if (grid > ctx->sm_count) grid = ctx->sm_count;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = ctx->use_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (layout == LLVQ_PLANES) {
-        if (no_weights) gemv_planes_kernel<true><<<grid, kThreads, smem, s>>>(p);
-        else gemv_planes_kernel<false><<<grid, kThreads, smem, s>>>(p);
-    } else {
-        gemv_onehot_kernel<<<grid, kThreads, smem, s>>>(p);
+        if (no_weights) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<true>, p);
+        return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false>, p);
     }
-    return cudaGetLastError();
+    cfg.numAttrs = 0;
+    return cudaLaunchKernelEx(&cfg, gemv_onehot_kernel, p);
 }
 
 cudaError_t launch_gemv_fp16(const __half *W, const __half *x, float *y, int64_t rows, int64_t k, cudaStream_t s) {

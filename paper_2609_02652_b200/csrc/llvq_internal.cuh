@@ -17,10 +17,6 @@ constexpr int kTileCells = 4;
 constexpr int kTileBytes = 1792;
 constexpr int kOneHotCellBytes = 640;  // 32 rows x 20 bytes
 
-// A GEMV work item is one row group times one "chunk" of consecutive tiles.  The chunk length
-// depends on nb only, so the order in which a row is summed never depends on the launch.
-constexpr int kChunkTiles = 3;
-
 struct DeviceTables {
     const uint64_t *base;            // num_classes + 1
     const ClassDesc *desc;           // num_classes
@@ -30,6 +26,7 @@ struct DeviceTables {
     const uint32_t *cls_parity;      // 512
     const float *cls_value;          // 512 x 8
     const uint8_t *cls_dist;         // 512 x 8
+    const float2 *cls_pack;          // 512 x {scale, parity bits}
     int weight_offset[25];
     int num_classes;
     uint64_t num_points;
@@ -42,19 +39,23 @@ struct GemvProblemDev {
     int rows;
     int group_begin;   // index of this matrix's first row group in the concatenation
     float gain0, gain1;
+    int qexp_base;     // log2 of this matrix's fixed-point quantum, before the exponent of max |x| is added
 };
 
 struct GemvParams {
     GemvProblemDev prob[LLVQ_MAX_GROUP];
     int nprob;
     const __half *x;
-    int nb, tiles, tail_cells, nchunk;
-    int total_groups, total_items;
-    float *partial;        // total_items x 32 floats (context scratch)
-    unsigned *counter;     // total_groups (context scratch, zero between launches)
+    int nb, tiles, tail_cells;
+    int units;             // units a row group: tiles, plus one for the nb mod 4 last columns
+    int total_groups;
+    long long total_units;
+    unsigned long long *accum;   // total_groups x 32 fixed-point row accumulators (context scratch, zero between launches)
     const float *cls_scale;
     const uint32_t *cls_parity;
     const float *cls_value;
+    const float2 *cls_pack;   // 512 x {2^21 / (4 sqrt m), parity pattern as bits}
+    int *error;               // set when a bounded wait ran out
 };
 
 }  // namespace llvq
@@ -64,9 +65,10 @@ struct llvq_ctx {
     llvq::HostTables host;
     llvq::DeviceTables dev;
     void *table_blob;        // one allocation holding every table
-    float *partial;
-    unsigned *counter;
-    size_t partial_floats, counter_slots;
+    unsigned long long *accum;   // reduction scratch: one 64-bit accumulator a row of the largest launch
+    size_t accum_slots;
+    int *error;              // device flag: a kernel's bounded wait ran out
+    int use_pdl;             // launch the GEMV with programmatic stream serialization
     int sm_count;
     int max_smem_optin;
 };

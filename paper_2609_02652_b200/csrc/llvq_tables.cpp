@@ -172,6 +172,11 @@ bool build_tables(HostTables &t) {
             t.cls_dist[c * 8 + l] = d.dist[l];
         }
     }
+    t.cls_pack.assign(kClassSlots * 2, 0u);
+    for (int c = 0; c < kClassSlots; c++) {
+        std::memcpy(&t.cls_pack[2 * c], &t.cls_scale[c], 4);
+        t.cls_pack[2 * c + 1] = t.cls_parity[c];
+    }
     t.base[all.size()] = running;
     t.num_points = running;
     return t.num_classes == 301 && t.num_points == 111043117458000ull;

@@ -13,7 +13,7 @@ constexpr int kClassSlots = 512;       // a 9-bit id can never index out of boun
 constexpr int kEmptyClass = 511;       // record of a code that names no point
 constexpr uint64_t kIndexBits = 47;
 
-// What the expander needs to un-rank an index inside one class.  48 bytes.
+// What the expander needs to un-rank an index inside one class.  40 bytes.
 struct ClassDesc {
     uint64_t perm_a;      // even: orderings of the support magnitudes; odd: orderings of all 24
     uint64_t perm_b;      // even: orderings of the off-support magnitudes; odd: 1
@@ -35,6 +35,7 @@ struct HostTables {
     std::vector<uint32_t> golay_by_message;// word of message k = XOR of generator rows in k
     std::vector<float> cls_scale;          // kClassSlots: 2^21 / (4 sqrt(shell)), 0 if unused
     std::vector<uint32_t> cls_parity;      // kClassSlots: parity * 0x00080008
+    std::vector<uint32_t> cls_pack;        // kClassSlots x 2: bits of cls_scale, then cls_parity
     std::vector<float> cls_value;          // kClassSlots * 8: dist[l] / (4 sqrt(shell)), l < 5
     std::vector<uint8_t> cls_dist;         // kClassSlots * 8: dist[l]
 };

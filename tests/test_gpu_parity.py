@@ -102,6 +102,7 @@ def test_gemv_every_row(B, ctx, oracle, layout, rows, k):
     case = make_case(rows, k, seed=rows + k)
     buf = B.expand(ctx, layout, case.d_codes, rows, case.nb)
     y = B.gemv(ctx, layout, buf, case.d_scale, GAIN, case.d_x, rows, case.nb * 24)
+    B.status(ctx)                      # no bounded wait ran out
     check_gemv(oracle, case, y)
     # a second launch on the same context finds the scratch clean
     y2 = B.gemv(ctx, layout, buf, case.d_scale, GAIN, case.d_x, rows, case.nb * 24)
