@@ -54,6 +54,9 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
     if (!ctx) return LLVQ_ECUDA;
     ctx->device = device;
     ctx->table_blob = nullptr; ctx->accum = nullptr; ctx->error = nullptr; ctx->use_pdl = 1;
+#ifdef LLVQ_TRACE
+    ctx->trace = nullptr; ctx->trace_launch = 0;
+#endif
     if (!build_tables(ctx->host)) { delete ctx; return LLVQ_EINVAL; }
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
@@ -133,6 +136,15 @@ int llvq_set_pdl(llvq_ctx *ctx, int enabled) {
     return LLVQ_OK;
 }
 
+#ifdef LLVQ_TRACE
+// debug builds only: eight 64-bit timestamps a warp a launch are stored at `buf`
+int llvq_trace_set(llvq_ctx *ctx, unsigned long long *buf) {
+    ctx->trace = buf;
+    ctx->trace_launch = 0;
+    return LLVQ_OK;
+}
+#endif
+
 int llvq_num_classes(const llvq_ctx *ctx) { return ctx ? ctx->host.num_classes : LLVQ_EINVAL; }
 
 uint64_t llvq_class_base(const llvq_ctx *ctx, int c) {
@@ -193,7 +205,7 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
         if (q.rows > ((int64_t)1 << 30)) return LLVQ_ESIZE;
         groups += (q.rows + kRowsPerGroup - 1) / kRowsPerGroup;
     }
-    if (groups > ((int64_t)1 << 26) || p.units > 2047) return LLVQ_ESIZE;
+    if (groups > ((int64_t)1 << 26) || p.units > 2047 || groups * p.units > 0x7fffffffll) return LLVQ_ESIZE;
     if ((size_t)groups * 32 > ctx->accum_slots) return LLVQ_ESIZE;
     if (!(gain_max < 3.0e38f)) return LLVQ_EINVAL;
     // quantum of the fixed-point row accumulators, per matrix so that grouping does not change it:
@@ -206,13 +218,17 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
         p.prob[i].qexp_base = ge + 5 - 39;
     }
     p.total_groups = (int)groups;
-    p.total_units = groups * p.units;
+    p.total_units = (int)(groups * p.units);
     p.accum = ctx->accum;
     p.cls_scale = ctx->dev.cls_scale;
     p.cls_parity = ctx->dev.cls_parity;
     p.cls_value = ctx->dev.cls_value;
     p.cls_pack = ctx->dev.cls_pack;
     p.error = ctx->error;
+#ifdef LLVQ_TRACE
+    p.trace = ctx->trace;
+    p.trace_launch = ctx->trace ? ctx->trace_launch++ : 0;
+#endif
     if (gemv_smem_bytes(layout, p.nb, n) + 1024 > (size_t)ctx->max_smem_optin) return LLVQ_ESIZE;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;

@@ -30,12 +30,42 @@
 // while the previous kernel drains.  Every wait is bounded.
 #include "llvq_internal.cuh"
 
+// Optional timeline (compiled in only with -DLLVQ_TRACE, never in the shipped library): lane 0 of
+// every warp stores the global timer at a few points of the kernel.
+#ifdef LLVQ_TRACE
+#define LLVQ_TRACE_POINT(i)                                                                                       \
+    if (p.trace && lane == 0) {                                                                                   \
+        unsigned long long t_;                                                                                    \
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                                    \
+        p.trace[(((size_t)p.trace_launch * gridDim.x + blockIdx.x) * kWarps + warp) * 128 + (i)] = t_;            \
+    }
+// per-unit timeline of every warp: slot 8 + 3*n + {0: wait begins, 1: data there, 2: decoded}, n < 40
+#define LLVQ_TRACE_UNIT(n, i)                                                                                     \
+    if (p.trace && lane == 0 && (n) < 40) {                                                                       \
+        unsigned long long t_;                                                                                    \
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                                    \
+        p.trace[(((size_t)p.trace_launch * gridDim.x + blockIdx.x) * kWarps + warp) * 128 + 8 + 3 * (n) + (i)] = t_; \
+    }
+#else
+#define LLVQ_TRACE_POINT(i)
+#define LLVQ_TRACE_UNIT(n, i)
+#endif
+
 namespace llvq {
 namespace {
 
-constexpr int kWarps = 16;                 // warps per CTA
+#ifndef LLVQ_WARPS
+#define LLVQ_WARPS 16
+#endif
+#ifndef LLVQ_SLOTS
+#define LLVQ_SLOTS 3
+#endif
+#ifndef LLVQ_MINB
+#define LLVQ_MINB 2
+#endif
+constexpr int kWarps = LLVQ_WARPS;         // warps per CTA
 constexpr int kThreads = kWarps * 32;
-constexpr int kSlots = 4;                  // ring slots per warp
+constexpr int kSlots = LLVQ_SLOTS;         // ring slots per warp
 constexpr uint32_t kPairMask = 0x80708070u;
 
 // fixed-point accumulator word: bits 53..63 count units, bits 0..52 sum the biased unit values
@@ -100,13 +130,13 @@ __device__ __forceinline__ int find_problem(const GemvParams &p, int group) {
 // exact power of two as a float, |e| < 126
 __device__ __forceinline__ float pow2f(int e) { return __int_as_float((127 + e) << 23); }
 
-// The contiguous range of units [u0, u1) of this warp; warps are numbered with the CTA index
-// fastest, so the ranges that are one unit longer spread over all multiprocessors.
-__device__ __forceinline__ void warp_range(const GemvParams &p, int warp, long long &u0, long long &u1) {
-    const long long warps = (long long)gridDim.x * kWarps, gw = (long long)warp * gridDim.x + blockIdx.x;
-    const long long base = p.total_units / warps, rem = p.total_units % warps;
-    u0 = gw * base + (gw < rem ? gw : rem);
-    u1 = u0 + base + (gw < rem ? 1 : 0);
+// The contiguous range of units [u0, u0 + n) of this warp; warps are numbered with the CTA index
+// fastest, so the ranges that are one unit longer spread over all multiprocessors.  The host
+// supplies total_units divided by the number of warps of the grid.
+__device__ __forceinline__ void warp_range(const GemvParams &p, int warp, int &u0, int &n) {
+    const int gw = warp * gridDim.x + blockIdx.x;
+    u0 = gw * p.units_base + min(gw, p.units_rem);
+    n = p.units_base + (gw < p.units_rem ? 1 : 0);
 }
 
 // Hands the warp's sum over `count` units of row group `group` to the row accumulators.
@@ -151,42 +181,35 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     return false;
 }
 
-// Position in the unit sequence: row group, unit inside it, the matrix it belongs to.
-struct Pos {
-    int group, k, q;
-    const uint8_t *grp;     // first byte of the row group's records
-};
+// Returns zero, but only once `v` is available: an address that adds this zero cannot be formed
+// before the loads that produced `v` have completed.
+__device__ __forceinline__ uint32_t settled(uint32_t v) {
+    uint32_t z;
+    asm volatile("and.b32 %0, %1, 0;" : "=r"(z) : "r"(v));
+    return z;
+}
 
-__device__ __forceinline__ void pos_set_group(const GemvParams &p, Pos &c, int cell_bytes) {
-    c.q = find_problem(p, c.group);
-    c.grp = p.prob[c.q].layout + (size_t)(c.group - p.prob[c.q].group_begin) * (size_t)p.nb * cell_bytes;
-}
-__device__ __forceinline__ void pos_init(const GemvParams &p, Pos &c, long long u, int cell_bytes) {
-    c.group = (int)(u / p.units);
-    c.k = (int)(u - (long long)c.group * p.units);
-    if (c.group < p.total_groups) pos_set_group(p, c, cell_bytes);
-}
-__device__ __forceinline__ void pos_next(const GemvParams &p, Pos &c, int cell_bytes) {
-    if (++c.k == p.units) {
-        c.k = 0;
-        c.group++;
-        if (c.group < p.total_groups) pos_set_group(p, c, cell_bytes);
-    }
+// First byte of a row group's records, and the matrix it belongs to.
+__device__ __forceinline__ const uint8_t *group_base(const GemvParams &p, int group, int cell_bytes, int &q) {
+    q = find_problem(p, group);
+    return p.prob[q].layout + (size_t)(group - p.prob[q].group_begin) * (size_t)p.nb * cell_bytes;
 }
 
 template <bool NO_WEIGHTS>
-__global__ void __launch_bounds__(kThreads, 2) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
+__global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
+    // shared memory: ring | per-matrix block constants (1024 x {scale * gain, parity}) | x | barriers
     unsigned char *ring = smem;
-    const float2 *cls = reinterpret_cast<const float2 *>(smem + kWarps * kSlots * kTileBytes);
-    const uint4 *xs = reinterpret_cast<const uint4 *>(smem + kWarps * kSlots * kTileBytes + kClassSlots * 8);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kWarps * kSlots * kTileBytes + kClassSlots * 8 + ((p.nb * 48 + 127) / 128) * 128);
+    float2 *tab = reinterpret_cast<float2 *>(smem + kWarps * kSlots * kTileBytes);
+    const uint4 *xs = reinterpret_cast<const uint4 *>(smem + kWarps * kSlots * kTileBytes + p.nprob * 8192);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kWarps * kSlots * kTileBytes + p.nprob * 8192 + ((p.nb * 48 + 127) / 128) * 128);
     uint32_t *xor_word = reinterpret_cast<uint32_t *>(bars + kWarps * kSlots + 1);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t my_ring = smem_addr(ring + warp * kSlots * kTileBytes);
     const uint32_t my_bar = smem_addr(bars + warp * kSlots);
     const uint32_t pro_bar = smem_addr(bars + kWarps * kSlots);
 
+    LLVQ_TRACE_POINT(0)
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kSlots; s++) mbar_init(my_bar + 8 * s, 1);
@@ -195,40 +218,53 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_planes_kernel(const __grid_c
     }
     __syncthreads();
 
-    long long u0, u1;
-    warp_range(p, warp, u0, u1);
-    Pos pi, pc;                            // issue side, consume side
-    pos_init(p, pi, u0, kCellBytes);
-    pc = pi;
-    long long ui = u0;
+    int u0, n_units;
+    warp_range(p, warp, u0, n_units);
+    // consume side: row group and unit inside it; issue side: a running source pointer
+    int group = u0 / p.units, k = u0 - group * p.units, q = 0;
+    const uint8_t *src = nullptr;
+    int ik = k, igroup = group, issued = 0;
+    if (n_units > 0) src = group_base(p, group, kCellBytes, q) + (size_t)(k < p.tiles ? k : p.tiles) * kTileBytes;
     const uint32_t tail_bytes = (uint32_t)p.tail_cells * kCellBytes;
 
-    auto issue = [&](int s) {
+    // issue the copy of the next unit into slot s (lane 0), then step the source
+    auto issue = [&](int s, uint32_t zero) {
+        const bool tile = ik < p.tiles;
+        const uint32_t bytes = tile ? (uint32_t)kTileBytes : tail_bytes;
         if (lane == 0) {
-            const bool tile = pi.k < p.tiles;
-            const uint32_t bytes = tile ? (uint32_t)kTileBytes : tail_bytes;
             mbar_expect(my_bar + 8 * s, bytes);
-            bulk_g2s(my_ring + s * kTileBytes, pi.grp + (size_t)(tile ? pi.k : p.tiles) * kTileBytes, bytes, my_bar + 8 * s);
+            bulk_g2s(my_ring + s * kTileBytes + zero, src, bytes, my_bar + 8 * s);
         }
-        pos_next(p, pi, kCellBytes);
-        ui++;
+        issued++;
+        src += bytes;                                  // a row group's units are contiguous, and so are a matrix's row groups
+        if (++ik == p.units) {
+            ik = 0;
+            igroup++;
+            if (igroup < p.total_groups && issued < n_units) { int qi; src = group_base(p, igroup, kCellBytes, qi); }
+        }
     };
 
     if (!NO_WEIGHTS) {
 #pragma unroll
         for (int s = 0; s < kSlots; s++)
-            if (ui < u1) issue(s);
+            if (issued < n_units) issue(s, 0u);
     }
-    if (tid == 0) {
-        mbar_expect(pro_bar, kClassSlots * 8 + p.nb * 48);
-        bulk_g2s(smem_addr(cls), p.cls_pack, kClassSlots * 8, pro_bar);
+    // block constants of every matrix of the launch: (class | gain << 9) -> {gain * 2^21 / (4 sqrt m), parity pattern}
+    for (int e = tid; e < p.nprob * 1024; e += kThreads) {
+        const float2 v = __ldg(p.cls_pack + (e & 511));
+        const GemvProblemDev &pe = p.prob[e >> 10];
+        tab[e] = make_float2(v.x * ((e & 512) ? pe.gain1 : pe.gain0), v.y);
     }
     // let the next kernel in the stream start its own prefetch, then wait for the previous one:
     // x, y and the reduction scratch may still be in use by it
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    LLVQ_TRACE_POINT(1)
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    if (tid == 0) bulk_g2s(smem_addr(xs), p.x, p.nb * 48, pro_bar);
-
+    LLVQ_TRACE_POINT(2)
+    if (tid == 0) {
+        mbar_expect(pro_bar, p.nb * 48);
+        bulk_g2s(smem_addr(xs), p.x, p.nb * 48, pro_bar);
+    }
     bool failed = !mbar_wait(pro_bar, 0);
     // every |x| is below 2^(e-14), e the biased exponent of the OR of all magnitudes
     int xexp;
@@ -238,42 +274,49 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_planes_kernel(const __grid_c
         for (int e = tid; e < p.nb * 12; e += kThreads) m |= xw[e];
         m = __reduce_or_sync(0xffffffffu, (m | (m >> 16)) & 0x7fffu);
         if (lane == 0 && m) atomicOr(xor_word, m);
-        __syncthreads();
+        __syncthreads();                               // also publishes the block constants
         xexp = max((int)(*xor_word >> 10), 1) - 14;
     }
+    LLVQ_TRACE_POINT(3)
 
     uint32_t phases = 0;
     int slot = 0, count = 0;
     long long sum = 0;
-    int qexp = xexp + p.prob[pc.q].qexp_base;
+    int qexp = xexp + p.prob[q].qexp_base;
     float inv_q = pow2f(-qexp);
+    const float2 *tq = tab + q * 1024;
 
-    for (long long u = u0; u < u1 && !failed; u++) {
-        const GemvProblemDev &pr = p.prob[pc.q];
+    for (int n = 0; n < n_units && !failed; n++) {
         float s = 0.f;
         if (!NO_WEIGHTS) {
             const uint32_t bar = my_bar + 8 * slot;
+            LLVQ_TRACE_UNIT(n, 0)
             if (!mbar_wait(bar, (phases >> slot) & 1u)) { failed = true; break; }
             phases ^= 1u << slot;
+            LLVQ_TRACE_UNIT(n, 1)
+            if (n == 0) { LLVQ_TRACE_POINT(4) }
             const unsigned char *buf = ring + (warp * kSlots + slot) * kTileBytes;
-            if (pc.k < p.tiles) {
+            if (k < p.tiles) {
                 const uint4 a0 = *reinterpret_cast<const uint4 *>(buf + 16 * lane);
                 const uint4 a1 = *reinterpret_cast<const uint4 *>(buf + 512 + 16 * lane);
                 const uint4 a2 = *reinterpret_cast<const uint4 *>(buf + 1024 + 16 * lane);
                 const uint2 hh = *reinterpret_cast<const uint2 *>(buf + 1536 + 8 * lane);
                 const uint32_t w0[4] = {a0.x, a0.y, a0.z, a0.w}, w1[4] = {a1.x, a1.y, a1.z, a1.w}, w2[4] = {a2.x, a2.y, a2.z, a2.w};
                 const uint32_t hd[4] = {hh.x & 0xffffu, hh.x >> 16, hh.y & 0xffffu, hh.y >> 16};
+                // The slot's words are in registers: refill it at once with the unit kSlots ahead, so
+                // that every slot but the one just read is in flight while this unit is decoded.  The
+                // copy's address is made to depend on the loaded words, which holds the copy back
+                // until the four shared-memory reads of the whole warp have completed.
+                if (issued < n_units) issue(slot, settled(a0.w ^ a1.w ^ a2.w ^ hh.y));
+                const uint4 *xc = xs + 12 * k;
 #pragma unroll
                 for (int c = 0; c < 4; c++) {
-                    const float2 k = cls[hd[c] & 511u];
-                    const float g = (hd[c] & 512u) ? pr.gain1 : pr.gain0;
-                    const float dot = block_dot(w0[c], w1[c], w2[c], __float_as_uint(k.y), xs + 3 * (4 * pc.k + c));
-                    s = fmaf(k.x * g, dot, s);
-                    if (c == 1) {
-                        // the slot's words are in registers: refill it with the unit kSlots ahead
-                        __syncwarp();
-                        if (ui < u1) issue(slot);
-                    }
+#ifdef LLVQ_STREAM_ONLY
+                    s += __uint_as_float((w0[c] ^ w1[c] ^ w2[c] ^ hd[c]) & 0x007fffffu);   // debug: bytes only, no decode
+#else
+                    const float2 kc = tq[hd[c] & 1023u];
+                    s = fmaf(kc.x, block_dot(w0[c], w1[c], w2[c], __float_as_uint(kc.y), xc + 3 * c), s);
+#endif
                 }
             } else {
                 uint32_t tw[3][3], th[3];
@@ -286,38 +329,45 @@ __global__ void __launch_bounds__(kThreads, 2) gemv_planes_kernel(const __grid_c
                         tw[c][2] = *reinterpret_cast<const uint32_t *>(cell + 256 + 4 * lane);
                         th[c] = *reinterpret_cast<const uint16_t *>(cell + 384 + 2 * lane);
                     }
+                if (issued < n_units)
+                    issue(slot, settled(tw[0][0] ^ tw[0][1] ^ tw[0][2] ^ th[0] ^ (p.tail_cells > 1 ? tw[1][2] ^ th[1] : 0u) ^
+                                        (p.tail_cells > 2 ? tw[2][2] ^ th[2] : 0u)));
+                const uint4 *xc = xs + 12 * p.tiles;
 #pragma unroll
                 for (int c = 0; c < 3; c++)
                     if (c < p.tail_cells) {
-                        const float2 k = cls[th[c] & 511u];
-                        const float g = (th[c] & 512u) ? pr.gain1 : pr.gain0;
-                        const float dot = block_dot(tw[c][0], tw[c][1], tw[c][2], __float_as_uint(k.y), xs + 3 * (4 * p.tiles + c));
-                        s = fmaf(k.x * g, dot, s);
+                        const float2 kc = tq[th[c] & 1023u];
+                        s = fmaf(kc.x, block_dot(tw[c][0], tw[c][1], tw[c][2], __float_as_uint(kc.y), xc + 3 * c), s);
                     }
-                __syncwarp();
-                if (ui < u1) issue(slot);
             }
             slot = (slot + 1 == kSlots) ? 0 : slot + 1;
         }
         sum += __float2ll_rn(s * inv_q) + kUnitBias;
         count++;
-        const int group = pc.group;
-        pos_next(p, pc, kCellBytes);
-        if (pc.k == 0 || u + 1 == u1) {
-            deliver(p, pr, group, lane, sum, count, qexp);
+        LLVQ_TRACE_UNIT(n, 2)
+        if (++k == p.units || n + 1 == n_units) {
+            if (n + 1 == n_units) { LLVQ_TRACE_POINT(6) }
+            deliver(p, p.prob[q], group, lane, sum, count, qexp);
             sum = 0;
             count = 0;
-            if (pc.group < p.total_groups) {
-                qexp = xexp + p.prob[pc.q].qexp_base;
-                inv_q = pow2f(-qexp);
+            if (k == p.units) {
+                k = 0;
+                group++;
+                if (group < p.total_groups) {
+                    q = find_problem(p, group);
+                    qexp = xexp + p.prob[q].qexp_base;
+                    inv_q = pow2f(-qexp);
+                    tq = tab + q * 1024;
+                }
             }
         }
     }
 
+    LLVQ_TRACE_POINT(5)
     if (failed) {
         // a wait ran out: report it, then give the copies still in flight a bounded chance to land
         if (lane == 0) atomicExch(p.error, 1);
-        const int pending = (int)min((long long)kSlots, ui - u0);     // generous: wait on every slot once
+        const int pending = min(kSlots, issued);       // generous: wait on every slot once
         for (int s = 0; s < pending; s++) {
             mbar_wait(my_bar + 8 * slot, (phases >> slot) & 1u);
             slot = (slot + 1 == kSlots) ? 0 : slot + 1;
@@ -346,19 +396,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_onehot_kernel(const __grid_c
     __syncthreads();
     const int xexp = max((int)(xor_word >> 10), 1) - 14;
 
-    long long u0, u1;
-    warp_range(p, warp, u0, u1);
-    Pos pc;
-    pos_init(p, pc, u0, kOneHotCellBytes);
+    int u0, n_units;
+    warp_range(p, warp, u0, n_units);
+    int group = u0 / p.units, k = u0 - group * p.units, q = 0;
+    const uint8_t *grp = n_units > 0 ? group_base(p, group, kOneHotCellBytes, q) : nullptr;
     long long sum = 0;
     int count = 0;
-    for (long long u = u0; u < u1; u++) {
-        const GemvProblemDev &pr = p.prob[pc.q];
+    for (int n = 0; n < n_units; n++) {
+        const GemvProblemDev &pr = p.prob[q];
         const int qexp = xexp + pr.qexp_base;
-        const int c0 = pc.k * kTileCells, c1 = pc.k < p.tiles ? c0 + kTileCells : p.nb;
+        const int c0 = k * kTileCells, c1 = k < p.tiles ? c0 + kTileCells : p.nb;
         float s = 0.f;
         for (int c = c0; c < c1; c++) {
-            const uint32_t *cell = reinterpret_cast<const uint32_t *>(pc.grp + (size_t)c * kOneHotCellBytes);
+            const uint32_t *cell = reinterpret_cast<const uint32_t *>(grp + (size_t)c * kOneHotCellBytes);
             uint32_t v[5];
 #pragma unroll
             for (int t = 0; t < 5; t++) v[t] = __ldcs(cell + 32 * t + lane);
@@ -371,12 +421,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_onehot_kernel(const __grid_c
         }
         sum += __float2ll_rn(s * pow2f(-qexp)) + kUnitBias;
         count++;
-        const int group = pc.group;
-        pos_next(p, pc, kOneHotCellBytes);
-        if (pc.k == 0 || u + 1 == u1) {
+        if (++k == p.units || n + 1 == n_units) {
             deliver(p, pr, group, lane, sum, count, qexp);
             sum = 0;
             count = 0;
+            if (k == p.units) {
+                k = 0;
+                group++;
+                if (group < p.total_groups) grp = group_base(p, group, kOneHotCellBytes, q);
+            }
         }
     }
 }
@@ -488,10 +541,9 @@ __global__ void __launch_bounds__(256) dequant_kernel(int layout, const uint8_t 
 }  // namespace
 
 size_t gemv_smem_bytes(int layout, int nb, int nprob) {
-    (void)nprob;
     const size_t xbytes = ((size_t)nb * 48 + 127) / 128 * 128;
     if (layout != LLVQ_PLANES) return xbytes;
-    return (size_t)kWarps * kSlots * kTileBytes + kClassSlots * 8 + xbytes + (kWarps * kSlots + 2) * 8;
+    return (size_t)kWarps * kSlots * kTileBytes + (size_t)nprob * 8192 + xbytes + (kWarps * kSlots + 2) * 8;
 }
 
 template <typename K>
@@ -509,11 +561,13 @@ int gemv_configure(const llvq_ctx *ctx) {
     return 0;
 }
 
-cudaError_t launch_gemv(const llvq_ctx *ctx, int layout, const GemvParams &p, bool no_weights, cudaStream_t s) {
+cudaError_t launch_gemv(const llvq_ctx *ctx, int layout, GemvParams &p, bool no_weights, cudaStream_t s) {
     const size_t smem = gemv_smem_bytes(layout, p.nb, p.nprob);
     // one CTA a multiprocessor; fewer only when there are fewer units than warps
-    long long grid = (p.total_units + kWarps - 1) / kWarps;
+    int grid = (p.total_units + kWarps - 1) / kWarps;
     if (grid > ctx->sm_count) grid = ctx->sm_count;
+    p.units_base = p.total_units / (grid * kWarps);
+    p.units_rem = p.total_units % (grid * kWarps);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kThreads);

@@ -49,13 +49,18 @@ struct GemvParams {
     int nb, tiles, tail_cells;
     int units;             // units a row group: tiles, plus one for the nb mod 4 last columns
     int total_groups;
-    long long total_units;
+    int total_units;       // total_groups * units
+    int units_base, units_rem;   // total_units divided by the warps of the grid (set at launch)
     unsigned long long *accum;   // total_groups x 32 fixed-point row accumulators (context scratch, zero between launches)
     const float *cls_scale;
     const uint32_t *cls_parity;
     const float *cls_value;
     const float2 *cls_pack;   // 512 x {2^21 / (4 sqrt m), parity pattern as bits}
     int *error;               // set when a bounded wait ran out
+#ifdef LLVQ_TRACE
+    unsigned long long *trace;   // timeline buffer (debug builds only)
+    int trace_launch;
+#endif
 };
 
 }  // namespace llvq
@@ -69,6 +74,10 @@ struct llvq_ctx {
     size_t accum_slots;
     int *error;              // device flag: a kernel's bounded wait ran out
     int use_pdl;             // launch the GEMV with programmatic stream serialization
+#ifdef LLVQ_TRACE
+    unsigned long long *trace;
+    int trace_launch;
+#endif
     int sm_count;
     int max_smem_optin;
 };
@@ -76,7 +85,7 @@ struct llvq_ctx {
 namespace llvq {
 cudaError_t launch_expand(const llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, int64_t nb,
                           void *out, uint32_t *bad_count, cudaStream_t s);
-cudaError_t launch_gemv(const llvq_ctx *ctx, int layout, const GemvParams &p, bool no_weights, cudaStream_t s);
+cudaError_t launch_gemv(const llvq_ctx *ctx, int layout, GemvParams &p, bool no_weights, cudaStream_t s);
 cudaError_t launch_gemv_fp16(const __half *W, const __half *x, float *y, int64_t rows, int64_t k, cudaStream_t s);
 cudaError_t launch_dequant(const llvq_ctx *ctx, int layout, const uint8_t *buf, const __half *row_scale, float g0, float g1,
                            __half *W, int64_t rows, int64_t nb, cudaStream_t s);
