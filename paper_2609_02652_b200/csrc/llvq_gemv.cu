@@ -279,99 +279,95 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     }
     LLVQ_TRACE_POINT(3)
 
-    uint32_t phases = 0;
-    int slot = 0, count = 0;
+    int count = 0, n = 0;
     long long sum = 0;
     int qexp = xexp + p.prob[q].qexp_base;
     float inv_q = pow2f(-qexp);
     const float2 *tq = tab + q * 1024;
+    uint32_t parity = 0;                               // every slot completes once a round of kSlots units
 
-    for (int n = 0; n < n_units && !failed; n++) {
-        float s = 0.f;
-        if (!NO_WEIGHTS) {
-            const uint32_t bar = my_bar + 8 * slot;
-            LLVQ_TRACE_UNIT(n, 0)
-            if (!mbar_wait(bar, (phases >> slot) & 1u)) { failed = true; break; }
-            phases ^= 1u << slot;
-            LLVQ_TRACE_UNIT(n, 1)
-            if (n == 0) { LLVQ_TRACE_POINT(4) }
-            const unsigned char *buf = ring + (warp * kSlots + slot) * kTileBytes;
-            if (k < p.tiles) {
-                const uint4 a0 = *reinterpret_cast<const uint4 *>(buf + 16 * lane);
-                const uint4 a1 = *reinterpret_cast<const uint4 *>(buf + 512 + 16 * lane);
-                const uint4 a2 = *reinterpret_cast<const uint4 *>(buf + 1024 + 16 * lane);
-                const uint2 hh = *reinterpret_cast<const uint2 *>(buf + 1536 + 8 * lane);
-                const uint32_t w0[4] = {a0.x, a0.y, a0.z, a0.w}, w1[4] = {a1.x, a1.y, a1.z, a1.w}, w2[4] = {a2.x, a2.y, a2.z, a2.w};
-                const uint32_t hd[4] = {hh.x & 0xffffu, hh.x >> 16, hh.y & 0xffffu, hh.y >> 16};
-                // The slot's words are in registers: refill it at once with the unit kSlots ahead, so
-                // that every slot but the one just read is in flight while this unit is decoded.  The
-                // copy's address is made to depend on the loaded words, which holds the copy back
-                // until the four shared-memory reads of the whole warp have completed.
-                if (issued < n_units) issue(slot, settled(a0.w ^ a1.w ^ a2.w ^ hh.y));
-                const uint4 *xc = xs + 12 * k;
+    while (n < n_units && !failed) {
 #pragma unroll
-                for (int c = 0; c < 4; c++) {
+        for (int slot = 0; slot < kSlots; slot++) {
+            if (n >= n_units) break;
+            float s = 0.f;
+            if (!NO_WEIGHTS) {
+                const uint32_t bar = my_bar + 8 * slot;
+                LLVQ_TRACE_UNIT(n, 0)
+                if (!mbar_wait(bar, parity)) { failed = true; break; }
+                LLVQ_TRACE_UNIT(n, 1)
+                if (n == 0) { LLVQ_TRACE_POINT(4) }
+                const unsigned char *buf = ring + (warp * kSlots + slot) * kTileBytes;
+                if (k < p.tiles) {
+                    const uint4 a0 = *reinterpret_cast<const uint4 *>(buf + 16 * lane);
+                    const uint4 a1 = *reinterpret_cast<const uint4 *>(buf + 512 + 16 * lane);
+                    const uint4 a2 = *reinterpret_cast<const uint4 *>(buf + 1024 + 16 * lane);
+                    const uint2 hh = *reinterpret_cast<const uint2 *>(buf + 1536 + 8 * lane);
+                    const uint32_t w0[4] = {a0.x, a0.y, a0.z, a0.w}, w1[4] = {a1.x, a1.y, a1.z, a1.w}, w2[4] = {a2.x, a2.y, a2.z, a2.w};
+                    const uint32_t hd[4] = {hh.x & 0xffffu, hh.x >> 16, hh.y & 0xffffu, hh.y >> 16};
+                    // The slot's words are in registers: refill it at once with the unit kSlots ahead, so
+                    // that every slot but the one just read is in flight while this unit is decoded.  The
+                    // copy's address is made to depend on the loaded words, which holds the copy back
+                    // until the four shared-memory reads of the whole warp have completed.
+                    if (issued < n_units) issue(slot, settled(a0.w ^ a1.w ^ a2.w ^ hh.y));
+                    const uint4 *xc = xs + 12 * k;
+#pragma unroll
+                    for (int c = 0; c < 4; c++) {
 #ifdef LLVQ_STREAM_ONLY
-                    s += __uint_as_float((w0[c] ^ w1[c] ^ w2[c] ^ hd[c]) & 0x007fffffu);   // debug: bytes only, no decode
+                        s += __uint_as_float((w0[c] ^ w1[c] ^ w2[c] ^ hd[c]) & 0x007fffffu);   // debug: bytes only, no decode
 #else
-                    const float2 kc = tq[hd[c] & 1023u];
-                    s = fmaf(kc.x, block_dot(w0[c], w1[c], w2[c], __float_as_uint(kc.y), xc + 3 * c), s);
+                        const float2 kc = tq[hd[c] & 1023u];
+                        s = fmaf(kc.x, block_dot(w0[c], w1[c], w2[c], __float_as_uint(kc.y), xc + 3 * c), s);
 #endif
-                }
-            } else {
-                uint32_t tw[3][3], th[3];
-#pragma unroll
-                for (int c = 0; c < 3; c++)
-                    if (c < p.tail_cells) {
+                    }
+                } else {
+                    // the nb mod 4 last block columns of the row group: rare, kept out of the unrolled path
+                    uint32_t guard = 0;
+                    const uint4 *xc = xs + 12 * p.tiles;
+#pragma unroll 1
+                    for (int c = 0; c < p.tail_cells; c++) {
                         const unsigned char *cell = buf + c * kCellBytes;
-                        tw[c][0] = *reinterpret_cast<const uint32_t *>(cell + 4 * lane);
-                        tw[c][1] = *reinterpret_cast<const uint32_t *>(cell + 128 + 4 * lane);
-                        tw[c][2] = *reinterpret_cast<const uint32_t *>(cell + 256 + 4 * lane);
-                        th[c] = *reinterpret_cast<const uint16_t *>(cell + 384 + 2 * lane);
+                        const uint32_t t0 = *reinterpret_cast<const uint32_t *>(cell + 4 * lane);
+                        const uint32_t t1 = *reinterpret_cast<const uint32_t *>(cell + 128 + 4 * lane);
+                        const uint32_t t2 = *reinterpret_cast<const uint32_t *>(cell + 256 + 4 * lane);
+                        const uint32_t th = *reinterpret_cast<const uint16_t *>(cell + 384 + 2 * lane);
+                        guard ^= t0 ^ t1 ^ t2 ^ th;
+                        const float2 kc = tq[th & 1023u];
+                        s = fmaf(kc.x, block_dot(t0, t1, t2, __float_as_uint(kc.y), xc + 3 * c), s);
                     }
-                if (issued < n_units)
-                    issue(slot, settled(tw[0][0] ^ tw[0][1] ^ tw[0][2] ^ th[0] ^ (p.tail_cells > 1 ? tw[1][2] ^ th[1] : 0u) ^
-                                        (p.tail_cells > 2 ? tw[2][2] ^ th[2] : 0u)));
-                const uint4 *xc = xs + 12 * p.tiles;
-#pragma unroll
-                for (int c = 0; c < 3; c++)
-                    if (c < p.tail_cells) {
-                        const float2 kc = tq[th[c] & 1023u];
-                        s = fmaf(kc.x, block_dot(tw[c][0], tw[c][1], tw[c][2], __float_as_uint(kc.y), xc + 3 * c), s);
-                    }
+                    if (issued < n_units) issue(slot, settled(guard));
+                }
             }
-            slot = (slot + 1 == kSlots) ? 0 : slot + 1;
-        }
-        sum += __float2ll_rn(s * inv_q) + kUnitBias;
-        count++;
-        LLVQ_TRACE_UNIT(n, 2)
-        if (++k == p.units || n + 1 == n_units) {
-            if (n + 1 == n_units) { LLVQ_TRACE_POINT(6) }
-            deliver(p, p.prob[q], group, lane, sum, count, qexp);
-            sum = 0;
-            count = 0;
-            if (k == p.units) {
-                k = 0;
-                group++;
-                if (group < p.total_groups) {
-                    q = find_problem(p, group);
-                    qexp = xexp + p.prob[q].qexp_base;
-                    inv_q = pow2f(-qexp);
-                    tq = tab + q * 1024;
+            sum += __float2ll_rn(s * inv_q) + kUnitBias;
+            count++;
+            LLVQ_TRACE_UNIT(n, 2)
+            n++;
+            if (++k == p.units || n == n_units) {
+                if (n == n_units) { LLVQ_TRACE_POINT(6) }
+                deliver(p, p.prob[q], group, lane, sum, count, qexp);
+                sum = 0;
+                count = 0;
+                if (k == p.units) {
+                    k = 0;
+                    group++;
+                    if (group < p.total_groups) {
+                        q = find_problem(p, group);
+                        qexp = xexp + p.prob[q].qexp_base;
+                        inv_q = pow2f(-qexp);
+                        tq = tab + q * 1024;
+                    }
                 }
             }
         }
+        parity ^= 1u;
     }
 
     LLVQ_TRACE_POINT(5)
     if (failed) {
         // a wait ran out: report it, then give the copies still in flight a bounded chance to land
+        // (a slot that is not pending returns at once or runs into the same bound)
         if (lane == 0) atomicExch(p.error, 1);
-        const int pending = min(kSlots, issued);       // generous: wait on every slot once
-        for (int s = 0; s < pending; s++) {
-            mbar_wait(my_bar + 8 * slot, (phases >> slot) & 1u);
-            slot = (slot + 1 == kSlots) ? 0 : slot + 1;
-        }
+        for (int s = 0; s < kSlots && s < issued; s++) mbar_wait(my_bar + 8 * s, parity);
     }
 }
 
