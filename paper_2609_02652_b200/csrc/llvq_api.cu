@@ -210,7 +210,8 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
     if (!(gain_max < 3.0e38f)) return LLVQ_EINVAL;
     // quantum of the fixed-point row accumulators, per matrix so that grouping does not change it:
     // a unit sums at most four blocks, each bounded by max|gain| * sqrt(24) * max|x| < 2^ge * 5 * 2^xe;
-    // 4 * 5 < 2^5, and the unit value is kept under 2^39 quanta (see deliver() in llvq_gemv.cu)
+    // 4 * 5 < 2^5, and the unit value is kept under 2^39 quanta (see deliver() in llvq_gemv.cu), which
+    // puts the quantum some 2^-32 below a typical unit sum: far finer than the f32 sums it collects
     for (int i = 0; i < n; i++) {
         const float gm = std::fmax(std::fabs(problems[i].gain[0]), std::fabs(problems[i].gain[1]));
         int ge = 0;

@@ -127,6 +127,13 @@ __device__ __forceinline__ int find_problem(const GemvParams &p, int group) {
     return q;
 }
 
+// running maximum of |fp16| over both halves of a word, kept as two 15-bit patterns
+__device__ __forceinline__ uint32_t max_abs_pair(uint32_t m, uint32_t x2) {
+    const uint32_t a = x2 & 0x7fff7fffu;
+    const __half2 r = __hmax2(*reinterpret_cast<const __half2 *>(&m), *reinterpret_cast<const __half2 *>(&a));
+    return *reinterpret_cast<const uint32_t *>(&r);
+}
+
 // exact power of two as a float, |e| < 126
 __device__ __forceinline__ float pow2f(int e) { return __int_as_float((127 + e) << 23); }
 
@@ -144,7 +151,7 @@ __device__ __forceinline__ void deliver(const GemvParams &p, const GemvProblemDe
                                         long long sum, int count, int qexp) {
     const int row = (group - pr.group_begin) * kRowsPerGroup + lane;
     if (row >= pr.rows) return;                      // padding rows of the last row group
-    const unsigned long long addend = (unsigned long long)sum + ((unsigned long long)count << kCountShift);
+    const unsigned long long addend = (unsigned long long)(sum + (long long)count * kUnitBias) + ((unsigned long long)count << kCountShift);
     unsigned long long *slot = p.accum + (size_t)group * 32 + lane;
     const unsigned long long old = atomicAdd(slot, addend);
     if ((int)(old >> kCountShift) + count == p.units) {
@@ -181,11 +188,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     return false;
 }
 
-// Returns zero, but only once `v` is available: an address that adds this zero cannot be formed
-// before the loads that produced `v` have completed.
-__device__ __forceinline__ uint32_t settled(uint32_t v) {
+// Returns zero, but only once its operands are available: an address that adds this zero cannot be
+// formed before the loads that produced them have completed.
+__device__ __forceinline__ uint32_t settled(uint32_t a, uint32_t b, uint32_t c) {
     uint32_t z;
-    asm volatile("and.b32 %0, %1, 0;" : "=r"(z) : "r"(v));
+    asm volatile("lop3.b32 %0, %1, %2, %3, 0x00;" : "=r"(z) : "r"(a), "r"(b), "r"(c));
     return z;
 }
 
@@ -227,14 +234,19 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     if (n_units > 0) src = group_base(p, group, kCellBytes, q) + (size_t)(k < p.tiles ? k : p.tiles) * kTileBytes;
     const uint32_t tail_bytes = (uint32_t)p.tail_cells * kCellBytes;
 
-    // issue the copy of the next unit into slot s (lane 0), then step the source
-    auto issue = [&](int s, uint32_t zero) {
-        const bool tile = ik < p.tiles;
-        const uint32_t bytes = tile ? (uint32_t)kTileBytes : tail_bytes;
-        if (lane == 0) {
-            mbar_expect(my_bar + 8 * s, bytes);
-            bulk_g2s(my_ring + s * kTileBytes + zero, src, bytes, my_bar + 8 * s);
-        }
+    // issue the copy of the next unit (lane 0 alone, by predicate) onto barrier `b` and buffer `dst`,
+    // then step the source
+    auto issue = [&](uint32_t b, uint32_t dst) {
+        const uint32_t bytes = ik < p.tiles ? (uint32_t)kTileBytes : tail_bytes;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.eq.u32 p, %0, 0;\n\t"
+            "@p mbarrier.arrive.expect_tx.shared::cta.b64 _, [%1], %2;\n\t"
+            "@p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%3], [%4], %2, [%1];\n\t}"
+            ::"r"(lane), "r"(b), "r"(bytes), "r"(dst), "l"(src));
+        // No "memory" clobber: the only memory the copy writes is the slot, whose last reads feed
+        // `dst` through settled() and whose next reads follow the next wait on `b`; a clobber here
+        // would pin every shared-memory read of the decode behind the copy.
         issued++;
         src += bytes;                                  // a row group's units are contiguous, and so are a matrix's row groups
         if (++ik == p.units) {
@@ -247,7 +259,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     if (!NO_WEIGHTS) {
 #pragma unroll
         for (int s = 0; s < kSlots; s++)
-            if (issued < n_units) issue(s, 0u);
+            if (issued < n_units) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
     }
     // block constants of every matrix of the launch: (class | gain << 9) -> {gain * 2^21 / (4 sqrt m), parity pattern}
     for (int e = tid; e < p.nprob * 1024; e += kThreads) {
@@ -266,100 +278,104 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         bulk_g2s(smem_addr(xs), p.x, p.nb * 48, pro_bar);
     }
     bool failed = !mbar_wait(pro_bar, 0);
-    // every |x| is below 2^(e-14), e the biased exponent of the OR of all magnitudes
+    // every |x| is below 2^(e-14), e the biased exponent of the largest magnitude (fp16 bit patterns
+    // of non-negative values order like integers)
     int xexp;
     {
         uint32_t m = 0;
         const uint32_t *xw = reinterpret_cast<const uint32_t *>(xs);
-        for (int e = tid; e < p.nb * 12; e += kThreads) m |= xw[e];
-        m = __reduce_or_sync(0xffffffffu, (m | (m >> 16)) & 0x7fffu);
-        if (lane == 0 && m) atomicOr(xor_word, m);
+        for (int e = tid; e < p.nb * 12; e += kThreads) m = max_abs_pair(m, xw[e]);
+        m = __reduce_max_sync(0xffffffffu, max(m & 0xffffu, m >> 16));
+        if (lane == 0 && m) atomicMax(xor_word, m);
         __syncthreads();                               // also publishes the block constants
         xexp = max((int)(*xor_word >> 10), 1) - 14;
     }
     LLVQ_TRACE_POINT(3)
 
-    int count = 0, n = 0;
-    long long sum = 0;
-    int qexp = xexp + p.prob[q].qexp_base;
-    float inv_q = pow2f(-qexp);
-    const float2 *tq = tab + q * 1024;
+    int n = 0;
     uint32_t parity = 0;                               // every slot completes once a round of kSlots units
+    uint32_t bar = my_bar;                             // barrier and buffer of the slot that is consumed next
+    const unsigned char *buf = ring + warp * kSlots * kTileBytes;
+    const unsigned char *const buf_end = buf + kSlots * kTileBytes;
+    const int tiles = p.tiles, units = p.units;
 
+    // A run is the stretch of units of one row group inside this warp's range: its units are summed
+    // in a register and handed over together.
     while (n < n_units && !failed) {
-#pragma unroll
-        for (int slot = 0; slot < kSlots; slot++) {
-            if (n >= n_units) break;
+        const GemvProblemDev &pr = p.prob[q];
+        const int qexp = xexp + pr.qexp_base;
+        const float inv_q = pow2f(-qexp);
+        const float2 *tq = tab + q * 1024;
+        const int run = min(units - k, n_units - n);
+        const int run_tiles = NO_WEIGHTS ? 0 : max(0, min(run, tiles - k));
+        const uint4 *xc = xs + 12 * k;
+        long long sum = 0;
+
+        for (int t = 0; t < run_tiles; t++, xc += 12) {
+            LLVQ_TRACE_UNIT(n + t, 0)
+            if (!mbar_wait(bar, parity)) { failed = true; break; }
+            LLVQ_TRACE_UNIT(n + t, 1)
+            const uint4 a0 = *reinterpret_cast<const uint4 *>(buf + 16 * lane);
+            const uint4 a1 = *reinterpret_cast<const uint4 *>(buf + 512 + 16 * lane);
+            const uint4 a2 = *reinterpret_cast<const uint4 *>(buf + 1024 + 16 * lane);
+            const uint2 hh = *reinterpret_cast<const uint2 *>(buf + 1536 + 8 * lane);
+            const uint32_t w0[4] = {a0.x, a0.y, a0.z, a0.w}, w1[4] = {a1.x, a1.y, a1.z, a1.w}, w2[4] = {a2.x, a2.y, a2.z, a2.w};
+            const uint32_t hd[4] = {hh.x & 0xffffu, hh.x >> 16, hh.y & 0xffffu, hh.y >> 16};
+            // The slot's words are in registers: refill it at once with the unit kSlots ahead, so
+            // that every slot but the one just read is in flight while this unit is decoded.  The
+            // copy's address is made to depend on the loaded words, which holds the copy back
+            // until the four shared-memory reads of the whole warp have completed.
+            if (issued < n_units) issue(bar, smem_addr(buf) + (settled(a0.w, a1.w, a2.w) | settled(hh.y, hh.x, a0.x)));
             float s = 0.f;
-            if (!NO_WEIGHTS) {
-                const uint32_t bar = my_bar + 8 * slot;
-                LLVQ_TRACE_UNIT(n, 0)
-                if (!mbar_wait(bar, parity)) { failed = true; break; }
-                LLVQ_TRACE_UNIT(n, 1)
-                if (n == 0) { LLVQ_TRACE_POINT(4) }
-                const unsigned char *buf = ring + (warp * kSlots + slot) * kTileBytes;
-                if (k < p.tiles) {
-                    const uint4 a0 = *reinterpret_cast<const uint4 *>(buf + 16 * lane);
-                    const uint4 a1 = *reinterpret_cast<const uint4 *>(buf + 512 + 16 * lane);
-                    const uint4 a2 = *reinterpret_cast<const uint4 *>(buf + 1024 + 16 * lane);
-                    const uint2 hh = *reinterpret_cast<const uint2 *>(buf + 1536 + 8 * lane);
-                    const uint32_t w0[4] = {a0.x, a0.y, a0.z, a0.w}, w1[4] = {a1.x, a1.y, a1.z, a1.w}, w2[4] = {a2.x, a2.y, a2.z, a2.w};
-                    const uint32_t hd[4] = {hh.x & 0xffffu, hh.x >> 16, hh.y & 0xffffu, hh.y >> 16};
-                    // The slot's words are in registers: refill it at once with the unit kSlots ahead, so
-                    // that every slot but the one just read is in flight while this unit is decoded.  The
-                    // copy's address is made to depend on the loaded words, which holds the copy back
-                    // until the four shared-memory reads of the whole warp have completed.
-                    if (issued < n_units) issue(slot, settled(a0.w ^ a1.w ^ a2.w ^ hh.y));
-                    const uint4 *xc = xs + 12 * k;
 #pragma unroll
-                    for (int c = 0; c < 4; c++) {
+            for (int c = 0; c < 4; c++) {
 #ifdef LLVQ_STREAM_ONLY
-                        s += __uint_as_float((w0[c] ^ w1[c] ^ w2[c] ^ hd[c]) & 0x007fffffu);   // debug: bytes only, no decode
+                s += __uint_as_float((w0[c] ^ w1[c] ^ w2[c] ^ hd[c]) & 0x007fffffu);   // debug: bytes only, no decode
 #else
-                        const float2 kc = tq[hd[c] & 1023u];
-                        s = fmaf(kc.x, block_dot(w0[c], w1[c], w2[c], __float_as_uint(kc.y), xc + 3 * c), s);
+                const float2 kc = tq[hd[c]];           // header bits 10..15 are zero
+                s = fmaf(kc.x, block_dot(w0[c], w1[c], w2[c], __float_as_uint(kc.y), xc + 3 * c), s);
 #endif
-                    }
-                } else {
-                    // the nb mod 4 last block columns of the row group: rare, kept out of the unrolled path
-                    uint32_t guard = 0;
-                    const uint4 *xc = xs + 12 * p.tiles;
-#pragma unroll 1
-                    for (int c = 0; c < p.tail_cells; c++) {
-                        const unsigned char *cell = buf + c * kCellBytes;
-                        const uint32_t t0 = *reinterpret_cast<const uint32_t *>(cell + 4 * lane);
-                        const uint32_t t1 = *reinterpret_cast<const uint32_t *>(cell + 128 + 4 * lane);
-                        const uint32_t t2 = *reinterpret_cast<const uint32_t *>(cell + 256 + 4 * lane);
-                        const uint32_t th = *reinterpret_cast<const uint16_t *>(cell + 384 + 2 * lane);
-                        guard ^= t0 ^ t1 ^ t2 ^ th;
-                        const float2 kc = tq[th & 1023u];
-                        s = fmaf(kc.x, block_dot(t0, t1, t2, __float_as_uint(kc.y), xc + 3 * c), s);
-                    }
-                    if (issued < n_units) issue(slot, settled(guard));
-                }
             }
-            sum += __float2ll_rn(s * inv_q) + kUnitBias;
-            count++;
-            LLVQ_TRACE_UNIT(n, 2)
-            n++;
-            if (++k == p.units || n == n_units) {
-                if (n == n_units) { LLVQ_TRACE_POINT(6) }
-                deliver(p, p.prob[q], group, lane, sum, count, qexp);
-                sum = 0;
-                count = 0;
-                if (k == p.units) {
-                    k = 0;
-                    group++;
-                    if (group < p.total_groups) {
-                        q = find_problem(p, group);
-                        qexp = xexp + p.prob[q].qexp_base;
-                        inv_q = pow2f(-qexp);
-                        tq = tab + q * 1024;
-                    }
-                }
-            }
+            sum += __float2ll_rn(s * inv_q);
+            LLVQ_TRACE_UNIT(n + t, 2)
+            bar += 8;
+            buf += kTileBytes;
+            if (buf == buf_end) { buf -= kSlots * kTileBytes; bar -= 8 * kSlots; parity ^= 1u; }
         }
-        parity ^= 1u;
+        if (failed) break;
+        if (!NO_WEIGHTS && run_tiles < run) {
+            // the run ends with the nb mod 4 last block columns of the row group: one cell at a time
+            if (!mbar_wait(bar, parity)) { failed = true; break; }
+            uint32_t guard = 0;
+            const uint4 *xt = xs + 12 * tiles;
+            float s = 0.f;
+#pragma unroll 1
+            for (int c = 0; c < p.tail_cells; c++) {
+                const unsigned char *cell = buf + c * kCellBytes;
+                const uint32_t t0 = *reinterpret_cast<const uint32_t *>(cell + 4 * lane);
+                const uint32_t t1 = *reinterpret_cast<const uint32_t *>(cell + 128 + 4 * lane);
+                const uint32_t t2 = *reinterpret_cast<const uint32_t *>(cell + 256 + 4 * lane);
+                const uint32_t th = *reinterpret_cast<const uint16_t *>(cell + 384 + 2 * lane);
+                guard |= settled(t0, t1, t2) | settled(th, t0, t1);
+                const float2 kc = tq[th];
+                s = fmaf(kc.x, block_dot(t0, t1, t2, __float_as_uint(kc.y), xt + 3 * c), s);
+            }
+            if (issued < n_units) issue(bar, smem_addr(buf) + guard);
+            sum += __float2ll_rn(s * inv_q);
+            bar += 8;
+            buf += kTileBytes;
+            if (buf == buf_end) { buf -= kSlots * kTileBytes; bar -= 8 * kSlots; parity ^= 1u; }
+        }
+        // with no records read (the control launch) every unit contributes zero
+        n += run;
+        k += run;
+        if (n == n_units) { LLVQ_TRACE_POINT(6) }
+        deliver(p, pr, group, lane, sum, run, qexp);
+        if (k == units) {
+            k = 0;
+            group++;
+            if (group < p.total_groups) q = find_problem(p, group);
+        }
     }
 
     LLVQ_TRACE_POINT(5)
@@ -384,11 +400,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_onehot_kernel(const __grid_c
     for (int e = tid; e < 3 * p.nb; e += kThreads) {
         const uint4 v = __ldg(xg + e);
         xs4[e] = v;
-        m |= v.x | v.y | v.z | v.w;
+        m = max_abs_pair(max_abs_pair(max_abs_pair(max_abs_pair(m, v.x), v.y), v.z), v.w);
     }
     __syncthreads();
-    m = __reduce_or_sync(0xffffffffu, (m | (m >> 16)) & 0x7fffu);
-    if (lane == 0 && m) atomicOr(&xor_word, m);
+    m = __reduce_max_sync(0xffffffffu, max(m & 0xffffu, m >> 16));
+    if (lane == 0 && m) atomicMax(&xor_word, m);
     __syncthreads();
     const int xexp = max((int)(xor_word >> 10), 1) - 14;
 
@@ -415,7 +431,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_onehot_kernel(const __grid_c
             const float val[5] = {lv.x, lv.y, lv.z, lv.w, l4};
             s = fmaf(g, onehot_dot(v, val, xs + 24 * c), s);
         }
-        sum += __float2ll_rn(s * pow2f(-qexp)) + kUnitBias;
+        sum += __float2ll_rn(s * pow2f(-qexp));
         count++;
         if (++k == p.units || n + 1 == n_units) {
             deliver(p, pr, group, lane, sum, count, qexp);
