@@ -30,6 +30,10 @@ sys.path.insert(0, ROOT)
 from paper_2609_02652_b200 import datagen  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
+# DRAM bytes (read + write) per algorithmic byte of gemv_planes_kernel, from one ncu capture of the
+# 8192 x 8192 launch (profiles/gemv_planes_kernel_config4_8192x8192.txt: 39.354 MB against 39.289 MB);
+# traffic grows in proportion to the records streamed, so a launch's traffic is its bytes times this.
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 39.3536 / 39.2888
 METRIC = "us_per_lattice_gemv"
 
 
@@ -210,6 +214,20 @@ def time_arm(fn_step, ncopies, steps, warmup):
     return e0.elapsed_time(e1) / steps
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """A multi-rank time is the slowest rank's (all-reduce MAX); a single process returns its own."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def us_per_gemv_of_job(ms_per_step: float, n_gemv: int, world: int) -> float:
+    """Every rank runs its own replica of the step: the job finishes world * n_gemv GEMVs a step time."""
+    return ms_per_step * 1e3 / (n_gemv * world)
+
+
 def reference_arm(args, wl):
     """Times the CPU oracle as it stands: each step decodes and multiplies a bounded sample."""
     from oracle import oracle as O
@@ -337,14 +355,11 @@ def main():
     if dist:
         dist.barrier()
     clocks = sampler.result()
-    if dist:
-        t = torch.tensor([ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, device)
 
     ms_per_step = ms / args.steps
     n_gemv = len(mats)
-    us_per_gemv = ms_per_step * 1e3 / n_gemv / world          # the job ran `world` replicas of the step in that time
+    us_per_gemv = us_per_gemv_of_job(ms_per_step, n_gemv, world)
     gbps = step_bytes / (ms_per_step * 1e-3) / 1e9            # per GPU
     per_shape = None
 
@@ -431,7 +446,9 @@ def main():
                        "l2": f"records rotate through {ncopies} distinct copies ({ncopies * layout_bytes / 1e6:.0f} MB) so no launch finds its records in L2",
                        "multi_gpu": "replicas only: each rank runs the whole step on its own copy", "seed": wl.seed},
             "gbps": gbps, "hbm_frac": gbps / peak, "bytes_per_step": step_bytes,
-            "roofline": {"bound": "hbm", "achieved": gbps, "peak": peak, "unit": "GB/s", "frac": gbps / peak, "traffic": None,
+            "roofline": {"bound": "hbm", "achieved": gbps, "peak": peak, "unit": "GB/s", "frac": gbps / peak,
+                         "traffic": step_bytes / launches_per_step * NCU_TRAFFIC_PER_ALGORITHMIC_BYTE,
+                         "traffic_note": "DRAM bytes per launch (mean over the step's launches): ncu capture of the 8192x8192 launch scaled by bytes",
                          "kernel": "gemv_planes_kernel", "peak_source": peak_src,
                          "how": "algorithmic bytes of a step / CUDA-event time of the step, averaged over its launches"},
             "cpu_baseline": cpu_baseline,
