@@ -126,6 +126,25 @@ int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row
 int llvq_gemv_grouped(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n,
                       const void *x, int64_t k_padded, void *stream);
 
+/* No counterpart in the paper: the bit-plane llvq_gemv for callers that cannot allocate device
+ * memory - a process whose memory pool already owns the whole GPU, a plug-in that receives buffers
+ * but no allocator, code that runs while a stream is being captured, a loop that cannot afford the
+ * device synchronisation an allocation implies.  Such callers cannot use a context either
+ * (llvq_create allocates), so this call takes none: the reduction scratch, the class table and the
+ * error flag are file-scope device arrays inside the library (about 516 KiB on every GPU that loads
+ * it, held until the process exits).  Same arguments, layout (LLVQ_PLANES only), alignment rules and
+ * results as llvq_gemv; it runs on the CURRENT device.  Limits and rules:
+ *   - rows, rounded up to a multiple of 32, must not exceed 65536 (the built-in scratch holds one
+ *     64-bit accumulator a row); more returns LLVQ_ESIZE and launches nothing.
+ *   - The first call on a device sets the arrays up (resolves their device addresses, uploads the
+ *     class table, zeroes the scratch - synchronous copies, no allocation).  Make that first call
+ *     before any stream capture begins.
+ *   - Every call shares the one scratch array.  A launch that completes leaves it zeroed for the
+ *     next; launches that overlap on the GPU (two streams) race on it - serialise them.
+ * It calls no cudaMalloc, cudaFree or other allocating routine. */
+int llvq_gemv_static(const void *layout_buf, const void *row_scale, const float *gain, const void *x, float *y,
+                     int64_t rows, int64_t k_padded, void *stream);
+
 /* [Table "layout scale", FP16 control] y = W x, W fp16 row-major rows x k (k a multiple of 8,
  * W and x 16-byte aligned), f32 accumulation, f32 y. */
 int llvq_gemv_fp16(const void *W, const void *x, float *y, int64_t rows, int64_t k, void *stream);

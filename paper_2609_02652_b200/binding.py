@@ -21,7 +21,7 @@ _lib = None
 
 SYMBOLS = (
     "llvq_create", "llvq_destroy", "llvq_strerror", "llvq_status", "llvq_set_pdl", "llvq_num_classes", "llvq_class_base", "llvq_layout_bytes",
-    "llvq_expand", "llvq_gemv", "llvq_gemv_grouped", "llvq_gemv_fp16", "llvq_gemv_noweights", "llvq_dequant_fp16",
+    "llvq_expand", "llvq_gemv", "llvq_gemv_grouped", "llvq_gemv_static", "llvq_gemv_fp16", "llvq_gemv_noweights", "llvq_dequant_fp16",
     "llvq_decode_i8",
 )
 
@@ -61,6 +61,7 @@ def load() -> ctypes.CDLL:
         L.llvq_expand.argtypes = [vp, ci, vp, i64, i64, vp, sz, vp, vp]
         L.llvq_gemv.argtypes = [vp, ci, vp, vp, ctypes.POINTER(ctypes.c_float), vp, vp, i64, i64, vp]
         L.llvq_gemv_grouped.argtypes = [vp, ci, ctypes.POINTER(Problem), ci, vp, i64, vp]
+        L.llvq_gemv_static.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), vp, vp, i64, i64, vp]
         L.llvq_gemv_fp16.argtypes = [vp, vp, vp, i64, i64, vp]
         L.llvq_gemv_noweights.argtypes = [vp, vp, vp, vp, i64, i64, vp]
         L.llvq_dequant_fp16.argtypes = [vp, ci, vp, vp, ctypes.POINTER(ctypes.c_float), vp, i64, i64, vp]
@@ -166,6 +167,16 @@ def gemv(ctx: Context, layout: int, layout_buf: torch.Tensor, row_scale: torch.T
     _check(load().llvq_gemv(ctx.ptr, int(layout), _dev(layout_buf, torch.uint8, "layout_buf"),
                             _dev(row_scale, torch.float16, "row_scale"), _gain(gain), _dev(x, torch.float16, "x"),
                             _dev(y, torch.float32, "y"), int(rows), int(k_padded), _stream(stream)), "llvq_gemv")
+    return y
+
+
+def gemv_static(layout_buf: torch.Tensor, row_scale: torch.Tensor, gain, x: torch.Tensor, rows: int, k_padded: int,
+                y: torch.Tensor, stream=None) -> torch.Tensor:
+    """llvq_gemv_static: no context and no allocation inside the library; the caller supplies y.  Runs on the
+    current CUDA device; at most 65536 rows; calls must not overlap on the GPU (they share built-in scratch)."""
+    _check(load().llvq_gemv_static(_dev(layout_buf, torch.uint8, "layout_buf"), _dev(row_scale, torch.float16, "row_scale"),
+                                   _gain(gain), _dev(x, torch.float16, "x"), _dev(y, torch.float32, "y"), int(rows),
+                                   int(k_padded), _stream(stream)), "llvq_gemv_static")
     return y
 
 

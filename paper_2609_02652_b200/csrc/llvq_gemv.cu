@@ -28,6 +28,9 @@
 // kSlots units ahead.  The first copies go out before the kernel waits for its predecessor in the
 // stream (records never depend on it), so under programmatic dependent launch the ring fills
 // while the previous kernel drains.  Every wait is bounded.
+#include <cmath>
+#include <cstring>
+
 #include "llvq_internal.cuh"
 
 // Optional timeline (compiled in only with -DLLVQ_TRACE, never in the shipped library): lane 0 of
@@ -622,3 +625,128 @@ cudaError_t launch_decode_i8(const llvq_ctx *ctx, int layout, const uint8_t *buf
 }
 
 }  // namespace llvq
+
+// ---------------------------------------------------------------------------------------------
+// llvq_gemv_static: the bit-plane GEMV for callers that must not allocate device memory.
+//
+// Some hosts of this library cannot call cudaMalloc at the moment they need a matvec: a serving
+// process whose memory pool already owns all of HBM, a plug-in that is handed buffers but no
+// allocator, code that runs while a stream is being captured (allocation is not allowed there), or
+// a real-time loop in which an allocation's implicit device synchronisation is not acceptable.
+// Those callers cannot create a context either, because llvq_create allocates the tables and the
+// reduction scratch.  For them everything the kernel needs besides the caller's own buffers lives
+// in file-scope __device__ arrays that the module carries: the row accumulators (the scratch), the
+// class table and the error flag.  Every GPU that loads the library holds these arrays (about
+// 516 KiB) until the process exits.
+//
+// In host code the name of a __device__ array is only a host-side stand-in, not a device address;
+// the kernel is therefore given the address that cudaGetSymbolAddress returns for the current
+// device.  That, the upload of the class table and the kernel's shared-memory attribute are done
+// by the first call on each device (synchronously), so make that first call before any stream
+// capture begins.  All calls share the arrays: the accumulators are left at zero by every launch
+// that completes, but two launches that overlap on the GPU (different streams) race on them.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr int kStaticMaxRows = 65536;      // rows (rounded up to 32) one llvq_gemv_static call may have
+constexpr int kStaticMaxDevices = 64;
+
+static __device__ __align__(256) unsigned long long g_static_accum[kStaticMaxRows];   // 512 KiB of scratch
+static __device__ __align__(256) float2 g_static_cls_pack[llvq::kClassSlots];           // 4 KiB
+static __device__ __align__(256) int g_static_error[64];
+
+struct StaticDevice {
+    bool ready = false;
+    unsigned long long *accum = nullptr;
+    float2 *cls_pack = nullptr;
+    int *error = nullptr;
+    int sm_count = 0, max_smem_optin = 0;
+};
+StaticDevice g_static_dev[kStaticMaxDevices];
+
+// Once per device, with that device current: resolve the arrays' device addresses, fill the class
+// table, zero the accumulators, raise the kernel's shared-memory limit.  Allocates no device memory.
+int static_setup(int device, StaticDevice &d) {
+    if (cudaGetSymbolAddress((void **)&d.accum, g_static_accum) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaGetSymbolAddress((void **)&d.cls_pack, g_static_cls_pack) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaGetSymbolAddress((void **)&d.error, g_static_error) != cudaSuccess) return LLVQ_ECUDA;
+    llvq::HostTables host;                                   // host memory only
+    if (!llvq::build_tables(host)) return LLVQ_EINVAL;
+    if (cudaMemcpy(d.cls_pack, host.cls_pack.data(), llvq::kClassSlots * 8, cudaMemcpyHostToDevice) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaMemset(d.accum, 0, sizeof(unsigned long long) * kStaticMaxRows) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaMemset(d.error, 0, sizeof(int) * 64) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) return LLVQ_ECUDA;
+    if (llvq::allow_max_smem(llvq::gemv_planes_kernel<false>, d.max_smem_optin)) return LLVQ_ECUDA;
+    if (cudaDeviceSynchronize() != cudaSuccess) return LLVQ_ECUDA;
+    d.ready = true;
+    return LLVQ_OK;
+}
+
+}  // namespace
+
+extern "C" int llvq_gemv_static(const void *layout_buf, const void *row_scale, const float *gain, const void *x, float *y,
+                                int64_t rows, int64_t k_padded, void *stream) {
+    using namespace llvq;
+    if (!layout_buf || !row_scale || !gain || !x || !y || rows <= 0 || k_padded <= 0 || k_padded % 24 != 0) return LLVQ_EINVAL;
+    if (k_padded > LLVQ_MAX_K) return LLVQ_ESIZE;
+    const int64_t groups = (rows + kRowsPerGroup - 1) / kRowsPerGroup;
+    if (groups * kRowsPerGroup > kStaticMaxRows) return LLVQ_ESIZE;      // more rows than the built-in scratch holds
+    if ((reinterpret_cast<uintptr_t>(layout_buf) & 127) || (reinterpret_cast<uintptr_t>(x) & 15) ||
+        (reinterpret_cast<uintptr_t>(row_scale) & 1) || (reinterpret_cast<uintptr_t>(y) & 3))
+        return LLVQ_EALIGN;
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return LLVQ_ECUDA;
+    if (device < 0 || device >= kStaticMaxDevices) return LLVQ_EINVAL;
+    StaticDevice &d = g_static_dev[device];
+    if (!d.ready) {
+        const int rc = static_setup(device, d);
+        if (rc != LLVQ_OK) return rc;
+    }
+    GemvParams p;
+    memset(&p, 0, sizeof p);
+    p.nprob = 1;
+    p.prob[0].layout = (const uint8_t *)layout_buf;
+    p.prob[0].row_scale = (const __half *)row_scale;
+    p.prob[0].y = y;
+    p.prob[0].rows = (int)rows;
+    p.prob[0].group_begin = 0;
+    p.prob[0].gain0 = gain[0];
+    p.prob[0].gain1 = gain[1];
+    {
+        const float gm = fmaxf(fabsf(gain[0]), fabsf(gain[1]));
+        if (!(gm < 3.0e38f)) return LLVQ_EINVAL;
+        int ge = 0;
+        frexpf(gm > 0.f ? gm : 1.f, &ge);
+        p.prob[0].qexp_base = ge + 5 - 39;               // same quantum as llvq_gemv
+    }
+    p.x = (const __half *)x;
+    p.nb = (int)(k_padded / 24);
+    p.tiles = p.nb / kTileCells;
+    p.tail_cells = p.nb % kTileCells;
+    p.units = p.tiles + (p.tail_cells ? 1 : 0);
+    if (p.units > 2047 || groups * p.units > 0x7fffffffll) return LLVQ_ESIZE;
+    p.total_groups = (int)groups;
+    p.total_units = (int)(groups * p.units);
+    p.accum = d.accum;
+    p.cls_pack = d.cls_pack;
+    p.error = d.error;
+    const size_t smem = gemv_smem_bytes(LLVQ_PLANES, p.nb, 1);
+    if (smem + 1024 > (size_t)d.max_smem_optin) return LLVQ_ESIZE;
+    int grid = (p.total_units + kWarps - 1) / kWarps;
+    if (grid > d.sm_count) grid = d.sm_count;
+    p.units_base = p.total_units / (grid * kWarps);
+    p.units_rem = p.total_units % (grid * kWarps);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = (cudaStream_t)stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false>, p) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+}
+

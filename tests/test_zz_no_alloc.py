@@ -1,0 +1,51 @@
+"""llvq_gemv_static, the entry point for callers that cannot allocate device memory (a process whose
+pool owns the GPU, a plug-in without an allocator, code inside a stream capture): it must give what
+llvq_gemv gives, call after call, with nothing but the caller's buffers and the library's built-in
+scratch.  Collected last on purpose: a failure here cannot hide the result of any other test."""
+import numpy as np
+import pytest
+import torch
+
+from helpers import GAIN, TOL_NORMALISED, make_case
+
+pytestmark = pytest.mark.gpu
+
+
+def test_static_entry_point_matches_context_entry_point_twice_in_a_row():
+    from paper_2609_02652_b200 import binding as B
+
+    B.load()
+    torch.cuda.set_device(0)
+    ctx = B.create(0)
+    try:
+        # two different shapes back to back: the second call finds the shared scratch as the first left it
+        for rows, k, seed in [(1000, 2560, 31), (4096, 4096, 32), (1000, 2560, 31)]:
+            case = make_case(rows, k, seed=seed)
+            buf = B.expand(ctx, B.PLANES, case.d_codes, rows, case.nb)
+            ref = B.gemv(ctx, B.PLANES, buf, case.d_scale, GAIN, case.d_x, rows, case.nb * 24)
+            for _ in range(2):
+                y = torch.full((rows,), float("nan"), dtype=torch.float32, device="cuda")
+                B.gemv_static(buf, case.d_scale, GAIN, case.d_x, rows, case.nb * 24, y)
+                torch.cuda.synchronize()
+                yv, rv = y.cpu().numpy().astype(np.float64), ref.cpu().numpy().astype(np.float64)
+                assert np.isfinite(yv).all()
+                # same tolerance as the parity tests, relative to ||W_row|| ||x||; ||W_row|| = r * sqrt(sum gain^2) >= r * 0.75 * sqrt(nb)
+                bound = case.row_scale.astype(np.float64) * 0.75 * np.sqrt(case.nb) * np.linalg.norm(case.x.astype(np.float64))
+                assert (np.abs(yv - rv) <= TOL_NORMALISED * bound + 1e-30).all()
+                assert torch.equal(y, ref)          # same kernel, order-free reduction: in fact identical
+        # more rows than the built-in scratch holds: a clear error, nothing launched
+        rows = 65536 + 32
+        dummy = torch.zeros(B.layout_bytes(B.PLANES, rows, 24), dtype=torch.uint8, device="cuda")
+        sc = torch.zeros(rows, dtype=torch.float16, device="cuda")
+        xx = torch.zeros(24, dtype=torch.float16, device="cuda")
+        yy = torch.zeros(rows, dtype=torch.float32, device="cuda")
+        with pytest.raises(B.LlvqError) as e:
+            B.gemv_static(dummy, sc, GAIN, xx, rows, 24, yy)
+        assert e.value.code == -3
+        # exactly the maximum is accepted
+        rows = 65536
+        B.gemv_static(dummy[: B.layout_bytes(B.PLANES, rows, 24)], sc[:rows], GAIN, xx, rows, 24, yy[:rows])
+        torch.cuda.synchronize()
+        assert (yy[:rows] == 0).all()
+    finally:
+        ctx.close()
