@@ -131,7 +131,11 @@ def make_copies(B, ctx, mats, layout, ncopies, device, grouped=True):
                 keys.append(k)
         for k in keys:
             members = [e for e in mats if (e["key"] if grouped else ("solo", e["m"].tensor_id)) == k]
-            x = members[0]["x"].to(device)
+            # x is the previous operator's output in a decoder: small and cache-resident.  One buffer a
+            # launch, shared by every copy of the records; only the records (and scales) rotate.
+            if ("x", k) not in first:
+                first[("x", k)] = members[0]["x"].to(device)
+            x = first[("x", k)]
             bufs = [first[e["m"].tensor_id] if c == 0 else first[e["m"].tensor_id].clone() for e in members]
             scales = [e["scale"].to(device) for e in members]
             ys = [torch.zeros(e["m"].rows, dtype=torch.float32, device=device) for e in members]
@@ -147,10 +151,11 @@ def run_step(B, ctx, layout, cp):
         B.gemv_grouped(ctx, layout, ln["problems"], ln["x"], ln["k_padded"])
 
 
-def verify(oracle, copies, threads):
-    """Every row of copy 0 against the f64 oracle. Returns (worst normalised error, oracle seconds, blocks)."""
-    worst, secs, blocks = 0.0, 0.0, 0
-    for ln in copies[0].launches:
+def verify(oracle, copies, threads, max_launches=None):
+    """Every row of copy 0 (of its first max_launches launches) against the f64 oracle.
+    Returns (worst normalised error, oracle seconds, blocks, GEMVs checked)."""
+    worst, secs, blocks, gemvs = 0.0, 0.0, 0, 0
+    for ln in copies[0].launches[:max_launches]:
         xh = ln["x"].cpu().numpy()
         for e, y in zip(ln["members"], ln["ys"]):
             m = e["m"]
@@ -166,7 +171,8 @@ def verify(oracle, copies, threads):
             if not (np.isfinite(yv).all() and ratio.max() <= 1e-4 and (yv[denom == 0] == 0).all()):
                 raise SystemExit(f"parity failure on {m.name}: normalised error {ratio.max():.3e}")
             worst = max(worst, float(ratio.max()))
-    return worst, secs, blocks
+            gemvs += 1
+    return worst, secs, blocks, gemvs
 
 
 def capture_graphs(B, ctx, layout, copies, total_steps, first_step=0, chunk=512):
@@ -272,6 +278,7 @@ def main():
     ap.add_argument("--no-arms", action="store_true", help="skip the one-hot / FP16 / no-weights comparison arms")
     ap.add_argument("--no-verify", action="store_true", help="skip the oracle check (profiling runs only)")
     ap.add_argument("--lean", action="store_true", help="profiling runs: no clock ramp, no end-to-end leg, no arms, no oracle check")
+    ap.add_argument("--no-pdl", action="store_true", help="launch the GEMV without programmatic dependent launch")
     ap.add_argument("--ungrouped", action="store_true", help="one launch a matrix instead of row-concatenated groups")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -301,6 +308,8 @@ def main():
 
     build.build()
     ctx = B.create(local)
+    if args.no_pdl:
+        B.set_pdl(ctx, False)
     peak, peak_src = measured_peaks()
 
     mats = build_inputs(wl, device)
@@ -330,10 +339,12 @@ def main():
     if not args.no_verify:
         from oracle import oracle as O
 
-        worst, osecs, oblocks = verify(O, copies, cores)
+        # the multi-layer stacks are checked (and the oracle timed) on their first layer; tests/ cover more layers
+        first_layer = 4 if len(mats) > 7 and not args.ungrouped else (7 if len(mats) > 7 else None)
+        worst, osecs, oblocks, ogemvs = verify(O, copies, cores, first_layer)
         if rank == 0:
-            cpu_baseline = {"value": osecs / len(mats) * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
-                            "sample": f"the whole step once ({oblocks} blocks, {len(mats)} GEMVs): index decode + f64 matvec",
+            cpu_baseline = {"value": osecs / ogemvs * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
+                            "sample": f"{ogemvs} GEMVs of the step once ({oblocks} of {wl.blocks} blocks): index decode + f64 matvec",
                             "blocks_per_s": oblocks / osecs}
 
     # warm-up: ramp the clocks, then W untimed steps, then exactly K timed steps
@@ -387,6 +398,8 @@ def main():
     e2e_us = (time.perf_counter() - t1) / e2e_steps * 1e6 / n_gemv / world
 
     arms = {}
+    if len(mats) > 7:
+        args.no_arms = True          # the comparison arms and per-shape timings are taken on the single-layer workloads
     if not args.no_arms and rank == 0:
         arm_steps = min(args.steps, 200)
         # per-matrix timings of the bit-plane kernel, one launch each
@@ -412,7 +425,7 @@ def main():
         torch.cuda.synchronize()
         if not args.no_verify:
             from oracle import oracle as O
-            verify(O, oh_copies, cores)
+            verify(O, oh_copies, cores, 4 if len(mats) > 7 and not args.ungrouped else None)
         t = time_arm(lambda i: run_step(B, ctx, B.ONEHOT, oh_copies[i % len(oh_copies)]), len(oh_copies), arm_steps, 3)
         ob = sum(gemv_bytes(e["m"].rows, e["m"].nb, 20) for e in mats)
         arms["onehot"] = {"us_per_gemv": t * 1e3 / n_gemv, "gbps": ob / (t * 1e-3) / 1e9, "frac": ob / (t * 1e-3) / 1e9 / peak, "bytes_per_block": 20}
@@ -443,7 +456,7 @@ def main():
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": f"config {wl.config}: {wl.name}", "gemvs_per_step": n_gemv, "launches_per_step": launches_per_step,
                        "layout": "bit planes, 14 B per 24 weights (4.67 b/w payload; the paper's 4.80 b/w label counts its f32 tail and scales)",
-                       "l2": f"records rotate through {ncopies} distinct copies ({ncopies * layout_bytes / 1e6:.0f} MB) so no launch finds its records in L2",
+                       "l2": f"records and scales rotate through {ncopies} distinct copies ({ncopies * layout_bytes / 1e6:.0f} MB) so no launch finds its records in L2; x (a few KB a launch) is one buffer, as in a decoder where it is the previous operator's output",
                        "multi_gpu": "replicas only: each rank runs the whole step on its own copy", "seed": wl.seed},
             "gbps": gbps, "hbm_frac": gbps / peak, "bytes_per_step": step_bytes,
             "roofline": {"bound": "hbm", "achieved": gbps, "peak": peak, "unit": "GB/s", "frac": gbps / peak,

@@ -151,7 +151,7 @@ __device__ __forceinline__ void warp_range(const GemvParams &p, int warp, int &u
 
 // Hands the warp's sum over `count` units of row group `group` to the row accumulators.
 __device__ __forceinline__ void deliver(const GemvParams &p, const GemvProblemDev &pr, int group, int lane,
-                                        long long sum, int count, int qexp) {
+                                        long long sum, int count, int qexp, float row_scale) {
     const int row = (group - pr.group_begin) * kRowsPerGroup + lane;
     if (row >= pr.rows) return;                      // padding rows of the last row group
     const unsigned long long addend = (unsigned long long)(sum + (long long)count * kUnitBias) + ((unsigned long long)count << kCountShift);
@@ -159,7 +159,7 @@ __device__ __forceinline__ void deliver(const GemvParams &p, const GemvProblemDe
     const unsigned long long old = atomicAdd(slot, addend);
     if ((int)(old >> kCountShift) + count == p.units) {
         const long long total = (long long)((old + addend) & kSumMask) - (long long)p.units * kUnitBias;
-        pr.y[row] = ((float)total * pow2f(qexp)) * __half2float(pr.row_scale[row]);
+        pr.y[row] = ((float)total * pow2f(qexp)) * row_scale;
         *slot = 0ull;                                // ready for the next launch on this context
     }
 }
@@ -169,13 +169,6 @@ __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -217,13 +210,12 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t my_ring = smem_addr(ring + warp * kSlots * kTileBytes);
     const uint32_t my_bar = smem_addr(bars + warp * kSlots);
-    const uint32_t pro_bar = smem_addr(bars + kWarps * kSlots);
 
     LLVQ_TRACE_POINT(0)
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kSlots; s++) mbar_init(my_bar + 8 * s, 1);
-        if (warp == 0) { mbar_init(pro_bar, 1); *xor_word = 0; }
+        if (warp == 0) *xor_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -273,24 +265,30 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     // let the next kernel in the stream start its own prefetch, then wait for the previous one:
     // x, y and the reduction scratch may still be in use by it
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // warm the L2 lines and the address translation of x while waiting; the values are read only
+    // after the wait, through L2, which is where the previous kernel's writes to x land
+    for (int e = tid * 128; e < p.nb * 48; e += kThreads * 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(p.x) + e));
     LLVQ_TRACE_POINT(1)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     LLVQ_TRACE_POINT(2)
-    if (tid == 0) {
-        mbar_expect(pro_bar, p.nb * 48);
-        bulk_g2s(smem_addr(xs), p.x, p.nb * 48, pro_bar);
-    }
-    bool failed = !mbar_wait(pro_bar, 0);
-    // every |x| is below 2^(e-14), e the biased exponent of the largest magnitude (fp16 bit patterns
-    // of non-negative values order like integers)
+    // x into shared memory, every thread a 16-byte piece (L2 hits after the prefetch), and on the way
+    // the largest |x|: every |x| is below 2^(e-14), e the biased exponent of the largest magnitude
+    // (fp16 bit patterns of non-negative values order like integers)
+    bool failed = false;
     int xexp;
     {
         uint32_t m = 0;
-        const uint32_t *xw = reinterpret_cast<const uint32_t *>(xs);
-        for (int e = tid; e < p.nb * 12; e += kThreads) m = max_abs_pair(m, xw[e]);
+        const uint4 *xg = reinterpret_cast<const uint4 *>(p.x);
+        uint4 *xw = const_cast<uint4 *>(xs);
+        for (int e = tid; e < p.nb * 3; e += kThreads) {
+            const uint4 v = __ldcg(xg + e);
+            xw[e] = v;
+            m = max_abs_pair(max_abs_pair(max_abs_pair(max_abs_pair(m, v.x), v.y), v.z), v.w);
+        }
         m = __reduce_max_sync(0xffffffffu, max(m & 0xffffu, m >> 16));
         if (lane == 0 && m) atomicMax(xor_word, m);
-        __syncthreads();                               // also publishes the block constants
+        __syncthreads();                               // publishes x, the maximum and the block constants
         xexp = max((int)(*xor_word >> 10), 1) - 14;
     }
     LLVQ_TRACE_POINT(3)
@@ -311,6 +309,10 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         const float2 *tq = tab + q * 1024;
         const int run = min(units - k, n_units - n);
         const int run_tiles = NO_WEIGHTS ? 0 : max(0, min(run, tiles - k));
+        // the row's scale is needed only by the arrival that finishes the row, but loading it now
+        // keeps a cold read off the tail of the kernel
+        const int row = (group - pr.group_begin) * kRowsPerGroup + lane;
+        const float row_scale = row < pr.rows ? __half2float(pr.row_scale[row]) : 0.f;
         const uint4 *xc = xs + 12 * k;
         long long sum = 0;
 
@@ -373,7 +375,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         n += run;
         k += run;
         if (n == n_units) { LLVQ_TRACE_POINT(6) }
-        deliver(p, pr, group, lane, sum, run, qexp);
+        deliver(p, pr, group, lane, sum, run, qexp, row_scale);
         if (k == units) {
             k = 0;
             group++;
@@ -437,7 +439,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_onehot_kernel(const __grid_c
         sum += __float2ll_rn(s * pow2f(-qexp));
         count++;
         if (++k == p.units || n + 1 == n_units) {
-            deliver(p, pr, group, lane, sum, count, qexp);
+            const int row = (group - pr.group_begin) * kRowsPerGroup + lane;
+            deliver(p, pr, group, lane, sum, count, qexp, row < pr.rows ? __half2float(pr.row_scale[row]) : 0.f);
             sum = 0;
             count = 0;
             if (k == p.units) {
