@@ -64,7 +64,7 @@ namespace {
 #define LLVQ_SLOTS 3
 #endif
 #ifndef LLVQ_MINB
-#define LLVQ_MINB 2
+#define LLVQ_MINB 1
 #endif
 constexpr int kWarps = LLVQ_WARPS;         // warps per CTA
 constexpr int kThreads = kWarps * 32;
@@ -88,7 +88,7 @@ __device__ __forceinline__ void fma_pair(float &lo, float &hi, uint32_t w, uint3
 
 // sum over the 24 coordinates of one block of (+-|x_i| * 2^-21) * x[i]
 __device__ __forceinline__ float block_dot(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t parity, const uint4 *xs) {
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    float a0 = 0.f, a1 = 0.f;
     const uint32_t w[3] = {w0, w1, w2};
 #pragma unroll
     for (int j = 0; j < 3; j++) {
@@ -98,10 +98,10 @@ __device__ __forceinline__ float block_dot(uint32_t w0, uint32_t w1, uint32_t w2
         for (int k = 0; k < 4; k++) {
             const uint32_t r = k ? __funnelshift_r(w[j], w[j], 4 * k) : w[j];
             const uint32_t v = (r & kPairMask) | parity;
-            if (k & 1) fma_pair(a2, a3, v, xp[k]); else fma_pair(a0, a1, v, xp[k]);
+            fma_pair(a0, a1, v, xp[k]);              // two chains of twelve: measured faster than four of six
         }
     }
-    return (a0 + a1) + (a2 + a3);
+    return a0 + a1;
 }
 
 // one-hot record: value = class table entry of the rank level, selected without indexing
