@@ -212,13 +212,24 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     const uint32_t my_bar = smem_addr(bars + warp * kSlots);
 
     LLVQ_TRACE_POINT(0)
+    // first the loads whose latency the rest of the prologue can cover: the class constants this
+    // thread will turn into block constants, and x on its way into L2 (its values are read only after
+    // the wait below, through L2, which is where the previous kernel's writes to x land)
+    const int tab_entries = p.nprob * 1024;
+    float2 cv[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+    for (int i = 0; i < 2; i++)
+        if (tid + i * kThreads < tab_entries) cv[i] = __ldg(p.cls_pack + ((tid + i * kThreads) & 511));
+    for (int e = tid * 128; e < p.nb * 48; e += kThreads * 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(p.x) + e));
+    // a warp's barriers are used by that warp alone: no block-wide synchronisation is needed for them
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kSlots; s++) mbar_init(my_bar + 8 * s, 1);
         if (warp == 0) *xor_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    __syncthreads();
+    __syncwarp();
 
     int u0, n_units;
     warp_range(p, warp, u0, n_units);
@@ -257,18 +268,14 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             if (issued < n_units) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
     }
     // block constants of every matrix of the launch: (class | gain << 9) -> {gain * 2^21 / (4 sqrt m), parity pattern}
-    for (int e = tid; e < p.nprob * 1024; e += kThreads) {
-        const float2 v = __ldg(p.cls_pack + (e & 511));
+    for (int e = tid, i = 0; e < tab_entries; e += kThreads, i++) {
+        const float2 v = i < 2 ? cv[i] : __ldg(p.cls_pack + (e & 511));
         const GemvProblemDev &pe = p.prob[e >> 10];
         tab[e] = make_float2(v.x * ((e & 512) ? pe.gain1 : pe.gain0), v.y);
     }
     // let the next kernel in the stream start its own prefetch, then wait for the previous one:
     // x, y and the reduction scratch may still be in use by it
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    // warm the L2 lines and the address translation of x while waiting; the values are read only
-    // after the wait, through L2, which is where the previous kernel's writes to x land
-    for (int e = tid * 128; e < p.nb * 48; e += kThreads * 128)
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(p.x) + e));
     LLVQ_TRACE_POINT(1)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     LLVQ_TRACE_POINT(2)
