@@ -85,10 +85,20 @@ __device__ __forceinline__ void fma_pair(float &lo, float &hi, uint32_t w, uint3
         : "+f"(lo), "+f"(hi)
         : "r"(w), "r"(x));
 }
+// the same with a zero addend: starts the two chains without clearing registers first
+__device__ __forceinline__ void mul_pair(float &lo, float &hi, uint32_t w, uint32_t x) {
+    asm("{\n\t.reg .f16 wl, wh, xl, xh;\n\t"
+        "mov.b32 {wl, wh}, %2;\n\t"
+        "mov.b32 {xl, xh}, %3;\n\t"
+        "fma.rn.f32.f16 %0, wl, xl, 0f00000000;\n\t"
+        "fma.rn.f32.f16 %1, wh, xh, 0f00000000;\n\t}"
+        : "=f"(lo), "=f"(hi)
+        : "r"(w), "r"(x));
+}
 
 // sum over the 24 coordinates of one block of (+-|x_i| * 2^-21) * x[i]
 __device__ __forceinline__ float block_dot(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t parity, const uint4 *xs) {
-    float a0 = 0.f, a1 = 0.f;
+    float a0, a1;
     const uint32_t w[3] = {w0, w1, w2};
 #pragma unroll
     for (int j = 0; j < 3; j++) {
@@ -98,7 +108,8 @@ __device__ __forceinline__ float block_dot(uint32_t w0, uint32_t w1, uint32_t w2
         for (int k = 0; k < 4; k++) {
             const uint32_t r = k ? __funnelshift_r(w[j], w[j], 4 * k) : w[j];
             const uint32_t v = (r & kPairMask) | parity;
-            fma_pair(a0, a1, v, xp[k]);              // two chains of twelve: measured faster than four of six
+            // two chains of twelve (measured faster than four of six)
+            if (j == 0 && k == 0) mul_pair(a0, a1, v, xp[k]); else fma_pair(a0, a1, v, xp[k]);
         }
     }
     return a0 + a1;
@@ -182,6 +193,29 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
     for (int i = 0; i < kSpinLimit; i++)
         if (mbar_try(bar, parity)) return true;
     return false;
+}
+
+// Ring reads through 32-bit shared-memory addresses.  Volatile: they must stay behind the wait on the
+// slot's barrier and ahead of the copy that refills the slot.
+__device__ __forceinline__ uint4 lds128(uint32_t a) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
 }
 
 // Returns zero, but only once its operands are available: an address that adds this zero cannot be
@@ -303,8 +337,9 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     int n = 0;
     uint32_t parity = 0;                               // every slot completes once a round of kSlots units
     uint32_t bar = my_bar;                             // barrier and buffer of the slot that is consumed next
-    const unsigned char *buf = ring + warp * kSlots * kTileBytes;
-    const unsigned char *const buf_end = buf + kSlots * kTileBytes;
+    uint32_t sbuf = my_ring;
+    const uint32_t sbuf_end = my_ring + kSlots * kTileBytes;
+    const uint32_t lane16 = 16 * lane, lane8 = 8 * lane;
     const int tiles = p.tiles, units = p.units;
 
     // A run is the stretch of units of one row group inside this warp's range: its units are summed
@@ -327,17 +362,17 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             LLVQ_TRACE_UNIT(n + t, 0)
             if (!mbar_wait(bar, parity)) { failed = true; break; }
             LLVQ_TRACE_UNIT(n + t, 1)
-            const uint4 a0 = *reinterpret_cast<const uint4 *>(buf + 16 * lane);
-            const uint4 a1 = *reinterpret_cast<const uint4 *>(buf + 512 + 16 * lane);
-            const uint4 a2 = *reinterpret_cast<const uint4 *>(buf + 1024 + 16 * lane);
-            const uint2 hh = *reinterpret_cast<const uint2 *>(buf + 1536 + 8 * lane);
+            const uint4 a0 = lds128(sbuf + lane16);
+            const uint4 a1 = lds128(sbuf + lane16 + 512);
+            const uint4 a2 = lds128(sbuf + lane16 + 1024);
+            const uint2 hh = lds64(sbuf + lane8 + 1536);
             const uint32_t w0[4] = {a0.x, a0.y, a0.z, a0.w}, w1[4] = {a1.x, a1.y, a1.z, a1.w}, w2[4] = {a2.x, a2.y, a2.z, a2.w};
             const uint32_t hd[4] = {hh.x & 0xffffu, hh.x >> 16, hh.y & 0xffffu, hh.y >> 16};
             // The slot's words are in registers: refill it at once with the unit kSlots ahead, so
             // that every slot but the one just read is in flight while this unit is decoded.  The
             // copy's address is made to depend on the loaded words, which holds the copy back
             // until the four shared-memory reads of the whole warp have completed.
-            if (issued < n_units) issue(bar, smem_addr(buf) + (settled(a0.w, a1.w, a2.w) | settled(hh.y, hh.x, a0.x)));
+            if (issued < n_units) issue(bar, sbuf + (settled(a0.w, a1.w, a2.w) | settled(hh.y, hh.x, a0.x)));
             float s = 0.f;
 #pragma unroll
             for (int c = 0; c < 4; c++) {
@@ -351,8 +386,11 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             sum += __float2ll_rn(s * inv_q);
             LLVQ_TRACE_UNIT(n + t, 2)
             bar += 8;
-            buf += kTileBytes;
-            if (buf == buf_end) { buf -= kSlots * kTileBytes; bar -= 8 * kSlots; parity ^= 1u; }
+            sbuf += kTileBytes;
+            const bool wrap = sbuf == sbuf_end;        // every slot completes once a round
+            sbuf = wrap ? my_ring : sbuf;
+            bar = wrap ? my_bar : bar;
+            parity ^= wrap ? 1u : 0u;
         }
         if (failed) break;
         if (!NO_WEIGHTS && run_tiles < run) {
@@ -363,20 +401,20 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             float s = 0.f;
 #pragma unroll 1
             for (int c = 0; c < p.tail_cells; c++) {
-                const unsigned char *cell = buf + c * kCellBytes;
-                const uint32_t t0 = *reinterpret_cast<const uint32_t *>(cell + 4 * lane);
-                const uint32_t t1 = *reinterpret_cast<const uint32_t *>(cell + 128 + 4 * lane);
-                const uint32_t t2 = *reinterpret_cast<const uint32_t *>(cell + 256 + 4 * lane);
-                const uint32_t th = *reinterpret_cast<const uint16_t *>(cell + 384 + 2 * lane);
+                const uint32_t cell = sbuf + c * kCellBytes;
+                const uint32_t t0 = lds32(cell + 4 * lane);
+                const uint32_t t1 = lds32(cell + 128 + 4 * lane);
+                const uint32_t t2 = lds32(cell + 256 + 4 * lane);
+                const uint32_t th = lds16(cell + 384 + 2 * lane);
                 guard |= settled(t0, t1, t2) | settled(th, t0, t1);
                 const float2 kc = tq[th];
                 s = fmaf(kc.x, block_dot(t0, t1, t2, __float_as_uint(kc.y), xt + 3 * c), s);
             }
-            if (issued < n_units) issue(bar, smem_addr(buf) + guard);
+            if (issued < n_units) issue(bar, sbuf + guard);
             sum += __float2ll_rn(s * inv_q);
             bar += 8;
-            buf += kTileBytes;
-            if (buf == buf_end) { buf -= kSlots * kTileBytes; bar -= 8 * kSlots; parity ^= 1u; }
+            sbuf += kTileBytes;
+            if (sbuf == sbuf_end) { sbuf = my_ring; bar = my_bar; parity ^= 1u; }
         }
         // with no records read (the control launch) every unit contributes zero
         n += run;
