@@ -48,7 +48,7 @@ def measured_peaks():
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML (read-only) while a region runs."""
 
-    def __init__(self, index: int, period: float = 0.005):
+    def __init__(self, index: int, period: float = 0.001):
         super().__init__(daemon=True)
         self.samples, self.reasons, self.stop_flag, self.max_mhz = [], set(), threading.Event(), None
         self.period, self.index, self.ok = period, index, False
