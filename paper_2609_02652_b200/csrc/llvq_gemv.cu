@@ -240,7 +240,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     float2 *tab = reinterpret_cast<float2 *>(smem + kWarps * kSlots * kTileBytes);
     const uint4 *xs = reinterpret_cast<const uint4 *>(smem + kWarps * kSlots * kTileBytes + p.nprob * 8192);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kWarps * kSlots * kTileBytes + p.nprob * 8192 + ((p.nb * 48 + 127) / 128) * 128);
-    uint32_t *xor_word = reinterpret_cast<uint32_t *>(bars + kWarps * kSlots + 1);
+    uint32_t *warp_max = reinterpret_cast<uint32_t *>(bars + kWarps * kSlots);     // one slot a warp
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t my_ring = smem_addr(ring + warp * kSlots * kTileBytes);
     const uint32_t my_bar = smem_addr(bars + warp * kSlots);
@@ -260,7 +260,6 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kSlots; s++) mbar_init(my_bar + 8 * s, 1);
-        if (warp == 0) *xor_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
@@ -327,10 +326,12 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             xw[e] = v;
             m = max_abs_pair(max_abs_pair(max_abs_pair(max_abs_pair(m, v.x), v.y), v.z), v.w);
         }
+        LLVQ_TRACE_POINT(4)
         m = __reduce_max_sync(0xffffffffu, max(m & 0xffffu, m >> 16));
-        if (lane == 0 && m) atomicMax(xor_word, m);
-        __syncthreads();                               // publishes x, the maximum and the block constants
-        xexp = max((int)(*xor_word >> 10), 1) - 14;
+        if (lane == 0) warp_max[warp] = m;             // plain stores: atomics on one word would serialise the warps
+        __syncthreads();                               // publishes x, the maxima and the block constants
+        m = warp_max[lane < kWarps ? lane : 0];
+        xexp = max((int)(__reduce_max_sync(0xffffffffu, m) >> 10), 1) - 14;
     }
     LLVQ_TRACE_POINT(3)
 
@@ -606,14 +607,17 @@ __global__ void __launch_bounds__(256) dequant_kernel(int layout, const uint8_t 
 size_t gemv_smem_bytes(int layout, int nb, int nprob) {
     const size_t xbytes = ((size_t)nb * 48 + 127) / 128 * 128;
     if (layout != LLVQ_PLANES) return xbytes;
-    return (size_t)kWarps * kSlots * kTileBytes + (size_t)nprob * 8192 + xbytes + (kWarps * kSlots + 2) * 8;
+    return (size_t)kWarps * kSlots * kTileBytes + (size_t)nprob * 8192 + xbytes + kWarps * kSlots * 8 + kWarps * 4 + 16;
 }
 
 template <typename K>
 static int allow_max_smem(K kernel, int optin) {
     cudaFuncAttributes a;
     if (cudaFuncGetAttributes(&a, kernel) != cudaSuccess) return -1;
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - (int)a.sharedSizeBytes) == cudaSuccess ? 0 : -1;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin - (int)a.sharedSizeBytes) != cudaSuccess) return -1;
+    // ask for the largest shared-memory carve-out, so that a CTA of the next kernel of the stream can
+    // settle beside a running one (programmatic dependent launch) whenever two of them fit
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) == cudaSuccess ? 0 : -1;
 }
 
 int gemv_configure(const llvq_ctx *ctx) {
