@@ -14,6 +14,21 @@ N13_PAPER = 280_974_212_784_720         # Sec. 2.4, "Invariant locks upstream"
 KISSING = 196_560                       # Sec. 2.4
 
 
+def _golden(name):
+    import os
+
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", name)
+
+
+def paper_constants():
+    out = {}
+    for line in open(_golden("paper_constants.txt")):
+        if line.strip() and not line.startswith("#"):
+            name, value, _cite = line.rstrip("\n").split("\t")
+            out[name] = int(value)
+    return out
+
+
 # ---------------------------------------------------------------- independent ingredients
 def golay_set():
     """All multiples of g(x) = x^11+x^10+x^6+x^5+x^4+x^2+1 of degree < 23, plus a parity bit."""
@@ -99,6 +114,42 @@ def test_class_count_and_totals(oracle):
         base += i["size"]
     keys = [(i["shell"], i["odd"], i["w"], tuple(i["mags"])) for i in infos]
     assert keys == sorted(keys) and len(set(keys)) == 301
+
+
+def test_against_the_values_the_paper_prints(oracle):
+    c = paper_constants()
+    assert oracle.total_points() == c["ball_points"] == N_PAPER
+    assert math.ceil(math.log2(c["ball_points"])) == c["index_bits"]
+    assert oracle.num_classes() == c["classes"]
+    infos = [oracle.class_info(k) for k in range(oracle.num_classes())]
+    assert len({i["shell"] for i in infos}) == c["shells"]
+    assert oracle.shell_count(2) == c["kissing_number"] == KISSING
+    assert max(i["ndist"] for i in infos) == c["max_levels_per_class"]
+    assert 9 + 1 + 24 + 3 * 24 == c["planes_payload_bits"] and c["planes_payload_bits"] <= 8 * c["planes_record_bytes"]
+    assert oracle.planes_bytes(32, 1) == 32 * c["planes_record_bytes"]
+    assert oracle.num_classes() <= c["class_table_slots"] and oracle.SENTINEL_CLASS < c["class_table_slots"]
+    try:
+        oracle.init_shells(13)
+        assert oracle.total_points() == c["points_through_shell_13"] == N13_PAPER
+    finally:
+        oracle.init_shells(12)
+
+
+def test_stored_index_examples_still_decode_the_same(oracle):
+    """Regression pin of the index order (the reading of Sec. 2.1): examples written by the oracle itself,
+    each also a lattice point of its class's shell and a fixed point of encode."""
+    n = 0
+    for line in open(_golden("index_examples.txt")):
+        if line.startswith("#"):
+            continue
+        idx, cls, coords = line.rstrip("\n").split("\t")
+        x = np.array([int(v) for v in coords.split()], dtype=np.int8)
+        c, got = oracle.decode(int(idx))
+        assert c == int(cls) and got.tolist() == x.tolist()
+        assert is_leech_point(x) and oracle.encode(x) == int(idx)
+        assert int((x.astype(int) ** 2).sum()) == 16 * oracle.class_info(c)["shell"]
+        n += 1
+    assert n >= 16
 
 
 def test_count_through_shell_13(oracle):
