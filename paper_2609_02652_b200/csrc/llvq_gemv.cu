@@ -49,9 +49,14 @@
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                                    \
         p.trace[(((size_t)p.trace_launch * gridDim.x + blockIdx.x) * kWarps + warp) * 128 + 8 + 3 * (n) + (i)] = t_; \
     }
+// SM cycle counter into slots 120..127
+#define LLVQ_TRACE_CLOCK(i)                                                                                       \
+    if (p.trace && lane == 0)                                                                                     \
+        p.trace[(((size_t)p.trace_launch * gridDim.x + blockIdx.x) * kWarps + warp) * 128 + 120 + (i)] = clock64();
 #else
 #define LLVQ_TRACE_POINT(i)
 #define LLVQ_TRACE_UNIT(n, i)
+#define LLVQ_TRACE_CLOCK(i)
 #endif
 
 namespace llvq {
@@ -254,8 +259,12 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
 #pragma unroll
     for (int i = 0; i < 2; i++)
         if (tid + i * kThreads < tab_entries) cv[i] = __ldg(p.cls_pack + ((tid + i * kThreads) & 511));
-    for (int e = tid * 128; e < p.nb * 48; e += kThreads * 128)
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char *>(p.x) + e));
+    for (int e = tid * 128; e < p.nb * 48; e += kThreads * 128) {
+        // a load whose value is thrown away: it brings the line into L2 and the translation into this
+        // multiprocessor's TLB, which a prefetch hint does not promise
+        uint32_t ignored;
+        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(ignored) : "l"(reinterpret_cast<const char *>(p.x) + e));
+    }
     // a warp's barriers are used by that warp alone: no block-wide synchronisation is needed for them
     if (lane == 0) {
 #pragma unroll
@@ -312,6 +321,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     LLVQ_TRACE_POINT(1)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     LLVQ_TRACE_POINT(2)
+    LLVQ_TRACE_CLOCK(0)
     // x into shared memory, every thread a 16-byte piece (L2 hits after the prefetch), and on the way
     // the largest |x|: every |x| is below 2^(e-14), e the biased exponent of the largest magnitude
     // (fp16 bit patterns of non-negative values order like integers)
@@ -321,12 +331,24 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         uint32_t m = 0;
         const uint4 *xg = reinterpret_cast<const uint4 *>(p.x);
         uint4 *xw = const_cast<uint4 *>(xs);
-        for (int e = tid; e < p.nb * 3; e += kThreads) {
-            const uint4 v = __ldcg(xg + e);
-            xw[e] = v;
-            m = max_abs_pair(max_abs_pair(max_abs_pair(max_abs_pair(m, v.x), v.y), v.z), v.w);
+        // all of a thread's loads go out before the first store, so their latencies overlap
+        const int nx = p.nb * 3;
+        for (int base = 0; base < nx; base += 4 * kThreads) {
+            uint4 v[4];
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+                const int e = base + i * kThreads + tid;
+                v[i] = e < nx ? __ldcg(xg + e) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+                const int e = base + i * kThreads + tid;
+                if (e < nx) xw[e] = v[i];
+                m = max_abs_pair(max_abs_pair(max_abs_pair(max_abs_pair(m, v[i].x), v[i].y), v[i].z), v[i].w);
+            }
         }
         LLVQ_TRACE_POINT(4)
+        LLVQ_TRACE_CLOCK(1)
         m = __reduce_max_sync(0xffffffffu, max(m & 0xffffu, m >> 16));
         if (lane == 0) warp_max[warp] = m;             // plain stores: atomics on one word would serialise the warps
         __syncthreads();                               // publishes x, the maxima and the block constants
@@ -334,6 +356,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         xexp = max((int)(__reduce_max_sync(0xffffffffu, m) >> 10), 1) - 14;
     }
     LLVQ_TRACE_POINT(3)
+    LLVQ_TRACE_CLOCK(2)
 
     int n = 0;
     uint32_t parity = 0;                               // every slot completes once a round of kSlots units
