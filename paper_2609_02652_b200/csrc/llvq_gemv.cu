@@ -653,9 +653,8 @@ int gemv_configure(const llvq_ctx *ctx) {
 
 cudaError_t launch_gemv(const llvq_ctx *ctx, int layout, GemvParams &p, bool no_weights, cudaStream_t s) {
     const size_t smem = gemv_smem_bytes(layout, p.nb, p.nprob);
-    // one CTA a multiprocessor; fewer only when there are fewer units than warps
-    int grid = (p.total_units + kWarps - 1) / kWarps;
-    if (grid > ctx->sm_count) grid = ctx->sm_count;
+    // one CTA a multiprocessor (warps are numbered CTA-first, so a short launch spreads over all of them)
+    int grid = p.total_units < ctx->sm_count ? p.total_units : ctx->sm_count;
     p.units_base = p.total_units / (grid * kWarps);
     p.units_rem = p.total_units % (grid * kWarps);
     cudaLaunchConfig_t cfg = {};
@@ -808,8 +807,7 @@ extern "C" int llvq_gemv_static(const void *layout_buf, const void *row_scale, c
     p.error = d.error;
     const size_t smem = gemv_smem_bytes(LLVQ_PLANES, p.nb, 1);
     if (smem + 1024 > (size_t)d.max_smem_optin) return LLVQ_ESIZE;
-    int grid = (p.total_units + kWarps - 1) / kWarps;
-    if (grid > d.sm_count) grid = d.sm_count;
+    int grid = p.total_units < d.sm_count ? p.total_units : d.sm_count;
     p.units_base = p.total_units / (grid * kWarps);
     p.units_rem = p.total_units % (grid * kWarps);
     cudaLaunchConfig_t cfg = {};
