@@ -198,3 +198,34 @@ def test_error_codes(B, ctx):
     # the context is still usable
     y = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, 96)
     assert torch.isfinite(y).all()
+
+
+def test_wide_matrix_many_groups_and_size_limits(B, ctx, oracle):
+    # a long row (1024 blocks, x of 48 KB in shared memory) and a launch over eight matrices
+    case = make_case(70, 24 * 1024, seed=41)
+    buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    y = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
+    B.status(ctx)
+    check_gemv(oracle, case, y)
+    cases = [make_case(32 + 17 * i, 24 * 40, seed=50, tensor_id=i) for i in range(8)]
+    for c in cases[1:]:
+        c.x, c.d_x = cases[0].x, cases[0].d_x
+    bufs = [B.expand(ctx, 0, c.d_codes, c.rows, c.nb) for c in cases]
+    gains = [(0.5 + 0.25 * i, 1.0 + 0.125 * i) for i in range(8)]
+    ys = [torch.full((c.rows,), float("nan"), dtype=torch.float32, device="cuda") for c in cases]
+    B.gemv_grouped(ctx, 0, [(b, c.d_scale, g, y, c.rows) for b, c, g, y in zip(bufs, cases, gains, ys)], cases[0].d_x, 24 * 40)
+    B.status(ctx)
+    for c, g, y in zip(cases, gains, ys):
+        check_gemv(oracle, c, y, gain=g)
+    # nine matrices, and an in-dimension whose x does not fit in shared memory beside the ring: refused, nothing launched
+    with pytest.raises(B.LlvqError) as e:
+        B.gemv_grouped(ctx, 0, [(bufs[0], cases[0].d_scale, GAIN, ys[0], cases[0].rows)] * 9, cases[0].d_x, 24 * 40)
+    assert e.value.code == -1
+    big_k = 98304
+    xx = torch.zeros(big_k, dtype=torch.float16, device="cuda")
+    with pytest.raises(B.LlvqError) as e:
+        B.gemv(ctx, 0, bufs[0], cases[0].d_scale, GAIN, xx, 32, big_k)
+    assert e.value.code == -3
+    # negative and zero gains are legal
+    y = B.gemv(ctx, 0, bufs[0], cases[0].d_scale, (-1.25, 0.0), cases[0].d_x, cases[0].rows, 24 * 40)
+    check_gemv(oracle, cases[0], y, gain=(-1.25, 0.0))
