@@ -229,3 +229,21 @@ def test_wide_matrix_many_groups_and_size_limits(B, ctx, oracle):
     # negative and zero gains are legal
     y = B.gemv(ctx, 0, bufs[0], cases[0].d_scale, (-1.25, 0.0), cases[0].d_x, cases[0].rows, 24 * 40)
     check_gemv(oracle, cases[0], y, gain=(-1.25, 0.0))
+
+
+@pytest.mark.parametrize("scale", [0.0, 6e-8, 1e-4, 3.0e3])
+def test_gemv_extreme_activation_ranges(B, ctx, oracle, scale):
+    """All-zero x, fp16-subnormal x, small x and x near the top of the fp16 range: the fixed-point quantum
+    follows max |x|, so the normalised error bound holds at every scale."""
+    case = make_case(96, 24 * 57, seed=77)
+    xs = (case.x.astype(np.float64) * scale).astype(np.float16)
+    if scale == 6e-8:
+        assert (np.abs(xs[xs != 0]) < 6.2e-5).all()          # every non-zero entry is an fp16 subnormal
+    case.x, case.d_x = xs, torch.from_numpy(xs).cuda()
+    buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    y = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
+    B.status(ctx)
+    if not xs.any():
+        assert (y == 0).all()
+    else:
+        check_gemv(oracle, case, y)
