@@ -86,9 +86,15 @@ const char *llvq_strerror(int code);
 
 /* Synchronises `stream` and reports whether any GEMV launched on this context since the last
  * call gave up on one of its bounded waits (LLVQ_ETIMEOUT; the flag and the scratch are then
- * reset).  Every wait inside the kernels - on an asynchronous copy or on the previous kernel -
- * has an iteration limit; none can spin forever. */
+ * reset).  Every wait inside the kernels on an asynchronous copy has a time limit of about a second;
+ * none can spin forever, and none traps. */
 int llvq_status(llvq_ctx *ctx, void *stream);
+
+/* Enqueues a one-warp kernel that waits, with a limit of about a millisecond, on a barrier nothing
+ * completes, and then raises the context's error flag exactly as a GEMV whose copy never arrived
+ * would: the next llvq_status returns LLVQ_ETIMEOUT, the one after LLVQ_OK.  Lets a caller (and the
+ * tests) check the failure path without any fault on the GPU. */
+int llvq_selftest_wait_limit(llvq_ctx *ctx, void *stream);
 
 /* The GEMV is launched with programmatic dependent launch (on by default): its record prefetch
  * starts while the previous kernel of the stream drains, and it waits for that kernel before it

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libllvq.so")
 _lib = None
 
 SYMBOLS = (
-    "llvq_create", "llvq_destroy", "llvq_strerror", "llvq_status", "llvq_set_pdl", "llvq_num_classes", "llvq_class_base", "llvq_layout_bytes",
+    "llvq_create", "llvq_destroy", "llvq_strerror", "llvq_status", "llvq_selftest_wait_limit", "llvq_set_pdl", "llvq_num_classes", "llvq_class_base", "llvq_layout_bytes",
     "llvq_expand", "llvq_gemv", "llvq_gemv_grouped", "llvq_gemv_static", "llvq_gemv_fp16", "llvq_gemv_noweights", "llvq_dequant_fp16",
     "llvq_decode_i8",
 )
@@ -55,6 +55,7 @@ def load() -> ctypes.CDLL:
         L.llvq_num_classes.argtypes = [vp]
         L.llvq_status.argtypes = [vp, vp]
         L.llvq_set_pdl.argtypes = [vp, ci]
+        L.llvq_selftest_wait_limit.argtypes = [vp, vp]
         L.llvq_class_base.argtypes = [vp, ci]
         L.llvq_class_base.restype = ctypes.c_uint64
         L.llvq_layout_bytes.argtypes = [ci, i64, i64, ctypes.POINTER(sz)]
@@ -129,6 +130,11 @@ def destroy(ctx: Context) -> None:
 def status(ctx: Context, stream=None) -> None:
     """Synchronises the stream; raises if a kernel on this context gave up on a bounded wait."""
     _check(load().llvq_status(ctx.ptr, _stream(stream)), "llvq_status")
+
+
+def selftest_wait_limit(ctx: Context, stream=None) -> None:
+    """Enqueues the bounded-wait self-test; the next status() raises LlvqError(-5)."""
+    _check(load().llvq_selftest_wait_limit(ctx.ptr, _stream(stream)), "llvq_selftest_wait_limit")
 
 
 def set_pdl(ctx: Context, enabled: bool) -> None:

@@ -130,6 +130,13 @@ int llvq_status(llvq_ctx *ctx, void *stream) {
     return LLVQ_OK;
 }
 
+int llvq_selftest_wait_limit(llvq_ctx *ctx, void *stream) {
+    if (!ctx) return LLVQ_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    return launch_wait_limit_selftest(ctx, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+}
+
 int llvq_set_pdl(llvq_ctx *ctx, int enabled) {
     if (!ctx) return LLVQ_EINVAL;
     ctx->use_pdl = enabled ? 1 : 0;

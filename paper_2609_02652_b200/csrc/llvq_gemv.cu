@@ -192,13 +192,19 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
                  : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Every wait is bounded: after kSpinLimit failed polls the caller records an error and winds down.
-constexpr int kSpinLimit = 1 << 22;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (int i = 0; i < kSpinLimit; i++)
+// Every wait is bounded in time: a poll that fails starts a clock, and once kWaitLimitCycles SM cycles
+// (about a second) have passed without the barrier completing, the caller records an error and winds
+// down.  The first poll reads no clock, so a wait that is already satisfied costs one instruction.
+constexpr long long kWaitLimitCycles = 2000000000ll;
+__device__ __forceinline__ bool mbar_wait_for(uint32_t bar, uint32_t parity, long long limit_cycles) {
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    do {
         if (mbar_try(bar, parity)) return true;
+    } while (clock64() - t0 < limit_cycles);
     return false;
 }
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) { return mbar_wait_for(bar, parity, kWaitLimitCycles); }
 
 // Ring reads through 32-bit shared-memory addresses.  Volatile: they must stay behind the wait on the
 // slot's barrier and ahead of the copy that refills the slot.
@@ -461,6 +467,19 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     }
 }
 
+// Exercises the wait limit without any fault: one warp waits, for about a millisecond, on a barrier
+// that nothing will ever complete, then reports through the same error flag the GEMV uses.
+__global__ void wait_limit_selftest_kernel(int *error) {
+    __shared__ __align__(8) uint64_t bar;
+    const uint32_t b = smem_addr(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (!mbar_wait_for(b, 0, 2000000ll) && threadIdx.x == 0) atomicExch(error, 1);
+}
+
 // One-hot comparison arm: same unit sequence, same reduction, records read with plain loads.
 __global__ void __launch_bounds__(kThreads, 1) gemv_onehot_kernel(const __grid_constant__ GemvParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -673,6 +692,11 @@ cudaError_t launch_gemv(const llvq_ctx *ctx, int layout, GemvParams &p, bool no_
     }
     cfg.numAttrs = 0;
     return cudaLaunchKernelEx(&cfg, gemv_onehot_kernel, p);
+}
+
+cudaError_t launch_wait_limit_selftest(const llvq_ctx *ctx, cudaStream_t s) {
+    wait_limit_selftest_kernel<<<1, 32, 0, s>>>(ctx->error);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_gemv_fp16(const __half *W, const __half *x, float *y, int64_t rows, int64_t k, cudaStream_t s) {

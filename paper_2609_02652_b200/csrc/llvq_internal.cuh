@@ -86,6 +86,7 @@ namespace llvq {
 cudaError_t launch_expand(const llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, int64_t nb,
                           void *out, uint32_t *bad_count, cudaStream_t s);
 cudaError_t launch_gemv(const llvq_ctx *ctx, int layout, GemvParams &p, bool no_weights, cudaStream_t s);
+cudaError_t launch_wait_limit_selftest(const llvq_ctx *ctx, cudaStream_t s);
 cudaError_t launch_gemv_fp16(const __half *W, const __half *x, float *y, int64_t rows, int64_t k, cudaStream_t s);
 cudaError_t launch_dequant(const llvq_ctx *ctx, int layout, const uint8_t *buf, const __half *row_scale, float g0, float g1,
                            __half *W, int64_t rows, int64_t nb, cudaStream_t s);

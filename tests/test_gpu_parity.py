@@ -247,3 +247,22 @@ def test_gemv_extreme_activation_ranges(B, ctx, oracle, scale):
         assert (y == 0).all()
     else:
         check_gemv(oracle, case, y)
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(B, oracle):
+    """No fault is injected: a one-warp kernel waits about a millisecond on a barrier nothing completes."""
+    ctx = B.create(0)
+    try:
+        B.status(ctx)
+        B.selftest_wait_limit(ctx)
+        with pytest.raises(B.LlvqError) as e:
+            B.status(ctx)
+        assert e.value.code == -5
+        B.status(ctx)                          # the flag was reset
+        case = make_case(100, 24 * 20, seed=3)
+        buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+        y = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
+        B.status(ctx)
+        check_gemv(oracle, case, y)
+    finally:
+        ctx.close()
