@@ -28,15 +28,31 @@
  * group", rows past the end are filled with the empty record, class id 511):
  *   LLVQ_PLANES  14 bytes a block [Sec. 3.2 "Planes14": class id 9 b, gain 1 b, sign mask 24 b,
  *                three binary planes of the per-coordinate level 3 x 24 b = 106 bits in 112].
- *                The level of a coordinate is |x_i| >> 1; the class fixes the parity of every
- *                magnitude, so |x_i| = 2 level + parity.  Per (row group, block column) "cell"
- *                and per row: a 16-bit header = class | gain << 9 and three 32-bit words; word j
- *                carries coordinates 8j..8j+7; coordinate 8j+2k+e (k = 0..3, e = 0..1) has level
- *                bit t at bit (4+t+16e+4k) mod 32 and its sign at bit (15+16e+4k) mod 32.  Four
- *                consecutive cells form a 1792-byte tile (row l: bytes 512j+16l = word j of the
- *                four cells, bytes 1536+8l = the four headers); the nb mod 4 last cells of a row
- *                group are stored alone, 448 bytes each (word j of row l at 128j+4l, header at
- *                384+2l).  A row group takes 448*nb bytes.
+ *                The class fixes the parity of every coordinate, so sign and level (|x_i| >> 1) of a
+ *                coordinate are stored as one four-bit code u_i = 8 + floor(x_i / 2): x_i = 2 (u_i - 8)
+ *                + parity.  Per block a 16-bit header = class | gain << 9 and 24 codes; the empty
+ *                record has u_i = 8.  The codes are laid out as the operand fragments of the integer
+ *                tensor-core instruction the GEMV uses (16 rows x 32 or 16 positions, a byte each once
+ *                the nibbles are split):
+ *                  row of a group r = 16 m + 8 e + g (m, e in {0,1}, g in 0..7); lane L = 4 g + t.
+ *                  A half-step is 16 rows (one m) of two block slots, 48 positions k: k < 24 is
+ *                  coordinate k of slot 0, else coordinate k - 24 of slot 1.  Lane L owns three words;
+ *                  nibble n = 2 i + c (i = 0..3, c = 0..1) of a word is bits 4n..4n+3:
+ *                    Wa: code of row (m, e=0, g) at position 16 c + 4 t + i
+ *                    Wb: code of row (m, e=1, g) at position 16 c + 4 t + i
+ *                    Wc: code of row (m, e=c, g) at position 32 + 4 t + i
+ *                  and lane pair P = 2 g + (t >> 1) owns one header word:
+ *                    header(row (m,0,g), slot t >> 1) | header(row (m,1,g), slot t >> 1) << 16.
+ *                  Tile = blocks 4T..4T+3 of a row group, 1792 bytes: half-step h = 2 s + m has slots
+ *                  4T+2s, 4T+2s+1; word w = 3 h + (0 Wa, 1 Wb, 2 Wc) of lane L at byte
+ *                  512 (w >> 2) + 16 L + 4 (w & 3); header word h of pair P at 1536 + 16 P + 4 h.
+ *                  The nb mod 4 blocks left over follow the tiles: if two or three, first a pair
+ *                  (896 bytes; half-steps m = 0,1 with the next two blocks as slots; word
+ *                  w = 3 m + (0,1,2) of lane L at 128 w + 4 L; header word m of pair P at
+ *                  768 + 8 P + 4 m); if one or three, last a single (448 bytes; one half-step whose
+ *                  slot s is rows 16 s..16 s+15 of the last block, i.e. "row (m,e,g), slot s" above
+ *                  reads row (s,e,g); word w of lane L at 128 w + 4 L; header word of pair P at
+ *                  384 + 4 P).  A row group takes 448*nb bytes.
  *   LLVQ_ONEHOT  20 bytes a block [Sec. 3.2 "Slot32": class id, gain, sign mask, one 24-bit
  *                one-hot mask per non-zero level].  Level = rank of |x_i| among the class's
  *                distinct magnitudes.  Per cell five arrays of 32 words (word t of row l at
@@ -64,7 +80,7 @@ extern "C" {
 #define LLVQ_ETIMEOUT (-5) /* a bounded wait inside a kernel ran out (llvq_status only)         */
 
 #define LLVQ_MAX_GROUP 8       /* matrices in one grouped launch                             */
-#define LLVQ_MAX_K 98304       /* largest k_padded the GEMV stages in shared memory          */
+#define LLVQ_MAX_K 98304       /* largest k_padded the GEMV accepts                          */
 
 typedef struct llvq_ctx llvq_ctx;
 
@@ -118,12 +134,14 @@ int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, 
                 void *layout_out, size_t out_bytes, uint32_t *bad_count, void *stream);
 
 /* [Sec. 2.3] y[row] = row_scale[row] * sum_b gain[g_b] / (4 sqrt(m_b)) * sum_i x_b,i * x[24b+i],
- * m_b the shell of block b's class, with f32 accumulation (the products of the small integer
- * coordinates with fp16 x are exact in f32).  gain is a HOST pointer to two floats.  x is fp16,
- * 16-byte aligned; y is f32; x must be finite.  A row is summed in chunks of blocks whose bounds
- * depend on nb alone; the chunk sums meet in a fixed-point accumulator (integer addition, exact
- * and order-free, finer than f32), so the result never depends on the launch geometry and a
- * grouped launch returns bit-identical rows. */
+ * m_b the shell of block b's class.  gain is a HOST pointer to two floats.  x is fp16, 16-byte
+ * aligned; y is f32; x must be finite.  LLVQ_PLANES: x is taken as fixed point on a scale set by
+ * the largest |x| (X_i = rint(x_i 2^F), |X_i| < 2^29; exact for every x_i within 2^-18 of the
+ * largest, rounded to within 2^-29 of the largest below that), the inner sums over a block are integer and
+ * exact, the per-block scale is applied in f32.  LLVQ_ONEHOT: f32 products and sums.  Either way a
+ * row is summed in pieces of at most four blocks whose bounds depend on nb alone; the pieces meet
+ * in a fixed-point accumulator (integer addition, exact and order-free, finer than f32), so the
+ * result never depends on the launch geometry and a grouped launch returns bit-identical rows. */
 int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row_scale,
               const float *gain, const void *x, float *y, int64_t rows, int64_t k_padded, void *stream);
 

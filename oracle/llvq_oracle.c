@@ -486,49 +486,108 @@ size_t llvqo_planes_bytes(int64_t rows, int64_t nb) { return (size_t)((rows + 31
 size_t llvqo_onehot_bytes(int64_t rows, int64_t nb) { return (size_t)((rows + 31) / 32) * (size_t)nb * 640u; }
 
 /*
- * Bit-plane layout, 14 bytes a block.  Rows are taken 32 at a time (a row group); rows past the
- * end are filled with the sentinel record.  The cell of (row group, block column b) holds, for
- * each of its 32 rows, three payload words and a 16-bit header:
- *   header  = class | gain << 9
- *   word j (j = 0,1,2) carries coordinates 8j .. 8j+7.  Coordinate 8j + 2k + e (pair k = 0..3,
- *   e = 0 low / 1 high) has its level bit t at bit (4 + t + 16 e + 4 k) mod 32 and its sign
- *   at bit (15 + 16 e + 4 k) mod 32.
- * Four consecutive cells of a row group form a 1792-byte tile: for row l, bytes 512 j + 16 l
- * hold word j of the four cells in order, bytes 1536 + 8 l their four headers.  The nb mod 4
- * cells left at the end of a row group are stored alone, 448 bytes each: word j of row l at
- * 128 j + 4 l, header at 384 + 2 l.  A row group occupies 448 nb bytes.
+ * 14-byte layout ("planes"): per block a 16-bit header = class | gain << 9 and 24 four-bit codes
+ * u_i = 8 + floor(x_i / 2), so x_i = 2 (u_i - 8) + parity of the class; the same 106 bits as the
+ * record's sign mask and three level planes (u_i = 8 + level for a positive coordinate,
+ * 8 - level - parity for a negative one).  The sentinel record has u_i = 8.
+ *
+ * Rows are taken 32 at a time (a row group; rows past the end hold the sentinel); row
+ * r = 16 m + 8 e + g with m, e in {0,1}, g in 0..7.  A lane is L = 4 g + t, t in 0..3.
+ *
+ * A half-step covers 16 rows (one m) of two block slots, 48 positions kappa: kappa < 24 is
+ * coordinate kappa of slot 0, otherwise coordinate kappa - 24 of slot 1.  Lane L owns three words;
+ * nibble n = 2 i + c (i = 0..3, c = 0..1) of a word sits at bits 4n .. 4n+3:
+ *   Wa: code of row (m, e=0, g) at position 16 c + 4 t + i
+ *   Wb: code of row (m, e=1, g) at position 16 c + 4 t + i
+ *   Wc: code of row (m, e=c, g) at position 32 + 4 t + i
+ * and lane pair P = 2 g + (t >> 1) owns one header word:
+ *   header(row (m,0,g), slot t >> 1) | header(row (m,1,g), slot t >> 1) << 16.
+ *
+ * Tile = blocks 4T .. 4T+3 of a row group, 1792 bytes: half-step h = 2 s + m has slots 4T+2s and
+ * 4T+2s+1; word w = 3 h + (0 Wa, 1 Wb, 2 Wc) of lane L at 512 (w >> 2) + 16 L + 4 (w & 3); header
+ * word h of pair P at 1536 + 16 P + 4 h.
+ * The c = nb mod 4 blocks left over follow the tiles, 448 c bytes:
+ *   c >= 2: a pair (896 bytes) for the next two blocks: half-steps m = 0,1 with those two blocks
+ *           as slots; word w = 3 m + (0,1,2) of lane L at 128 w + 4 L; header word m of pair P at
+ *           768 + 8 P + 4 m.
+ *   c odd:  a single (448 bytes) for the last block: one half-step whose slot s is rows
+ *           16 s .. 16 s + 15 of that block (read "row (m,e,g), slot s" above as row (s,e,g));
+ *           word w of lane L at 128 w + 4 L; header word of pair P at 384 + 4 P.
+ * A row group occupies 448 nb bytes.
  */
+typedef struct { const uint8_t *code; const uint16_t *hdr; int64_t nb; } group_t;   /* code[(r*nb+b)*24+i], hdr[r*nb+b] */
+
+/* code at position kappa of a half-step: rows 16 m + 8 e + g of blocks b0 (slot 0) and b1 (slot 1);
+ * in a single (b1 < 0) the slot picks the row half instead */
+static uint32_t hs_code(const group_t *G, int64_t b0, int64_t b1, int m, int e, int g, int kappa) {
+    int slot = kappa / 24, i = kappa % 24;
+    int row = (b1 < 0) ? 16 * slot + 8 * e + g : 16 * m + 8 * e + g;
+    int64_t b = (b1 < 0) ? b0 : (slot ? b1 : b0);
+    return G->code[((size_t)row * G->nb + b) * 24 + i];
+}
+static uint32_t hs_header(const group_t *G, int64_t b0, int64_t b1, int m, int e, int g, int slot) {
+    int row = (b1 < 0) ? 16 * slot + 8 * e + g : 16 * m + 8 * e + g;
+    int64_t b = (b1 < 0) ? b0 : (slot ? b1 : b0);
+    return G->hdr[(size_t)row * G->nb + b];
+}
+/* the three words of lane (g, t) and the header word of its pair */
+static void hs_words(const group_t *G, int64_t b0, int64_t b1, int m, int g, int t, uint32_t w[3], uint32_t *hw) {
+    w[0] = w[1] = w[2] = 0;
+    for (int i = 0; i < 4; i++)
+        for (int c = 0; c < 2; c++) {
+            int n = 2 * i + c;
+            w[0] |= hs_code(G, b0, b1, m, 0, g, 16 * c + 4 * t + i) << (4 * n);
+            w[1] |= hs_code(G, b0, b1, m, 1, g, 16 * c + 4 * t + i) << (4 * n);
+            w[2] |= hs_code(G, b0, b1, m, c, g, 32 + 4 * t + i) << (4 * n);
+        }
+    *hw = hs_header(G, b0, b1, m, 0, g, t >> 1) | hs_header(G, b0, b1, m, 1, g, t >> 1) << 16;
+}
+
 void llvqo_pack_planes(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t *out) {
-    int64_t ngroups = (rows + 31) / 32, nfull = nb / 4;
+    int64_t ngroups = (rows + 31) / 32, ntiles = nb / 4, left = nb % 4;
+    uint8_t *code = malloc((size_t)32 * nb * 24);
+    uint16_t *hdr = malloc((size_t)32 * nb * 2);
     for (int64_t rg = 0; rg < ngroups; rg++) {
-        uint8_t *grp = out + (size_t)rg * (size_t)nb * 448u;
-        for (int l = 0; l < 32; l++) {
-            int64_t row = rg * 32 + l;
+        for (int r = 0; r < 32; r++)
             for (int64_t b = 0; b < nb; b++) {
-                record_t r;
-                if (row < rows) make_record(codes[row * nb + b], &r);
-                else { memset(&r, 0, sizeof r); r.cls = SENTINEL_CLASS; }
-                uint32_t word[3] = {0, 0, 0};
-                for (int i = 0; i < NCOORD; i++) {
-                    int j = i / 8, k = (i % 8) / 2, e = i % 2;
-                    for (int t = 0; t < 3; t++)
-                        if ((r.plane[t] >> i) & 1) word[j] |= 1u << ((4 + t + 16 * e + 4 * k) % 32);
-                    if ((r.smask >> i) & 1) word[j] |= 1u << ((15 + 16 * e + 4 * k) % 32);
+                record_t rec;
+                int64_t row = rg * 32 + r;
+                if (row < rows) make_record(codes[row * nb + b], &rec);
+                else { memset(&rec, 0, sizeof rec); rec.cls = SENTINEL_CLASS; }
+                int parity = rec.cls == SENTINEL_CLASS ? 0 : (rec.x[0] & 1);
+                for (int i = 0; i < NCOORD; i++) code[((size_t)r * nb + b) * 24 + i] = (uint8_t)(8 + (rec.x[i] - parity) / 2);
+                hdr[(size_t)r * nb + b] = (uint16_t)(rec.cls | (rec.gain << 9));
+            }
+        group_t G = {code, hdr, nb};
+        uint8_t *grp = out + (size_t)rg * (size_t)nb * 448u;
+        uint32_t w[3], hw;
+        for (int g = 0; g < 8; g++)
+            for (int t = 0; t < 4; t++) {
+                int L = 4 * g + t, P = 2 * g + (t >> 1);
+                for (int64_t T = 0; T < ntiles; T++)
+                    for (int h = 0; h < 4; h++) {
+                        hs_words(&G, 4 * T + 2 * (h >> 1), 4 * T + 2 * (h >> 1) + 1, h & 1, g, t, w, &hw);
+                        uint8_t *tile = grp + (size_t)T * 1792u;
+                        for (int q = 0; q < 3; q++) { int k = 3 * h + q; memcpy(tile + 512 * (k >> 2) + 16 * L + 4 * (k & 3), &w[q], 4); }
+                        memcpy(tile + 1536 + 16 * P + 4 * h, &hw, 4);
+                    }
+                uint8_t *rest = grp + (size_t)ntiles * 1792u;
+                if (left >= 2) {
+                    for (int m = 0; m < 2; m++) {
+                        hs_words(&G, 4 * ntiles, 4 * ntiles + 1, m, g, t, w, &hw);
+                        for (int q = 0; q < 3; q++) memcpy(rest + 128 * (3 * m + q) + 4 * L, &w[q], 4);
+                        memcpy(rest + 768 + 8 * P + 4 * m, &hw, 4);
+                    }
+                    rest += 896;
                 }
-                uint16_t hdr = (uint16_t)(r.cls | (r.gain << 9));
-                if (b < nfull * 4) {
-                    uint8_t *tile = grp + (size_t)(b / 4) * 1792u;
-                    int q = (int)(b % 4);
-                    for (int j = 0; j < 3; j++) memcpy(tile + 512 * j + 16 * l + 4 * q, &word[j], 4);
-                    memcpy(tile + 1536 + 8 * l + 2 * q, &hdr, 2);
-                } else {
-                    uint8_t *cell = grp + (size_t)nfull * 1792u + (size_t)(b - nfull * 4) * 448u;
-                    for (int j = 0; j < 3; j++) memcpy(cell + 128 * j + 4 * l, &word[j], 4);
-                    memcpy(cell + 384 + 2 * l, &hdr, 2);
+                if (left & 1) {
+                    hs_words(&G, nb - 1, -1, 0, g, t, w, &hw);
+                    for (int q = 0; q < 3; q++) memcpy(rest + 128 * q + 4 * L, &w[q], 4);
+                    memcpy(rest + 384 + 4 * P, &hw, 4);
                 }
             }
-        }
     }
+    free(code); free(hdr);
 }
 
 /*

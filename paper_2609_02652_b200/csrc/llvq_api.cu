@@ -237,10 +237,11 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
     p.trace = ctx->trace;
     p.trace_launch = ctx->trace ? ctx->trace_launch++ : 0;
 #endif
-    if (gemv_smem_bytes(layout, p.nb, n) + 1024 > (size_t)ctx->max_smem_optin) return LLVQ_ESIZE;
+    const GemvLaunch g = gemv_plan(layout, p, ctx->sm_count);
+    if (g.smem + 1024 > (size_t)ctx->max_smem_optin) return LLVQ_ESIZE;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
-    return launch_gemv(ctx, layout, p, no_weights, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+    return launch_gemv(layout, p, g, no_weights, ctx->use_pdl != 0, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
 }
 
 int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row_scale, const float *gain, const void *x,

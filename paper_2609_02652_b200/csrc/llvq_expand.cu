@@ -109,35 +109,47 @@ __device__ bool decode_code(uint64_t code, const DeviceTables &T, Decoded &d) {
     return true;
 }
 
-// word j of the bit-plane record: coordinate 8j+2k+e -> level at (4+16e+4k) mod 32, sign at (15+16e+4k) mod 32
-__device__ __forceinline__ uint32_t planes_word(const Decoded &d, int j) {
+// word j of a block's codes in coordinate order: nibble n = code of coordinate 8j+n, u = 8 + floor(x / 2)
+__device__ __forceinline__ uint32_t code_word(const Decoded &d, int j) {
     uint32_t w = 0;
 #pragma unroll
     for (int n = 0; n < 8; n++) {
-        const int k = n >> 1, e = n & 1, i = 8 * j + n;
-        const uint32_t level = ((d.mag[j] >> (4 * n)) & 15u) >> 1;
-        w |= level << ((4 + 16 * e + 4 * k) & 31);
-        w |= ((d.smask >> i) & 1u) << ((15 + 16 * e + 4 * k) & 31);
+        const uint32_t a = (d.mag[j] >> (4 * n)) & 15u;
+        const bool neg = (d.smask >> (8 * j + n)) & 1u;
+        const uint32_t u = neg ? 8u - (a >> 1) - (a & 1u) : 8u + (a >> 1);
+        w |= u << (4 * n);
     }
     return w;
 }
 
+// nibbles 0..3 of h go to nibbles 0, 2, 4, 6
+__device__ __forceinline__ uint32_t spread4(uint32_t h) {
+    h &= 0xffffu;
+    h = (h | (h << 8)) & 0x00ff00ffu;
+    return (h | (h << 4)) & 0x0f0f0f0fu;
+}
+
+// One warp writes one piece of a row group: a tile (four blocks), the pair after the tiles or the
+// single at the end (see include/llvq.h).  First every lane decodes the blocks of its own row into
+// shared memory in coordinate order, then lane 4g+t gathers the words it owns in the layout.
 __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, const uint64_t *__restrict__ codes, int64_t rows, int64_t nb,
                                                             uint8_t *__restrict__ out, uint32_t *bad_count) {
-    const int64_t tiles = nb / kTileCells, tail = nb % kTileCells, units = tiles + tail;
+    __shared__ uint32_t nat_all[8][4][4][32];              // [warp][block of the piece][word 0..2, header][row]
+    const int64_t tiles = nb / kTileCells, left = nb % kTileCells;
+    const int64_t pieces = tiles + (left >= 2 ? 1 : 0) + (left & 1);
     const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int lane = (int)(gid & 31);
-    const int64_t unit_id = gid >> 5;
+    const int64_t piece_id = gid >> 5;
     const int64_t groups = (rows + kRowsPerGroup - 1) / kRowsPerGroup;
-    if (unit_id >= groups * units) return;
-    const int64_t rg = unit_id / units, u = unit_id % units;
+    if (piece_id >= groups * pieces) return;               // whole warps leave together
+    uint32_t (*nat)[4][32] = nat_all[threadIdx.x >> 5];
+    const int64_t rg = piece_id / pieces, u = piece_id % pieces;
     const int64_t row = rg * kRowsPerGroup + lane;
     uint8_t *grp = out + (size_t)rg * (size_t)nb * kCellBytes;
-    const bool full = u < tiles;
-    const int ncell = full ? kTileCells : 1;
-    const int64_t b0 = full ? u * kTileCells : tiles * kTileCells + (u - tiles);
-    uint32_t w[3][4];
-    uint32_t hdr[4];
+    const bool is_tile = u < tiles;
+    const bool is_pair = !is_tile && left >= 2 && u == tiles;
+    const int ncell = is_tile ? 4 : (is_pair ? 2 : 1);
+    const int64_t b0 = is_tile ? u * kTileCells : (is_pair ? tiles * kTileCells : nb - 1);
     int bad = 0;
 #pragma unroll 1
     for (int q = 0; q < ncell; q++) {
@@ -147,24 +159,55 @@ __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, cons
         } else {
             d.cls = kEmptyClass; d.gain = 0; d.smask = 0; d.mag[0] = d.mag[1] = d.mag[2] = 0;
         }
-#pragma unroll
-        for (int qq = 0; qq < 4; qq++)
-            if (qq == q) {
-                w[0][qq] = planes_word(d, 0); w[1][qq] = planes_word(d, 1); w[2][qq] = planes_word(d, 2);
-                hdr[qq] = (uint32_t)d.cls | ((uint32_t)d.gain << 9);
-            }
+        nat[q][0][lane] = code_word(d, 0); nat[q][1][lane] = code_word(d, 1); nat[q][2][lane] = code_word(d, 2);
+        nat[q][3][lane] = (uint32_t)d.cls | ((uint32_t)d.gain << 9);
     }
-    if (full) {
+    __syncwarp();
+    const int g = lane >> 2, t = lane & 3;
+    const bool single = !is_tile && !is_pair;
+    // four codes of row (m, e, g) starting at position kappa0 (a multiple of 4) of the half-step whose slots are blocks q0, q0+1
+    auto quad = [&](int q0, int m, int e, int kappa0) -> uint32_t {
+        const int slot = kappa0 / 24, i0 = kappa0 % 24;
+        const int r = single ? 16 * slot + 8 * e + g : 16 * m + 8 * e + g;
+        const int q = single ? q0 : q0 + slot;
+        return nat[q][i0 >> 3][r] >> (16 * ((i0 >> 2) & 1));
+    };
+    auto header = [&](int q0, int m, int e, int slot) -> uint32_t {
+        const int r = single ? 16 * slot + 8 * e + g : 16 * m + 8 * e + g;
+        return nat[single ? q0 : q0 + slot][3][r];
+    };
+    auto half_step = [&](int q0, int m, uint32_t w[3], uint32_t &hw) {
+        w[0] = spread4(quad(q0, m, 0, 4 * t)) | spread4(quad(q0, m, 0, 16 + 4 * t)) << 4;
+        w[1] = spread4(quad(q0, m, 1, 4 * t)) | spread4(quad(q0, m, 1, 16 + 4 * t)) << 4;
+        w[2] = spread4(quad(q0, m, 0, 32 + 4 * t)) | spread4(quad(q0, m, 1, 32 + 4 * t)) << 4;
+        hw = header(q0, m, 0, t >> 1) | header(q0, m, 1, t >> 1) << 16;
+    };
+    if (is_tile) {
+        uint32_t w[12], hw[4];
+#pragma unroll
+        for (int h = 0; h < 4; h++) half_step(2 * (h >> 1), h & 1, w + 3 * h, hw[h]);
         uint8_t *tile = grp + (size_t)u * kTileBytes;
 #pragma unroll
         for (int j = 0; j < 3; j++)
-            *reinterpret_cast<uint4 *>(tile + 512 * j + 16 * lane) = make_uint4(w[j][0], w[j][1], w[j][2], w[j][3]);
-        *reinterpret_cast<uint2 *>(tile + 1536 + 8 * lane) = make_uint2(hdr[0] | (hdr[1] << 16), hdr[2] | (hdr[3] << 16));
-    } else {
-        uint8_t *cell = grp + (size_t)tiles * kTileBytes + (size_t)(u - tiles) * kCellBytes;
+            *reinterpret_cast<uint4 *>(tile + 512 * j + 16 * lane) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
+        if ((t & 1) == 0) *reinterpret_cast<uint4 *>(tile + 1536 + 16 * (lane >> 1)) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+    } else if (is_pair) {
+        uint8_t *pair = grp + (size_t)tiles * kTileBytes;
 #pragma unroll
-        for (int j = 0; j < 3; j++) *reinterpret_cast<uint32_t *>(cell + 128 * j + 4 * lane) = w[j][0];
-        *reinterpret_cast<uint16_t *>(cell + 384 + 2 * lane) = (uint16_t)hdr[0];
+        for (int m = 0; m < 2; m++) {
+            uint32_t w[3], hw;
+            half_step(0, m, w, hw);
+#pragma unroll
+            for (int q = 0; q < 3; q++) *reinterpret_cast<uint32_t *>(pair + 128 * (3 * m + q) + 4 * lane) = w[q];
+            if ((t & 1) == 0) *reinterpret_cast<uint32_t *>(pair + 768 + 8 * (lane >> 1) + 4 * m) = hw;
+        }
+    } else {
+        uint8_t *one = grp + (size_t)tiles * kTileBytes + (left == 3 ? 2 * kCellBytes : 0);
+        uint32_t w[3], hw;
+        half_step(0, 0, w, hw);
+#pragma unroll
+        for (int q = 0; q < 3; q++) *reinterpret_cast<uint32_t *>(one + 128 * q + 4 * lane) = w[q];
+        if ((t & 1) == 0) *reinterpret_cast<uint32_t *>(one + 384 + 4 * (lane >> 1)) = hw;
     }
     if (bad && bad_count) atomicAdd(bad_count, (uint32_t)bad);
 }
@@ -211,8 +254,9 @@ cudaError_t launch_expand(const llvq_ctx *ctx, int layout, const uint64_t *codes
                           void *out, uint32_t *bad_count, cudaStream_t s) {
     const int64_t groups = (rows + kRowsPerGroup - 1) / kRowsPerGroup;
     if (layout == LLVQ_PLANES) {
-        const int64_t units = nb / kTileCells + nb % kTileCells;
-        const int64_t threads = groups * units * 32;
+        const int64_t left = nb % kTileCells;
+        const int64_t pieces = nb / kTileCells + (left >= 2 ? 1 : 0) + (left & 1);
+        const int64_t threads = groups * pieces * 32;
         const int64_t blocks = (threads + 255) / 256;
         expand_planes_kernel<<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count);
     } else {

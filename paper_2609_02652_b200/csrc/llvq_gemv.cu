@@ -1,33 +1,39 @@
 // The fused dequantize-plus-matvec (paper Sec. 2.3, "The kernel"), re-designed for sm_100a.
 //
-// Geometry.  A lane owns a row: the 32 lanes of a warp work on the 32 rows of one row group and
-// walk the same block columns together, so every read of x is a shared-memory broadcast and no
-// shuffle reduction is needed.  The records of a launch form one sequence of units - a unit is a
-// tile of four block columns of a row group, or the row group's last nb mod 4 columns - and the
-// sequence is cut into equal contiguous ranges, one per warp of a grid of one CTA a
-// multiprocessor, so every warp streams the same number of bytes (give or take one unit).
+// Arithmetic.  A block contributes scale * sum_i x_i * x[24b+i] with x_i = 2 u_i + (parity - 16), u_i the
+// four-bit code the record stores.  The activations are taken as fixed point, X_i = rint(x_i * 2^F) with F
+// set by the largest |x| of the call, and 2 X_i is split into four balanced 8-bit limbs.  The inner sum then
+// is an integer contraction that the tensor cores do exactly: mma.sync m16n8k32 / m16n8k16, u8 x s8 -> s32.
+// A is 16 rows x 48 positions (two block slots of 24 coordinates) of codes, one byte each once the two nibbles
+// of a payload byte are split (one shift, two ANDs a word: the whole decode); B is block-diagonal, its eight
+// columns the four limbs of slot 0 and the four limbs of slot 1, so one accumulator tile holds, for 16 rows,
+// the two blocks' sums limb by limb.  Per (row, block) the limbs are recombined in integers, the offset term
+// (parity - 16) * sum_i X_i is added from a per-block sum prepared with x, and one float multiply-add applies
+// gain[g] / (4 sqrt m), looked up by the header.  Every lane runs the same instructions whatever its class.
 //
-// Reduction.  The float sum of a unit (at most four blocks, fixed order) is converted to fixed
-// point and from there on everything is integer: a warp adds its units of a row group in a
-// 64-bit register and hands the sum, with the number of units it covers, to the row's 64-bit
-// accumulator in the context's scratch by one atomic add.  Integer addition is exact and
-// order-free, so a row's result does not depend on how the units were dealt or on which warp
-// arrives last; the arrival that completes the unit count converts the total back to float,
-// applies the row scale, writes y and clears the accumulator.  The quantum is 2^-39 of a bound on
-// a unit's sum derived from max |x| and the gain, i.e. far below f32 resolution.
+// Geometry.  A warp works on the 32 rows of a row group, 16 at a time; the records are stored as the
+// instruction's operand fragments (include/llvq.h), so a lane's 128-bit shared-memory reads are its A
+// registers.  The records of a launch form one sequence of units - a unit is a tile of four block columns of
+// a row group, or the row group's last nb mod 4 columns - ordered panel by panel (a panel is about sixteen
+// consecutive unit columns of every row group).  The sequence is cut into equal contiguous ranges, one per
+// warp of a grid of one CTA a multiprocessor, warps numbered CTA by CTA: every warp streams the same number of
+// bytes (give or take one unit), and a CTA's units lie in one or two panels, so it prepares only that part
+// of x.
 //
-// Decode.  One rotate and one three-input logic op turn a payload word into a pair of fp16 bit
-// patterns whose value is (+-)|x_i| * 2^-21 (a subnormal built in place: level bits at [6:4],
-// the class parity or-ed in at bit 3, the sign at bit 15).  A mixed-precision fused multiply-add
-// (fp16 x fp16 + f32, one instruction) accumulates the exact product with the fp16 activation.
-// Per block one multiply applies gain[g] * 2^21 / (4 sqrt m), looked up by the class id.  Every
-// lane runs the same instructions whatever its class.
+// Reduction.  After a unit the four lanes that share a row add their shares (two shuffles, fixed order), the
+// float sum of the unit (at most four blocks) is converted to fixed point and from there on everything is
+// integer: a warp adds its units of a row group in a 64-bit register and hands the sum, with the number of
+// units it covers, to the row's 64-bit accumulator in the context's scratch by one atomic add.  Integer
+// addition is exact and order-free, so a row's result does not depend on how the units were dealt or on which
+// warp arrives last; the arrival that completes the unit count converts the total back to float, applies the
+// row scale, writes y and clears the accumulator.  The quantum is 2^-39 of a bound on a unit's sum derived
+// from max |x| and the gain, i.e. far below f32 resolution.
 //
-// Memory.  Each warp streams its units through a private ring of 1792-byte shared-memory slots
-// filled by bulk asynchronous copies (cp.async.bulk, completion on an mbarrier) that lane 0 issues
-// kSlots units ahead.  The first copies go out before the kernel waits for its predecessor in the
-// stream (records never depend on it), so under programmatic dependent launch the ring fills
-// while the previous kernel drains.  Every wait is bounded.
+// Memory.  Each warp streams its units through a private ring of 1792-byte shared-memory slots filled by bulk
+// asynchronous copies (cp.async.bulk, completion on an mbarrier) that lane 0 issues kSlots units ahead.  The
+// first copies go out before the kernel waits for its predecessor in the stream (records never depend on
+// it), so under programmatic dependent launch the ring fills while the previous kernel drains.  Every wait is
+// bounded.
 #include <cmath>
 #include <cstring>
 
@@ -74,7 +80,6 @@ namespace {
 constexpr int kWarps = LLVQ_WARPS;         // warps per CTA
 constexpr int kThreads = kWarps * 32;
 constexpr int kSlots = LLVQ_SLOTS;         // ring slots per warp
-constexpr uint32_t kPairMask = 0x80708070u;
 
 // fixed-point accumulator word: bits 53..63 count units, bits 0..52 sum the biased unit values
 constexpr int kCountShift = 53;
@@ -90,36 +95,6 @@ __device__ __forceinline__ void fma_pair(float &lo, float &hi, uint32_t w, uint3
         : "+f"(lo), "+f"(hi)
         : "r"(w), "r"(x));
 }
-// the same with a zero addend: starts the two chains without clearing registers first
-__device__ __forceinline__ void mul_pair(float &lo, float &hi, uint32_t w, uint32_t x) {
-    asm("{\n\t.reg .f16 wl, wh, xl, xh;\n\t"
-        "mov.b32 {wl, wh}, %2;\n\t"
-        "mov.b32 {xl, xh}, %3;\n\t"
-        "fma.rn.f32.f16 %0, wl, xl, 0f00000000;\n\t"
-        "fma.rn.f32.f16 %1, wh, xh, 0f00000000;\n\t}"
-        : "=f"(lo), "=f"(hi)
-        : "r"(w), "r"(x));
-}
-
-// sum over the 24 coordinates of one block of (+-|x_i| * 2^-21) * x[i]
-__device__ __forceinline__ float block_dot(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t parity, const uint4 *xs) {
-    float a0, a1;
-    const uint32_t w[3] = {w0, w1, w2};
-#pragma unroll
-    for (int j = 0; j < 3; j++) {
-        const uint4 xv = xs[j];                      // x[8j .. 8j+7] as four fp16 pairs (broadcast read)
-        const uint32_t xp[4] = {xv.x, xv.y, xv.z, xv.w};
-#pragma unroll
-        for (int k = 0; k < 4; k++) {
-            const uint32_t r = k ? __funnelshift_r(w[j], w[j], 4 * k) : w[j];
-            const uint32_t v = (r & kPairMask) | parity;
-            // two chains of twelve (measured faster than four of six)
-            if (j == 0 && k == 0) mul_pair(a0, a1, v, xp[k]); else fma_pair(a0, a1, v, xp[k]);
-        }
-    }
-    return a0 + a1;
-}
-
 // one-hot record: value = class table entry of the rank level, selected without indexing
 __device__ __forceinline__ float onehot_dot(const uint32_t v[5], const float *__restrict__ val, const __half *xs) {
     const uint32_t smask = v[0], m1 = v[1], m2 = v[2], m3 = v[3], m4 = v[4];
@@ -180,6 +155,38 @@ __device__ __forceinline__ void deliver(const GemvParams &p, const GemvProblemDe
     }
 }
 
+// The same in two halves, so that a warp does not sit out the atomic's round trip between two runs: hand_over
+// sends the sum and remembers what the answer will mean, settle (called at the next hand-over, or at the end)
+// reads the answer and, if this arrival completed the row, writes y and clears the accumulator.
+struct Handed {
+    unsigned long long old, addend;
+    unsigned long long *slot;     // null: nothing is pending
+    float *y;
+    float yscale;
+    int count;
+};
+__device__ __forceinline__ void settle(const GemvParams &p, Handed &h) {
+    if (h.slot == nullptr) return;
+    if ((int)(h.old >> kCountShift) + h.count == p.units) {
+        const long long total = (long long)((h.old + h.addend) & kSumMask) - (long long)p.units * kUnitBias;
+        *h.y = (float)total * h.yscale;
+        *h.slot = 0ull;                              // ready for the next launch on this context
+    }
+    h.slot = nullptr;
+}
+__device__ __forceinline__ void hand_over(const GemvParams &p, const GemvProblemDev &pr, int group, int lane, long long sum,
+                                          int count, int qexp, float row_scale, Handed &h) {
+    settle(p, h);
+    const int row = (group - pr.group_begin) * kRowsPerGroup + lane;
+    if (row >= pr.rows) return;                      // padding rows of the last row group
+    h.addend = (unsigned long long)(sum + (long long)count * kUnitBias) + ((unsigned long long)count << kCountShift);
+    h.slot = p.accum + (size_t)group * 32 + lane;
+    h.old = atomicAdd(h.slot, h.addend);
+    h.y = pr.y + row;
+    h.yscale = pow2f(qexp) * row_scale;
+    h.count = count;
+}
+
 // ---- asynchronous copies: global -> shared, completion counted on an mbarrier in shared memory
 __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -213,22 +220,11 @@ __device__ __forceinline__ uint4 lds128(uint32_t a) {
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
     return v;
 }
-__device__ __forceinline__ uint2 lds64(uint32_t a) {
-    uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
-    return v;
-}
 __device__ __forceinline__ uint32_t lds32(uint32_t a) {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
     return v;
 }
-__device__ __forceinline__ uint32_t lds16(uint32_t a) {
-    uint32_t v;
-    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(a));
-    return v;
-}
-
 // Returns zero, but only once its operands are available: an address that adds this zero cannot be
 // formed before the loads that produced them have completed.
 __device__ __forceinline__ uint32_t settled(uint32_t a, uint32_t b, uint32_t c) {
@@ -243,35 +239,194 @@ __device__ __forceinline__ const uint8_t *group_base(const GemvParams &p, int gr
     return p.prob[q].layout + (size_t)(group - p.prob[q].group_begin) * (size_t)p.nb * cell_bytes;
 }
 
+// ---- integer tensor-core contraction: D (16 rows x 8 columns, s32) = A (16 x k, u8) * B (k x 8, s8) [+ D]
+__device__ __forceinline__ void mma_k32(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+                 : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(0));
+}
+__device__ __forceinline__ void mma_k16(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+    asm("mma.sync.aligned.m16n8k16.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                 : "r"(a0), "r"(a1), "r"(b0));
+}
+
+// Bytes of x in shared memory, one record a block: four planes of 24 bytes (plane l = limb l of the 24
+// fixed-point activations, doubled), a zero word at 96, and at 100 and 104 the two halves of the block's
+// activation sum (see stage_x).
+constexpr int kXRecBytes = 112;
+
+// Offsets of this lane's operand words inside the two x records of a half-step (or, one = true, inside
+// the single record both slots of the row group's last half-step share).  B is block-diagonal: column
+// n = lane >> 2 carries limb n & 3 of slot n >> 2, and is zero at the positions of the other slot.
+struct LaneOffsets { uint32_t b0, b1, b2, xs; };
+__device__ __forceinline__ LaneOffsets lane_offsets(int lane, bool one) {
+    const int g = lane >> 2, t = lane & 3, l = g & 3;
+    const uint32_t zero = 96, second = one ? 0 : kXRecBytes;
+    LaneOffsets o;
+    if (g < 4) {
+        o.b0 = 24 * l + 4 * t;                                  // positions 4t..4t+3: slot 0, coordinates 4t..
+        o.b1 = t < 2 ? 24 * l + 16 + 4 * t : zero;              // positions 16+4t..: slot 0 up to 23, then slot 1
+        o.b2 = zero;                                            // positions 32+4t..: slot 1
+    } else {
+        o.b0 = zero;
+        o.b1 = t >= 2 ? second + 24 * l + 4 * (t - 2) : zero;
+        o.b2 = second + 24 * l + 8 + 4 * t;
+    }
+    o.xs = (one ? 0 : kXRecBytes * (t >> 1)) + 100 + 4 * (t & 1);
+    return o;
+}
+
+// Shared-memory reads with a constant byte offset folded into the instruction.  Volatile, so that the
+// compiler never moves one out of the branch that guards it: an address formed for a unit this CTA does not
+// own may lie outside its shared memory.
+template <int OFF>
+__device__ __forceinline__ uint32_t lds32_at(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(a), "n"(OFF));
+    return v;
+}
+__device__ __forceinline__ float2 lds_f2(uint32_t a) {
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a));
+    return v;
+}
+
+// The B operand of one step (two block slots) for this lane, and its share of the slots' activation sum.
+struct StepX { uint32_t b0, b1, b2; int xsum; };
+// a.* are this lane's four addresses for the records at the start of a tile; OFF selects the step
+template <int OFF>
+__device__ __forceinline__ StepX load_step(const LaneOffsets &a) {
+    StepX s;
+    s.b0 = lds32_at<OFF>(a.b0); s.b1 = lds32_at<OFF>(a.b1); s.b2 = lds32_at<OFF>(a.b2);
+    s.xsum = (int)lds32_at<OFF>(a.xs);
+    return s;
+}
+
+// One half-step: 16 rows x 2 block slots.  wa, wb, wc are this lane's three payload words, h0 and h1 the
+// headers of its two rows for slot (lane & 3) >> 1, sx the step's operand.  Adds to r0 (row g of the 16) and r1
+// (row g + 8) this lane's share of scale * sum_i x_i * X_i, X the fixed-point activations: its share is the
+// limb pair (lane & 1) of slot (lane & 3) >> 1.  FIRST: r0 and r1 are written, not added to.
+template <bool FIRST>
+__device__ __forceinline__ void half_step(uint32_t wa, uint32_t wb, uint32_t wc, uint32_t h0, uint32_t h1, const StepX &sx, uint32_t tq,
+                                          float &r0, float &r1) {
+    constexpr uint32_t kNib = 0x0f0f0f0fu;
+    int d[4];
+    mma_k32(d, wa & kNib, wb & kNib, (wa >> 4) & kNib, (wb >> 4) & kNib, sx.b0, sx.b1);
+    mma_k16(d, wc & kNib, (wc >> 4) & kNib, sx.b2);
+    const float2 k0 = lds_f2(tq + (h0 << 3)), k1 = lds_f2(tq + (h1 << 3));     // h0, h1: headers of rows g and g + 8
+    // sum_i x_i X_i = sum_i u_i (2 X_i) + (parity - 16) sum_i X_i, limb pair by limb pair, in integers
+    const int e0 = __float_as_int(k0.y) * sx.xsum + (d[0] + 256 * d[1]);
+    const int e1 = __float_as_int(k1.y) * sx.xsum + (d[2] + 256 * d[3]);
+    if (FIRST) { r0 = (float)e0 * k0.x; r1 = (float)e1 * k1.x; }
+    else { r0 = fmaf((float)e0, k0.x, r0); r1 = fmaf((float)e1, k1.x, r1); }
+}
+
+// x (fp16) -> records.  X_i = rint(x_i * 2^F) with F chosen from the largest |x| so that |X_i| < 2^29; the
+// record of a block stores the four balanced limbs of 2 X_i (2 X_i = sum_l limb_l 256^l, limbs in -128..127)
+// plane by plane, and the block's sum of the X_i split in two, sum = s0 + 65536 s1.  An item is eight coordinates (one 128-bit piece of x): item e belongs to block e / 3.
+// The three items of a block add their shares of s0 and s1 with shared-memory atomics; the words were zeroed
+// before.  `rec` is the shared-memory address of the block's record.
+__device__ __forceinline__ void convert_item(const uint4 &v, int third, uint32_t rec, float scale) {
+    const uint32_t hv[4] = {v.x, v.y, v.z, v.w};
+    uint32_t w[8];
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&hv[i]));
+        const int z0 = __float2int_rn(f.x * scale), z1 = __float2int_rn(f.y * scale);
+        w[2 * i] = ((uint32_t)(2 * z0) + 0x80808080u) ^ 0x80808080u;       // bytes = balanced limbs of 2 X
+        w[2 * i + 1] = ((uint32_t)(2 * z1) + 0x80808080u) ^ 0x80808080u;
+    }
+    uint32_t pl[4][2];
+    int limb_sum[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int hlf = 0; hlf < 2; hlf++) {
+        const uint32_t a = w[4 * hlf], b = w[4 * hlf + 1], c = w[4 * hlf + 2], dd = w[4 * hlf + 3];
+        const uint32_t t0 = __byte_perm(a, b, 0x5140), t1 = __byte_perm(c, dd, 0x5140);   // limbs 0,1 of a,b / c,d
+        const uint32_t t2 = __byte_perm(a, b, 0x7362), t3 = __byte_perm(c, dd, 0x7362);   // limbs 2,3
+        pl[0][hlf] = __byte_perm(t0, t1, 0x5410); pl[1][hlf] = __byte_perm(t0, t1, 0x7632);
+        pl[2][hlf] = __byte_perm(t2, t3, 0x5410); pl[3][hlf] = __byte_perm(t2, t3, 0x7632);
+#pragma unroll
+        for (int l = 0; l < 4; l++) limb_sum[l] = __dp4a((int)pl[l][hlf], 0x01010101, limb_sum[l]);
+    }
+#pragma unroll
+    for (int l = 0; l < 4; l++)
+        asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(rec + 24 * l + 8 * third), "r"(pl[l][0]), "r"(pl[l][1]) : "memory");
+    // this item's sum of 2 X is a0 + 65536 a1; it is even, and so is a0; if a1 is odd one unit of it moves to
+    // a0, and then both halve exactly: the item adds a0 / 2 and a1 / 2 to the block's s0 and s1
+    int a0 = limb_sum[0] + 256 * limb_sum[1], a1 = limb_sum[2] + 256 * limb_sum[3];
+    a0 += (a1 & 1) << 16;
+    asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(rec + 100), "r"(a0 >> 1) : "memory");
+    asm volatile("red.shared.add.s32 [%0], %1;" ::"r"(rec + 104), "r"(a1 >> 1) : "memory");
+}
+
+// ---- the order of work.  A unit is a tile of a row group or its leftover blocks (column p.tiles).  Units
+// are numbered panel by panel: a panel is p.panel consecutive unit columns (the last panel may be narrower)
+// of every row group; inside a panel row group by row group, inside a row group by column.  The sequence is
+// cut into equal contiguous ranges, one per warp, warps numbered CTA by CTA: a CTA's range then lies in one
+// or two panels, so it needs only those panels' part of x, while a warp still meets several consecutive
+// units of one row group (a run), which it sums in registers.
+struct Cursor {
+    int panel, group, col, end;      // end = first column past the panel
+};
+// n / d for 0 <= n < 2^31, 0 < d: a float estimate and two fix-ups (a 32-bit integer division costs more than
+// everything else a warp does before it waits)
+__host__ __device__ inline int small_div(int n, int d) {
+#ifdef __CUDA_ARCH__
+    int q = (int)(__int2float_rz(n) * __frcp_rz(__int2float_ru(d)));       // never above the true quotient
+    int r = n - q * d;
+    while (r >= d) { q++; r -= d; }
+    return q;
+#else
+    return n / d;
+#endif
+}
+__host__ __device__ inline int panel_of_unit(const GemvParams &p, int f) {
+    const int j = small_div(f, p.total_groups * p.panel);
+    return j < p.npanels ? j : p.npanels - 1;
+}
+__device__ __forceinline__ Cursor locate(const GemvParams &p, int f) {
+    Cursor c;
+    c.panel = panel_of_unit(p, f);
+    const int first = c.panel * p.panel;
+    c.end = min(first + p.panel, p.units);
+    const int r = f - c.panel * (p.total_groups * p.panel), w = c.end - first;
+    c.group = small_div(r, w);
+    c.col = first + (r - c.group * w);
+    return c;
+}
+// steps over n units of the current row group's stretch; true if the row group changed
+__device__ __forceinline__ bool advance(const GemvParams &p, Cursor &c, int n) {
+    c.col += n;
+    if (c.col < c.end) return false;
+    c.group++;
+    if (c.group == p.total_groups) {
+        c.group = 0;
+        c.panel++;
+        c.end = min(c.end + p.panel, p.units);
+    }
+    c.col = c.panel * p.panel;
+    return true;
+}
+// first unit of warp gw when total = base * warps + rem units are dealt out, the first rem warps taking one more
+__host__ __device__ inline int first_unit_of_warp(int base, int rem, int gw) { return gw * base + (gw < rem ? gw : rem); }
+
 template <bool NO_WEIGHTS>
 __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
-    // shared memory: ring | per-matrix block constants (1024 x {scale * gain, parity}) | x | barriers
+    // shared memory: ring | per-matrix block constants (1024 x {gain / (4 sqrt m), parity - 16}) | x records | barriers
     unsigned char *ring = smem;
     float2 *tab = reinterpret_cast<float2 *>(smem + kWarps * kSlots * kTileBytes);
-    const uint4 *xs = reinterpret_cast<const uint4 *>(smem + kWarps * kSlots * kTileBytes + p.nprob * 8192);
-    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + kWarps * kSlots * kTileBytes + p.nprob * 8192 + ((p.nb * 48 + 127) / 128) * 128);
+    unsigned char *xrec = smem + kWarps * kSlots * kTileBytes + p.nprob * 8192;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(xrec + ((p.xblocks * kXRecBytes + 127) / 128) * 128);
     uint32_t *warp_max = reinterpret_cast<uint32_t *>(bars + kWarps * kSlots);     // one slot a warp
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t my_ring = smem_addr(ring + warp * kSlots * kTileBytes);
     const uint32_t my_bar = smem_addr(bars + warp * kSlots);
 
     LLVQ_TRACE_POINT(0)
-    // first the loads whose latency the rest of the prologue can cover: the class constants this
-    // thread will turn into block constants, and x on its way into L2 (its values are read only after
-    // the wait below, through L2, which is where the previous kernel's writes to x land)
-    const int tab_entries = p.nprob * 1024;
-    float2 cv[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-    for (int i = 0; i < 2; i++)
-        if (tid + i * kThreads < tab_entries) cv[i] = __ldg(p.cls_pack + ((tid + i * kThreads) & 511));
-    for (int e = tid * 128; e < p.nb * 48; e += kThreads * 128) {
-        // a load whose value is thrown away: it brings the line into L2 and the translation into this
-        // multiprocessor's TLB, which a prefetch hint does not promise
-        uint32_t ignored;
-        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(ignored) : "l"(reinterpret_cast<const char *>(p.x) + e));
-    }
-    // a warp's barriers are used by that warp alone: no block-wide synchronisation is needed for them
+    // a warp's barriers are used by that warp alone: no block-wide synchronisation is needed for them; they
+    // are set up before any load is in flight, so that the fence has nothing to wait for
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kSlots; s++) mbar_init(my_bar + 8 * s, 1);
@@ -279,43 +434,98 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     }
     __syncwarp();
 
-    int u0, n_units;
-    warp_range(p, warp, u0, n_units);
-    // consume side: row group and unit inside it; issue side: a running source pointer
-    int group = u0 / p.units, k = u0 - group * p.units, q = 0;
-    const uint8_t *src = nullptr;
-    int ik = k, igroup = group, issued = 0;
-    if (n_units > 0) src = group_base(p, group, kCellBytes, q) + (size_t)(k < p.tiles ? k : p.tiles) * kTileBytes;
+    // then the loads whose latency the rest of the prologue can cover:
+    // the class constants this
+    // thread will turn into block constants, and x on its way into L2 (its values are read only after
+    // the wait below, through L2, which is where the previous kernel's writes to x land)
+    const int tab_entries = p.nprob * 1024;
+    float2 cv[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+    for (int i = 0; i < 2; i++)
+        if (tid + i * kThreads < tab_entries) cv[i] = __ldg(p.cls_pack + ((tid + i * kThreads) & 511));
+    uint32_t warm = 0;
+    for (int e = tid * 128; e < p.nb * 48; e += kThreads * 128) {
+        // a load whose value is not used: it brings the line into L2 and the translation into this
+        // multiprocessor's TLB, which a prefetch hint does not promise.  The register stays claimed until
+        // after the wait (settled() below), so nothing stalls on the load's return before then.
+        uint32_t w;
+        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(w) : "l"(reinterpret_cast<const char *>(p.x) + e));
+        warm |= w;
+    }
+    // this warp's units, and the blocks of x this CTA's units touch
+    const int gw = blockIdx.x * kWarps + warp;
+    const int u0 = first_unit_of_warp(p.units_base, p.units_rem, gw);
+    const int n_units = p.units_base + (gw < p.units_rem ? 1 : 0);
+    const int cta_u0 = first_unit_of_warp(p.units_base, p.units_rem, blockIdx.x * kWarps);
+    const int cta_u1 = first_unit_of_warp(p.units_base, p.units_rem, (blockIdx.x + 1) * kWarps);
+    const int blk_lo = panel_of_unit(p, cta_u0) * p.panel * kTileCells;
+    const int blk_hi = min(p.nb, (panel_of_unit(p, max(cta_u1 - 1, cta_u0)) + 1) * p.panel * kTileCells);
+    const uint32_t xs0 = smem_addr(xrec) - (uint32_t)blk_lo * kXRecBytes;     // address of block 0's record, were it there
+
+    // consume side and issue side walk the same sequence of units
+    Cursor cc = locate(p, u0), ic = cc;
+    int q = 0;
+    const uint8_t *isrc = nullptr;                     // first byte of the issue side's row group
+    if (n_units > 0) isrc = group_base(p, ic.group, kCellBytes, q);
     const uint32_t tail_bytes = (uint32_t)p.tail_cells * kCellBytes;
 
     // issue the copy of the next unit (lane 0 alone, by predicate) onto barrier `b` and buffer `dst`,
     // then step the source
+    // The issue side's walk: inext is the next unit's first byte, ileft the units left in its stretch of its
+    // row group.  next() hands out the unit's source and size and steps on.
+    struct Walk {
+        Cursor c;
+        const uint8_t *next;
+        int left, done;
+    };
+    const int n_tiles_total = p.tiles;
+    Walk iw;
+    iw.c = ic;
+    iw.next = isrc + (size_t)ic.col * kTileBytes;      // the leftover blocks follow the last tile
+    iw.left = ic.end - ic.col;
+    iw.done = 0;
+    auto walk_next = [&](Walk &w, const uint8_t *&src, uint32_t &bytes) {
+        src = w.next;
+        bytes = w.c.col < n_tiles_total ? (uint32_t)kTileBytes : tail_bytes;
+        w.done++;
+        w.next += kTileBytes;
+        w.c.col++;
+        if (--w.left == 0) {                           // rare: the stretch ends, the next one starts elsewhere
+            w.c.col--;
+            advance(p, w.c, 1);
+            if (w.done < n_units) {
+                int qi;
+                w.next = group_base(p, w.c.group, kCellBytes, qi) + (size_t)w.c.col * kTileBytes;
+            }
+            w.left = w.c.end - w.c.col;
+        }
+    };
+    // issue the copy of the next unit (lane 0 alone, by predicate) onto barrier `b` and buffer `dst`
+    const int my_issues = lane == 0 ? n_units : 0;     // lanes other than 0 never issue
     auto issue = [&](uint32_t b, uint32_t dst) {
-        const uint32_t bytes = ik < p.tiles ? (uint32_t)kTileBytes : tail_bytes;
+        const int done = iw.done;
+        const uint8_t *src;
+        uint32_t bytes;
+        walk_next(iw, src, bytes);
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "setp.eq.u32 p, %0, 0;\n\t"
-            "@p mbarrier.arrive.expect_tx.shared::cta.b64 _, [%1], %2;\n\t"
-            "@p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%3], [%4], %2, [%1];\n\t}"
-            ::"r"(lane), "r"(b), "r"(bytes), "r"(dst), "l"(src));
+            "setp.lt.s32 p, %0, %1;\n\t"
+            "@p mbarrier.arrive.expect_tx.shared::cta.b64 _, [%2], %3;\n\t"
+            "@p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%4], [%5], %3, [%2];\n\t}"
+            ::"r"(done), "r"(my_issues), "r"(b), "r"(bytes), "r"(dst), "l"(src));
         // No "memory" clobber: the only memory the copy writes is the slot, whose last reads feed
         // `dst` through settled() and whose next reads follow the next wait on `b`; a clobber here
         // would pin every shared-memory read of the decode behind the copy.
-        issued++;
-        src += bytes;                                  // a row group's units are contiguous, and so are a matrix's row groups
-        if (++ik == p.units) {
-            ik = 0;
-            igroup++;
-            if (igroup < p.total_groups && issued < n_units) { int qi; src = group_base(p, igroup, kCellBytes, qi); }
-        }
     };
 
     if (!NO_WEIGHTS) {
 #pragma unroll
-        for (int s = 0; s < kSlots; s++)
-            if (issued < n_units) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
+        for (int s = 0; s < kSlots; s++) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
     }
-    // block constants of every matrix of the launch: (class | gain << 9) -> {gain * 2^21 / (4 sqrt m), parity pattern}
+    // the zero word and the two sums of every x record this CTA will fill
+    for (int b = tid; b < blk_hi - blk_lo; b += kThreads)
+        asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(smem_addr(xrec) + b * kXRecBytes + 96), "r"(0) : "memory");
+    // block constants of every matrix of the launch: (class | gain << 9) -> {gain / (4 sqrt m), parity - 16}
     for (int e = tid, i = 0; e < tab_entries; e += kThreads, i++) {
         const float2 v = i < 2 ? cv[i] : __ldg(p.cls_pack + (e & 511));
         const GemvProblemDev &pe = p.prob[e >> 10];
@@ -328,17 +538,19 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     asm volatile("griddepcontrol.wait;" ::: "memory");
     LLVQ_TRACE_POINT(2)
     LLVQ_TRACE_CLOCK(0)
-    // x into shared memory, every thread a 16-byte piece (L2 hits after the prefetch), and on the way
-    // the largest |x|: every |x| is below 2^(e-14), e the biased exponent of the largest magnitude
-    // (fp16 bit patterns of non-negative values order like integers)
+    // One pass over x finds the largest |x| (fp16 bit patterns of non-negative values order like integers):
+    // every |x| is below 2^xexp, xexp = e - 14 with e the biased exponent of the largest magnitude.  The
+    // pieces of x this CTA needs stay in registers meanwhile and then become fixed-point records on the scale
+    // 2^(29 - xexp).
     bool failed = false;
     int xexp;
     {
-        uint32_t m = 0;
+        uint32_t m = settled(warm, warm, warm);
         const uint4 *xg = reinterpret_cast<const uint4 *>(p.x);
-        uint4 *xw = const_cast<uint4 *>(xs);
-        // all of a thread's loads go out before the first store, so their latencies overlap
-        const int nx = p.nb * 3;
+        const int nx = p.nb * 3, e_lo = 3 * blk_lo, e_hi = 3 * blk_hi;
+        const bool one_each = e_hi - e_lo <= kThreads;         // then no thread meets two of the pieces wanted
+        uint4 mine = make_uint4(0u, 0u, 0u, 0u);
+        int mine_e = -1;
         for (int base = 0; base < nx; base += 4 * kThreads) {
             uint4 v[4];
 #pragma unroll
@@ -349,17 +561,24 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
 #pragma unroll
             for (int i = 0; i < 4; i++) {
                 const int e = base + i * kThreads + tid;
-                if (e < nx) xw[e] = v[i];
                 m = max_abs_pair(max_abs_pair(max_abs_pair(max_abs_pair(m, v[i].x), v[i].y), v[i].z), v[i].w);
+                if (e >= e_lo && e < e_hi) { mine = v[i]; mine_e = e; }
             }
         }
-        LLVQ_TRACE_POINT(4)
-        LLVQ_TRACE_CLOCK(1)
         m = __reduce_max_sync(0xffffffffu, max(m & 0xffffu, m >> 16));
-        if (lane == 0) warp_max[warp] = m;             // plain stores: atomics on one word would serialise the warps
-        __syncthreads();                               // publishes x, the maxima and the block constants
+            if (lane == 0) warp_max[warp] = m;             // plain stores: atomics on one word would serialise the warps
+        __syncthreads();                               // publishes the maxima, the block constants and the zeroed sums
         m = warp_max[lane < kWarps ? lane : 0];
         xexp = max((int)(__reduce_max_sync(0xffffffffu, m) >> 10), 1) - 14;
+        LLVQ_TRACE_POINT(4)
+        LLVQ_TRACE_CLOCK(1)
+        const float scale = pow2f(29 - xexp);
+        if (one_each) {
+            if (mine_e >= 0) convert_item(mine, mine_e % 3, xs0 + (uint32_t)(mine_e / 3) * kXRecBytes, scale);
+        } else {
+            for (int e = e_lo + tid; e < e_hi; e += kThreads) convert_item(__ldcg(xg + e), e % 3, xs0 + (uint32_t)(e / 3) * kXRecBytes, scale);
+        }
+        __syncthreads();                               // publishes the x records
     }
     LLVQ_TRACE_POINT(3)
     LLVQ_TRACE_CLOCK(2)
@@ -369,52 +588,76 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     uint32_t bar = my_bar;                             // barrier and buffer of the slot that is consumed next
     uint32_t sbuf = my_ring;
     const uint32_t sbuf_end = my_ring + kSlots * kTileBytes;
-    const uint32_t lane16 = 16 * lane, lane8 = 8 * lane;
-    const int tiles = p.tiles, units = p.units;
+    const uint32_t lane16 = 16 * lane, lane4 = 4 * lane, pair16 = 16 * (lane >> 1);
+    const int tiles = p.tiles;
+    const LaneOffsets lo = lane_offsets(lane, false);
+    const bool odd_lane = lane & 1, high_lane = lane & 2;
+    const float limb_scale = odd_lane ? 65536.f : 1.f;     // this lane's limb pair: 256^0,1 or 256^2,3
+    const int my_row = (lane >> 2) + 8 * (lane & 3);       // the row of the group this lane ends up with
+    const uint32_t tab0 = smem_addr(tab);
+    q = n_units > 0 ? find_problem(p, cc.group) : 0;
 
+    // Sums the quad's shares: acc[r] of lane 4g+t is the share of row g + 8r; afterwards lane 4g+t
+    // holds the whole sum of row g + 8t.  Fixed order, so the result does not depend on the launch.
+    auto quad_sum = [&](const float (&acc)[4]) -> float {
+        const float send0 = high_lane ? acc[0] : acc[2], send1 = high_lane ? acc[1] : acc[3];
+        const float keep0 = high_lane ? acc[2] : acc[0], keep1 = high_lane ? acc[3] : acc[1];
+        const float r0 = (keep0 + __shfl_xor_sync(0xffffffffu, send0, 2)) * limb_scale;
+        const float r1 = (keep1 + __shfl_xor_sync(0xffffffffu, send1, 2)) * limb_scale;
+        return (odd_lane ? r1 : r0) + __shfl_xor_sync(0xffffffffu, odd_lane ? r0 : r1, 1);
+    };
+
+    Handed handed;
+    handed.slot = nullptr;
     // A run is the stretch of units of one row group inside this warp's range: its units are summed
     // in a register and handed over together.
-    while (n < n_units && !failed) {
+    while (n < n_units) {
         const GemvProblemDev &pr = p.prob[q];
+        // quantum of the row accumulator: 2^qexp in units of y / row_scale; a lane's sums are in units of 2^(xexp - 29)
         const int qexp = xexp + pr.qexp_base;
-        const float inv_q = pow2f(-qexp);
-        const float2 *tq = tab + q * 1024;
-        const int run = min(units - k, n_units - n);
-        const int run_tiles = NO_WEIGHTS ? 0 : max(0, min(run, tiles - k));
+        const float inv_q = pow2f(-29 - pr.qexp_base);
+        const uint32_t tq = tab0 + q * 8192;
+        const int run = min(cc.end - cc.col, n_units - n);
+        const int run_tiles = NO_WEIGHTS ? 0 : max(0, min(run, tiles - cc.col));
         // the row's scale is needed only by the arrival that finishes the row, but loading it now
         // keeps a cold read off the tail of the kernel
-        const int row = (group - pr.group_begin) * kRowsPerGroup + lane;
+        const int row = (cc.group - pr.group_begin) * kRowsPerGroup + my_row;
         const float row_scale = row < pr.rows ? __half2float(pr.row_scale[row]) : 0.f;
-        const uint4 *xc = xs + 12 * k;
+        // this lane's addresses in the x records of the run's first tile
+        const uint32_t xk = xs0 + (uint32_t)cc.col * (4 * kXRecBytes);
+        LaneOffsets xa = {xk + lo.b0, xk + lo.b1, xk + lo.b2, xk + lo.xs};
         long long sum = 0;
 
-        for (int t = 0; t < run_tiles; t++, xc += 12) {
+#pragma unroll 1
+        for (int t = 0; t < run_tiles; t++) {
             LLVQ_TRACE_UNIT(n + t, 0)
-            if (!mbar_wait(bar, parity)) { failed = true; break; }
+            if (!mbar_try(bar, parity)) {
+                if (!mbar_wait(bar, parity)) { failed = true; break; }
+            }
             LLVQ_TRACE_UNIT(n + t, 1)
             const uint4 a0 = lds128(sbuf + lane16);
             const uint4 a1 = lds128(sbuf + lane16 + 512);
             const uint4 a2 = lds128(sbuf + lane16 + 1024);
-            const uint2 hh = lds64(sbuf + lane8 + 1536);
-            const uint32_t w0[4] = {a0.x, a0.y, a0.z, a0.w}, w1[4] = {a1.x, a1.y, a1.z, a1.w}, w2[4] = {a2.x, a2.y, a2.z, a2.w};
-            const uint32_t hd[4] = {hh.x & 0xffffu, hh.x >> 16, hh.y & 0xffffu, hh.y >> 16};
+            const uint4 hh = lds128(sbuf + pair16 + 1536);
             // The slot's words are in registers: refill it at once with the unit kSlots ahead, so
             // that every slot but the one just read is in flight while this unit is decoded.  The
             // copy's address is made to depend on the loaded words, which holds the copy back
             // until the four shared-memory reads of the whole warp have completed.
-            if (issued < n_units) issue(bar, sbuf + (settled(a0.w, a1.w, a2.w) | settled(hh.y, hh.x, a0.x)));
-            float s = 0.f;
-#pragma unroll
-            for (int c = 0; c < 4; c++) {
+            issue(bar, sbuf + (settled(a0.w, a1.w, a2.w) | settled(hh.w, hh.x, a0.x)));
+            float acc[4];
 #ifdef LLVQ_STREAM_ONLY
-                s += __uint_as_float((w0[c] ^ w1[c] ^ w2[c] ^ hd[c]) & 0x007fffffu);   // debug: bytes only, no decode
+            acc[0] = __uint_as_float((a0.x ^ a1.y ^ a2.z ^ hh.w) & 0x007fffffu);   // debug: bytes only, no decode
+            acc[1] = acc[2] = acc[3] = 0.f;
 #else
-                const float2 kc = tq[hd[c]];           // header bits 10..15 are zero
-                s = fmaf(kc.x, block_dot(w0[c], w1[c], w2[c], __float_as_uint(kc.y), xc + 3 * c), s);
+            const StepX s0 = load_step<0>(xa), s1 = load_step<2 * kXRecBytes>(xa);
+            half_step<true>(a0.x, a0.y, a0.z, hh.x & 0xffffu, hh.x >> 16, s0, tq, acc[0], acc[1]);
+            half_step<true>(a0.w, a1.x, a1.y, hh.y & 0xffffu, hh.y >> 16, s0, tq, acc[2], acc[3]);
+            half_step<false>(a1.z, a1.w, a2.x, hh.z & 0xffffu, hh.z >> 16, s1, tq, acc[0], acc[1]);
+            half_step<false>(a2.y, a2.z, a2.w, hh.w & 0xffffu, hh.w >> 16, s1, tq, acc[2], acc[3]);
 #endif
-            }
-            sum += __float2ll_rn(s * inv_q);
+            sum += __float2ll_rn(quad_sum(acc) * inv_q);
             LLVQ_TRACE_UNIT(n + t, 2)
+            xa.b0 += 4 * kXRecBytes; xa.b1 += 4 * kXRecBytes; xa.b2 += 4 * kXRecBytes; xa.xs += 4 * kXRecBytes;
             bar += 8;
             sbuf += kTileBytes;
             const bool wrap = sbuf == sbuf_end;        // every slot completes once a round
@@ -424,46 +667,57 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         }
         if (failed) break;
         if (!NO_WEIGHTS && run_tiles < run) {
-            // the run ends with the nb mod 4 last block columns of the row group: one cell at a time
+            // the run ends with the nb mod 4 last block columns of the row group: a pair, a single, or both
             if (!mbar_wait(bar, parity)) { failed = true; break; }
-            uint32_t guard = 0;
-            const uint4 *xt = xs + 12 * tiles;
-            float s = 0.f;
-#pragma unroll 1
-            for (int c = 0; c < p.tail_cells; c++) {
-                const uint32_t cell = sbuf + c * kCellBytes;
-                const uint32_t t0 = lds32(cell + 4 * lane);
-                const uint32_t t1 = lds32(cell + 128 + 4 * lane);
-                const uint32_t t2 = lds32(cell + 256 + 4 * lane);
-                const uint32_t th = lds16(cell + 384 + 2 * lane);
-                guard |= settled(t0, t1, t2) | settled(th, t0, t1);
-                const float2 kc = tq[th];
-                s = fmaf(kc.x, block_dot(t0, t1, t2, __float_as_uint(kc.y), xt + 3 * c), s);
+            uint32_t guard = 0, piece = sbuf;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint32_t xt = xs0 + (uint32_t)tiles * (4 * kXRecBytes);
+            if (p.tail_cells >= 2) {
+                const LaneOffsets ta = {xt + lo.b0, xt + lo.b1, xt + lo.b2, xt + lo.xs};
+                const StepX st = load_step<0>(ta);
+#pragma unroll
+                for (int m = 0; m < 2; m++) {
+                    const uint32_t wa = lds32(piece + 128 * (3 * m) + lane4), wb = lds32(piece + 128 * (3 * m + 1) + lane4);
+                    const uint32_t wc = lds32(piece + 128 * (3 * m + 2) + lane4), hw = lds32(piece + 768 + 8 * (lane >> 1) + 4 * m);
+                    guard |= settled(wa, wb, wc) | settled(hw, wa, wb);
+                    half_step<false>(wa, wb, wc, hw & 0xffffu, hw >> 16, st, tq, acc[2 * m], acc[2 * m + 1]);
+                }
+                piece += 2 * kCellBytes;
             }
-            if (issued < n_units) issue(bar, sbuf + guard);
-            sum += __float2ll_rn(s * inv_q);
+            if (p.tail_cells & 1) {
+                // one block: the slots of this half-step are the two halves of the row group
+                const uint32_t xl = xs0 + (uint32_t)(p.nb - 1) * kXRecBytes;
+                const LaneOffsets l1 = lane_offsets(lane, true);
+                const LaneOffsets ta = {xl + l1.b0, xl + l1.b1, xl + l1.b2, xl + l1.xs};
+                const StepX st = load_step<0>(ta);
+                const uint32_t wa = lds32(piece + lane4), wb = lds32(piece + 128 + lane4);
+                const uint32_t wc = lds32(piece + 256 + lane4), hw = lds32(piece + 384 + 4 * (lane >> 1));
+                guard |= settled(wa, wb, wc) | settled(hw, wa, wb);
+                float c0, c1;
+                half_step<true>(wa, wb, wc, hw & 0xffffu, hw >> 16, st, tq, c0, c1);
+                acc[0] += high_lane ? 0.f : c0; acc[1] += high_lane ? 0.f : c1;
+                acc[2] += high_lane ? c0 : 0.f; acc[3] += high_lane ? c1 : 0.f;
+            }
+            issue(bar, sbuf + guard);
+            sum += __float2ll_rn(quad_sum(acc) * inv_q);
             bar += 8;
             sbuf += kTileBytes;
             if (sbuf == sbuf_end) { sbuf = my_ring; bar = my_bar; parity ^= 1u; }
         }
         // with no records read (the control launch) every unit contributes zero
         n += run;
-        k += run;
         if (n == n_units) { LLVQ_TRACE_POINT(6) }
-        deliver(p, pr, group, lane, sum, run, qexp, row_scale);
-        if (k == units) {
-            k = 0;
-            group++;
-            if (group < p.total_groups) q = find_problem(p, group);
-        }
+        hand_over(p, pr, cc.group, my_row, sum, run, qexp, row_scale, handed);
+        if (advance(p, cc, run) && cc.panel < p.npanels) q = find_problem(p, cc.group);
     }
+    settle(p, handed);
 
     LLVQ_TRACE_POINT(5)
     if (failed) {
         // a wait ran out: report it, then give the copies still in flight a bounded chance to land
         // (a slot that is not pending returns at once or runs into the same bound)
         if (lane == 0) atomicExch(p.error, 1);
-        for (int s = 0; s < kSlots && s < issued; s++) mbar_wait(my_bar + 8 * s, parity);
+        for (int s = 0; s < kSlots && s < min(iw.done, n_units); s++) mbar_wait(my_bar + 8 * s, parity);
     }
 }
 
@@ -564,20 +818,44 @@ __global__ void __launch_bounds__(256) gemv_fp16_kernel(const __half *__restrict
     if (lane == 0) y[row] = s;
 }
 
-// ---- helpers reading a record back: thread = (row group, block column, lane)
-__device__ __forceinline__ void read_planes_record(const uint8_t *buf, int64_t nb, int64_t rg, int64_t b, int lane,
-                                                   uint32_t w[3], uint32_t &hdr) {
-    const int64_t tiles = nb / kTileCells;
+// ---- helpers reading a record back: thread = (row group, block column, row of the group)
+// The 24 codes (c[j] = codes of coordinates 8j..8j+7, a nibble each) and the header of one block of one row,
+// found from the layout's description in include/llvq.h: which piece, half-step, lane, word and nibble.
+__device__ __forceinline__ void read_planes_record(const uint8_t *buf, int64_t nb, int64_t rg, int64_t b, int r,
+                                                   uint32_t c[3], uint32_t &hdr) {
+    const int64_t tiles = nb / kTileCells, left = nb % kTileCells;
     const uint8_t *grp = buf + (size_t)rg * (size_t)nb * kCellBytes;
-    if (b < tiles * kTileCells) {
-        const uint8_t *tile = grp + (size_t)(b / kTileCells) * kTileBytes;
-        const int q = (int)(b % kTileCells);
-        for (int j = 0; j < 3; j++) w[j] = *reinterpret_cast<const uint32_t *>(tile + 512 * j + 16 * lane + 4 * q);
-        hdr = *reinterpret_cast<const uint16_t *>(tile + 1536 + 8 * lane + 2 * q);
+    const int m = r >> 4, e = (r >> 3) & 1, g = r & 7;
+    const int64_t j = b - tiles * kTileCells;
+    const uint8_t *base;
+    int slot, kind, h = 0;                         // kind 0 tile, 1 pair, 2 single
+    if (j < 0) {
+        base = grp + (size_t)(b / kTileCells) * kTileBytes;
+        slot = (int)(b & 1); h = 2 * (int)((b % kTileCells) >> 1) + m; kind = 0;
+    } else if (left >= 2 && j < 2) {
+        base = grp + (size_t)tiles * kTileBytes; slot = (int)j; kind = 1;
     } else {
-        const uint8_t *cell = grp + (size_t)tiles * kTileBytes + (size_t)(b - tiles * kTileCells) * kCellBytes;
-        for (int j = 0; j < 3; j++) w[j] = *reinterpret_cast<const uint32_t *>(cell + 128 * j + 4 * lane);
-        hdr = *reinterpret_cast<const uint16_t *>(cell + 384 + 2 * lane);
+        base = grp + (size_t)tiles * kTileBytes + (left == 3 ? 2 * kCellBytes : 0); slot = m; kind = 2;
+    }
+    auto word = [&](int q, int lane) -> uint32_t {
+        const int k = 3 * h + q;
+        const uint8_t *a = kind == 0 ? base + 512 * (k >> 2) + 16 * lane + 4 * (k & 3)
+                         : kind == 1 ? base + 128 * (3 * m + q) + 4 * lane
+                                     : base + 128 * q + 4 * lane;
+        return *reinterpret_cast<const uint32_t *>(a);
+    };
+    const int pair = 2 * g + slot;
+    const uint32_t hw = *reinterpret_cast<const uint32_t *>(kind == 0 ? base + 1536 + 16 * pair + 4 * h
+                                                            : kind == 1 ? base + 768 + 8 * pair + 4 * m
+                                                                        : base + 384 + 4 * pair);
+    hdr = (hw >> (16 * e)) & 0xffffu;
+    c[0] = c[1] = c[2] = 0;
+    for (int i = 0; i < 24; i++) {
+        const int kappa = 24 * slot + i;
+        uint32_t w; int nib;
+        if (kappa < 32) { w = word(e, 4 * g + ((kappa & 15) >> 2)); nib = 2 * (kappa & 3) + (kappa >> 4); }
+        else { w = word(2, 4 * g + ((kappa - 32) >> 2)); nib = 2 * (kappa & 3) + e; }
+        c[i >> 3] |= ((w >> (4 * nib)) & 15u) << (4 * (i & 7));
     }
 }
 
@@ -585,17 +863,11 @@ __device__ __forceinline__ void read_planes_record(const uint8_t *buf, int64_t n
 __device__ __forceinline__ void record_coords(int layout, const uint8_t *buf, int64_t nb, int64_t rg, int64_t b, int lane,
                                               const uint32_t *cls_parity, const uint8_t *cls_dist, int &cls, int &gain, int x[24]) {
     if (layout == LLVQ_PLANES) {
-        uint32_t w[3], hdr;
-        read_planes_record(buf, nb, rg, b, lane, w, hdr);
+        uint32_t c[3], hdr;
+        read_planes_record(buf, nb, rg, b, lane, c, hdr);
         cls = (int)(hdr & 511u); gain = (int)((hdr >> 9) & 1u);
         const int par = cls_parity[cls] ? 1 : 0;
-        for (int i = 0; i < 24; i++) {
-            const int j = i >> 3, k = (i & 7) >> 1, e = i & 1;
-            const uint32_t r = __funnelshift_r(w[j], w[j], 4 * k);
-            const int level = (int)((r >> (4 + 16 * e)) & 7u);
-            const int a = (cls == kEmptyClass) ? 0 : 2 * level + par;
-            x[i] = ((r >> (15 + 16 * e)) & 1u) ? -a : a;
-        }
+        for (int i = 0; i < 24; i++) x[i] = 2 * ((int)((c[i >> 3] >> (4 * (i & 7))) & 15u) - 8) + par;
     } else {
         const uint32_t *cell = reinterpret_cast<const uint32_t *>(buf + ((size_t)rg * (size_t)nb + (size_t)b) * kOneHotCellBytes);
         uint32_t v[5];
@@ -646,10 +918,32 @@ __global__ void __launch_bounds__(256) dequant_kernel(int layout, const uint8_t 
 
 }  // namespace
 
-size_t gemv_smem_bytes(int layout, int nb, int nprob) {
-    const size_t xbytes = ((size_t)nb * 48 + 127) / 128 * 128;
-    if (layout != LLVQ_PLANES) return xbytes;
-    return (size_t)kWarps * kSlots * kTileBytes + (size_t)nprob * 8192 + xbytes + kWarps * kSlots * 8 + kWarps * 4 + 16;
+GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
+    GemvLaunch g;
+    // one CTA a multiprocessor
+    g.grid = p.total_units < sm_count ? p.total_units : sm_count;
+    p.units_base = p.total_units / (g.grid * kWarps);
+    p.units_rem = p.total_units % (g.grid * kWarps);
+    if (layout != LLVQ_PLANES) {
+        g.smem = ((size_t)p.nb * 48 + 127) / 128 * 128;
+        return g;
+    }
+    // panels of about sixteen unit columns, as equal as they come
+    const int want = (p.units + 8) / 16 > 1 ? (p.units + 8) / 16 : 1;
+    p.panel = (p.units + want - 1) / want;
+    p.npanels = (p.units + p.panel - 1) / p.panel;
+    // the widest stretch of x a CTA meets: its units lie in consecutive panels
+    p.xblocks = 0;
+    for (int c = 0; c < g.grid; c++) {
+        const int f0 = first_unit_of_warp(p.units_base, p.units_rem, c * kWarps), f1 = first_unit_of_warp(p.units_base, p.units_rem, (c + 1) * kWarps);
+        const int lo = panel_of_unit(p, f0) * p.panel * kTileCells;
+        int hi = (panel_of_unit(p, f1 - 1 > f0 ? f1 - 1 : f0) + 1) * p.panel * kTileCells;
+        if (hi > p.nb) hi = p.nb;
+        if (hi - lo > p.xblocks) p.xblocks = hi - lo;
+    }
+    const size_t xbytes = ((size_t)p.xblocks * kXRecBytes + 127) / 128 * 128;
+    g.smem = (size_t)kWarps * kSlots * kTileBytes + (size_t)p.nprob * 8192 + xbytes + kWarps * kSlots * 8 + kWarps * 4 + 16;
+    return g;
 }
 
 template <typename K>
@@ -670,20 +964,15 @@ int gemv_configure(const llvq_ctx *ctx) {
     return 0;
 }
 
-cudaError_t launch_gemv(const llvq_ctx *ctx, int layout, GemvParams &p, bool no_weights, cudaStream_t s) {
-    const size_t smem = gemv_smem_bytes(layout, p.nb, p.nprob);
-    // one CTA a multiprocessor (warps are numbered CTA-first, so a short launch spreads over all of them)
-    int grid = p.total_units < ctx->sm_count ? p.total_units : ctx->sm_count;
-    p.units_base = p.total_units / (grid * kWarps);
-    p.units_rem = p.total_units % (grid * kWarps);
+cudaError_t launch_gemv(int layout, const GemvParams &p, const GemvLaunch &g, bool no_weights, bool pdl, cudaStream_t s) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid);
+    cfg.gridDim = dim3((unsigned)g.grid);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
+    cfg.dynamicSmemBytes = g.smem;
     cfg.stream = s;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = ctx->use_pdl ? 1 : 0;
+    attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (layout == LLVQ_PLANES) {
@@ -829,21 +1118,8 @@ extern "C" int llvq_gemv_static(const void *layout_buf, const void *row_scale, c
     p.accum = d.accum;
     p.cls_pack = d.cls_pack;
     p.error = d.error;
-    const size_t smem = gemv_smem_bytes(LLVQ_PLANES, p.nb, 1);
-    if (smem + 1024 > (size_t)d.max_smem_optin) return LLVQ_ESIZE;
-    int grid = p.total_units < d.sm_count ? p.total_units : d.sm_count;
-    p.units_base = p.total_units / (grid * kWarps);
-    p.units_rem = p.total_units % (grid * kWarps);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = (cudaStream_t)stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false>, p) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+    const llvq::GemvLaunch g = llvq::gemv_plan(LLVQ_PLANES, p, d.sm_count);
+    if (g.smem + 1024 > (size_t)d.max_smem_optin) return LLVQ_ESIZE;
+    return llvq::launch_gemv(LLVQ_PLANES, p, g, false, true, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
 }
 

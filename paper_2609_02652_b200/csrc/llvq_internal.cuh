@@ -10,7 +10,7 @@
 
 namespace llvq {
 
-// Geometry of the bit-plane layout (see include/llvq.h).
+// Geometry of the 14-byte layout (see include/llvq.h).
 constexpr int kRowsPerGroup = 32;
 constexpr int kCellBytes = 448;        // 32 rows x 14 bytes
 constexpr int kTileCells = 4;
@@ -26,7 +26,7 @@ struct DeviceTables {
     const uint32_t *cls_parity;      // 512
     const float *cls_value;          // 512 x 8
     const uint8_t *cls_dist;         // 512 x 8
-    const float2 *cls_pack;          // 512 x {scale, parity bits}
+    const float2 *cls_pack;          // 512 x {1 / (4 sqrt m), int parity - 16 as bits}
     int weight_offset[25];
     int num_classes;
     uint64_t num_points;
@@ -50,12 +50,14 @@ struct GemvParams {
     int units;             // units a row group: tiles, plus one for the nb mod 4 last columns
     int total_groups;
     int total_units;       // total_groups * units
-    int units_base, units_rem;   // total_units divided by the warps of the grid (set at launch)
+    int units_base, units_rem;   // total_units divided by the warps of the grid (set by gemv_plan; the one-hot arm's order)
+    int panel, npanels;          // unit columns a panel, panels (set by gemv_plan; the 14-byte layout's order of work)
+    int xblocks;                 // most blocks of x any CTA needs (set by gemv_plan)
     unsigned long long *accum;   // total_groups x 32 fixed-point row accumulators (context scratch, zero between launches)
     const float *cls_scale;
     const uint32_t *cls_parity;
     const float *cls_value;
-    const float2 *cls_pack;   // 512 x {2^21 / (4 sqrt m), parity pattern as bits}
+    const float2 *cls_pack;   // 512 x {1 / (4 sqrt m), int parity - 16 as bits}
     int *error;               // set when a bounded wait ran out
 #ifdef LLVQ_TRACE
     unsigned long long *trace;   // timeline buffer (debug builds only)
@@ -85,13 +87,18 @@ struct llvq_ctx {
 namespace llvq {
 cudaError_t launch_expand(const llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, int64_t nb,
                           void *out, uint32_t *bad_count, cudaStream_t s);
-cudaError_t launch_gemv(const llvq_ctx *ctx, int layout, GemvParams &p, bool no_weights, cudaStream_t s);
+struct GemvLaunch {
+    int grid;
+    size_t smem;
+};
+// Completes the launch geometry in `p` (order of work, shares of x) and returns grid and dynamic shared memory.
+GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count);
+cudaError_t launch_gemv(int layout, const GemvParams &p, const GemvLaunch &g, bool no_weights, bool pdl, cudaStream_t s);
 cudaError_t launch_wait_limit_selftest(const llvq_ctx *ctx, cudaStream_t s);
 cudaError_t launch_gemv_fp16(const __half *W, const __half *x, float *y, int64_t rows, int64_t k, cudaStream_t s);
 cudaError_t launch_dequant(const llvq_ctx *ctx, int layout, const uint8_t *buf, const __half *row_scale, float g0, float g1,
                            __half *W, int64_t rows, int64_t nb, cudaStream_t s);
 cudaError_t launch_decode_i8(const llvq_ctx *ctx, int layout, const uint8_t *buf, int8_t *coords, uint16_t *class_ids,
                              int64_t rows, int64_t nb, cudaStream_t s);
-size_t gemv_smem_bytes(int layout, int nb, int nprob);
 int gemv_configure(const llvq_ctx *ctx);   // sets the kernels' shared-memory attributes once
 }  // namespace llvq

@@ -174,8 +174,10 @@ bool build_tables(HostTables &t) {
     }
     t.cls_pack.assign(kClassSlots * 2, 0u);
     for (int c = 0; c < kClassSlots; c++) {
-        std::memcpy(&t.cls_pack[2 * c], &t.cls_scale[c], 4);
-        t.cls_pack[2 * c + 1] = t.cls_parity[c];
+        const float inv_norm = t.cls_scale[c] * (1.0f / 2097152.0f);      // exact: a power of two
+        std::memcpy(&t.cls_pack[2 * c], &inv_norm, 4);
+        const int32_t offset = t.cls_scale[c] != 0.f ? (t.cls_parity[c] ? 1 : 0) - 16 : 0;   // x_i = 2 u_i + offset
+        std::memcpy(&t.cls_pack[2 * c + 1], &offset, 4);
     }
     t.base[all.size()] = running;
     t.num_points = running;

@@ -35,7 +35,7 @@ struct HostTables {
     std::vector<uint32_t> golay_by_message;// word of message k = XOR of generator rows in k
     std::vector<float> cls_scale;          // kClassSlots: 2^21 / (4 sqrt(shell)), 0 if unused
     std::vector<uint32_t> cls_parity;      // kClassSlots: parity * 0x00080008
-    std::vector<uint32_t> cls_pack;        // kClassSlots x 2: bits of cls_scale, then cls_parity
+    std::vector<uint32_t> cls_pack;        // kClassSlots x 2: bits of float 1 / (4 sqrt(shell)), then int parity - 16
     std::vector<float> cls_value;          // kClassSlots * 8: dist[l] / (4 sqrt(shell)), l < 5
     std::vector<uint8_t> cls_dist;         // kClassSlots * 8: dist[l]
 };

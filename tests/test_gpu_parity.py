@@ -201,7 +201,7 @@ def test_error_codes(B, ctx):
 
 
 def test_wide_matrix_many_groups_and_size_limits(B, ctx, oracle):
-    # a long row (1024 blocks, x of 48 KB in shared memory) and a launch over eight matrices
+    # a long row (1024 blocks) and a launch over eight matrices
     case = make_case(70, 24 * 1024, seed=41)
     buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
     y = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
@@ -217,15 +217,21 @@ def test_wide_matrix_many_groups_and_size_limits(B, ctx, oracle):
     B.status(ctx)
     for c, g, y in zip(cases, gains, ys):
         check_gemv(oracle, c, y, gain=g)
-    # nine matrices, and an in-dimension whose x does not fit in shared memory beside the ring: refused, nothing launched
+    # nine matrices, and an in-dimension above the documented maximum: refused, nothing launched
     with pytest.raises(B.LlvqError) as e:
         B.gemv_grouped(ctx, 0, [(bufs[0], cases[0].d_scale, GAIN, ys[0], cases[0].rows)] * 9, cases[0].d_x, 24 * 40)
     assert e.value.code == -1
-    big_k = 98304
+    big_k = 98304 + 24
     xx = torch.zeros(big_k, dtype=torch.float16, device="cuda")
     with pytest.raises(B.LlvqError) as e:
         B.gemv(ctx, 0, bufs[0], cases[0].d_scale, GAIN, xx, 32, big_k)
     assert e.value.code == -3
+    # the maximum itself works: 4096 blocks a row, one more than the tiles of 1023 columns would hold
+    case = make_case(40, 98304, seed=43)
+    buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    y = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
+    B.status(ctx)
+    check_gemv(oracle, case, y)
     # negative and zero gains are legal
     y = B.gemv(ctx, 0, bufs[0], cases[0].d_scale, (-1.25, 0.0), cases[0].d_x, cases[0].rows, 24 * 40)
     check_gemv(oracle, cases[0], y, gain=(-1.25, 0.0))

@@ -257,30 +257,46 @@ def test_worked_examples_derived_by_hand(oracle):
 
 # ---------------------------------------------------------------- records and layouts
 def _unpack_planes_cell(buf, nb, row, b):
-    """Reader of the bit-plane layout written from its description (not from the packer)."""
-    rg, l = divmod(row, 32)
+    """Reader of the 14-byte layout written from its description, in the direction opposite to the packer's:
+    from (row, block, coordinate) to the byte and nibble that hold its code."""
+    rg, r = divmod(row, 32)
+    m, e, g = r // 16, (r // 8) % 2, r % 8
     grp = rg * nb * 448
-    nfull = nb // 4
-    if b < nfull * 4:
-        t, q = divmod(b, 4)
-        base = grp + t * 1792
-        words = [int.from_bytes(buf[base + 512 * j + 16 * l + 4 * q: base + 512 * j + 16 * l + 4 * q + 4].tobytes(), "little") for j in range(3)]
-        hdr = int.from_bytes(buf[base + 1536 + 8 * l + 2 * q: base + 1536 + 8 * l + 2 * q + 2].tobytes(), "little")
-    else:
-        base = grp + nfull * 1792 + (b - nfull * 4) * 448
-        words = [int.from_bytes(buf[base + 128 * j + 4 * l: base + 128 * j + 4 * l + 4].tobytes(), "little") for j in range(3)]
-        hdr = int.from_bytes(buf[base + 384 + 2 * l: base + 384 + 2 * l + 2].tobytes(), "little")
+    ntiles, left = divmod(nb, 4)
+
+    def word(off):
+        return int.from_bytes(buf[off: off + 4].tobytes(), "little")
+
+    j = b - 4 * ntiles
+    if j < 0:                                   # inside a tile
+        base = grp + (b // 4) * 1792
+        slot, h = b % 2, 2 * ((b % 4) // 2) + m
+        addr = lambda q, lane: base + 512 * ((3 * h + q) >> 2) + 16 * lane + 4 * ((3 * h + q) & 3)
+        hdr_word = word(base + 1536 + 16 * (2 * g + slot) + 4 * h)
+    elif left >= 2 and j < 2:                   # the pair after the tiles
+        base = grp + ntiles * 1792
+        slot = j
+        addr = lambda q, lane: base + 128 * (3 * m + q) + 4 * lane
+        hdr_word = word(base + 768 + 8 * (2 * g + slot) + 4 * m)
+    else:                                       # the single at the very end: the slot is the row half
+        base = grp + ntiles * 1792 + (896 if left == 3 else 0)
+        slot = m
+        addr = lambda q, lane: base + 128 * q + 4 * lane
+        hdr_word = word(base + 384 + 4 * (2 * g + slot))
+    hdr = (hdr_word >> (16 * e)) & 0xFFFF
     cls, gain = hdr & 511, (hdr >> 9) & 1
     assert hdr >> 10 == 0
-    level, sign = [0] * 24, [0] * 24
-    for j, w in enumerate(words):
-        for k in range(4):
-            r = ((w >> (4 * k)) | (w << (32 - 4 * k))) & 0xFFFFFFFF
-            for e in range(2):
-                i = 8 * j + 2 * k + e
-                level[i] = (r >> (4 + 16 * e)) & 7
-                sign[i] = (r >> (15 + 16 * e)) & 1
-    return cls, gain, level, sign
+    codes = []
+    for i in range(24):
+        kappa = 24 * slot + i
+        if kappa < 32:
+            c, t, ii = kappa // 16, (kappa % 16) // 4, kappa % 4
+            w = word(addr(e, 4 * g + t))        # Wa for e = 0, Wb for e = 1
+        else:
+            c, t, ii = e, (kappa - 32) // 4, (kappa - 32) % 4
+            w = word(addr(2, 4 * g + t))        # Wc: the nibble column picks the row
+        codes.append((w >> (4 * (2 * ii + c))) & 15)
+    return cls, gain, codes
 
 
 def _codes(oracle, rows, nb, seed):
@@ -289,7 +305,7 @@ def _codes(oracle, rows, nb, seed):
     return datagen.make_codes(rows, nb, seed).numpy().astype(np.uint64)
 
 
-@pytest.mark.parametrize("rows,nb", [(32, 4), (40, 7), (3, 1), (64, 9)])
+@pytest.mark.parametrize("rows,nb", [(32, 4), (40, 7), (3, 1), (64, 9), (33, 2), (20, 6), (50, 3)])
 def test_planes_layout_round_trip(oracle, rows, nb):
     codes = _codes(oracle, rows, nb, seed=5)
     codes[0] = N_PAPER                       # a code that names no point
@@ -298,15 +314,19 @@ def test_planes_layout_round_trip(oracle, rows, nb):
     xs, cls = oracle.decode_batch(codes)
     for row in range(((rows + 31) // 32) * 32):
         for b in range(nb):
-            c, g, level, sign = _unpack_planes_cell(buf, nb, row, b)
+            c, g, u = _unpack_planes_cell(buf, nb, row, b)
             if row >= rows or cls[row * nb + b] < 0:
-                assert c == 511 and g == 0 and not any(level) and not any(sign)
+                assert c == 511 and g == 0 and u == [8] * 24
                 continue
             code = int(codes[row * nb + b])
             assert c == cls[row * nb + b] and g == code >> 47
             par = oracle.class_info(c)["odd"]
-            x = [(-1 if s else 1) * (2 * lv + par) for lv, s in zip(level, sign)]
-            assert x == xs[row * nb + b].tolist()
+            assert [2 * (v - 8) + par for v in u] == xs[row * nb + b].tolist()
+            # the same 106 bits as the record's sign mask and level planes
+            rec = oracle.record(code)
+            for i, v in enumerate(u):
+                level = sum(((rec["planes"][t] >> i) & 1) << t for t in range(3))
+                assert v == (8 - level - par if (rec["smask"] >> i) & 1 else 8 + level)
 
 
 @pytest.mark.parametrize("rows,nb", [(32, 3), (37, 5)])
