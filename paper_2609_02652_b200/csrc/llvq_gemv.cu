@@ -72,7 +72,7 @@ namespace {
 #define LLVQ_WARPS 16
 #endif
 #ifndef LLVQ_SLOTS
-#define LLVQ_SLOTS 3
+#define LLVQ_SLOTS 2
 #endif
 #ifndef LLVQ_MINB
 #define LLVQ_MINB 1
@@ -80,6 +80,10 @@ namespace {
 constexpr int kWarps = LLVQ_WARPS;         // warps per CTA
 constexpr int kThreads = kWarps * 32;
 constexpr int kSlots = LLVQ_SLOTS;         // ring slots per warp
+#ifndef LLVQ_EARLY
+#define LLVQ_EARLY 1
+#endif
+constexpr int kEarlySlots = LLVQ_EARLY;    // slots filled before the wait for the previous kernel; the rest once x is being prepared
 
 // fixed-point accumulator word: bits 53..63 count units, bits 0..52 sum the biased unit values
 constexpr int kCountShift = 53;
@@ -114,6 +118,7 @@ __device__ __forceinline__ float onehot_dot(const uint32_t v[5], const float *__
 }
 
 __device__ __forceinline__ int find_problem(const GemvParams &p, int group) {
+    if (p.nprob == 1) return 0;                      // the common launch: one matrix
     int q = 0;
 #pragma unroll
     for (int i = 1; i < LLVQ_MAX_GROUP; i++)
@@ -520,7 +525,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
 
     if (!NO_WEIGHTS) {
 #pragma unroll
-        for (int s = 0; s < kSlots; s++) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
+        for (int s = 0; s < kEarlySlots; s++) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
     }
     // the zero word and the two sums of every x record this CTA will fill
     for (int b = tid; b < blk_hi - blk_lo; b += kThreads)
@@ -577,6 +582,10 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             if (mine_e >= 0) convert_item(mine, mine_e % 3, xs0 + (uint32_t)(mine_e / 3) * kXRecBytes, scale);
         } else {
             for (int e = e_lo + tid; e < e_hi; e += kThreads) convert_item(__ldcg(xg + e), e % 3, xs0 + (uint32_t)(e / 3) * kXRecBytes, scale);
+        }
+        if (!NO_WEIGHTS) {
+#pragma unroll
+            for (int s = kEarlySlots; s < kSlots; s++) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
         }
         __syncthreads();                               // publishes the x records
     }
