@@ -31,9 +31,9 @@ from paper_2609_02652_b200 import datagen  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) per algorithmic byte of gemv_planes_kernel, from one ncu capture of the
-# 8192 x 8192 launch (profiles/gemv_planes_kernel_config4_8192x8192.txt: 39.354 MB against 39.289 MB);
+# 8192 x 8192 launch (profiles/gemv_planes_kernel_config4_8192x8192.txt: 39.365 MB against 39.289 MB);
 # traffic grows in proportion to the records streamed, so a launch's traffic is its bytes times this.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 39.3536 / 39.2888
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 39.3651 / 39.2888
 METRIC = "us_per_lattice_gemv"
 
 
@@ -402,7 +402,7 @@ def main():
         args.no_arms = True          # the comparison arms and per-shape timings are taken on the single-layer workloads
     if not args.no_arms and rank == 0:
         arm_steps = min(args.steps, 200)
-        # per-matrix timings of the bit-plane kernel, one launch each
+        # per-matrix timings of the 14-byte-layout kernel, one launch each
         per_shape = {}
         for li, ln in enumerate(copies[0].launches):
             for mi, m in enumerate(ln["mats"]):
@@ -453,9 +453,9 @@ def main():
         line = {
             "metric": METRIC, "value": us_per_gemv, "unit": "us", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
+            "dtype": "u8 x s8 -> s32 (tensor cores), f32 block scale, int64 row sums", "data": "synthetic",
             "config": {"workload": f"config {wl.config}: {wl.name}", "gemvs_per_step": n_gemv, "launches_per_step": launches_per_step,
-                       "layout": "bit planes, 14 B per 24 weights (4.67 b/w payload; the paper's 4.80 b/w label counts its f32 tail and scales)",
+                       "layout": "Planes14: 14 B per 24 weights - class, gain, 24 four-bit sign+level codes (4.67 b/w payload; the paper's 4.80 b/w label counts its f32 tail and scales)",
                        "l2": f"records and scales rotate through {ncopies} distinct copies ({ncopies * layout_bytes / 1e6:.0f} MB) so no launch finds its records in L2; x (a few KB a launch) is one buffer, as in a decoder where it is the previous operator's output",
                        "multi_gpu": "replicas only: each rank runs the whole step on its own copy", "seed": wl.seed},
             "gbps": gbps, "hbm_frac": gbps / peak, "bytes_per_step": step_bytes,

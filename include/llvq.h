@@ -150,7 +150,7 @@ int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row
 int llvq_gemv_grouped(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n,
                       const void *x, int64_t k_padded, void *stream);
 
-/* No counterpart in the paper: the bit-plane llvq_gemv for callers that cannot allocate device
+/* No counterpart in the paper: the LLVQ_PLANES llvq_gemv for callers that cannot allocate device
  * memory - a process whose memory pool already owns the whole GPU, a plug-in that receives buffers
  * but no allocator, code that runs while a stream is being captured, a loop that cannot afford the
  * device synchronisation an allocation implies.  Such callers cannot use a context either

@@ -157,7 +157,7 @@ def onehot_bytes(rows: int, nb: int) -> int:
 
 
 def pack_planes(codes: np.ndarray, rows: int, nb: int) -> np.ndarray:
-    """Expected bytes of the bit-plane layout (14 B a block) for a rows x nb matrix of codes."""
+    """Expected bytes of the 14-byte layout (LLVQ_PLANES) for a rows x nb matrix of codes."""
     codes = np.ascontiguousarray(codes, dtype=np.uint64).ravel()
     assert codes.size == rows * nb
     out = np.zeros(planes_bytes(rows, nb), np.uint8)

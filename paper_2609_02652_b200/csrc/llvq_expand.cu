@@ -1,6 +1,6 @@
 // The expander (paper Sec. 2.2, "Unfolding at load time"): one pass that turns every 48-bit code
 // word into its decoded-field record - class id, gain bit, sign mask, per-coordinate level - in
-// the bit-plane or the one-hot layout.  Integer arithmetic only, so the output is bit-exact.
+// the 14-byte or the one-hot layout.  Integer arithmetic only, so the output is bit-exact.
 //
 // The index splits as the paper states it (Sec. 2.1: classes first, then arrangements and signs
 // inside a class, as a mixed-radix number).  The digit order used here:

@@ -1023,7 +1023,7 @@ cudaError_t launch_decode_i8(const llvq_ctx *ctx, int layout, const uint8_t *buf
 }  // namespace llvq
 
 // ---------------------------------------------------------------------------------------------
-// llvq_gemv_static: the bit-plane GEMV for callers that must not allocate device memory.
+// llvq_gemv_static: the 14-byte-layout GEMV for callers that must not allocate device memory.
 //
 // Some hosts of this library cannot call cudaMalloc at the moment they need a matvec: a serving
 // process whose memory pool already owns all of HBM, a plug-in that is handed buffers but no
