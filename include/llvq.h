@@ -154,14 +154,14 @@ int llvq_gemv_grouped(llvq_ctx *ctx, int layout, const llvq_problem *problems, i
  * memory - a process whose memory pool already owns the whole GPU, a plug-in that receives buffers
  * but no allocator, code that runs while a stream is being captured, a loop that cannot afford the
  * device synchronisation an allocation implies.  Such callers cannot use a context either
- * (llvq_create allocates), so this call takes none: the reduction scratch, the class table and the
- * error flag are file-scope device arrays inside the library (about 516 KiB on every GPU that loads
- * it, held until the process exits).  Same arguments, layout (LLVQ_PLANES only), alignment rules and
+ * (llvq_create allocates), so this call takes none: the reduction scratch and the error flag are
+ * file-scope device arrays inside the library (about 512 KiB on every GPU that loads it, held
+ * until the process exits).  Same arguments, layout (LLVQ_PLANES only), alignment rules and
  * results as llvq_gemv; it runs on the CURRENT device.  Limits and rules:
  *   - rows, rounded up to a multiple of 32, must not exceed 65536 (the built-in scratch holds one
  *     64-bit accumulator a row); more returns LLVQ_ESIZE and launches nothing.
- *   - The first call on a device sets the arrays up (resolves their device addresses, uploads the
- *     class table, zeroes the scratch - synchronous copies, no allocation).  Make that first call
+ *   - The first call on a device sets the arrays up (resolves their device addresses, zeroes the
+ *     scratch - synchronous, no allocation).  Make that first call
  *     before any stream capture begins.
  *   - Every call shares the one scratch array.  A launch that completes leaves it zeroed for the
  *     next; launches that overlap on the GPU (two streams) race on it - serialise them.

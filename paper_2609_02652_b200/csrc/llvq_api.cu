@@ -232,6 +232,9 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
     p.cls_parity = ctx->dev.cls_parity;
     p.cls_value = ctx->dev.cls_value;
     p.cls_pack = ctx->dev.cls_pack;
+    std::memcpy(p.cls_shell_nibbles, ctx->host.cls_shell_nibbles, sizeof p.cls_shell_nibbles);
+    std::memcpy(p.cls_odd_bits, ctx->host.cls_odd_bits, sizeof p.cls_odd_bits);
+    std::memcpy(p.shell_inv_norm, ctx->host.shell_inv_norm, sizeof p.shell_inv_norm);
     p.error = ctx->error;
 #ifdef LLVQ_TRACE
     p.trace = ctx->trace;

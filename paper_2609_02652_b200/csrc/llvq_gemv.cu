@@ -440,14 +440,9 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     __syncwarp();
 
     // then the loads whose latency the rest of the prologue can cover:
-    // the class constants this
-    // thread will turn into block constants, and x on its way into L2 (its values are read only after
-    // the wait below, through L2, which is where the previous kernel's writes to x land)
+    // x on its way into L2 (its values are read only after the wait below, through L2, which is where the
+    // previous kernel's writes to x land)
     const int tab_entries = p.nprob * 1024;
-    float2 cv[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-#pragma unroll
-    for (int i = 0; i < 2; i++)
-        if (tid + i * kThreads < tab_entries) cv[i] = __ldg(p.cls_pack + ((tid + i * kThreads) & 511));
     uint32_t warm = 0;
     for (int e = tid * 128; e < p.nb * 48; e += kThreads * 128) {
         // a load whose value is not used: it brings the line into L2 and the translation into this
@@ -530,11 +525,14 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     // the zero word and the two sums of every x record this CTA will fill
     for (int b = tid; b < blk_hi - blk_lo; b += kThreads)
         asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(smem_addr(xrec) + b * kXRecBytes + 96), "r"(0) : "memory");
-    // block constants of every matrix of the launch: (class | gain << 9) -> {gain / (4 sqrt m), parity - 16}
-    for (int e = tid, i = 0; e < tab_entries; e += kThreads, i++) {
-        const float2 v = i < 2 ? cv[i] : __ldg(p.cls_pack + (e & 511));
+    // block constants of every matrix of the launch: (class | gain << 9) -> {gain / (4 sqrt m), parity - 16},
+    // from the class constants in the kernel's parameters
+    for (int e = tid; e < tab_entries; e += kThreads) {
+        const int c = e & 511;
+        const uint32_t shell = (p.cls_shell_nibbles[c >> 3] >> (4 * (c & 7))) & 15u;
+        const int odd = (int)((p.cls_odd_bits[c >> 5] >> (c & 31)) & 1u);
         const GemvProblemDev &pe = p.prob[e >> 10];
-        tab[e] = make_float2(v.x * ((e & 512) ? pe.gain1 : pe.gain0), v.y);
+        tab[e] = make_float2(p.shell_inv_norm[shell] * ((e & 512) ? pe.gain1 : pe.gain0), __int_as_float(shell ? odd - 16 : 0));
     }
     // let the next kernel in the stream start its own prefetch, then wait for the previous one:
     // x, y and the reduction scratch may still be in use by it
@@ -1031,13 +1029,13 @@ cudaError_t launch_decode_i8(const llvq_ctx *ctx, int layout, const uint8_t *buf
 // a real-time loop in which an allocation's implicit device synchronisation is not acceptable.
 // Those callers cannot create a context either, because llvq_create allocates the tables and the
 // reduction scratch.  For them everything the kernel needs besides the caller's own buffers lives
-// in file-scope __device__ arrays that the module carries: the row accumulators (the scratch), the
-// class table and the error flag.  Every GPU that loads the library holds these arrays (about
-// 516 KiB) until the process exits.
+// in file-scope __device__ arrays that the module carries: the row accumulators (the scratch) and
+// the error flag; the class constants travel in the kernel's parameters.  Every GPU that loads the
+// library holds these arrays (about 512 KiB) until the process exits.
 //
 // In host code the name of a __device__ array is only a host-side stand-in, not a device address;
 // the kernel is therefore given the address that cudaGetSymbolAddress returns for the current
-// device.  That, the upload of the class table and the kernel's shared-memory attribute are done
+// device.  That, the zeroing of the scratch and the kernel's shared-memory attribute are done
 // by the first call on each device (synchronously), so make that first call before any stream
 // capture begins.  All calls share the arrays: the accumulators are left at zero by every launch
 // that completes, but two launches that overlap on the GPU (different streams) race on them.
@@ -1048,27 +1046,28 @@ constexpr int kStaticMaxRows = 65536;      // rows (rounded up to 32) one llvq_g
 constexpr int kStaticMaxDevices = 64;
 
 static __device__ __align__(256) unsigned long long g_static_accum[kStaticMaxRows];   // 512 KiB of scratch
-static __device__ __align__(256) float2 g_static_cls_pack[llvq::kClassSlots];           // 4 KiB
 static __device__ __align__(256) int g_static_error[64];
 
 struct StaticDevice {
     bool ready = false;
     unsigned long long *accum = nullptr;
-    float2 *cls_pack = nullptr;
+    uint32_t cls_shell_nibbles[64], cls_odd_bits[16];      // class constants (host copies, handed to every launch)
+    float shell_inv_norm[16];
     int *error = nullptr;
     int sm_count = 0, max_smem_optin = 0;
 };
 StaticDevice g_static_dev[kStaticMaxDevices];
 
-// Once per device, with that device current: resolve the arrays' device addresses, fill the class
-// table, zero the accumulators, raise the kernel's shared-memory limit.  Allocates no device memory.
+// Once per device, with that device current: resolve the arrays' device addresses, build the class
+// constants on the host, zero the accumulators, raise the kernel's shared-memory limit.  Allocates no device memory.
 int static_setup(int device, StaticDevice &d) {
     if (cudaGetSymbolAddress((void **)&d.accum, g_static_accum) != cudaSuccess) return LLVQ_ECUDA;
-    if (cudaGetSymbolAddress((void **)&d.cls_pack, g_static_cls_pack) != cudaSuccess) return LLVQ_ECUDA;
     if (cudaGetSymbolAddress((void **)&d.error, g_static_error) != cudaSuccess) return LLVQ_ECUDA;
     llvq::HostTables host;                                   // host memory only
     if (!llvq::build_tables(host)) return LLVQ_EINVAL;
-    if (cudaMemcpy(d.cls_pack, host.cls_pack.data(), llvq::kClassSlots * 8, cudaMemcpyHostToDevice) != cudaSuccess) return LLVQ_ECUDA;
+    memcpy(d.cls_shell_nibbles, host.cls_shell_nibbles, sizeof d.cls_shell_nibbles);
+    memcpy(d.cls_odd_bits, host.cls_odd_bits, sizeof d.cls_odd_bits);
+    memcpy(d.shell_inv_norm, host.shell_inv_norm, sizeof d.shell_inv_norm);
     if (cudaMemset(d.accum, 0, sizeof(unsigned long long) * kStaticMaxRows) != cudaSuccess) return LLVQ_ECUDA;
     if (cudaMemset(d.error, 0, sizeof(int) * 64) != cudaSuccess) return LLVQ_ECUDA;
     if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return LLVQ_ECUDA;
@@ -1125,7 +1124,9 @@ extern "C" int llvq_gemv_static(const void *layout_buf, const void *row_scale, c
     p.total_groups = (int)groups;
     p.total_units = (int)(groups * p.units);
     p.accum = d.accum;
-    p.cls_pack = d.cls_pack;
+    memcpy(p.cls_shell_nibbles, d.cls_shell_nibbles, sizeof p.cls_shell_nibbles);
+    memcpy(p.cls_odd_bits, d.cls_odd_bits, sizeof p.cls_odd_bits);
+    memcpy(p.shell_inv_norm, d.shell_inv_norm, sizeof p.shell_inv_norm);
     p.error = d.error;
     const llvq::GemvLaunch g = llvq::gemv_plan(LLVQ_PLANES, p, d.sm_count);
     if (g.smem + 1024 > (size_t)d.max_smem_optin) return LLVQ_ESIZE;

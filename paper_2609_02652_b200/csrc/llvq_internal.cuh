@@ -58,6 +58,11 @@ struct GemvParams {
     const uint32_t *cls_parity;
     const float *cls_value;
     const float2 *cls_pack;   // 512 x {1 / (4 sqrt m), int parity - 16 as bits}
+    // the class constants the 14-byte GEMV needs, in the parameters themselves (no load from global memory
+    // stands between a CTA's start and its block-constant table)
+    uint32_t cls_shell_nibbles[64];   // nibble c & 7 of word c >> 3: shell of class c, 0 if unused
+    uint32_t cls_odd_bits[16];        // bit c & 31 of word c >> 5: odd type
+    float shell_inv_norm[16];         // [m] = 1 / (4 sqrt m)
     int *error;               // set when a bounded wait ran out
 #ifdef LLVQ_TRACE
     unsigned long long *trace;   // timeline buffer (debug builds only)

@@ -172,6 +172,13 @@ bool build_tables(HostTables &t) {
             t.cls_dist[c * 8 + l] = d.dist[l];
         }
     }
+    std::memset(t.cls_shell_nibbles, 0, sizeof t.cls_shell_nibbles);
+    std::memset(t.cls_odd_bits, 0, sizeof t.cls_odd_bits);
+    for (int m = 0; m < 16; m++) t.shell_inv_norm[m] = (m >= 2 && m <= 12) ? (float)(1.0 / (4.0 * std::sqrt((double)m))) : 0.f;
+    for (size_t c = 0; c < all.size(); c++) {
+        t.cls_shell_nibbles[c >> 3] |= (uint32_t)all[c].shell << (4 * (c & 7));
+        if (all[c].odd) t.cls_odd_bits[c >> 5] |= 1u << (c & 31);
+    }
     t.cls_pack.assign(kClassSlots * 2, 0u);
     for (int c = 0; c < kClassSlots; c++) {
         const float inv_norm = t.cls_scale[c] * (1.0f / 2097152.0f);      // exact: a power of two
