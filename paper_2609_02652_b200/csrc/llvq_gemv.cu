@@ -477,6 +477,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         Cursor c;
         const uint8_t *next;
         int left, done;
+        uint32_t bytes;       // size of the next unit
     };
     const int n_tiles_total = p.tiles;
     Walk iw;
@@ -484,13 +485,10 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     iw.next = isrc + (size_t)ic.col * kTileBytes;      // the leftover blocks follow the last tile
     iw.left = ic.end - ic.col;
     iw.done = 0;
-    auto walk_next = [&](Walk &w, const uint8_t *&src, uint32_t &bytes) {
-        src = w.next;
-        bytes = w.c.col < n_tiles_total ? (uint32_t)kTileBytes : tail_bytes;
-        w.done++;
-        w.next += kTileBytes;
-        w.c.col++;
-        if (--w.left == 0) {                           // rare: the stretch ends, the next one starts elsewhere
+    iw.bytes = ic.col < n_tiles_total ? (uint32_t)kTileBytes : tail_bytes;
+    // the stretch ends or its last unit is the leftover one: the next unit starts elsewhere or has another size
+    auto walk_turn = [&](Walk &w) {
+        if (w.left == 0) {
             w.c.col--;
             advance(p, w.c, 1);
             if (w.done < n_units) {
@@ -499,6 +497,15 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             }
             w.left = w.c.end - w.c.col;
         }
+        w.bytes = w.c.col < n_tiles_total ? (uint32_t)kTileBytes : tail_bytes;
+    };
+    auto walk_next = [&](Walk &w, const uint8_t *&src, uint32_t &bytes) {
+        src = w.next;
+        bytes = w.bytes;
+        w.done++;
+        w.next += kTileBytes;
+        w.c.col++;
+        if (--w.left <= 1) walk_turn(w);               // rare: at most twice a stretch
     };
     // issue the copy of the next unit (lane 0 alone, by predicate) onto barrier `b` and buffer `dst`
     const int my_issues = lane == 0 ? n_units : 0;     // lanes other than 0 never issue
