@@ -413,9 +413,6 @@ __device__ __forceinline__ bool advance(const GemvParams &p, Cursor &c, int n) {
     c.col = c.panel * p.panel;
     return true;
 }
-// first unit of warp gw when total = base * warps + rem units are dealt out, the first rem warps taking one more
-__host__ __device__ inline int first_unit_of_warp(int base, int rem, int gw) { return gw * base + (gw < rem ? gw : rem); }
-
 template <bool NO_WEIGHTS>
 __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
@@ -453,11 +450,11 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         warm |= w;
     }
     // this warp's units, and the blocks of x this CTA's units touch
-    const int gw = blockIdx.x * kWarps + warp;
-    const int u0 = first_unit_of_warp(p.units_base, p.units_rem, gw);
-    const int n_units = p.units_base + (gw < p.units_rem ? 1 : 0);
-    const int cta_u0 = first_unit_of_warp(p.units_base, p.units_rem, blockIdx.x * kWarps);
-    const int cta_u1 = first_unit_of_warp(p.units_base, p.units_rem, (blockIdx.x + 1) * kWarps);
+    // the CTA's units come from the host's plan; its warps share them evenly, the earlier warps taking the odd ones
+    const int cta_u0 = p.cta_first[blockIdx.x], cta_u1 = p.cta_first[blockIdx.x + 1];
+    const int cta_n = cta_u1 - cta_u0;
+    const int u0 = cta_u0 + (warp * cta_n + kWarps - 1) / kWarps;
+    const int n_units = cta_u0 + ((warp + 1) * cta_n + kWarps - 1) / kWarps - u0;
     const int blk_lo = panel_of_unit(p, cta_u0) * p.panel * kTileCells;
     const int blk_hi = min(p.nb, (panel_of_unit(p, max(cta_u1 - 1, cta_u0)) + 1) * p.panel * kTileCells);
     const uint32_t xs0 = smem_addr(xrec) - (uint32_t)blk_lo * kXRecBytes;     // address of block 0's record, were it there
@@ -946,10 +943,31 @@ GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
     const int want = (p.units + 8) / 16 > 1 ? (p.units + 8) / 16 : 1;
     p.panel = (p.units + want - 1) / want;
     p.npanels = (p.units + p.panel - 1) / p.panel;
+    // Shares of the CTAs.  CTAs start in index order as multiprocessors come free, the first ones while the
+    // previous kernel of the stream is still finishing, so the first CTAs can afford more units than the last:
+    // the share falls linearly from mean + lead to mean - lead.
+    if (g.grid > kMaxGridCtas) g.grid = kMaxGridCtas;
+    {
+        const double mean = (double)p.total_units / g.grid;
+        double lead = 10.0;                            // units: about half a microsecond of a multiprocessor's streaming (measured optimum 9-12)
+        if (lead > 0.6 * mean) lead = 0.6 * mean;
+        const double skew = mean > 0 ? lead / mean : 0.0;
+        double acc = 0.0;
+        p.cta_first[0] = 0;
+        for (int c = 0; c < g.grid; c++) {
+            const double w = g.grid > 1 ? 1.0 + skew * (1.0 - 2.0 * c / (g.grid - 1)) : 1.0;
+            acc += mean * w;
+            int f = (int)(acc + 0.5);
+            if (f < p.cta_first[c]) f = p.cta_first[c];
+            if (f > p.total_units) f = p.total_units;
+            p.cta_first[c + 1] = f;
+        }
+        p.cta_first[g.grid] = p.total_units;
+    }
     // the widest stretch of x a CTA meets: its units lie in consecutive panels
     p.xblocks = 0;
     for (int c = 0; c < g.grid; c++) {
-        const int f0 = first_unit_of_warp(p.units_base, p.units_rem, c * kWarps), f1 = first_unit_of_warp(p.units_base, p.units_rem, (c + 1) * kWarps);
+        const int f0 = p.cta_first[c], f1 = p.cta_first[c + 1];
         const int lo = panel_of_unit(p, f0) * p.panel * kTileCells;
         int hi = (panel_of_unit(p, f1 - 1 > f0 ? f1 - 1 : f0) + 1) * p.panel * kTileCells;
         if (hi > p.nb) hi = p.nb;

@@ -16,6 +16,7 @@ constexpr int kCellBytes = 448;        // 32 rows x 14 bytes
 constexpr int kTileCells = 4;
 constexpr int kTileBytes = 1792;
 constexpr int kOneHotCellBytes = 640;  // 32 rows x 20 bytes
+constexpr int kMaxGridCtas = 256;      // the GEMV launches one CTA a multiprocessor; more multiprocessors than this share the work of 256
 
 struct DeviceTables {
     const uint64_t *base;            // num_classes + 1
@@ -53,6 +54,7 @@ struct GemvParams {
     int units_base, units_rem;   // total_units divided by the warps of the grid (set by gemv_plan; the one-hot arm's order)
     int panel, npanels;          // unit columns a panel, panels (set by gemv_plan; the 14-byte layout's order of work)
     int xblocks;                 // most blocks of x any CTA needs (set by gemv_plan)
+    int cta_first[kMaxGridCtas + 1];   // first unit of every CTA of the grid, and the total (set by gemv_plan)
     unsigned long long *accum;   // total_groups x 32 fixed-point row accumulators (context scratch, zero between launches)
     const float *cls_scale;
     const uint32_t *cls_parity;
