@@ -940,7 +940,10 @@ GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
         return g;
     }
     // panels of about sixteen unit columns, as equal as they come
-    const int want = (p.units + 8) / 16 > 1 ? (p.units + 8) / 16 : 1;
+#ifndef LLVQ_PANEL
+#define LLVQ_PANEL 16
+#endif
+    const int want = (p.units + LLVQ_PANEL / 2) / LLVQ_PANEL > 1 ? (p.units + LLVQ_PANEL / 2) / LLVQ_PANEL : 1;
     p.panel = (p.units + want - 1) / want;
     p.npanels = (p.units + p.panel - 1) / p.panel;
     // Shares of the CTAs.  CTAs start in index order as multiprocessors come free, the first ones while the
