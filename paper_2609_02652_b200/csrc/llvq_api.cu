@@ -64,12 +64,11 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
     ctx->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
 
     const HostTables &h = ctx->host;
-    struct Part { const void *src; size_t bytes; size_t off; } parts[9] = {
+    struct Part { const void *src; size_t bytes; size_t off; } parts[8] = {
         {h.base.data(), h.base.size() * 8, 0},          {h.desc.data(), h.desc.size() * sizeof(ClassDesc), 0},
         {h.golay_by_weight.data(), 4096 * 4, 0},        {h.golay_by_message.data(), 4096 * 4, 0},
         {h.cls_scale.data(), kClassSlots * 4, 0},       {h.cls_parity.data(), kClassSlots * 4, 0},
-        {h.cls_value.data(), kClassSlots * 8 * 4, 0},   {h.cls_dist.data(), kClassSlots * 8, 0},
-        {h.cls_pack.data(), kClassSlots * 8, 0}};
+        {h.cls_value.data(), kClassSlots * 8 * 4, 0},   {h.cls_dist.data(), kClassSlots * 8, 0}};
     size_t total = 0;
     for (auto &p : parts) { p.off = total; total += round_up(p.bytes, 256); }
     if (cudaMalloc(&ctx->table_blob, total) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
@@ -88,7 +87,6 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
     d.cls_parity = (const uint32_t *)(blob + parts[5].off);
     d.cls_value = (const float *)(blob + parts[6].off);
     d.cls_dist = (const uint8_t *)(blob + parts[7].off);
-    d.cls_pack = (const float2 *)(blob + parts[8].off);
     std::memcpy(d.weight_offset, h.weight_offset, sizeof d.weight_offset);
     d.num_classes = h.num_classes;
     d.num_points = h.num_points;
@@ -231,7 +229,6 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
     p.cls_scale = ctx->dev.cls_scale;
     p.cls_parity = ctx->dev.cls_parity;
     p.cls_value = ctx->dev.cls_value;
-    p.cls_pack = ctx->dev.cls_pack;
     std::memcpy(p.cls_shell_nibbles, ctx->host.cls_shell_nibbles, sizeof p.cls_shell_nibbles);
     std::memcpy(p.cls_odd_bits, ctx->host.cls_odd_bits, sizeof p.cls_odd_bits);
     std::memcpy(p.shell_inv_norm, ctx->host.shell_inv_norm, sizeof p.shell_inv_norm);

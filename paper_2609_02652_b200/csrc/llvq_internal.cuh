@@ -27,7 +27,6 @@ struct DeviceTables {
     const uint32_t *cls_parity;      // 512
     const float *cls_value;          // 512 x 8
     const uint8_t *cls_dist;         // 512 x 8
-    const float2 *cls_pack;          // 512 x {1 / (4 sqrt m), int parity - 16 as bits}
     int weight_offset[25];
     int num_classes;
     uint64_t num_points;
@@ -59,7 +58,6 @@ struct GemvParams {
     const float *cls_scale;
     const uint32_t *cls_parity;
     const float *cls_value;
-    const float2 *cls_pack;   // 512 x {1 / (4 sqrt m), int parity - 16 as bits}
     // the class constants the 14-byte GEMV needs, in the parameters themselves (no load from global memory
     // stands between a CTA's start and its block-constant table)
     uint32_t cls_shell_nibbles[64];   // nibble c & 7 of word c >> 3: shell of class c, 0 if unused

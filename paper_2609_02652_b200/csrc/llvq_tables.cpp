@@ -179,13 +179,6 @@ bool build_tables(HostTables &t) {
         t.cls_shell_nibbles[c >> 3] |= (uint32_t)all[c].shell << (4 * (c & 7));
         if (all[c].odd) t.cls_odd_bits[c >> 5] |= 1u << (c & 31);
     }
-    t.cls_pack.assign(kClassSlots * 2, 0u);
-    for (int c = 0; c < kClassSlots; c++) {
-        const float inv_norm = t.cls_scale[c] * (1.0f / 2097152.0f);      // exact: a power of two
-        std::memcpy(&t.cls_pack[2 * c], &inv_norm, 4);
-        const int32_t offset = t.cls_scale[c] != 0.f ? (t.cls_parity[c] ? 1 : 0) - 16 : 0;   // x_i = 2 u_i + offset
-        std::memcpy(&t.cls_pack[2 * c + 1], &offset, 4);
-    }
     t.base[all.size()] = running;
     t.num_points = running;
     return t.num_classes == 301 && t.num_points == 111043117458000ull;

@@ -35,8 +35,8 @@ struct HostTables {
     std::vector<uint32_t> golay_by_message;// word of message k = XOR of generator rows in k
     std::vector<float> cls_scale;          // kClassSlots: 2^21 / (4 sqrt(shell)), 0 if unused
     std::vector<uint32_t> cls_parity;      // kClassSlots: parity * 0x00080008
-    std::vector<uint32_t> cls_pack;        // kClassSlots x 2: bits of float 1 / (4 sqrt(shell)), then int parity - 16
-    // the same, small enough to travel in kernel parameters:
+    // the class constants of the 14-byte GEMV, small enough to travel in kernel parameters
+    // (x_i = 2 u_i + parity - 16, scale 1 / (4 sqrt(shell))):
     uint32_t cls_shell_nibbles[64];        // nibble c & 7 of word c >> 3: shell of class c (2..12), 0 if unused
     uint32_t cls_odd_bits[16];             // bit c & 31 of word c >> 5: class c is of the odd type
     float shell_inv_norm[16];              // [m] = 1 / (4 sqrt(m)) for m = 2..12, else 0

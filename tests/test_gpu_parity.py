@@ -272,3 +272,25 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(B, oracle
         check_gemv(oracle, case, y)
     finally:
         ctx.close()
+
+
+def test_gemv_fixed_point_activations_inside_one_vector(B, ctx, oracle):
+    """The 14-byte GEMV takes x as fixed point on a scale set by the largest |x| (include/llvq.h): entries within
+    2^-18 of the largest are exact, smaller ones are rounded to within 2^-29 of the largest.  One huge entry among
+    small ones: the result stays within that bound of the f64 oracle, row by row, and the normalised bar holds."""
+    case = make_case(128, 24 * 41, seed=91)
+    xs = (case.x.astype(np.float64) * 2.0**-12).astype(np.float16)          # |x| around 2^-12
+    xs[500] = np.float16(40000.0)                                           # and one entry 2^27 times larger
+    case.x, case.d_x = xs, torch.from_numpy(xs).cuda()
+    buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    y = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
+    B.status(ctx)
+    y_ref, wnorm, abssum = oracle.matvec(case.codes, case.rows, case.nb, case.row_scale, GAIN, case.x)
+    err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref)
+    xnorm = float(np.linalg.norm(xs.astype(np.float64)))
+    assert (err <= 1e-4 * wnorm * xnorm).all()
+    # every coordinate's activation is off by at most 2^-29 * 65536 (the largest is below 2^16); the weights of a
+    # row are at most |w_i| each, so the row is off by at most that times sum |w_i|, plus f32 rounding of the sums
+    W = oracle.dequant(case.codes, case.rows, case.nb, case.row_scale, GAIN)
+    bound = 2.0**-29 * 65536.0 * np.abs(W).sum(axis=1) + 2.0**-22 * abssum
+    assert (err <= bound).all(), float(np.max(err / bound))
