@@ -436,7 +436,6 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     }
     __syncwarp();
 
-    // then the loads whose latency the rest of the prologue can cover:
     // x on its way into L2 (its values are read only after the wait below, through L2, which is where the
     // previous kernel's writes to x land)
     const int tab_entries = p.nprob * 1024;
@@ -449,8 +448,8 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(w) : "l"(reinterpret_cast<const char *>(p.x) + e));
         warm |= w;
     }
-    // this warp's units, and the blocks of x this CTA's units touch
-    // the CTA's units come from the host's plan; its warps share them evenly, the earlier warps taking the odd ones
+    // The CTA's units come from the host's plan; its warps share them evenly (the odd ones spread over the
+    // warps).  The blocks of x the CTA's units touch are those of the panels its range lies in.
     const int cta_u0 = p.cta_first[blockIdx.x], cta_u1 = p.cta_first[blockIdx.x + 1];
     const int cta_n = cta_u1 - cta_u0;
     const int u0 = cta_u0 + (warp * cta_n + kWarps - 1) / kWarps;
@@ -466,8 +465,6 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     if (n_units > 0) isrc = group_base(p, ic.group, kCellBytes, q);
     const uint32_t tail_bytes = (uint32_t)p.tail_cells * kCellBytes;
 
-    // issue the copy of the next unit (lane 0 alone, by predicate) onto barrier `b` and buffer `dst`,
-    // then step the source
     // The issue side's walk: inext is the next unit's first byte, ileft the units left in its stretch of its
     // row group.  next() hands out the unit's source and size and steps on.
     struct Walk {
