@@ -374,20 +374,17 @@ __device__ __forceinline__ void convert_item(const uint4 &v, int third, uint32_t
 struct Cursor {
     int panel, group, col, end;      // end = first column past the panel
 };
-// n / d for 0 <= n < 2^31, 0 < d: a float estimate and two fix-ups (a 32-bit integer division costs more than
-// everything else a warp does before it waits)
-__host__ __device__ inline int small_div(int n, int d) {
+__host__ __device__ inline int fast_div(int n, const FastDiv &f, int d) {
 #ifdef __CUDA_ARCH__
-    int q = (int)(__int2float_rz(n) * __frcp_rz(__int2float_ru(d)));       // never above the true quotient
-    int r = n - q * d;
-    while (r >= d) { q++; r -= d; }
-    return q;
+    (void)d;
+    return f.mul ? (int)(__umulhi((uint32_t)n, f.mul) >> f.shift) : n;
 #else
+    (void)f;
     return n / d;
 #endif
 }
 __host__ __device__ inline int panel_of_unit(const GemvParams &p, int f) {
-    const int j = small_div(f, p.total_groups * p.panel);
+    const int j = fast_div(f, p.div_panel_units, p.total_groups * p.panel);
     return j < p.npanels ? j : p.npanels - 1;
 }
 __device__ __forceinline__ Cursor locate(const GemvParams &p, int f) {
@@ -396,7 +393,7 @@ __device__ __forceinline__ Cursor locate(const GemvParams &p, int f) {
     const int first = c.panel * p.panel;
     c.end = min(first + p.panel, p.units);
     const int r = f - c.panel * (p.total_groups * p.panel), w = c.end - first;
-    c.group = small_div(r, w);
+    c.group = c.panel == p.npanels - 1 ? fast_div(r, p.div_last, w) : fast_div(r, p.div_panel, w);
     c.col = first + (r - c.group * w);
     return c;
 }
@@ -427,6 +424,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     const uint32_t my_bar = smem_addr(bars + warp * kSlots);
 
     LLVQ_TRACE_POINT(0)
+    LLVQ_TRACE_CLOCK(7)
     // a warp's barriers are used by that warp alone: no block-wide synchronisation is needed for them; they
     // are set up before any load is in flight, so that the fence has nothing to wait for
     if (lane == 0) {
@@ -436,6 +434,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     }
     __syncwarp();
 
+    LLVQ_TRACE_CLOCK(3)
     // x on its way into L2 (its values are read only after the wait below, through L2, which is where the
     // previous kernel's writes to x land)
     const int tab_entries = p.nprob * 1024;
@@ -458,6 +457,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     const int blk_hi = min(p.nb, (panel_of_unit(p, max(cta_u1 - 1, cta_u0)) + 1) * p.panel * kTileCells);
     const uint32_t xs0 = smem_addr(xrec) - (uint32_t)blk_lo * kXRecBytes;     // address of block 0's record, were it there
 
+    LLVQ_TRACE_CLOCK(4)
     // consume side and issue side walk the same sequence of units
     Cursor cc = locate(p, u0), ic = cc;
     int q = 0;
@@ -523,18 +523,8 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
 #pragma unroll
         for (int s = 0; s < kEarlySlots; s++) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
     }
-    // the zero word and the two sums of every x record this CTA will fill
-    for (int b = tid; b < blk_hi - blk_lo; b += kThreads)
-        asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(smem_addr(xrec) + b * kXRecBytes + 96), "r"(0) : "memory");
-    // block constants of every matrix of the launch: (class | gain << 9) -> {gain / (4 sqrt m), parity - 16},
-    // from the class constants in the kernel's parameters
-    for (int e = tid; e < tab_entries; e += kThreads) {
-        const int c = e & 511;
-        const uint32_t shell = (p.cls_shell_nibbles[c >> 3] >> (4 * (c & 7))) & 15u;
-        const int odd = (int)((p.cls_odd_bits[c >> 5] >> (c & 31)) & 1u);
-        const GemvProblemDev &pe = p.prob[e >> 10];
-        tab[e] = make_float2(p.shell_inv_norm[shell] * ((e & 512) ? pe.gain1 : pe.gain0), __int_as_float(shell ? odd - 16 : 0));
-    }
+    LLVQ_TRACE_CLOCK(5)
+    LLVQ_TRACE_CLOCK(6)
     // let the next kernel in the stream start its own prefetch, then wait for the previous one:
     // x, y and the reduction scratch may still be in use by it
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -562,6 +552,21 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                 const int e = base + i * kThreads + tid;
                 v[i] = e < nx ? __ldcg(xg + e) : make_uint4(0u, 0u, 0u, 0u);
             }
+            if (base == 0) {
+                // while the first loads are on their way: what the loop needs besides x
+            // the zero word and the two sums of every x record this CTA will fill
+            for (int b = tid; b < blk_hi - blk_lo; b += kThreads)
+                asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(smem_addr(xrec) + b * kXRecBytes + 96), "r"(0) : "memory");
+            // block constants of every matrix of the launch: (class | gain << 9) -> {gain / (4 sqrt m), parity - 16},
+            // from the class constants in the kernel's parameters
+            for (int e = tid; e < tab_entries; e += kThreads) {
+                const int c = e & 511;
+                const uint32_t shell = (p.cls_shell_nibbles[c >> 3] >> (4 * (c & 7))) & 15u;
+                const int odd = (int)((p.cls_odd_bits[c >> 5] >> (c & 31)) & 1u);
+                const GemvProblemDev &pe = p.prob[e >> 10];
+                tab[e] = make_float2(p.shell_inv_norm[shell] * ((e & 512) ? pe.gain1 : pe.gain0), __int_as_float(shell ? odd - 16 : 0));
+            }
+            }
 #pragma unroll
             for (int i = 0; i < 4; i++) {
                 const int e = base + i * kThreads + tid;
@@ -570,7 +575,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             }
         }
         m = __reduce_max_sync(0xffffffffu, max(m & 0xffffu, m >> 16));
-            if (lane == 0) warp_max[warp] = m;             // plain stores: atomics on one word would serialise the warps
+        if (lane == 0) warp_max[warp] = m;             // plain stores: atomics on one word would serialise the warps
         __syncthreads();                               // publishes the maxima, the block constants and the zeroed sums
         m = warp_max[lane < kWarps ? lane : 0];
         xexp = max((int)(__reduce_max_sync(0xffffffffu, m) >> 10), 1) - 14;
@@ -943,6 +948,9 @@ GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
     const int want = (p.units + LLVQ_PANEL / 2) / LLVQ_PANEL > 1 ? (p.units + LLVQ_PANEL / 2) / LLVQ_PANEL : 1;
     p.panel = (p.units + want - 1) / want;
     p.npanels = (p.units + p.panel - 1) / p.panel;
+    p.div_panel_units = make_fastdiv((uint32_t)(p.total_groups * p.panel));
+    p.div_panel = make_fastdiv((uint32_t)p.panel);
+    p.div_last = make_fastdiv((uint32_t)(p.units - (p.npanels - 1) * p.panel));
     // Shares of the CTAs.  CTAs start in index order as multiprocessors come free, the first ones while the
     // previous kernel of the stream is still finishing, so the first CTAs can afford more units than the last:
     // the share falls linearly from mean + lead to mean - lead.

@@ -32,6 +32,21 @@ struct DeviceTables {
     uint64_t num_points;
 };
 
+// n / d by one multiply-high and one shift, for 0 <= n < 2^31 and a divisor fixed per launch
+// (mul = floor(2^(31+l) / d) + 1, shift = l - 1, l = ceil(log2 d); mul = 0 stands for d = 1)
+struct FastDiv {
+    uint32_t mul, shift;
+};
+inline FastDiv make_fastdiv(uint32_t d) {
+    FastDiv f = {0u, 0u};
+    if (d <= 1) return f;
+    uint32_t l = 0;
+    while ((1ull << l) < d) l++;
+    f.mul = (uint32_t)(((1ull << (31 + l)) / d) + 1);
+    f.shift = l - 1;
+    return f;
+}
+
 struct GemvProblemDev {
     const uint8_t *layout;
     const __half *row_scale;
@@ -52,6 +67,7 @@ struct GemvParams {
     int total_units;       // total_groups * units
     int units_base, units_rem;   // total_units divided by the warps of the grid (set by gemv_plan; the one-hot arm's order)
     int panel, npanels;          // unit columns a panel, panels (set by gemv_plan; the 14-byte layout's order of work)
+    FastDiv div_panel_units, div_panel, div_last;   // by total_groups * panel, by panel, by the last panel's width
     int xblocks;                 // most blocks of x any CTA needs (set by gemv_plan)
     int cta_first[kMaxGridCtas + 1];   // first unit of every CTA of the grid, and the total (set by gemv_plan)
     unsigned long long *accum;   // total_groups x 32 fixed-point row accumulators (context scratch, zero between launches)
