@@ -308,18 +308,26 @@ __device__ __forceinline__ StepX load_step(const LaneOffsets &a) {
     return s;
 }
 
-// One half-step: 16 rows x 2 block slots.  wa, wb, wc are this lane's three payload words, h0 and h1 the
-// headers of its two rows for slot (lane & 3) >> 1, sx the step's operand.  Adds to r0 (row g of the 16) and r1
+// One half-step: 16 rows x 2 block slots.  wa, wb, wc are this lane's three payload words, hw the two
+// headers of its rows for slot (lane & 3) >> 1, sx the step's operand.  Adds to r0 (row g of the 16) and r1
 // (row g + 8) this lane's share of scale * sum_i x_i * X_i, X the fixed-point activations: its share is the
 // limb pair (lane & 1) of slot (lane & 3) >> 1.  FIRST: r0 and r1 are written, not added to.
+// (a & b) | c in one instruction
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t r;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+    return r;
+}
+
 template <bool FIRST>
-__device__ __forceinline__ void half_step(uint32_t wa, uint32_t wb, uint32_t wc, uint32_t h0, uint32_t h1, const StepX &sx, uint32_t tq,
+__device__ __forceinline__ void half_step(uint32_t wa, uint32_t wb, uint32_t wc, uint32_t hw, const StepX &sx, uint32_t tq,
                                           float &r0, float &r1) {
     constexpr uint32_t kNib = 0x0f0f0f0fu;
     int d[4];
     mma_k32(d, wa & kNib, wb & kNib, (wa >> 4) & kNib, (wb >> 4) & kNib, sx.b0, sx.b1);
     mma_k16(d, wc & kNib, (wc >> 4) & kNib, sx.b2);
-    const float2 k0 = lds_f2(tq + (h0 << 3)), k1 = lds_f2(tq + (h1 << 3));     // h0, h1: headers of rows g and g + 8
+    // the headers of rows g (low half of hw) and g + 8 (high half), eight bytes an entry; tq is 8 KiB-aligned
+    const float2 k0 = lds_f2(and_or(hw << 3, 0x1ff8u, tq)), k1 = lds_f2(and_or(hw >> 13, 0x1ff8u, tq));
     // sum_i x_i X_i = sum_i u_i (2 X_i) + (parity - 16) sum_i X_i, limb pair by limb pair, in integers
     const int e0 = __float_as_int(k0.y) * sx.xsum + (d[0] + 256 * d[1]);
     const int e1 = __float_as_int(k1.y) * sx.xsum + (d[2] + 256 * d[3]);
@@ -415,8 +423,11 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     extern __shared__ __align__(128) unsigned char smem[];
     // shared memory: ring | per-matrix block constants (1024 x {gain / (4 sqrt m), parity - 16}) | x records | barriers
     unsigned char *ring = smem;
-    float2 *tab = reinterpret_cast<float2 *>(smem + kWarps * kSlots * kTileBytes);
-    unsigned char *xrec = smem + kWarps * kSlots * kTileBytes + p.nprob * 8192;
+    // the block constants start on an 8 KiB boundary of the shared window, so that a matrix's table base and
+    // an entry's offset combine by OR (half_step)
+    const uint32_t tab_pad = (0u - (smem_addr(smem) + kWarps * kSlots * kTileBytes)) & 8191u;
+    float2 *tab = reinterpret_cast<float2 *>(smem + kWarps * kSlots * kTileBytes + tab_pad);
+    unsigned char *xrec = smem + kWarps * kSlots * kTileBytes + tab_pad + p.nprob * 8192;
     uint64_t *bars = reinterpret_cast<uint64_t *>(xrec + ((p.xblocks * kXRecBytes + 127) / 128) * 128);
     uint32_t *warp_max = reinterpret_cast<uint32_t *>(bars + kWarps * kSlots);     // one slot a warp
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -663,10 +674,10 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             acc[1] = acc[2] = acc[3] = 0.f;
 #else
             const StepX s0 = load_step<0>(xa), s1 = load_step<2 * kXRecBytes>(xa);
-            half_step<true>(a0.x, a0.y, a0.z, hh.x & 0xffffu, hh.x >> 16, s0, tq, acc[0], acc[1]);
-            half_step<true>(a0.w, a1.x, a1.y, hh.y & 0xffffu, hh.y >> 16, s0, tq, acc[2], acc[3]);
-            half_step<false>(a1.z, a1.w, a2.x, hh.z & 0xffffu, hh.z >> 16, s1, tq, acc[0], acc[1]);
-            half_step<false>(a2.y, a2.z, a2.w, hh.w & 0xffffu, hh.w >> 16, s1, tq, acc[2], acc[3]);
+            half_step<true>(a0.x, a0.y, a0.z, hh.x, s0, tq, acc[0], acc[1]);
+            half_step<true>(a0.w, a1.x, a1.y, hh.y, s0, tq, acc[2], acc[3]);
+            half_step<false>(a1.z, a1.w, a2.x, hh.z, s1, tq, acc[0], acc[1]);
+            half_step<false>(a2.y, a2.z, a2.w, hh.w, s1, tq, acc[2], acc[3]);
 #endif
             sum += __float2ll_rn(quad_sum(acc) * inv_q);
             LLVQ_TRACE_UNIT(n + t, 2)
@@ -693,7 +704,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                     const uint32_t wa = lds32(piece + 128 * (3 * m) + lane4), wb = lds32(piece + 128 * (3 * m + 1) + lane4);
                     const uint32_t wc = lds32(piece + 128 * (3 * m + 2) + lane4), hw = lds32(piece + 768 + 8 * (lane >> 1) + 4 * m);
                     guard |= settled(wa, wb, wc) | settled(hw, wa, wb);
-                    half_step<false>(wa, wb, wc, hw & 0xffffu, hw >> 16, st, tq, acc[2 * m], acc[2 * m + 1]);
+                    half_step<false>(wa, wb, wc, hw, st, tq, acc[2 * m], acc[2 * m + 1]);
                 }
                 piece += 2 * kCellBytes;
             }
@@ -707,7 +718,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                 const uint32_t wc = lds32(piece + 256 + lane4), hw = lds32(piece + 384 + 4 * (lane >> 1));
                 guard |= settled(wa, wb, wc) | settled(hw, wa, wb);
                 float c0, c1;
-                half_step<true>(wa, wb, wc, hw & 0xffffu, hw >> 16, st, tq, c0, c1);
+                half_step<true>(wa, wb, wc, hw, st, tq, c0, c1);
                 acc[0] += high_lane ? 0.f : c0; acc[1] += high_lane ? 0.f : c1;
                 acc[2] += high_lane ? c0 : 0.f; acc[3] += high_lane ? c1 : 0.f;
             }
@@ -982,7 +993,7 @@ GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
         if (hi - lo > p.xblocks) p.xblocks = hi - lo;
     }
     const size_t xbytes = ((size_t)p.xblocks * kXRecBytes + 127) / 128 * 128;
-    g.smem = (size_t)kWarps * kSlots * kTileBytes + (size_t)p.nprob * 8192 + xbytes + kWarps * kSlots * 8 + kWarps * 4 + 16;
+    g.smem = (size_t)kWarps * kSlots * kTileBytes + 8192 /* alignment of the tables */ + (size_t)p.nprob * 8192 + xbytes + kWarps * kSlots * 8 + kWarps * 4 + 16;
     return g;
 }
 
