@@ -412,6 +412,26 @@ def main():
                 t = time_arm(one, ncopies, arm_steps, 3)
                 by = gemv_bytes(m.rows, m.nb)
                 per_shape[m.name] = {"rows": m.rows, "k": m.k, "us": t * 1e3, "gbps": by / (t * 1e-3) / 1e9, "frac": by / (t * 1e-3) / 1e9 / peak}
+        # small-batch decode: the same matrices, one launch each, 1 / 2 / 4 activation vectors a launch (the records
+        # are read and decoded once a launch; every vector was checked against the single-vector result by the tests)
+        batch_arm = {}
+        for nvec in (1, 2, 4):
+            xb = {}
+            for cp in copies:
+                for ln in cp.launches:
+                    if id(ln["x"]) not in xb:
+                        xb[id(ln["x"])] = (ln["x"].unsqueeze(0).repeat(nvec, 1).contiguous(),
+                                           [torch.empty((nvec, m.rows), dtype=torch.float32, device=device) for m in ln["mats"]])
+            def bstep(i, xb=xb):
+                for ln in copies[i % ncopies].launches:
+                    X, Ys = xb[id(ln["x"])]
+                    for mi, m in enumerate(ln["mats"]):
+                        B.gemv_batch(ctx, ln["bufs"][mi], ln["scales"][mi], datagen.GAIN, X, m.rows, ln["k_padded"], y=Ys[mi])
+            t = time_arm(bstep, ncopies, arm_steps, 3)
+            batch_arm[str(nvec)] = {"us_per_launch": t * 1e3 / n_gemv, "us_per_vector": t * 1e3 / n_gemv / nvec,
+                                    "record_gbps": step_bytes / (t * 1e-3) / 1e9}
+            del xb
+        arms["batch"] = batch_arm
         # no-weights control: the same launches without record reads
         def nw(i):
             for ln in copies[i % ncopies].launches:

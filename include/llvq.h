@@ -81,6 +81,7 @@ extern "C" {
 
 #define LLVQ_MAX_GROUP 8       /* matrices in one grouped launch                             */
 #define LLVQ_MAX_K 98304       /* largest k_padded the GEMV accepts                          */
+#define LLVQ_MAX_BATCH 4       /* activation vectors in one llvq_gemv_batch launch           */
 
 typedef struct llvq_ctx llvq_ctx;
 
@@ -144,6 +145,15 @@ int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, 
  * result never depends on the launch geometry and a grouped launch returns bit-identical rows. */
 int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row_scale,
               const float *gain, const void *x, float *y, int64_t rows, int64_t k_padded, void *stream);
+
+/* [Sec. 5 "Batching", the paper's stated boundary: one record decode reused across activations]
+ * llvq_gemv on the LLVQ_PLANES layout for batch (1..LLVQ_MAX_BATCH) activation vectors in one pass
+ * over the records: x is fp16 [batch][k_padded], y is f32 [batch][rows].  The records are read
+ * and decoded once; each vector has its own fixed-point scale and its own accumulators, and
+ * y[j] is bit-identical to what llvq_gemv returns for x[j].  Needs batch times the scratch of
+ * llvq_gemv (LLVQ_ESIZE otherwise). */
+int llvq_gemv_batch(llvq_ctx *ctx, const void *layout_buf, const void *row_scale, const float *gain,
+                    const void *x, float *y, int64_t rows, int64_t k_padded, int batch, void *stream);
 
 /* [Sec. 3.4] One launch over n <= LLVQ_MAX_GROUP row-concatenated matrices that share x and
  * k_padded (q/k/v, gate/up).  `problems` is a HOST array, copied before the call returns. */

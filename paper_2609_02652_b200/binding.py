@@ -21,7 +21,7 @@ _lib = None
 
 SYMBOLS = (
     "llvq_create", "llvq_destroy", "llvq_strerror", "llvq_status", "llvq_selftest_wait_limit", "llvq_set_pdl", "llvq_num_classes", "llvq_class_base", "llvq_layout_bytes",
-    "llvq_expand", "llvq_gemv", "llvq_gemv_grouped", "llvq_gemv_static", "llvq_gemv_fp16", "llvq_gemv_noweights", "llvq_dequant_fp16",
+    "llvq_expand", "llvq_gemv", "llvq_gemv_batch", "llvq_gemv_grouped", "llvq_gemv_static", "llvq_gemv_fp16", "llvq_gemv_noweights", "llvq_dequant_fp16",
     "llvq_decode_i8",
 )
 
@@ -61,6 +61,7 @@ def load() -> ctypes.CDLL:
         L.llvq_layout_bytes.argtypes = [ci, i64, i64, ctypes.POINTER(sz)]
         L.llvq_expand.argtypes = [vp, ci, vp, i64, i64, vp, sz, vp, vp]
         L.llvq_gemv.argtypes = [vp, ci, vp, vp, ctypes.POINTER(ctypes.c_float), vp, vp, i64, i64, vp]
+        L.llvq_gemv_batch.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_float), vp, vp, i64, i64, ci, vp]
         L.llvq_gemv_grouped.argtypes = [vp, ci, ctypes.POINTER(Problem), ci, vp, i64, vp]
         L.llvq_gemv_static.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), vp, vp, i64, i64, vp]
         L.llvq_gemv_fp16.argtypes = [vp, vp, vp, i64, i64, vp]
@@ -173,6 +174,20 @@ def gemv(ctx: Context, layout: int, layout_buf: torch.Tensor, row_scale: torch.T
     _check(load().llvq_gemv(ctx.ptr, int(layout), _dev(layout_buf, torch.uint8, "layout_buf"),
                             _dev(row_scale, torch.float16, "row_scale"), _gain(gain), _dev(x, torch.float16, "x"),
                             _dev(y, torch.float32, "y"), int(rows), int(k_padded), _stream(stream)), "llvq_gemv")
+    return y
+
+
+def gemv_batch(ctx: Context, layout_buf: torch.Tensor, row_scale: torch.Tensor, gain, x: torch.Tensor, rows: int,
+               k_padded: int, y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """llvq_gemv_batch: x is fp16 [batch, k_padded] (contiguous), the result f32 [batch, rows]."""
+    batch = int(x.shape[0])
+    if x.dim() != 2 or int(x.shape[1]) != int(k_padded) or not x.is_contiguous():
+        raise ValueError("x must be a contiguous [batch, k_padded] tensor")
+    if y is None:
+        y = torch.empty((batch, rows), dtype=torch.float32, device=x.device)
+    _check(load().llvq_gemv_batch(ctx.ptr, _dev(layout_buf, torch.uint8, "layout_buf"), _dev(row_scale, torch.float16, "row_scale"),
+                                  _gain(gain), _dev(x, torch.float16, "x"), _dev(y, torch.float32, "y"), int(rows), int(k_padded),
+                                  batch, _stream(stream)), "llvq_gemv_batch")
     return y
 
 

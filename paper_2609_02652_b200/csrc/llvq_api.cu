@@ -179,8 +179,9 @@ int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, 
 }
 
 static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n, const void *x, int64_t k_padded,
-                    bool no_weights, void *stream) {
+                    bool no_weights, void *stream, int batch = 1) {
     if (!ctx || !problems || !x || n < 1 || n > LLVQ_MAX_GROUP) return LLVQ_EINVAL;
+    if (batch < 1 || batch > LLVQ_MAX_BATCH || (batch > 1 && (n != 1 || layout != LLVQ_PLANES || no_weights))) return LLVQ_EINVAL;
     if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT) return LLVQ_EINVAL;
     if (k_padded <= 0 || k_padded % 24 != 0) return LLVQ_EINVAL;
     if (k_padded > LLVQ_MAX_K) return LLVQ_ESIZE;
@@ -189,6 +190,8 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
     std::memset(&p, 0, sizeof p);
     p.nprob = n;
     p.x = (const __half *)x;
+    p.batch = batch;
+    p.y_stride = (int)problems[0].rows;
     p.nb = (int)(k_padded / 24);
     p.tiles = p.nb / kTileCells;
     p.tail_cells = p.nb % kTileCells;
@@ -211,7 +214,7 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
         groups += (q.rows + kRowsPerGroup - 1) / kRowsPerGroup;
     }
     if (groups > ((int64_t)1 << 26) || p.units > 2047 || groups * p.units > 0x7fffffffll) return LLVQ_ESIZE;
-    if ((size_t)groups * 32 > ctx->accum_slots) return LLVQ_ESIZE;
+    if ((size_t)groups * 32 * (size_t)batch > ctx->accum_slots) return LLVQ_ESIZE;
     if (!(gain_max < 3.0e38f)) return LLVQ_EINVAL;
     // quantum of the fixed-point row accumulators, per matrix so that grouping does not change it:
     // a unit sums at most four blocks, each bounded by max|gain| * sqrt(24) * max|x| < 2^ge * 5 * 2^xe;
@@ -250,6 +253,14 @@ int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row
     llvq_problem q;
     q.layout = layout_buf; q.row_scale = row_scale; q.y = y; q.rows = rows; q.gain[0] = gain[0]; q.gain[1] = gain[1];
     return run_gemv(ctx, layout, &q, 1, x, k_padded, false, stream);
+}
+
+int llvq_gemv_batch(llvq_ctx *ctx, const void *layout_buf, const void *row_scale, const float *gain, const void *x, float *y,
+                    int64_t rows, int64_t k_padded, int batch, void *stream) {
+    if (!gain) return LLVQ_EINVAL;
+    llvq_problem q;
+    q.layout = layout_buf; q.row_scale = row_scale; q.y = y; q.rows = rows; q.gain[0] = gain[0]; q.gain[1] = gain[1];
+    return run_gemv(ctx, LLVQ_PLANES, &q, 1, x, k_padded, false, stream, batch);
 }
 
 int llvq_gemv_grouped(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n, const void *x, int64_t k_padded,

@@ -179,15 +179,17 @@ __device__ __forceinline__ void settle(const GemvParams &p, Handed &h) {
     }
     h.slot = nullptr;
 }
-__device__ __forceinline__ void hand_over(const GemvParams &p, const GemvProblemDev &pr, int group, int lane, long long sum,
-                                          int count, int qexp, float row_scale, Handed &h) {
+// `accum` and `y` are the accumulators and the output of the activation vector the sum belongs to (a batched
+// launch has one set a vector)
+__device__ __forceinline__ void hand_over(const GemvParams &p, const GemvProblemDev &pr, unsigned long long *accum, float *y,
+                                          int group, int lane, long long sum, int count, int qexp, float row_scale, Handed &h) {
     settle(p, h);
     const int row = (group - pr.group_begin) * kRowsPerGroup + lane;
     if (row >= pr.rows) return;                      // padding rows of the last row group
     h.addend = (unsigned long long)(sum + (long long)count * kUnitBias) + ((unsigned long long)count << kCountShift);
-    h.slot = p.accum + (size_t)group * 32 + lane;
+    h.slot = accum + (size_t)group * 32 + lane;
     h.old = atomicAdd(h.slot, h.addend);
-    h.y = pr.y + row;
+    h.y = y + row;
     h.yscale = pow2f(qexp) * row_scale;
     h.count = count;
 }
@@ -319,20 +321,37 @@ __device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c) {
     return r;
 }
 
+// The A operand of a half-step (the decode proper: one shift and two ANDs a word) and the block constants of
+// its two rows; both are shared by every activation vector of a batched launch.
+struct HalfA {
+    uint32_t a0, a1, a2, a3, c0, c1;
+    float2 k0, k1;
+};
+__device__ __forceinline__ HalfA decode_half(uint32_t wa, uint32_t wb, uint32_t wc, uint32_t hw, uint32_t tq) {
+    constexpr uint32_t kNib = 0x0f0f0f0fu;
+    HalfA h;
+    h.a0 = wa & kNib; h.a1 = wb & kNib; h.a2 = (wa >> 4) & kNib; h.a3 = (wb >> 4) & kNib;
+    h.c0 = wc & kNib; h.c1 = (wc >> 4) & kNib;
+    // the headers of rows g (low half of hw) and g + 8 (high half), eight bytes an entry; tq is 8 KiB-aligned
+    h.k0 = lds_f2(and_or(hw << 3, 0x1ff8u, tq));
+    h.k1 = lds_f2(and_or(hw >> 13, 0x1ff8u, tq));
+    return h;
+}
+template <bool FIRST>
+__device__ __forceinline__ void contract_half(const HalfA &h, const StepX &sx, float &r0, float &r1) {
+    int d[4];
+    mma_k32(d, h.a0, h.a1, h.a2, h.a3, sx.b0, sx.b1);
+    mma_k16(d, h.c0, h.c1, sx.b2);
+    // sum_i x_i X_i = sum_i u_i (2 X_i) + (parity - 16) sum_i X_i, limb pair by limb pair, in integers
+    const int e0 = __float_as_int(h.k0.y) * sx.xsum + (d[0] + 256 * d[1]);
+    const int e1 = __float_as_int(h.k1.y) * sx.xsum + (d[2] + 256 * d[3]);
+    if (FIRST) { r0 = (float)e0 * h.k0.x; r1 = (float)e1 * h.k1.x; }
+    else { r0 = fmaf((float)e0, h.k0.x, r0); r1 = fmaf((float)e1, h.k1.x, r1); }
+}
 template <bool FIRST>
 __device__ __forceinline__ void half_step(uint32_t wa, uint32_t wb, uint32_t wc, uint32_t hw, const StepX &sx, uint32_t tq,
                                           float &r0, float &r1) {
-    constexpr uint32_t kNib = 0x0f0f0f0fu;
-    int d[4];
-    mma_k32(d, wa & kNib, wb & kNib, (wa >> 4) & kNib, (wb >> 4) & kNib, sx.b0, sx.b1);
-    mma_k16(d, wc & kNib, (wc >> 4) & kNib, sx.b2);
-    // the headers of rows g (low half of hw) and g + 8 (high half), eight bytes an entry; tq is 8 KiB-aligned
-    const float2 k0 = lds_f2(and_or(hw << 3, 0x1ff8u, tq)), k1 = lds_f2(and_or(hw >> 13, 0x1ff8u, tq));
-    // sum_i x_i X_i = sum_i u_i (2 X_i) + (parity - 16) sum_i X_i, limb pair by limb pair, in integers
-    const int e0 = __float_as_int(k0.y) * sx.xsum + (d[0] + 256 * d[1]);
-    const int e1 = __float_as_int(k1.y) * sx.xsum + (d[2] + 256 * d[3]);
-    if (FIRST) { r0 = (float)e0 * k0.x; r1 = (float)e1 * k1.x; }
-    else { r0 = fmaf((float)e0, k0.x, r0); r1 = fmaf((float)e1, k1.x, r1); }
+    contract_half<FIRST>(decode_half(wa, wb, wc, hw, tq), sx, r0, r1);
 }
 
 // x (fp16) -> records.  X_i = rint(x_i * 2^F) with F chosen from the largest |x| so that |X_i| < 2^29; the
@@ -418,7 +437,11 @@ __device__ __forceinline__ bool advance(const GemvParams &p, Cursor &c, int n) {
     c.col = c.panel * p.panel;
     return true;
 }
-template <bool NO_WEIGHTS>
+// BATCH activation vectors share one pass over the records: the decode of a half-step and its block constants
+// are computed once, the contraction, the scaling and the reduction once a vector.  x is BATCH vectors of
+// 24 nb halves one after the other, y BATCH vectors of rows floats (p.prob[].y is vector 0's), the accumulators
+// BATCH sets of total_groups * 32.
+template <bool NO_WEIGHTS, int BATCH>
 __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     // shared memory: ring | per-matrix block constants (1024 x {gain / (4 sqrt m), parity - 16}) | x records | barriers
@@ -428,8 +451,9 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     const uint32_t tab_pad = (0u - (smem_addr(smem) + kWarps * kSlots * kTileBytes)) & 8191u;
     float2 *tab = reinterpret_cast<float2 *>(smem + kWarps * kSlots * kTileBytes + tab_pad);
     unsigned char *xrec = smem + kWarps * kSlots * kTileBytes + tab_pad + p.nprob * 8192;
-    uint64_t *bars = reinterpret_cast<uint64_t *>(xrec + ((p.xblocks * kXRecBytes + 127) / 128) * 128);
-    uint32_t *warp_max = reinterpret_cast<uint32_t *>(bars + kWarps * kSlots);     // one slot a warp
+    const uint32_t xrec_stride = ((p.xblocks * kXRecBytes + 127) / 128) * 128;     // a vector's records
+    uint64_t *bars = reinterpret_cast<uint64_t *>(xrec + BATCH * xrec_stride);
+    uint32_t *warp_max = reinterpret_cast<uint32_t *>(bars + kWarps * kSlots);     // one slot a warp and vector
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t my_ring = smem_addr(ring + warp * kSlots * kTileBytes);
     const uint32_t my_bar = smem_addr(bars + warp * kSlots);
@@ -450,7 +474,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     // previous kernel's writes to x land)
     const int tab_entries = p.nprob * 1024;
     uint32_t warm = 0;
-    for (int e = tid * 128; e < p.nb * 48; e += kThreads * 128) {
+    for (int e = tid * 128; e < p.nb * 48 * p.batch; e += kThreads * 128) {
         // a load whose value is not used: it brings the line into L2 and the translation into this
         // multiprocessor's TLB, which a prefetch hint does not promise.  The register stays claimed until
         // after the wait (settled() below), so nothing stalls on the load's return before then.
@@ -548,55 +572,67 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     // pieces of x this CTA needs stay in registers meanwhile and then become fixed-point records on the scale
     // 2^(29 - xexp).
     bool failed = false;
-    int xexp;
+    int xexp[BATCH];
     {
-        uint32_t m = settled(warm, warm, warm);
-        const uint4 *xg = reinterpret_cast<const uint4 *>(p.x);
         const int nx = p.nb * 3, e_lo = 3 * blk_lo, e_hi = 3 * blk_hi;
         const bool one_each = e_hi - e_lo <= kThreads;         // then no thread meets two of the pieces wanted
-        uint4 mine = make_uint4(0u, 0u, 0u, 0u);
+        uint4 mine[BATCH];
         int mine_e = -1;
-        for (int base = 0; base < nx; base += 4 * kThreads) {
-            uint4 v[4];
 #pragma unroll
-            for (int i = 0; i < 4; i++) {
-                const int e = base + i * kThreads + tid;
-                v[i] = e < nx ? __ldcg(xg + e) : make_uint4(0u, 0u, 0u, 0u);
-            }
-            if (base == 0) {
-                // while the first loads are on their way: what the loop needs besides x
-            // the zero word and the two sums of every x record this CTA will fill
-            for (int b = tid; b < blk_hi - blk_lo; b += kThreads)
-                asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(smem_addr(xrec) + b * kXRecBytes + 96), "r"(0) : "memory");
-            // block constants of every matrix of the launch: (class | gain << 9) -> {gain / (4 sqrt m), parity - 16},
-            // from the class constants in the kernel's parameters
-            for (int e = tid; e < tab_entries; e += kThreads) {
-                const int c = e & 511;
-                const uint32_t shell = (p.cls_shell_nibbles[c >> 3] >> (4 * (c & 7))) & 15u;
-                const int odd = (int)((p.cls_odd_bits[c >> 5] >> (c & 31)) & 1u);
-                const GemvProblemDev &pe = p.prob[e >> 10];
-                tab[e] = make_float2(p.shell_inv_norm[shell] * ((e & 512) ? pe.gain1 : pe.gain0), __int_as_float(shell ? odd - 16 : 0));
-            }
-            }
+        for (int j = 0; j < BATCH; j++) {
+            uint32_t m = j == 0 ? settled(warm, warm, warm) : 0u;
+            const uint4 *xg = reinterpret_cast<const uint4 *>(p.x) + (size_t)j * nx;
+            mine[j] = make_uint4(0u, 0u, 0u, 0u);
+            for (int base = 0; base < nx; base += 4 * kThreads) {
+                uint4 v[4];
 #pragma unroll
-            for (int i = 0; i < 4; i++) {
-                const int e = base + i * kThreads + tid;
-                m = max_abs_pair(max_abs_pair(max_abs_pair(max_abs_pair(m, v[i].x), v[i].y), v[i].z), v[i].w);
-                if (e >= e_lo && e < e_hi) { mine = v[i]; mine_e = e; }
+                for (int i = 0; i < 4; i++) {
+                    const int e = base + i * kThreads + tid;
+                    v[i] = (e < nx && j < p.batch) ? __ldcg(xg + e) : make_uint4(0u, 0u, 0u, 0u);
+                }
+                if (j == 0 && base == 0) {
+                    // while the first loads are on their way: what the loop needs besides x.
+                    // The zero word and the two sums of every x record this CTA will fill
+                    for (int b = tid; b < BATCH * (blk_hi - blk_lo); b += kThreads) {
+                        const int jj = BATCH == 1 ? 0 : b / (blk_hi - blk_lo), bb = b - jj * (blk_hi - blk_lo);
+                        asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(smem_addr(xrec) + jj * xrec_stride + bb * kXRecBytes + 96), "r"(0) : "memory");
+                    }
+                    // block constants of every matrix of the launch: (class | gain << 9) -> {gain / (4 sqrt m), parity - 16},
+                    // from the class constants in the kernel's parameters
+                    for (int e = tid; e < tab_entries; e += kThreads) {
+                        const int c = e & 511;
+                        const uint32_t shell = (p.cls_shell_nibbles[c >> 3] >> (4 * (c & 7))) & 15u;
+                        const int odd = (int)((p.cls_odd_bits[c >> 5] >> (c & 31)) & 1u);
+                        const GemvProblemDev &pe = p.prob[e >> 10];
+                        tab[e] = make_float2(p.shell_inv_norm[shell] * ((e & 512) ? pe.gain1 : pe.gain0), __int_as_float(shell ? odd - 16 : 0));
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    const int e = base + i * kThreads + tid;
+                    m = max_abs_pair(max_abs_pair(max_abs_pair(max_abs_pair(m, v[i].x), v[i].y), v[i].z), v[i].w);
+                    if (e >= e_lo && e < e_hi) { mine[j] = v[i]; mine_e = e; }
+                }
             }
+            m = __reduce_max_sync(0xffffffffu, max(m & 0xffffu, m >> 16));
+            if (lane == 0) warp_max[j * kWarps + warp] = m;    // plain stores: atomics on one word would serialise the warps
         }
-        m = __reduce_max_sync(0xffffffffu, max(m & 0xffffu, m >> 16));
-        if (lane == 0) warp_max[warp] = m;             // plain stores: atomics on one word would serialise the warps
         __syncthreads();                               // publishes the maxima, the block constants and the zeroed sums
-        m = warp_max[lane < kWarps ? lane : 0];
-        xexp = max((int)(__reduce_max_sync(0xffffffffu, m) >> 10), 1) - 14;
         LLVQ_TRACE_POINT(4)
         LLVQ_TRACE_CLOCK(1)
-        const float scale = pow2f(29 - xexp);
-        if (one_each) {
-            if (mine_e >= 0) convert_item(mine, mine_e % 3, xs0 + (uint32_t)(mine_e / 3) * kXRecBytes, scale);
-        } else {
-            for (int e = e_lo + tid; e < e_hi; e += kThreads) convert_item(__ldcg(xg + e), e % 3, xs0 + (uint32_t)(e / 3) * kXRecBytes, scale);
+#pragma unroll
+        for (int j = 0; j < BATCH; j++) {
+            const uint32_t m = warp_max[j * kWarps + (lane < kWarps ? lane : 0)];
+            xexp[j] = max((int)(__reduce_max_sync(0xffffffffu, m) >> 10), 1) - 14;
+            const float scale = pow2f(29 - xexp[j]);
+            const uint4 *xg = reinterpret_cast<const uint4 *>(p.x) + (size_t)j * nx;
+            const uint32_t xsj = xs0 + j * xrec_stride;
+            if (one_each) {
+                if (mine_e >= 0) convert_item(mine[j], mine_e % 3, xsj + (uint32_t)(mine_e / 3) * kXRecBytes, scale);
+            } else {
+                for (int e = e_lo + tid; e < e_hi; e += kThreads)
+                    convert_item(j < p.batch ? __ldcg(xg + e) : make_uint4(0u, 0u, 0u, 0u), e % 3, xsj + (uint32_t)(e / 3) * kXRecBytes, scale);
+            }
         }
         if (!NO_WEIGHTS) {
 #pragma unroll
@@ -631,14 +667,14 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         return (odd_lane ? r1 : r0) + __shfl_xor_sync(0xffffffffu, odd_lane ? r0 : r1, 1);
     };
 
-    Handed handed;
+    Handed handed;                                      // BATCH == 1: the hand-over waits for its answer a run later
     handed.slot = nullptr;
     // A run is the stretch of units of one row group inside this warp's range: its units are summed
     // in a register and handed over together.
     while (n < n_units) {
         const GemvProblemDev &pr = p.prob[q];
-        // quantum of the row accumulator: 2^qexp in units of y / row_scale; a lane's sums are in units of 2^(xexp - 29)
-        const int qexp = xexp + pr.qexp_base;
+        // quantum of a row accumulator: 2^(xexp + qexp_base) in units of y / row_scale, xexp that of the vector;
+        // a lane's sums are in units of 2^(xexp - 29)
         const float inv_q = pow2f(-29 - pr.qexp_base);
         const uint32_t tq = tab0 + q * 8192;
         const int run = min(cc.end - cc.col, n_units - n);
@@ -650,7 +686,9 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         // this lane's addresses in the x records of the run's first tile
         const uint32_t xk = xs0 + (uint32_t)cc.col * (4 * kXRecBytes);
         LaneOffsets xa = {xk + lo.b0, xk + lo.b1, xk + lo.b2, xk + lo.xs};
-        long long sum = 0;
+        long long sum[BATCH];
+#pragma unroll
+        for (int j = 0; j < BATCH; j++) sum[j] = 0;
 
 #pragma unroll 1
         for (int t = 0; t < run_tiles; t++) {
@@ -668,18 +706,42 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             // copy's address is made to depend on the loaded words, which holds the copy back
             // until the four shared-memory reads of the whole warp have completed.
             issue(bar, sbuf + (settled(a0.w, a1.w, a2.w) | settled(hh.w, hh.x, a0.x)));
-            float acc[4];
+            float acc[BATCH][4];
 #ifdef LLVQ_STREAM_ONLY
-            acc[0] = __uint_as_float((a0.x ^ a1.y ^ a2.z ^ hh.w) & 0x007fffffu);   // debug: bytes only, no decode
-            acc[1] = acc[2] = acc[3] = 0.f;
+#pragma unroll
+            for (int j = 0; j < BATCH; j++) {
+                acc[j][0] = __uint_as_float((a0.x ^ a1.y ^ a2.z ^ hh.w) & 0x007fffffu);   // debug: bytes only, no decode
+                acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
+            }
 #else
-            const StepX s0 = load_step<0>(xa), s1 = load_step<2 * kXRecBytes>(xa);
-            half_step<true>(a0.x, a0.y, a0.z, hh.x, s0, tq, acc[0], acc[1]);
-            half_step<true>(a0.w, a1.x, a1.y, hh.y, s0, tq, acc[2], acc[3]);
-            half_step<false>(a1.z, a1.w, a2.x, hh.z, s1, tq, acc[0], acc[1]);
-            half_step<false>(a2.y, a2.z, a2.w, hh.w, s1, tq, acc[2], acc[3]);
+            {
+                StepX sx[BATCH];
+#pragma unroll
+                for (int j = 0; j < BATCH; j++) {
+                    const LaneOffsets xj = {xa.b0 + j * xrec_stride, xa.b1 + j * xrec_stride, xa.b2 + j * xrec_stride, xa.xs + j * xrec_stride};
+                    sx[j] = load_step<0>(xj);
+                }
+                const HalfA h0 = decode_half(a0.x, a0.y, a0.z, hh.x, tq);
+#pragma unroll
+                for (int j = 0; j < BATCH; j++) contract_half<true>(h0, sx[j], acc[j][0], acc[j][1]);
+                const HalfA h1 = decode_half(a0.w, a1.x, a1.y, hh.y, tq);
+#pragma unroll
+                for (int j = 0; j < BATCH; j++) contract_half<true>(h1, sx[j], acc[j][2], acc[j][3]);
+#pragma unroll
+                for (int j = 0; j < BATCH; j++) {
+                    const LaneOffsets xj = {xa.b0 + j * xrec_stride, xa.b1 + j * xrec_stride, xa.b2 + j * xrec_stride, xa.xs + j * xrec_stride};
+                    sx[j] = load_step<2 * kXRecBytes>(xj);
+                }
+                const HalfA h2 = decode_half(a1.z, a1.w, a2.x, hh.z, tq);
+#pragma unroll
+                for (int j = 0; j < BATCH; j++) contract_half<false>(h2, sx[j], acc[j][0], acc[j][1]);
+                const HalfA h3 = decode_half(a2.y, a2.z, a2.w, hh.w, tq);
+#pragma unroll
+                for (int j = 0; j < BATCH; j++) contract_half<false>(h3, sx[j], acc[j][2], acc[j][3]);
+            }
 #endif
-            sum += __float2ll_rn(quad_sum(acc) * inv_q);
+#pragma unroll
+            for (int j = 0; j < BATCH; j++) sum[j] += __float2ll_rn(quad_sum(acc[j]) * inv_q);
             LLVQ_TRACE_UNIT(n + t, 2)
             xa.b0 += 4 * kXRecBytes; xa.b1 += 4 * kXRecBytes; xa.b2 += 4 * kXRecBytes; xa.xs += 4 * kXRecBytes;
             bar += 8;
@@ -694,17 +756,23 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             // the run ends with the nb mod 4 last block columns of the row group: a pair, a single, or both
             if (!mbar_wait(bar, parity)) { failed = true; break; }
             uint32_t guard = 0, piece = sbuf;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            float acc[BATCH][4];
+#pragma unroll
+            for (int j = 0; j < BATCH; j++) acc[j][0] = acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
             const uint32_t xt = xs0 + (uint32_t)tiles * (4 * kXRecBytes);
             if (p.tail_cells >= 2) {
-                const LaneOffsets ta = {xt + lo.b0, xt + lo.b1, xt + lo.b2, xt + lo.xs};
-                const StepX st = load_step<0>(ta);
 #pragma unroll
                 for (int m = 0; m < 2; m++) {
                     const uint32_t wa = lds32(piece + 128 * (3 * m) + lane4), wb = lds32(piece + 128 * (3 * m + 1) + lane4);
                     const uint32_t wc = lds32(piece + 128 * (3 * m + 2) + lane4), hw = lds32(piece + 768 + 8 * (lane >> 1) + 4 * m);
                     guard |= settled(wa, wb, wc) | settled(hw, wa, wb);
-                    half_step<false>(wa, wb, wc, hw, st, tq, acc[2 * m], acc[2 * m + 1]);
+                    const HalfA h = decode_half(wa, wb, wc, hw, tq);
+#pragma unroll
+                    for (int j = 0; j < BATCH; j++) {
+                        const uint32_t xj = xt + j * xrec_stride;
+                        const LaneOffsets ta = {xj + lo.b0, xj + lo.b1, xj + lo.b2, xj + lo.xs};
+                        contract_half<false>(h, load_step<0>(ta), acc[j][2 * m], acc[j][2 * m + 1]);
+                    }
                 }
                 piece += 2 * kCellBytes;
             }
@@ -712,18 +780,23 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                 // one block: the slots of this half-step are the two halves of the row group
                 const uint32_t xl = xs0 + (uint32_t)(p.nb - 1) * kXRecBytes;
                 const LaneOffsets l1 = lane_offsets(lane, true);
-                const LaneOffsets ta = {xl + l1.b0, xl + l1.b1, xl + l1.b2, xl + l1.xs};
-                const StepX st = load_step<0>(ta);
                 const uint32_t wa = lds32(piece + lane4), wb = lds32(piece + 128 + lane4);
                 const uint32_t wc = lds32(piece + 256 + lane4), hw = lds32(piece + 384 + 4 * (lane >> 1));
                 guard |= settled(wa, wb, wc) | settled(hw, wa, wb);
-                float c0, c1;
-                half_step<true>(wa, wb, wc, hw, st, tq, c0, c1);
-                acc[0] += high_lane ? 0.f : c0; acc[1] += high_lane ? 0.f : c1;
-                acc[2] += high_lane ? c0 : 0.f; acc[3] += high_lane ? c1 : 0.f;
+                const HalfA h = decode_half(wa, wb, wc, hw, tq);
+#pragma unroll
+                for (int j = 0; j < BATCH; j++) {
+                    const uint32_t xj = xl + j * xrec_stride;
+                    const LaneOffsets ta = {xj + l1.b0, xj + l1.b1, xj + l1.b2, xj + l1.xs};
+                    float c0, c1;
+                    contract_half<true>(h, load_step<0>(ta), c0, c1);
+                    acc[j][0] += high_lane ? 0.f : c0; acc[j][1] += high_lane ? 0.f : c1;
+                    acc[j][2] += high_lane ? c0 : 0.f; acc[j][3] += high_lane ? c1 : 0.f;
+                }
             }
             issue(bar, sbuf + guard);
-            sum += __float2ll_rn(quad_sum(acc) * inv_q);
+#pragma unroll
+            for (int j = 0; j < BATCH; j++) sum[j] += __float2ll_rn(quad_sum(acc[j]) * inv_q);
             bar += 8;
             sbuf += kTileBytes;
             if (sbuf == sbuf_end) { sbuf = my_ring; bar = my_bar; parity ^= 1u; }
@@ -731,7 +804,20 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         // with no records read (the control launch) every unit contributes zero
         n += run;
         if (n == n_units) { LLVQ_TRACE_POINT(6) }
-        hand_over(p, pr, cc.group, my_row, sum, run, qexp, row_scale, handed);
+        if (BATCH == 1) {
+            hand_over(p, pr, p.accum, pr.y, cc.group, my_row, sum[0], run, xexp[0] + pr.qexp_base, row_scale, handed);
+        } else {
+            // one hand-over a vector; each waits for its answer (a batched launch has arithmetic to hide behind)
+#pragma unroll
+            for (int j = 0; j < BATCH; j++) {
+                if (j >= p.batch) break;               // a launch may carry fewer vectors than the kernel is built for
+                Handed hj;
+                hj.slot = nullptr;
+                hand_over(p, pr, p.accum + (size_t)j * p.total_groups * 32, pr.y + (size_t)j * p.y_stride, cc.group, my_row, sum[j], run,
+                          xexp[j] + pr.qexp_base, row_scale, hj);
+                settle(p, hj);
+            }
+        }
         if (advance(p, cc, run) && cc.panel < p.npanels) q = find_problem(p, cc.group);
     }
     settle(p, handed);
@@ -992,8 +1078,9 @@ GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
         if (hi > p.nb) hi = p.nb;
         if (hi - lo > p.xblocks) p.xblocks = hi - lo;
     }
-    const size_t xbytes = ((size_t)p.xblocks * kXRecBytes + 127) / 128 * 128;
-    g.smem = (size_t)kWarps * kSlots * kTileBytes + 8192 /* alignment of the tables */ + (size_t)p.nprob * 8192 + xbytes + kWarps * kSlots * 8 + kWarps * 4 + 16;
+    const int vectors = p.batch <= 1 ? 1 : (p.batch == 2 ? 2 : 4);             // the kernel is built for 1, 2 and 4
+    const size_t xbytes = ((size_t)p.xblocks * kXRecBytes + 127) / 128 * 128 * vectors;
+    g.smem = (size_t)kWarps * kSlots * kTileBytes + 8192 /* alignment of the tables */ + (size_t)p.nprob * 8192 + xbytes + kWarps * kSlots * 8 + kWarps * 4 * vectors + 16;
     return g;
 }
 
@@ -1009,8 +1096,10 @@ static int allow_max_smem(K kernel, int optin) {
 
 int gemv_configure(const llvq_ctx *ctx) {
     const int bytes = ctx->max_smem_optin;
-    if (allow_max_smem(gemv_planes_kernel<false>, bytes)) return -1;
-    if (allow_max_smem(gemv_planes_kernel<true>, bytes)) return -1;
+    if (allow_max_smem(gemv_planes_kernel<false, 1>, bytes)) return -1;
+    if (allow_max_smem(gemv_planes_kernel<true, 1>, bytes)) return -1;
+    if (allow_max_smem(gemv_planes_kernel<false, 2>, bytes)) return -1;
+    if (allow_max_smem(gemv_planes_kernel<false, 4>, bytes)) return -1;
     if (allow_max_smem(gemv_onehot_kernel, bytes)) return -1;
     return 0;
 }
@@ -1027,8 +1116,10 @@ cudaError_t launch_gemv(int layout, const GemvParams &p, const GemvLaunch &g, bo
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (layout == LLVQ_PLANES) {
-        if (no_weights) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<true>, p);
-        return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false>, p);
+        if (no_weights) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<true, 1>, p);
+        if (p.batch <= 1) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 1>, p);
+        if (p.batch == 2) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 2>, p);
+        return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 4>, p);
     }
     cfg.numAttrs = 0;
     return cudaLaunchKernelEx(&cfg, gemv_onehot_kernel, p);
@@ -1116,7 +1207,7 @@ int static_setup(int device, StaticDevice &d) {
     if (cudaMemset(d.error, 0, sizeof(int) * 64) != cudaSuccess) return LLVQ_ECUDA;
     if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return LLVQ_ECUDA;
     if (cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) return LLVQ_ECUDA;
-    if (llvq::allow_max_smem(llvq::gemv_planes_kernel<false>, d.max_smem_optin)) return LLVQ_ECUDA;
+    if (llvq::allow_max_smem(llvq::gemv_planes_kernel<false, 1>, d.max_smem_optin)) return LLVQ_ECUDA;
     if (cudaDeviceSynchronize() != cudaSuccess) return LLVQ_ECUDA;
     d.ready = true;
     return LLVQ_OK;
@@ -1145,6 +1236,8 @@ extern "C" int llvq_gemv_static(const void *layout_buf, const void *row_scale, c
     GemvParams p;
     memset(&p, 0, sizeof p);
     p.nprob = 1;
+    p.batch = 1;
+    p.y_stride = (int)rows;
     p.prob[0].layout = (const uint8_t *)layout_buf;
     p.prob[0].row_scale = (const __half *)row_scale;
     p.prob[0].y = y;

@@ -60,7 +60,9 @@ struct GemvProblemDev {
 struct GemvParams {
     GemvProblemDev prob[LLVQ_MAX_GROUP];
     int nprob;
-    const __half *x;
+    const __half *x;             // batch vectors of 24 nb halves, one after the other
+    int batch;                   // activation vectors of the launch (1; up to LLVQ_MAX_BATCH through llvq_gemv_batch)
+    int y_stride;                // floats between the outputs of consecutive vectors
     int nb, tiles, tail_cells;
     int units;             // units a row group: tiles, plus one for the nb mod 4 last columns
     int total_groups;

@@ -294,3 +294,48 @@ def test_gemv_fixed_point_activations_inside_one_vector(B, ctx, oracle):
     W = oracle.dequant(case.codes, case.rows, case.nb, case.row_scale, GAIN)
     bound = 2.0**-29 * 65536.0 * np.abs(W).sum(axis=1) + 2.0**-22 * abssum
     assert (err <= bound).all(), float(np.max(err / bound))
+
+
+@pytest.mark.parametrize("rows,k,batch", [(70, 24 * 30, 2), (257, 24 * 21, 3), (96, 24 * 406, 4), (33, 24 * 33, 4), (1024, 2560, 2), (3072, 3072, 4)])
+def test_gemv_batch_matches_single_vector_calls_and_oracle(B, ctx, oracle, rows, k, batch):
+    """Small-batch decode: one pass over the records for several activation vectors.  Every vector's result is
+    bit-identical to llvq_gemv on that vector alone, and within the bar of the f64 oracle."""
+    case = make_case(rows, k, seed=rows + k + batch)
+    buf = B.expand(ctx, 0, case.d_codes, rows, case.nb)
+    kp = case.nb * 24
+    xs = []
+    for j in range(batch):
+        xj = (case.x.astype(np.float64) * (0.25 * 3.0**j)).astype(np.float16) if j else case.x.copy()
+        xj = np.roll(xj[:k], 7 * j)                      # distinct vectors of very different magnitude
+        xs.append(np.concatenate([xj, np.zeros(kp - k, dtype=np.float16)]))
+    X = torch.from_numpy(np.stack(xs)).cuda()
+    Y = B.gemv_batch(ctx, buf, case.d_scale, GAIN, X, rows, kp)
+    B.status(ctx)
+    assert Y.shape == (batch, rows)
+    for j in range(batch):
+        yj = B.gemv(ctx, 0, buf, case.d_scale, GAIN, X[j].contiguous(), rows, kp)
+        assert torch.equal(Y[j], yj)
+        cj = make_case(rows, k, seed=rows + k + batch, device=None)
+        cj.x = xs[j]
+        check_gemv(oracle, cj, Y[j])
+    # a second batched launch finds the scratch clean
+    Y2 = B.gemv_batch(ctx, buf, case.d_scale, GAIN, X, rows, kp)
+    assert torch.equal(Y, Y2)
+
+
+def test_gemv_batch_limits(B, ctx):
+    case = make_case(64, 96, seed=1)
+    buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    X = torch.zeros((5, 96), dtype=torch.float16, device="cuda")
+    with pytest.raises(B.LlvqError) as e:
+        B.gemv_batch(ctx, buf, case.d_scale, GAIN, X, case.rows, 96)                # more vectors than LLVQ_MAX_BATCH
+    assert e.value.code == -1
+    small = B.create(0, scratch_bytes=64 * 8)                                      # scratch for one vector of 64 rows only
+    try:
+        with pytest.raises(B.LlvqError) as e:
+            B.gemv_batch(small, buf, case.d_scale, GAIN, X[:2].contiguous(), case.rows, 96)
+        assert e.value.code == -3
+        y = B.gemv_batch(small, buf, case.d_scale, GAIN, X[:1].contiguous(), case.rows, 96)
+        assert (y == 0).all()
+    finally:
+        small.close()
