@@ -81,7 +81,7 @@ extern "C" {
 
 #define LLVQ_MAX_GROUP 8       /* matrices in one grouped launch                             */
 #define LLVQ_MAX_K 98304       /* largest k_padded the GEMV accepts                          */
-#define LLVQ_MAX_BATCH 4       /* activation vectors in one llvq_gemv_batch launch           */
+#define LLVQ_MAX_BATCH 8       /* activation vectors in one llvq_gemv_batch call             */
 
 typedef struct llvq_ctx llvq_ctx;
 
@@ -148,10 +148,11 @@ int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row
 
 /* [Sec. 5 "Batching", the paper's stated boundary: one record decode reused across activations]
  * llvq_gemv on the LLVQ_PLANES layout for batch (1..LLVQ_MAX_BATCH) activation vectors in one pass
- * over the records: x is fp16 [batch][k_padded], y is f32 [batch][rows].  The records are read
- * and decoded once; each vector has its own fixed-point scale and its own accumulators, and
- * y[j] is bit-identical to what llvq_gemv returns for x[j].  Needs batch times the scratch of
- * llvq_gemv (LLVQ_ESIZE otherwise). */
+ * over the records: x is fp16 [batch][k_padded], y is f32 [batch][rows].  Up to four vectors share
+ * one pass (the records are read and decoded once for them); five to eight take two passes.  Each
+ * vector has its own fixed-point scale and its own accumulators, and y[j] is bit-identical to what
+ * llvq_gemv returns for x[j].  Needs min(batch, 4) times the scratch of llvq_gemv (LLVQ_ESIZE
+ * otherwise). */
 int llvq_gemv_batch(llvq_ctx *ctx, const void *layout_buf, const void *row_scale, const float *gain,
                     const void *x, float *y, int64_t rows, int64_t k_padded, int batch, void *stream);
 

@@ -178,10 +178,12 @@ int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, 
     return launch_expand(ctx, layout, codes, rows, nb, layout_out, bad_count, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
 }
 
+constexpr int kVectorsPerPass = 4;      // activation vectors one launch of the GEMV kernel carries
+
 static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n, const void *x, int64_t k_padded,
                     bool no_weights, void *stream, int batch = 1) {
     if (!ctx || !problems || !x || n < 1 || n > LLVQ_MAX_GROUP) return LLVQ_EINVAL;
-    if (batch < 1 || batch > LLVQ_MAX_BATCH || (batch > 1 && (n != 1 || layout != LLVQ_PLANES || no_weights))) return LLVQ_EINVAL;
+    if (batch < 1 || batch > kVectorsPerPass || (batch > 1 && (n != 1 || layout != LLVQ_PLANES || no_weights))) return LLVQ_EINVAL;
     if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT) return LLVQ_EINVAL;
     if (k_padded <= 0 || k_padded % 24 != 0) return LLVQ_EINVAL;
     if (k_padded > LLVQ_MAX_K) return LLVQ_ESIZE;
@@ -257,10 +259,18 @@ int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row
 
 int llvq_gemv_batch(llvq_ctx *ctx, const void *layout_buf, const void *row_scale, const float *gain, const void *x, float *y,
                     int64_t rows, int64_t k_padded, int batch, void *stream) {
-    if (!gain) return LLVQ_EINVAL;
-    llvq_problem q;
-    q.layout = layout_buf; q.row_scale = row_scale; q.y = y; q.rows = rows; q.gain[0] = gain[0]; q.gain[1] = gain[1];
-    return run_gemv(ctx, LLVQ_PLANES, &q, 1, x, k_padded, false, stream, batch);
+    if (!gain || !y || !x || batch < 1 || batch > LLVQ_MAX_BATCH || rows <= 0 || k_padded <= 0) return LLVQ_EINVAL;
+    // the kernel carries up to four vectors a pass; a larger batch is that many passes over the records, one
+    // after the other on the stream (they share the context's scratch)
+    for (int first = 0; first < batch; first += kVectorsPerPass) {
+        const int n = batch - first < kVectorsPerPass ? batch - first : kVectorsPerPass;
+        llvq_problem q;
+        q.layout = layout_buf; q.row_scale = row_scale; q.y = y + (size_t)first * (size_t)rows; q.rows = rows;
+        q.gain[0] = gain[0]; q.gain[1] = gain[1];
+        const int rc = run_gemv(ctx, LLVQ_PLANES, &q, 1, (const __half *)x + (size_t)first * (size_t)k_padded, k_padded, false, stream, n);
+        if (rc != LLVQ_OK) return rc;
+    }
+    return LLVQ_OK;
 }
 
 int llvq_gemv_grouped(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n, const void *x, int64_t k_padded,

@@ -296,7 +296,7 @@ def test_gemv_fixed_point_activations_inside_one_vector(B, ctx, oracle):
     assert (err <= bound).all(), float(np.max(err / bound))
 
 
-@pytest.mark.parametrize("rows,k,batch", [(70, 24 * 30, 2), (257, 24 * 21, 3), (96, 24 * 406, 4), (33, 24 * 33, 4), (1024, 2560, 2), (3072, 3072, 4)])
+@pytest.mark.parametrize("rows,k,batch", [(70, 24 * 30, 2), (257, 24 * 21, 3), (96, 24 * 406, 4), (33, 24 * 33, 4), (1024, 2560, 2), (3072, 3072, 4), (130, 24 * 50, 7), (64, 24 * 9, 8)])
 def test_gemv_batch_matches_single_vector_calls_and_oracle(B, ctx, oracle, rows, k, batch):
     """Small-batch decode: one pass over the records for several activation vectors.  Every vector's result is
     bit-identical to llvq_gemv on that vector alone, and within the bar of the f64 oracle."""
@@ -326,7 +326,7 @@ def test_gemv_batch_matches_single_vector_calls_and_oracle(B, ctx, oracle, rows,
 def test_gemv_batch_limits(B, ctx):
     case = make_case(64, 96, seed=1)
     buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
-    X = torch.zeros((5, 96), dtype=torch.float16, device="cuda")
+    X = torch.zeros((9, 96), dtype=torch.float16, device="cuda")
     with pytest.raises(B.LlvqError) as e:
         B.gemv_batch(ctx, buf, case.d_scale, GAIN, X, case.rows, 96)                # more vectors than LLVQ_MAX_BATCH
     assert e.value.code == -1
