@@ -339,3 +339,30 @@ def test_gemv_batch_limits(B, ctx):
         assert (y == 0).all()
     finally:
         small.close()
+
+
+def test_gemv_random_shapes_grouped_and_batched(B, ctx, oracle):
+    """Thirty seeded random shapes (rows 1..700, 1..260 blocks a row: every leftover count, row groups that end
+    mid-group, launches smaller and larger than the grid), each through a plain, a grouped and a batched launch."""
+    rng = np.random.default_rng(20260925)
+    for it in range(30):
+        rows = int(rng.integers(1, 700))
+        nb = int(rng.integers(1, 260))
+        case = make_case(rows, 24 * nb, seed=1000 + it)
+        buf = B.expand(ctx, 0, case.d_codes, rows, nb)
+        gain = (float(rng.uniform(0.25, 2.0)), float(rng.uniform(0.25, 2.0)))
+        y = B.gemv(ctx, 0, buf, case.d_scale, gain, case.d_x, rows, 24 * nb)
+        check_gemv(oracle, case, y, gain=gain)
+        # the same matrix as the second member of a group, behind a matrix of another height
+        other = make_case(int(rng.integers(1, 300)), 24 * nb, seed=2000 + it, tensor_id=1)
+        other.d_x = case.d_x
+        bo = B.expand(ctx, 0, other.d_codes, other.rows, nb)
+        yo = torch.empty(other.rows, dtype=torch.float32, device="cuda")
+        yg = torch.full((rows,), float("nan"), dtype=torch.float32, device="cuda")
+        B.gemv_grouped(ctx, 0, [(bo, other.d_scale, GAIN, yo, other.rows), (buf, case.d_scale, gain, yg, rows)], case.d_x, 24 * nb)
+        assert torch.equal(y, yg)
+        # and as vector 1 of a batch of three
+        X = torch.stack([other.d_x.flip(0), case.d_x, (case.d_x.float() * 0.5).half()]).contiguous()
+        Y = B.gemv_batch(ctx, buf, case.d_scale, gain, X, rows, 24 * nb)
+        assert torch.equal(Y[1], y)
+    B.status(ctx)
