@@ -280,6 +280,8 @@ def main():
     ap.add_argument("--lean", action="store_true", help="profiling runs: no clock ramp, no end-to-end leg, no arms, no oracle check")
     ap.add_argument("--no-pdl", action="store_true", help="launch the GEMV without programmatic dependent launch")
     ap.add_argument("--ungrouped", action="store_true", help="one launch a matrix instead of row-concatenated groups")
+    ap.add_argument("--profile-batch", type=int, default=0,
+                    help="profiling runs: only launch llvq_gemv_batch with this many activation vectors, one launch a matrix, and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.lean:
@@ -320,6 +322,19 @@ def main():
     copies = make_copies(B, ctx, mats, B.PLANES, ncopies, device, grouped=not args.ungrouped)
     torch.cuda.synchronize()
     launches_per_step = len(copies[0].launches)
+
+    if args.profile_batch:
+        # a few batched launches for a profiler to capture; nothing is measured here
+        nvec = args.profile_batch
+        for i in range(args.warmup + args.steps):
+            for ln in copies[i % ncopies].launches:
+                X = ln["x"].unsqueeze(0).repeat(nvec, 1).contiguous()
+                for mi, m in enumerate(ln["mats"]):
+                    B.gemv_batch(ctx, ln["bufs"][mi], ln["scales"][mi], datagen.GAIN, X, m.rows, ln["k_padded"])
+        torch.cuda.synchronize()
+        B.status(ctx)
+        print(json.dumps({"profile": "llvq_gemv_batch", "vectors": nvec, "config": wl.name, "launches": (args.warmup + args.steps) * len(mats)}))
+        return
 
     # expander throughput (load-time step, outside the timed region)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
