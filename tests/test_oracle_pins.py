@@ -421,3 +421,25 @@ def test_generator_draws_valid_shell_uniform_indices(oracle):
     g = (codes >> np.uint64(47)).astype(int)
     assert 0.45 < g.mean() < 0.55 and g.max() == 1
     assert (datagen.make_codes(64, 128, 0, start=100, count=50).numpy() == datagen.make_codes(64, 128, 0).numpy()[100:150]).all()
+
+
+def test_planes_layout_worked_example_by_hand(oracle):
+    """One row, one block, index 0 (x = 0,...,0,4,4; class 0), written out by hand from the layout's description.
+    Codes: u = 8 everywhere except coordinates 22 and 23, where u = 8 + 4/2 = 10.  With one block the piece is a single:
+    row 0 is (m,e,g) = (0,0,0), its slot is its row half 0, so coordinate i sits at position i.  Positions 22 and 23
+    are 16*1 + 4*1 + 2 and 16*1 + 4*1 + 3: column c = 1, t = 1, i = 2 and 3, i.e. nibbles 2*2+1 = 5 and 2*3+1 = 7
+    of word Wa of lane 4*0 + 1, which is stored at byte 128*0 + 4*1.  Every other nibble of the 448 bytes of payload
+    is 8 (row 0's other codes and the empty records of rows 1..31).  Headers: pair 2*0 + 0 holds row 0 (class 0,
+    gain 0) in its low half and row 8 (empty: 511) in its high half, at byte 384; all other halves are 511."""
+    buf = oracle.pack_planes(np.array([0], dtype=np.uint64), 1, 1)
+    assert buf.size == 448
+    words = buf.view(np.uint32)
+    expect = np.full(112, 0x88888888, dtype=np.uint32)
+    expect[1] = 0xA8A88888
+    expect[96:] = 0x01FF01FF
+    expect[96] = 0x01FF0000
+    assert (words == expect).all()
+    # with the gain bit set only the header changes: class | 1 << 9
+    buf2 = oracle.pack_planes(np.array([1 << 47], dtype=np.uint64), 1, 1).view(np.uint32)
+    expect[96] = 0x01FF0200
+    assert (buf2 == expect).all()
