@@ -6,6 +6,8 @@
  *   llvq_expand      [Sec. 2.2 "Unfolding at load time"]  48-bit block codes -> in-memory records
  *   llvq_gemv        [Sec. 2.3 "The kernel"]               records, row scales, x -> y
  *   llvq_gemv_grouped[Sec. 3.4 "Attribution": row-concatenated q/k/v and gate/up launches]
+ *   llvq_gemv_batch  [Sec. 5 "Batching"]                  the same for 2..8 activation vectors a pass
+ *   llvq_gemv_static                                      llvq_gemv without a context or any allocation
  *   llvq_gemv_fp16, llvq_gemv_noweights [Sec. 3.2, Table "layout scale": the FP16 control and the
  *                    no-weights control that prices the launch geometry]
  *   llvq_dequant_fp16, llvq_decode_i8: helpers that feed the FP16 arm and the bit-exact decode check.
