@@ -34,6 +34,10 @@ L2_BYTES = 126 * 1024 * 1024
 # 8192 x 8192 launch (profiles/gemv_planes_kernel_config4_8192x8192.txt: 39.365 MB against 39.289 MB);
 # traffic grows in proportion to the records streamed, so a launch's traffic is its bytes times this.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 39.3651 / 39.2888
+# from the same capture: 5 847 216 warp instructions for 87 552 block columns (32 rows x 24 weights each), and the share
+# of issue slots busy over the launch
+NCU_WARP_INSTR_PER_CELL = 5847216 / 87552
+NCU_ISSUE_BUSY_PCT = 56.5
 METRIC = "us_per_lattice_gemv"
 
 
@@ -498,6 +502,10 @@ def main():
                          "traffic": step_bytes / launches_per_step * NCU_TRAFFIC_PER_ALGORITHMIC_BYTE,
                          "traffic_note": "DRAM bytes per launch (mean over the step's launches): ncu capture of the 8192x8192 launch scaled by bytes",
                          "kernel": "gemv_planes_kernel", "peak_source": peak_src,
+                         # the competing ceiling, from the ncu capture in profiles/ (8192 x 8192 launch): instruction issue
+                         "secondary": {"bound": "issue", "warp_instructions_per_block_column": NCU_WARP_INSTR_PER_CELL,
+                                       "issue_slots_busy_pct": NCU_ISSUE_BUSY_PCT,
+                                       "source": "profiles/gemv_planes_kernel_config4_8192x8192.txt"},
                          "how": "algorithmic bytes of a step / CUDA-event time of the step, averaged over its launches"},
             "cpu_baseline": cpu_baseline,
             "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
