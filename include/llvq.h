@@ -158,6 +158,13 @@ int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row
 int llvq_gemv_batch(llvq_ctx *ctx, const void *layout_buf, const void *row_scale, const float *gain,
                     const void *x, float *y, int64_t rows, int64_t k_padded, int batch, void *stream);
 
+/* Host query and test hook (no GPU needed): the launch plan llvq_gemv / llvq_gemv_grouped / llvq_gemv_batch
+ * (batch <= 4: one pass) would use on a device with sm_count multiprocessors for n matrices of rows[i] rows.
+ * out (host, out_len >= 8 + grid + 1 int32): grid, dynamic shared memory bytes, units a row group (tiles of
+ * four blocks, plus one for leftover blocks), total units, unit columns a panel, panels, most blocks of x a
+ * CTA prepares, row groups; then the first unit of every CTA and the total. */
+int llvq_gemv_plan(int sm_count, const int64_t *rows, int n, int64_t k_padded, int batch, int32_t *out, int out_len);
+
 /* [Sec. 3.4] One launch over n <= LLVQ_MAX_GROUP row-concatenated matrices that share x and
  * k_padded (q/k/v, gate/up).  `problems` is a HOST array, copied before the call returns. */
 int llvq_gemv_grouped(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n,

@@ -21,7 +21,7 @@ _lib = None
 
 SYMBOLS = (
     "llvq_create", "llvq_destroy", "llvq_strerror", "llvq_status", "llvq_selftest_wait_limit", "llvq_set_pdl", "llvq_num_classes", "llvq_class_base", "llvq_layout_bytes",
-    "llvq_expand", "llvq_gemv", "llvq_gemv_batch", "llvq_gemv_grouped", "llvq_gemv_static", "llvq_gemv_fp16", "llvq_gemv_noweights", "llvq_dequant_fp16",
+    "llvq_expand", "llvq_gemv", "llvq_gemv_batch", "llvq_gemv_plan", "llvq_gemv_grouped", "llvq_gemv_static", "llvq_gemv_fp16", "llvq_gemv_noweights", "llvq_dequant_fp16",
     "llvq_decode_i8",
 )
 
@@ -61,6 +61,7 @@ def load() -> ctypes.CDLL:
         L.llvq_layout_bytes.argtypes = [ci, i64, i64, ctypes.POINTER(sz)]
         L.llvq_expand.argtypes = [vp, ci, vp, i64, i64, vp, sz, vp, vp]
         L.llvq_gemv.argtypes = [vp, ci, vp, vp, ctypes.POINTER(ctypes.c_float), vp, vp, i64, i64, vp]
+        L.llvq_gemv_plan.argtypes = [ci, ctypes.POINTER(ctypes.c_int64), ci, i64, ci, ctypes.POINTER(ctypes.c_int32), ci]
         L.llvq_gemv_batch.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_float), vp, vp, i64, i64, ci, vp]
         L.llvq_gemv_grouped.argtypes = [vp, ci, ctypes.POINTER(Problem), ci, vp, i64, vp]
         L.llvq_gemv_static.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_float), vp, vp, i64, i64, vp]
@@ -189,6 +190,17 @@ def gemv_batch(ctx: Context, layout_buf: torch.Tensor, row_scale: torch.Tensor, 
                                   _gain(gain), _dev(x, torch.float16, "x"), _dev(y, torch.float32, "y"), int(rows), int(k_padded),
                                   batch, _stream(stream)), "llvq_gemv_batch")
     return y
+
+
+def gemv_plan(sm_count: int, rows, k_padded: int, batch: int = 1) -> dict:
+    """llvq_gemv_plan: the launch plan for matrices of `rows` rows each (a host query, no GPU needed)."""
+    rows = list(rows)
+    arr = (ctypes.c_int64 * len(rows))(*rows)
+    out = (ctypes.c_int32 * (8 + 256 + 1))()
+    _check(load().llvq_gemv_plan(int(sm_count), arr, len(rows), int(k_padded), int(batch), out, len(out)), "llvq_gemv_plan")
+    grid = out[0]
+    return dict(grid=grid, smem=out[1], units=out[2], total_units=out[3], panel=out[4], npanels=out[5], xblocks=out[6],
+                groups=out[7], cta_first=[out[8 + c] for c in range(grid + 1)])
 
 
 def gemv_static(layout_buf: torch.Tensor, row_scale: torch.Tensor, gain, x: torch.Tensor, rows: int, k_padded: int,

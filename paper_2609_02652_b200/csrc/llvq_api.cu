@@ -180,6 +180,36 @@ int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, 
 
 constexpr int kVectorsPerPass = 4;      // activation vectors one launch of the GEMV kernel carries
 
+int llvq_gemv_plan(int sm_count, const int64_t *rows, int n, int64_t k_padded, int batch, int32_t *out, int out_len) {
+    if (!rows || !out || n < 1 || n > LLVQ_MAX_GROUP || sm_count < 1 || batch < 1 || batch > kVectorsPerPass) return LLVQ_EINVAL;
+    if (k_padded <= 0 || k_padded % 24 != 0) return LLVQ_EINVAL;
+    if (k_padded > LLVQ_MAX_K) return LLVQ_ESIZE;
+    GemvParams p;
+    std::memset(&p, 0, sizeof p);
+    p.nprob = n;
+    p.batch = batch;
+    p.nb = (int)(k_padded / 24);
+    p.tiles = p.nb / kTileCells;
+    p.tail_cells = p.nb % kTileCells;
+    p.units = p.tiles + (p.tail_cells ? 1 : 0);
+    int64_t groups = 0;
+    for (int i = 0; i < n; i++) {
+        if (rows[i] <= 0 || rows[i] > ((int64_t)1 << 30)) return LLVQ_EINVAL;
+        p.prob[i].group_begin = (int)groups;
+        p.prob[i].rows = (int)rows[i];
+        groups += (rows[i] + kRowsPerGroup - 1) / kRowsPerGroup;
+    }
+    if (groups > ((int64_t)1 << 26) || p.units > 2047 || groups * p.units > 0x7fffffffll) return LLVQ_ESIZE;
+    p.total_groups = (int)groups;
+    p.total_units = (int)(groups * p.units);
+    const GemvLaunch g = gemv_plan(LLVQ_PLANES, p, sm_count);
+    if (out_len < 8 + g.grid + 1) return LLVQ_ESIZE;
+    out[0] = g.grid; out[1] = (int32_t)g.smem; out[2] = p.units; out[3] = p.total_units;
+    out[4] = p.panel; out[5] = p.npanels; out[6] = p.xblocks; out[7] = p.total_groups;
+    for (int c = 0; c <= g.grid; c++) out[8 + c] = p.cta_first[c];
+    return LLVQ_OK;
+}
+
 static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n, const void *x, int64_t k_padded,
                     bool no_weights, void *stream, int batch = 1) {
     if (!ctx || !problems || !x || n < 1 || n > LLVQ_MAX_GROUP) return LLVQ_EINVAL;

@@ -55,3 +55,61 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/libllvq.so")
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         binding.load()
+
+
+def _plan_invariants(plan, sm_count, rows, k_padded, batch):
+    nb = k_padded // 24
+    tiles, left = divmod(nb, 4)
+    units = tiles + (1 if left else 0)
+    groups = sum((r + 31) // 32 for r in rows)
+    total = groups * units
+    assert plan["units"] == units and plan["groups"] == groups and plan["total_units"] == total
+    grid = plan["grid"]
+    assert 1 <= grid <= min(sm_count, 256) and grid <= max(total, 1)
+    cf = plan["cta_first"]
+    assert cf[0] == 0 and cf[-1] == total and all(a <= b for a, b in zip(cf, cf[1:]))
+    # the first CTAs lead: shares never grow with the CTA index by more than the rounding, and stay within
+    # ten units (or 60 % of the mean) of the mean
+    shares = [b - a for a, b in zip(cf, cf[1:])]
+    mean = total / grid
+    lead = min(10.0, 0.6 * mean)
+    assert all(abs(s - mean) <= lead + 1.5 for s in shares[:-1])
+    assert all(shares[i + 1] <= shares[i] + 1 for i in range(len(shares) - 2))
+    # panels tile the unit columns; the x blocks a CTA prepares are those of the panels its units lie in
+    P, npan = plan["panel"], plan["npanels"]
+    assert P >= 1 and (npan - 1) * P < units <= npan * P
+    def panel_of(f):
+        return min(f // (groups * P), npan - 1)
+    need = 0
+    for a, b in zip(cf, cf[1:]):
+        lo = panel_of(a) * P * 4
+        hi = min(nb, (panel_of(max(b - 1, a)) + 1) * P * 4)
+        need = max(need, hi - lo)
+        # every unit of the CTA lies in those panels
+        for f in (a, max(b - 1, a)):
+            j = panel_of(f)
+            assert lo <= j * P * 4 and min(nb, (j + 1) * P * 4) <= hi
+    assert plan["xblocks"] == need <= nb
+    vectors = 1 if batch == 1 else (2 if batch == 2 else 4)
+    assert plan["smem"] >= 16 * 2 * 1792 + len(rows) * 8192 + vectors * need * 112
+    assert plan["smem"] + 1024 <= 227 * 1024
+
+
+def test_launch_plan_invariants():
+    """The host-side planner of the GEMV (no GPU): CTA shares, panels, shared-memory need."""
+    from paper_2609_02652_b200 import binding
+
+    cases = [(148, [8192], 8208, 1), (148, [4096, 1024, 1024], 2568, 1), (148, [9728, 9728], 2568, 1), (148, [2560], 9744, 1),
+             (148, [1], 24, 1), (148, [33], 48, 1), (148, [70], 24 * 1024, 1), (148, [40], 98304, 1), (148, [24576], 4104, 4),
+             (132, [5120], 17424, 2), (300, [100000], 4104, 1), (8, [3072], 3072, 1), (148, [32 + 17 * i for i in range(8)], 960, 1)]
+    for sm, rows, k, batch in cases:
+        _plan_invariants(binding.gemv_plan(sm, rows, k, batch), sm, rows, k, batch)
+    # argument checks
+    with pytest.raises(binding.LlvqError):
+        binding.gemv_plan(148, [8192], 8209)
+    with pytest.raises(binding.LlvqError):
+        binding.gemv_plan(148, [8192], 98304 + 24)
+    with pytest.raises(binding.LlvqError):
+        binding.gemv_plan(148, [8192] * 9, 8208)
+    with pytest.raises(binding.LlvqError):
+        binding.gemv_plan(148, [8192], 8208, batch=5)
