@@ -366,3 +366,20 @@ def test_gemv_random_shapes_grouped_and_batched(B, ctx, oracle):
         Y = B.gemv_batch(ctx, buf, case.d_scale, gain, X, rows, 24 * nb)
         assert torch.equal(Y[1], y)
     B.status(ctx)
+
+
+def test_gemv_without_programmatic_dependent_launch(B, oracle):
+    """llvq_set_pdl(0): the same kernel as an ordinary launch; same bits."""
+    ctx = B.create(0)
+    try:
+        case = make_case(300, 24 * 77, seed=21)
+        buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+        y1 = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
+        B.set_pdl(ctx, False)
+        y2 = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
+        y3 = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
+        B.status(ctx)
+        assert torch.equal(y1, y2) and torch.equal(y2, y3)
+        check_gemv(oracle, case, y2)
+    finally:
+        ctx.close()
