@@ -559,6 +559,22 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         for (int s = 0; s < kEarlySlots; s++) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
     }
     LLVQ_TRACE_CLOCK(5)
+    // what the loop needs that does not depend on the previous kernel: this lane's constants, and the scale of
+    // its row in the first run (the scales, like the records, are the caller's weights)
+    const uint32_t lane16 = 16 * lane, lane4 = 4 * lane, pair16 = 16 * (lane >> 1);
+    const int tiles = p.tiles;
+    const LaneOffsets lo = lane_offsets(lane, false);
+    const bool odd_lane = lane & 1, high_lane = lane & 2;
+    const float limb_scale = odd_lane ? 65536.f : 1.f;     // this lane's limb pair: 256^0,1 or 256^2,3
+    const int my_row = (lane >> 2) + 8 * (lane & 3);       // the row of the group this lane ends up with
+    const uint32_t tab0 = smem_addr(tab);
+    q = n_units > 0 ? find_problem(p, cc.group) : 0;
+    float first_row_scale = 0.f;
+    if (n_units > 0) {
+        const GemvProblemDev &p0 = p.prob[q];
+        const int row0 = (cc.group - p0.group_begin) * kRowsPerGroup + my_row;
+        if (row0 < p0.rows) first_row_scale = __half2float(p0.row_scale[row0]);
+    }
     LLVQ_TRACE_CLOCK(6)
     // let the next kernel in the stream start its own prefetch, then wait for the previous one:
     // x, y and the reduction scratch may still be in use by it
@@ -648,14 +664,6 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     uint32_t bar = my_bar;                             // barrier and buffer of the slot that is consumed next
     uint32_t sbuf = my_ring;
     const uint32_t sbuf_end = my_ring + kSlots * kTileBytes;
-    const uint32_t lane16 = 16 * lane, lane4 = 4 * lane, pair16 = 16 * (lane >> 1);
-    const int tiles = p.tiles;
-    const LaneOffsets lo = lane_offsets(lane, false);
-    const bool odd_lane = lane & 1, high_lane = lane & 2;
-    const float limb_scale = odd_lane ? 65536.f : 1.f;     // this lane's limb pair: 256^0,1 or 256^2,3
-    const int my_row = (lane >> 2) + 8 * (lane & 3);       // the row of the group this lane ends up with
-    const uint32_t tab0 = smem_addr(tab);
-    q = n_units > 0 ? find_problem(p, cc.group) : 0;
 
     // Sums the quad's shares: acc[r] of lane 4g+t is the share of row g + 8r; afterwards lane 4g+t
     // holds the whole sum of row g + 8t.  Fixed order, so the result does not depend on the launch.
@@ -682,7 +690,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         // the row's scale is needed only by the arrival that finishes the row, but loading it now
         // keeps a cold read off the tail of the kernel
         const int row = (cc.group - pr.group_begin) * kRowsPerGroup + my_row;
-        const float row_scale = row < pr.rows ? __half2float(pr.row_scale[row]) : 0.f;
+        const float row_scale = n == 0 ? first_row_scale : (row < pr.rows ? __half2float(pr.row_scale[row]) : 0.f);
         // this lane's addresses in the x records of the run's first tile
         const uint32_t xk = xs0 + (uint32_t)cc.col * (4 * kXRecBytes);
         LaneOffsets xa = {xk + lo.b0, xk + lo.b1, xk + lo.b2, xk + lo.xs};
