@@ -696,3 +696,80 @@ void llvqo_decode_batch(const uint64_t *codes, int64_t n, int8_t *x, int32_t *cl
         if (cls[i] < 0) memset(x + i * NCOORD, 0, NCOORD);
     }
 }
+
+/* ------------------------------------------------------------------------------------ */
+/* Activation rotation (Sec. 2.3: a separate kernel rotates the activation first, a        */
+/* Walsh--Hadamard transform; Sec. 5 "The rotated basis and the shared-memory wall").       */
+/* ------------------------------------------------------------------------------------ */
+/*
+ * The definition written out, block by block:
+ *     y[B c + k] = (1 / sqrt(B)) * sum_{i < B} (-1)^popcount(i & k) * s_i * x[B c + i],
+ * the Sylvester (natural-order) Hadamard matrix H_B[k][i] = (-1)^popcount(k & i), normalised
+ * so that the rotation is orthogonal.  B^2 operations a block: no fast transform here.
+ *
+ * Readings (the paper names the transform and nothing else about it):
+ *   - Lengths that are not powers of two (2560, 9728, 17408 ...): the rotation is block
+ *     diagonal, B the largest power of two that divides n (at most 16384) unless the caller
+ *     names a smaller power of two.
+ *   - Order: natural (Sylvester) order; scale 1 / sqrt(B).
+ *   - An optional sign flip s_i = -1 per input coordinate ahead of the transform (the usual
+ *     randomised form of an incoherence rotation); none when `negate` is NULL.
+ *   - Input and output are FP16, as the GEMV reads them.  The sum is taken exactly (every
+ *     FP16 value is a multiple of 2^-24, so the sum is an integer in that unit), scaled in
+ *     f64 and rounded once to FP16, to nearest even: the output is the correctly rounded
+ *     value of the definition whenever the block's sum of |x| stays below 2^29.
+ */
+static uint16_t double_to_half(double v) {
+    uint16_t sign = (uint16_t)(signbit(v) ? 0x8000 : 0);
+    double a = fabs(v);
+    if (isnan(a)) return (uint16_t)(sign | 0x7E00);
+    if (a == 0.0) return sign;
+    if (isinf(a)) return (uint16_t)(sign | 0x7C00);
+    int e;
+    (void)frexp(a, &e);                       /* a = m 2^e, 1/2 <= m < 1: leading bit at 2^(e-1) */
+    int q = (e - 1 < -14 ? -14 : e - 1) - 10; /* weight of the last kept bit */
+    double r = rint(ldexp(a, -q));            /* exact scaling; ties to even in the default mode */
+    if (r >= 2048.0) { r = 1024.0; q += 1; }
+    if (r < 1024.0) return (uint16_t)(sign | (uint16_t)r);            /* subnormal, q = -24 */
+    int biased = q + 10 + 15;
+    if (biased >= 31) return (uint16_t)(sign | 0x7C00);
+    return (uint16_t)(sign | (biased << 10) | ((int)r - 1024));
+}
+uint16_t llvqo_double_to_half(double v) { return double_to_half(v); }
+
+int64_t llvqo_rotate_block(int64_t n, int64_t block) {
+    if (n <= 0) return 0;
+    if (block == 0) {
+        block = 1;
+        while (block < 16384 && n % (2 * block) == 0) block *= 2;
+        return block;
+    }
+    if (block < 1 || block > 16384 || (block & (block - 1)) || n % block) return 0;
+    return block;
+}
+
+/* x[n], out[n] FP16 bit patterns; negate[n] bytes (non-zero = flip the sign of x_i) or NULL.
+ * Returns the block length used, 0 if `block` is not a power of two that divides n. */
+int64_t llvqo_rotate(const uint16_t *x, int64_t n, int64_t block, const uint8_t *negate, uint16_t *out) {
+    int64_t B = llvqo_rotate_block(n, block);
+    if (B == 0) return 0;
+    double scale = ldexp(1.0 / sqrt((double)B), -24);
+    int64_t *t = (int64_t *)malloc((size_t)B * sizeof(int64_t));
+    for (int64_t c = 0; c < n / B; c++) {
+        for (int64_t i = 0; i < B; i++) {
+            uint16_t h = x[B * c + i];
+            int e = (h >> 10) & 31, f = h & 1023;
+            int64_t v = e == 0 ? (int64_t)f : (int64_t)(f + 1024) << (e - 1);   /* |x_i| in units of 2^-24 */
+            if (h >> 15) v = -v;
+            if (negate && negate[B * c + i]) v = -v;
+            t[i] = v;
+        }
+        for (int64_t k = 0; k < B; k++) {
+            __int128 s = 0;
+            for (int64_t i = 0; i < B; i++) s += (__builtin_popcountll((unsigned long long)(i & k)) & 1) ? -t[i] : t[i];
+            out[B * c + k] = double_to_half((double)s * scale);
+        }
+    }
+    free(t);
+    return B;
+}

@@ -72,6 +72,12 @@ def lib() -> ctypes.CDLL:
             L.llvqo_matvec.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, vp, ci]
             L.llvqo_matvec.restype = None
             L.llvqo_decode_batch.argtypes = [vp, i64, vp, vp]
+            L.llvqo_rotate.argtypes = [vp, i64, i64, vp, vp]
+            L.llvqo_rotate.restype = i64
+            L.llvqo_rotate_block.argtypes = [i64, i64]
+            L.llvqo_rotate_block.restype = i64
+            L.llvqo_double_to_half.argtypes = [ctypes.c_double]
+            L.llvqo_double_to_half.restype = ctypes.c_uint16
             L.llvqo_decode_batch.restype = None
             L.llvqo_init()
             _lib = L
@@ -197,3 +203,28 @@ def matvec(codes, rows, nb, row_scale_f16, gain, x_f16, nthreads: int = 1):
     ab = np.zeros(rows, np.float64)
     lib().llvqo_matvec(_ptr(codes), rows, nb, _ptr(rs), _ptr(g), _ptr(xv), _ptr(y), _ptr(wn), _ptr(ab), int(nthreads))
     return y, wn, ab
+
+
+def rotate_block(n: int, block: int = 0) -> int:
+    """Block length of the rotation of an n-vector: `block`, or the largest power of two (<= 16384) dividing n."""
+    return int(lib().llvqo_rotate_block(int(n), int(block)))
+
+
+def double_to_half_bits(v: float) -> int:
+    """FP16 bit pattern of a double rounded to nearest even (the rounding step of `rotate`)."""
+    return int(lib().llvqo_double_to_half(float(v)))
+
+
+def rotate(x_f16, block: int = 0, negate=None) -> np.ndarray:
+    """Block-diagonal normalised Walsh-Hadamard rotation of an FP16 vector, by the definition (Sec. 2.3, Sec. 5).
+
+    y[B c + k] = sum_i (-1)^popcount(i & k) s_i x[B c + i] / sqrt(B), summed exactly and rounded once to FP16.
+    """
+    xv = np.ascontiguousarray(x_f16, dtype=np.float16).ravel().view(np.uint16)
+    out = np.zeros(xv.size, np.uint16)
+    ng = None if negate is None else np.ascontiguousarray(np.asarray(negate) != 0, dtype=np.uint8)
+    assert ng is None or ng.size == xv.size
+    B = lib().llvqo_rotate(_ptr(xv), xv.size, int(block), None if ng is None else _ptr(ng), _ptr(out))
+    if B == 0:
+        raise ValueError("block must be a power of two (<= 16384) that divides the length")
+    return out.view(np.float16)

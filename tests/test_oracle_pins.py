@@ -443,3 +443,103 @@ def test_planes_layout_worked_example_by_hand(oracle):
     buf2 = oracle.pack_planes(np.array([1 << 47], dtype=np.uint64), 1, 1).view(np.uint32)
     expect[96] = 0x01FF0200
     assert (buf2 == expect).all()
+
+
+# ---------------------------------------------------------------- activation rotation (Sec. 2.3, Sec. 5)
+def _oracle():
+    from oracle import oracle as O
+
+    return O
+
+
+def test_rotation_rounding_step_matches_numpy_float16():
+    """The oracle's f64 -> FP16 rounding against numpy's conversion: ties, subnormals, overflow, random values."""
+    O = _oracle()
+    rng = np.random.default_rng(5)
+    vals = [0.0, -0.0, 1.0, -1.0, 65504.0, 65519.9, 65520.0, 1e6, -1e6, 2.0 ** -24, 2.0 ** -25, 2.0 ** -25 * 1.0000001,
+            3 * 2.0 ** -25, 2.0 ** -14, 2.0 ** -14 - 2.0 ** -25, 1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 1.0 + 2.0 ** -11 + 2.0 ** -30,
+            2047.5, 2048.5, 2049.5, 0.1, -0.3]
+    vals += list(rng.normal(size=4000) * np.exp(rng.uniform(-18, 11, size=4000)))
+    # exact ties in every binade: (2 m + 1) / 2 quanta
+    for e in range(-14, 16):
+        for m in (1024, 1025, 1536, 2046, 2047):
+            vals.append((2 * m + 1) * 2.0 ** (e - 11))
+    with np.errstate(over="ignore"):
+        want = np.array(vals, np.float64).astype(np.float16).view(np.uint16)
+    got = np.array([O.double_to_half_bits(v) for v in vals], np.uint16)
+    np.testing.assert_array_equal(got, want)
+
+
+def test_rotation_worked_examples_by_hand():
+    """H_4 (1,2,3,4) / 2 = (5,-1,-2,0); a unit vector returns a column of H_B / sqrt(B); a constant lands on k = 0."""
+    O = _oracle()
+    y = O.rotate(np.array([1, 2, 3, 4], np.float16))
+    np.testing.assert_array_equal(y.astype(np.float64), [5.0, -1.0, -2.0, 0.0])
+    for B, j in ((8, 5), (64, 37), (256, 255)):
+        x = np.zeros(B, np.float16)
+        x[j] = 3.0
+        y = O.rotate(x).astype(np.float64)
+        sign = np.array([(-1) ** bin(j & k).count("1") for k in range(B)], np.float64)
+        want = (3.0 * sign / math.sqrt(B)).astype(np.float16).astype(np.float64)
+        np.testing.assert_array_equal(y, want)
+    y = O.rotate(np.full(1024, 0.5, np.float16)).astype(np.float64)
+    assert y[0] == 16.0 and not y[1:].any()
+    # block length 1 is the identity, and so is any length whose largest power-of-two divisor is 1
+    x = np.arange(7, dtype=np.float16) - 3
+    np.testing.assert_array_equal(O.rotate(x), x)
+    np.testing.assert_array_equal(O.rotate(np.arange(8, dtype=np.float16), block=1), np.arange(8, dtype=np.float16))
+
+
+def test_rotation_block_rule():
+    O = _oracle()
+    # the lengths of the paper's activations: hidden and intermediate sizes of the 4B / 8B / 14B / 32B models
+    assert [O.rotate_block(n) for n in (2560, 9728, 4096, 12288, 5120, 17408, 25600, 24, 98304, 7)] == \
+        [512, 512, 4096, 4096, 1024, 1024, 1024, 8, 16384, 1]
+    assert O.rotate_block(2560, 128) == 128
+    for n, b in ((2560, 1024), (4096, 3), (4096, 32768), (100, 8), (0, 0)):
+        assert O.rotate_block(n, b) == 0
+    with pytest.raises(ValueError):
+        O.rotate(np.zeros(24, np.float16), block=16)
+
+
+@pytest.mark.parametrize("n,block", [(24, 0), (96, 0), (2560, 0), (2560, 64), (4096, 0), (9728, 0), (1536, 512)])
+def test_rotation_against_scipy_hadamard_and_invariants(n, block):
+    """The definition against scipy's Hadamard matrix (a library routine the oracle does not call), plus
+    orthogonality: the norm is kept and applying the rotation twice returns x, both up to FP16 rounding."""
+    import scipy.linalg
+
+    O = _oracle()
+    rng = np.random.default_rng(n + block)
+    x = rng.normal(size=n).astype(np.float16)
+    neg = rng.integers(0, 2, size=n).astype(np.uint8) if block else None
+    B = O.rotate_block(n, block)
+    y = O.rotate(x, block, neg)
+    H = scipy.linalg.hadamard(B).astype(np.float64) if B > 1 else np.ones((1, 1))
+    xs = x.astype(np.float64) * (1.0 if neg is None else 1.0 - 2.0 * neg)
+    want = (xs.reshape(n // B, B) @ H.T / math.sqrt(B)).ravel()
+    # f64 matmul of these sizes carries ~1e-13 of error: compare before rounding, then the rounding itself
+    assert np.abs(y.astype(np.float64) - want).max() <= np.abs(want).max() * 2.0 ** -11 + 1e-12
+    same = want.astype(np.float16) == y
+    assert same.mean() > 0.999                       # the few others sit on a rounding boundary of the matmul's error
+    np.testing.assert_array_less(np.abs(y[~same].astype(np.float64) - want[~same]), np.abs(want[~same]) * 2.0 ** -10 + 2.0 ** -24)
+    nx, ny = np.linalg.norm(xs), np.linalg.norm(y.astype(np.float64))
+    assert abs(nx - ny) <= 2.0 ** -10 * nx
+    if neg is None:
+        back = O.rotate(y, block).astype(np.float64)
+        assert np.abs(back - x.astype(np.float64)).max() <= 2.0 ** -9 * max(1.0, np.abs(want).max())
+
+
+def test_rotation_is_exact_where_floats_would_round():
+    """A large and a tiny value in one block: the exact sum keeps both (an f32 butterfly would lose the small one)."""
+    O = _oracle()
+    x = np.zeros(4, np.float16)
+    x[0], x[1] = 2048.0, 2.0 ** -14
+    y = O.rotate(x).astype(np.float64)
+    # (2048 +- 2^-14) / 2 rounds to 1024 in FP16; with x0 = 0 the small value alone survives
+    np.testing.assert_array_equal(y, [1024.0, 1024.0, 1024.0, 1024.0])
+    x[0] = 0
+    np.testing.assert_array_equal(O.rotate(x).astype(np.float64), np.array([1, -1, 1, -1]) * 2.0 ** -15)
+    # cancellation: two large values cancel exactly and leave the small one (k = 0 and k = 2); where they add,
+    # (2000 +- 2^-10) / 2 rounds to 1000
+    x = np.array([1000.0, -1000.0, 2.0 ** -10, 0.0], np.float16)
+    np.testing.assert_array_equal(O.rotate(x).astype(np.float64), [2.0 ** -11, 1000.0, -(2.0 ** -11), 1000.0])
