@@ -8,6 +8,7 @@
  *   llvq_gemv_grouped[Sec. 3.4 "Attribution": row-concatenated q/k/v and gate/up launches]
  *   llvq_gemv_batch  [Sec. 5 "Batching"]                  the same for 2..8 activation vectors a pass
  *   llvq_gemv_static                                      llvq_gemv without a context or any allocation
+ *   llvq_rotate      [Sec. 2.3, Sec. 5 "The rotated basis"] Walsh-Hadamard rotation of x ahead of a projection
  *   llvq_gemv_fp16, llvq_gemv_noweights [Sec. 3.2, Table "layout scale": the FP16 control and the
  *                    no-weights control that prices the launch geometry]
  *   llvq_dequant_fp16, llvq_decode_i8: helpers that feed the FP16 arm and the bit-exact decode check.
@@ -197,6 +198,32 @@ int llvq_gemv_fp16(const void *W, const void *x, float *y, int64_t rows, int64_t
  * grid, shared memory, x staging, reduction and epilogue - with no record read; y = 0. */
 int llvq_gemv_noweights(llvq_ctx *ctx, const void *row_scale, const void *x, float *y,
                         int64_t rows, int64_t k_padded, void *stream);
+
+/* [Sec. 2.3: the activation is rotated by a kernel of its own ahead of the matvec; Sec. 5, the
+ * paragraph on the rotated basis: a Walsh-Hadamard transform, which every consumer of the stored
+ * weights applies.]  y = rotation of x, both fp16 vectors of n entries (n a multiple of 8, both
+ * 16-byte aligned; y may be x):
+ *     y[B c + k] = (1 / sqrt(B)) * sum_{i < B} (-1)^popcount(i & k) * s_i * x[B c + i],
+ * the natural-order (Sylvester) Hadamard matrix on each block of B consecutive coordinates.
+ *   - block: B, a power of two <= 16384 that divides n; 0 = the largest such power of two
+ *     (512 for n = 2560 or 9728, 4096 for n = 4096 or 12288, 1024 for n = 17408 or 25600).
+ *     The paper names the transform only: the block-diagonal form for lengths that are not powers
+ *     of two, the order and the scale are this library's reading.
+ *   - negate_bits: optional (may be null).  Bit i & 31 of word i >> 5 set = s_i = -1, the sign
+ *     flip of a randomised rotation; ceil(n / 32) words, 4-byte aligned.  Null = no flips.
+ *   - Arithmetic: the sums are exact (64-bit integers in units of 2^-24); the result is scaled in
+ *     f64 and rounded once to fp16, to nearest even.  While a block's sum of |x| is below 2^29 the
+ *     output is the correctly rounded value of the formula, bit for bit whatever the launch.
+ *     x must be finite.  A value beyond the fp16 range rounds to infinity.
+ *   - The launch is a link of the same programmatic-dependent-launch chain as the GEMV
+ *     (llvq_set_pdl): the GEMV enqueued after it on the stream sets up while it runs.
+ * Errors: LLVQ_EINVAL (null pointer, n <= 0 or not a multiple of 8, block not acceptable),
+ * LLVQ_EALIGN, LLVQ_ESIZE (n > 2^40), LLVQ_ECUDA. */
+int llvq_rotate(llvq_ctx *ctx, const void *x, void *y, const uint32_t *negate_bits, int64_t n,
+                int64_t block, void *stream);
+
+/* Host query: the block length llvq_rotate uses for (n, block); 0 if it would refuse them. */
+int64_t llvq_rotate_block(int64_t n, int64_t block);
 
 /* Decoded weights as fp16, W[row*k_padded + 24b + i] = fp16(row_scale * gain[g] * x_i / (4 sqrt m))
  * (product formed in f32, rounded once).  Feeds llvq_gemv_fp16. */

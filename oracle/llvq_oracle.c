@@ -698,8 +698,8 @@ void llvqo_decode_batch(const uint64_t *codes, int64_t n, int8_t *x, int32_t *cl
 }
 
 /* ------------------------------------------------------------------------------------ */
-/* Activation rotation (Sec. 2.3: a separate kernel rotates the activation first, a        */
-/* Walsh--Hadamard transform; Sec. 5 "The rotated basis and the shared-memory wall").       */
+/* Activation rotation: the Walsh-Hadamard transform applied to the activation ahead of   */
+/* every projection (Sec. 2.3, the kernel; Sec. 5, the paragraph on the rotated basis).     */
 /* ------------------------------------------------------------------------------------ */
 /*
  * The definition written out, block by block:

@@ -22,7 +22,7 @@ _lib = None
 SYMBOLS = (
     "llvq_create", "llvq_destroy", "llvq_strerror", "llvq_status", "llvq_selftest_wait_limit", "llvq_set_pdl", "llvq_num_classes", "llvq_class_base", "llvq_layout_bytes",
     "llvq_expand", "llvq_gemv", "llvq_gemv_batch", "llvq_gemv_plan", "llvq_gemv_grouped", "llvq_gemv_static", "llvq_gemv_fp16", "llvq_gemv_noweights", "llvq_dequant_fp16",
-    "llvq_decode_i8",
+    "llvq_decode_i8", "llvq_rotate", "llvq_rotate_block",
 )
 
 
@@ -69,8 +69,11 @@ def load() -> ctypes.CDLL:
         L.llvq_gemv_noweights.argtypes = [vp, vp, vp, vp, i64, i64, vp]
         L.llvq_dequant_fp16.argtypes = [vp, ci, vp, vp, ctypes.POINTER(ctypes.c_float), vp, i64, i64, vp]
         L.llvq_decode_i8.argtypes = [vp, ci, vp, vp, vp, i64, i64, vp]
+        L.llvq_rotate.argtypes = [vp, vp, vp, vp, i64, i64, vp]
+        L.llvq_rotate_block.argtypes = [i64, i64]
+        L.llvq_rotate_block.restype = i64
         for name in SYMBOLS:
-            if name not in ("llvq_destroy", "llvq_strerror", "llvq_class_base"):
+            if name not in ("llvq_destroy", "llvq_strerror", "llvq_class_base", "llvq_rotate_block"):
                 getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -237,6 +240,22 @@ def gemv_fp16(W: torch.Tensor, x: torch.Tensor, rows: int, k: int, y: torch.Tens
         y = torch.empty(rows, dtype=torch.float32, device=x.device)
     _check(load().llvq_gemv_fp16(_dev(W, torch.float16, "W"), _dev(x, torch.float16, "x"), _dev(y, torch.float32, "y"),
                                  int(rows), int(k), _stream(stream)), "llvq_gemv_fp16")
+    return y
+
+
+def rotate_block(n: int, block: int = 0) -> int:
+    """Block length `rotate` uses for a vector of n entries (0 if it would refuse them).  Host query."""
+    return int(load().llvq_rotate_block(int(n), int(block)))
+
+
+def rotate(ctx: Context, x: torch.Tensor, block: int = 0, negate_bits: torch.Tensor | None = None,
+           y: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """llvq_rotate: block-diagonal Walsh-Hadamard rotation of the fp16 vector x; `negate_bits` int32 words, bit i = flip x_i."""
+    if y is None:
+        y = torch.empty_like(x)
+    _check(load().llvq_rotate(ctx.ptr, _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"),
+                              None if negate_bits is None else _dev(negate_bits, torch.int32, "negate_bits"),
+                              int(x.numel()), int(block), _stream(stream)), "llvq_rotate")
     return y
 
 

@@ -7,7 +7,7 @@ import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-SOURCES = ["llvq_api.cu", "llvq_expand.cu", "llvq_gemv.cu", "llvq_tables.cpp"]
+SOURCES = ["llvq_api.cu", "llvq_expand.cu", "llvq_gemv.cu", "llvq_rotate.cu", "llvq_tables.cpp"]
 LIB = os.path.join(HERE, "libllvq.so")
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "shared"]

@@ -99,7 +99,7 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
         llvq_destroy(ctx);
         return LLVQ_ECUDA;
     }
-    if (gemv_configure(ctx) != 0 || cudaDeviceSynchronize() != cudaSuccess) { llvq_destroy(ctx); return LLVQ_ECUDA; }
+    if (gemv_configure(ctx) != 0 || rotate_configure() != 0 || cudaDeviceSynchronize() != cudaSuccess) { llvq_destroy(ctx); return LLVQ_ECUDA; }
     *out = ctx;
     return LLVQ_OK;
 }
@@ -320,6 +320,23 @@ int llvq_gemv_fp16(const void *W, const void *x, float *y, int64_t rows, int64_t
     if (!aligned(W, 16) || !aligned(x, 16) || !aligned(y, 4)) return LLVQ_EALIGN;
     if ((rows + 7) / 8 > 0x7fffffffll) return LLVQ_ESIZE;
     return launch_gemv_fp16((const __half *)W, (const __half *)x, y, rows, k, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+}
+
+int64_t llvq_rotate_block(int64_t n, int64_t block) {
+    const int l = rotate_block_log2(n, block);
+    return l < 0 ? 0 : (int64_t)1 << l;
+}
+
+int llvq_rotate(llvq_ctx *ctx, const void *x, void *y, const uint32_t *negate_bits, int64_t n, int64_t block, void *stream) {
+    if (!ctx || !x || !y || n <= 0 || n % 8 != 0) return LLVQ_EINVAL;
+    const int l = rotate_block_log2(n, block);
+    if (l < 0) return LLVQ_EINVAL;
+    if (!aligned(x, 16) || !aligned(y, 16) || !aligned(negate_bits, 4)) return LLVQ_EALIGN;
+    if (n > ((int64_t)1 << 40)) return LLVQ_ESIZE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    return launch_rotate((const __half *)x, (__half *)y, negate_bits, n, l, ctx->use_pdl != 0, (cudaStream_t)stream) == cudaSuccess
+               ? LLVQ_OK : LLVQ_ECUDA;
 }
 
 int llvq_dequant_fp16(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row_scale, const float *gain, void *W,

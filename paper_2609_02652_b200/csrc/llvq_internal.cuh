@@ -124,4 +124,11 @@ cudaError_t launch_dequant(const llvq_ctx *ctx, int layout, const uint8_t *buf, 
 cudaError_t launch_decode_i8(const llvq_ctx *ctx, int layout, const uint8_t *buf, int8_t *coords, uint16_t *class_ids,
                              int64_t rows, int64_t nb, cudaStream_t s);
 int gemv_configure(const llvq_ctx *ctx);   // sets the kernels' shared-memory attributes once
+
+// activation rotation: blocks of at most 2^14 coordinates (64-bit partial sums in 128 KiB of shared memory)
+constexpr int kRotMaxBlockLog2 = 14;
+int rotate_block_log2(int64_t n, int64_t block);   // log2 of the block length used, -1 if `block` is not acceptable
+int rotate_configure();                            // sets the kernel's shared-memory attribute once a device
+cudaError_t launch_rotate(const __half *x, __half *y, const uint32_t *negate, int64_t n, int block_log2, bool pdl,
+                          cudaStream_t s);
 }  // namespace llvq
