@@ -455,6 +455,35 @@ def main():
                                     "record_gbps": step_bytes / (t * 1e-3) / 1e9}
             del xb
         arms["batch"] = batch_arm
+        # activation rotation ahead of every projection (the served order: the weights live in the rotated basis, so
+        # each projection's input is rotated first).  The rotation acts on the k real entries of x; the zero padding
+        # passes through.  Three timings: the rotation inside the GEMV's own launch (llvq_gemv_rotated), the
+        # rotation as a kernel of its own ahead of each GEMV (llvq_rotate, the paper's arrangement), and those
+        # rotation kernels alone.
+        xr = {}
+        for cp in copies:
+            for ln in cp.launches:
+                if id(ln["x"]) not in xr:
+                    xr[id(ln["x"])] = ln["x"].clone()
+        def rot_fused(i):
+            for ln in copies[i % ncopies].launches:
+                B.gemv_rotated(ctx, ln["problems"], ln["x"], ln["k_padded"], n=ln["mats"][0].k)
+        def rot_two(i):
+            for ln in copies[i % ncopies].launches:
+                k = ln["mats"][0].k
+                B.rotate(ctx, ln["x"][:k], y=xr[id(ln["x"])][:k])
+                B.gemv_grouped(ctx, B.PLANES, ln["problems"], xr[id(ln["x"])], ln["k_padded"])
+        def rot_only(i):
+            for ln in copies[i % ncopies].launches:
+                k = ln["mats"][0].k
+                B.rotate(ctx, ln["x"][:k], y=xr[id(ln["x"])][:k])
+        t_f = time_arm(rot_fused, ncopies, arm_steps, 3)
+        t_2 = time_arm(rot_two, ncopies, arm_steps, 3)
+        t_0 = time_arm(rot_only, ncopies, arm_steps, 3)
+        n_launch = len(copies[0].launches)
+        arms["rotated"] = {"us_per_gemv_fused": t_f * 1e3 / n_gemv, "us_per_gemv_two_launches": t_2 * 1e3 / n_gemv,
+                           "us_per_rotation_alone": t_0 * 1e3 / n_launch, "rotations_per_step": n_launch,
+                           "block_lengths": sorted({int(B.rotate_block(ln["mats"][0].k)) for ln in copies[0].launches})}
         # no-weights control: the same launches without record reads
         def nw(i):
             for ln in copies[i % ncopies].launches:

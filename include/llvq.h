@@ -9,6 +9,7 @@
  *   llvq_gemv_batch  [Sec. 5 "Batching"]                  the same for 2..8 activation vectors a pass
  *   llvq_gemv_static                                      llvq_gemv without a context or any allocation
  *   llvq_rotate      [Sec. 2.3, Sec. 5 "The rotated basis"] Walsh-Hadamard rotation of x ahead of a projection
+ *   llvq_gemv_rotated                                     the same rotation inside the GEMV's own launch
  *   llvq_gemv_fp16, llvq_gemv_noweights [Sec. 3.2, Table "layout scale": the FP16 control and the
  *                    no-weights control that prices the launch geometry]
  *   llvq_dequant_fp16, llvq_decode_i8: helpers that feed the FP16 arm and the bit-exact decode check.
@@ -97,6 +98,14 @@ typedef struct {
     float gain[2];          /* centroid chosen by each block's gain bit [Sec. 2.1]           */
 } llvq_problem;
 
+/* The rotation of x that llvq_gemv_rotated applies (the arguments of llvq_rotate). */
+typedef struct llvq_rotation {
+    const uint32_t *negate_bits; /* device, may be null: bit i & 31 of word i >> 5 set = x_i negated first */
+    int64_t n;                   /* entries of x that are rotated: a multiple of the block length, <= k_padded;
+                                    the entries after them (the zero padding) pass through */
+    int64_t block;               /* block length, a power of two in 8..16384 that divides n; 0 = the largest */
+} llvq_rotation;
+
 /* Builds the class, index-base and Golay tables on the host, uploads them to `device`, and
  * allocates the context's reduction scratch (scratch_bytes; 0 = default 8 MiB, eight bytes a row
  * of the largest launch, rows rounded up to 32 per matrix).  Synchronous. */
@@ -170,6 +179,20 @@ int llvq_gemv_plan(int sm_count, const int64_t *rows, int n, int64_t k_padded, i
  * k_padded (q/k/v, gate/up).  `problems` is a HOST array, copied before the call returns. */
 int llvq_gemv_grouped(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n,
                       const void *x, int64_t k_padded, void *stream);
+
+/* [Sec. 2.3 and Sec. 5, the rotated basis] llvq_gemv_grouped(LLVQ_PLANES) on the rotated activation, in one
+ * launch: y = W * rotate(x).  The paper runs the rotation as a kernel of its own ahead of every projection,
+ * one thread block holding the whole activation; here every CTA of the GEMV rotates, in its prologue, the
+ * rotation blocks that meet its part of x, with llvq_rotate's arithmetic: the values that enter the matvec are
+ * bit for bit the FP16 values llvq_rotate(x, rotation->n, rotation->block, rotation->negate_bits) would store,
+ * so y agrees with llvq_rotate followed by llvq_gemv_grouped to within the GEMV's fixed-point quantum (the
+ * scale of that quantum comes from ||x||_2, which bounds every rotated entry, instead of from the largest
+ * entry).  x itself is not modified.  The blocks a CTA rotates must fit its shared memory beside the GEMV's
+ * own: block lengths up to 4096 always do; a longer block may return LLVQ_ESIZE (rotate with llvq_rotate then).
+ * Errors: those of llvq_gemv_grouped; LLVQ_EINVAL also for a null rotation, n not a positive multiple of 8
+ * or above k_padded, a block that is not acceptable or shorter than 8. */
+int llvq_gemv_rotated(llvq_ctx *ctx, const llvq_problem *problems, int n, const void *x, int64_t k_padded,
+                      const llvq_rotation *rotation, void *stream);
 
 /* No counterpart in the paper: the LLVQ_PLANES llvq_gemv for callers that cannot allocate device
  * memory - a process whose memory pool already owns the whole GPU, a plug-in that receives buffers

@@ -22,7 +22,7 @@ _lib = None
 SYMBOLS = (
     "llvq_create", "llvq_destroy", "llvq_strerror", "llvq_status", "llvq_selftest_wait_limit", "llvq_set_pdl", "llvq_num_classes", "llvq_class_base", "llvq_layout_bytes",
     "llvq_expand", "llvq_gemv", "llvq_gemv_batch", "llvq_gemv_plan", "llvq_gemv_grouped", "llvq_gemv_static", "llvq_gemv_fp16", "llvq_gemv_noweights", "llvq_dequant_fp16",
-    "llvq_decode_i8", "llvq_rotate", "llvq_rotate_block",
+    "llvq_decode_i8", "llvq_rotate", "llvq_rotate_block", "llvq_gemv_rotated",
 )
 
 
@@ -36,6 +36,10 @@ class LlvqError(RuntimeError):
 class Problem(ctypes.Structure):
     _fields_ = [("layout", ctypes.c_void_p), ("row_scale", ctypes.c_void_p), ("y", ctypes.c_void_p),
                 ("rows", ctypes.c_int64), ("gain", ctypes.c_float * 2)]
+
+
+class Rotation(ctypes.Structure):
+    _fields_ = [("negate_bits", ctypes.c_void_p), ("n", ctypes.c_int64), ("block", ctypes.c_int64)]
 
 
 def load() -> ctypes.CDLL:
@@ -70,6 +74,7 @@ def load() -> ctypes.CDLL:
         L.llvq_dequant_fp16.argtypes = [vp, ci, vp, vp, ctypes.POINTER(ctypes.c_float), vp, i64, i64, vp]
         L.llvq_decode_i8.argtypes = [vp, ci, vp, vp, vp, i64, i64, vp]
         L.llvq_rotate.argtypes = [vp, vp, vp, vp, i64, i64, vp]
+        L.llvq_gemv_rotated.argtypes = [vp, ctypes.POINTER(Problem), ci, vp, i64, ctypes.POINTER(Rotation), vp]
         L.llvq_rotate_block.argtypes = [i64, i64]
         L.llvq_rotate_block.restype = i64
         for name in SYMBOLS:
@@ -233,6 +238,15 @@ def gemv_grouped(ctx: Context, layout: int, problems, x: torch.Tensor, k_padded:
     arr = problems if isinstance(problems, ctypes.Array) else make_problems(problems)
     _check(load().llvq_gemv_grouped(ctx.ptr, int(layout), arr, len(arr), _dev(x, torch.float16, "x"), int(k_padded),
                                     _stream(stream)), "llvq_gemv_grouped")
+
+
+def gemv_rotated(ctx: Context, problems, x: torch.Tensor, k_padded: int, n: int, block: int = 0,
+                 negate_bits: torch.Tensor | None = None, stream=None) -> None:
+    """llvq_gemv_rotated: the grouped 14-byte-layout GEMV on rotate(x[:n]) (the rest of x passes through), one launch."""
+    arr = problems if isinstance(problems, ctypes.Array) else make_problems(problems)
+    rot = Rotation(None if negate_bits is None else _dev(negate_bits, torch.int32, "negate_bits"), int(n), int(block))
+    _check(load().llvq_gemv_rotated(ctx.ptr, arr, len(arr), _dev(x, torch.float16, "x"), int(k_padded), ctypes.byref(rot),
+                                    _stream(stream)), "llvq_gemv_rotated")
 
 
 def gemv_fp16(W: torch.Tensor, x: torch.Tensor, rows: int, k: int, y: torch.Tensor | None = None, stream=None) -> torch.Tensor:

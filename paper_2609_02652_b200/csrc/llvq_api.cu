@@ -211,7 +211,7 @@ int llvq_gemv_plan(int sm_count, const int64_t *rows, int n, int64_t k_padded, i
 }
 
 static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n, const void *x, int64_t k_padded,
-                    bool no_weights, void *stream, int batch = 1) {
+                    bool no_weights, void *stream, int batch = 1, const llvq_rotation *rot = nullptr) {
     if (!ctx || !problems || !x || n < 1 || n > LLVQ_MAX_GROUP) return LLVQ_EINVAL;
     if (batch < 1 || batch > kVectorsPerPass || (batch > 1 && (n != 1 || layout != LLVQ_PLANES || no_weights))) return LLVQ_EINVAL;
     if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT) return LLVQ_EINVAL;
@@ -268,6 +268,17 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
     std::memcpy(p.cls_odd_bits, ctx->host.cls_odd_bits, sizeof p.cls_odd_bits);
     std::memcpy(p.shell_inv_norm, ctx->host.shell_inv_norm, sizeof p.shell_inv_norm);
     p.error = ctx->error;
+    if (rot) {
+        // the rotation acts on the first rot->n entries of x; what follows (the padding) passes through
+        if (layout != LLVQ_PLANES || no_weights || batch != 1 || rot->n <= 0 || rot->n > k_padded || rot->n % 8 != 0) return LLVQ_EINVAL;
+        const int l = rotate_block_log2(rot->n, rot->block);
+        if (l < 3) return LLVQ_EINVAL;                 // blocks shorter than eight: rotate with llvq_rotate instead
+        if (!aligned(rot->negate_bits, 4)) return LLVQ_EALIGN;
+        p.rot_log2 = l;
+        p.rot_n = (int)rot->n;
+        p.rot_negate = rot->negate_bits;
+        p.rot_scale = std::ldexp(1.0 / std::sqrt((double)((int64_t)1 << l)), -24);
+    }
 #ifdef LLVQ_TRACE
     p.trace = ctx->trace;
     p.trace_launch = ctx->trace ? ctx->trace_launch++ : 0;
@@ -306,6 +317,12 @@ int llvq_gemv_batch(llvq_ctx *ctx, const void *layout_buf, const void *row_scale
 int llvq_gemv_grouped(llvq_ctx *ctx, int layout, const llvq_problem *problems, int n, const void *x, int64_t k_padded,
                       void *stream) {
     return run_gemv(ctx, layout, problems, n, x, k_padded, false, stream);
+}
+
+int llvq_gemv_rotated(llvq_ctx *ctx, const llvq_problem *problems, int n, const void *x, int64_t k_padded,
+                      const llvq_rotation *rotation, void *stream) {
+    if (!rotation) return LLVQ_EINVAL;
+    return run_gemv(ctx, LLVQ_PLANES, problems, n, x, k_padded, false, stream, 1, rotation);
 }
 
 int llvq_gemv_noweights(llvq_ctx *ctx, const void *row_scale, const void *x, float *y, int64_t rows, int64_t k_padded,

@@ -38,6 +38,7 @@
 #include <cstring>
 
 #include "llvq_internal.cuh"
+#include "llvq_rotate.cuh"
 
 // Optional timeline (compiled in only with -DLLVQ_TRACE, never in the shipped library): lane 0 of
 // every warp stores the global timer at a few points of the kernel.
@@ -441,7 +442,9 @@ __device__ __forceinline__ bool advance(const GemvParams &p, Cursor &c, int n) {
 // are computed once, the contraction, the scaling and the reduction once a vector.  x is BATCH vectors of
 // 24 nb halves one after the other, y BATCH vectors of rows floats (p.prob[].y is vector 0's), the accumulators
 // BATCH sets of total_groups * 32.
-template <bool NO_WEIGHTS, int BATCH>
+// ROTATE: x is rotated on its way into the records (llvq_gemv_rotated): every CTA rotates the Walsh-Hadamard
+// blocks of x that its share of the matrix touches, exactly as the rotation kernel does, and rounds them to FP16.
+template <bool NO_WEIGHTS, int BATCH, bool ROTATE = false>
 __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
     extern __shared__ __align__(128) unsigned char smem[];
     // shared memory: ring | per-matrix block constants (1024 x {gain / (4 sqrt m), parity - 16}) | x records | barriers
@@ -454,6 +457,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     const uint32_t xrec_stride = ((p.xblocks * kXRecBytes + 127) / 128) * 128;     // a vector's records
     uint64_t *bars = reinterpret_cast<uint64_t *>(xrec + BATCH * xrec_stride);
     uint32_t *warp_max = reinterpret_cast<uint32_t *>(bars + kWarps * kSlots);     // one slot a warp and vector
+    long long *rot = reinterpret_cast<long long *>(warp_max + BATCH * kWarps);     // ROTATE: the exact sums of this CTA's blocks of x
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t my_ring = smem_addr(ring + warp * kSlots * kTileBytes);
     const uint32_t my_bar = smem_addr(bars + warp * kSlots);
@@ -491,6 +495,16 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     const int blk_lo = panel_of_unit(p, cta_u0) * p.panel * kTileCells;
     const int blk_hi = min(p.nb, (panel_of_unit(p, max(cta_u1 - 1, cta_u0)) + 1) * p.panel * kTileCells);
     const uint32_t xs0 = smem_addr(xrec) - (uint32_t)blk_lo * kXRecBytes;     // address of block 0's record, were it there
+
+    // ROTATE: the coordinates [c_lo, c_hi) this CTA rotates are the whole rotation blocks that meet its blocks of x
+    int c_lo = 0, c_hi = 0;
+    if (ROTATE) {
+        const int mask = (1 << p.rot_log2) - 1;
+        c_lo = min(p.rot_n, (24 * blk_lo) & ~mask);
+        c_hi = min(p.rot_n, (24 * blk_hi + mask) & ~mask);
+        if (p.rot_negate)       // the sign flips are the caller's constants: on their way before the wait
+            for (int w = (c_lo >> 5) + tid; w < ((c_hi + 31) >> 5); w += kThreads) warm |= __ldg(p.rot_negate + w);
+    }
 
     LLVQ_TRACE_CLOCK(4)
     // consume side and issue side walk the same sequence of units
@@ -589,7 +603,86 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     // 2^(29 - xexp).
     bool failed = false;
     int xexp[BATCH];
-    {
+    if constexpr (ROTATE) {
+        // The rotated vector's largest magnitude is not known before it is rotated, but every rotated coordinate is
+        // a unit-norm combination of its block, so |x'_k| <= ||x||_2: the scan sums the squares instead of taking
+        // the maximum, and the fixed-point scale follows from that bound (a few bits coarser than the maximum
+        // would give, of 29).  In the same pass the pieces of this CTA's rotation blocks become integers, take
+        // their first three stages in registers and go to shared memory; the later stages follow there; the
+        // rounded FP16 values - bit for bit those of the rotation kernel - become the fixed-point records.
+        const int nx = p.nb * 3, e_lo = 3 * blk_lo, e_hi = 3 * blk_hi;
+        const bool one_each = e_hi - e_lo <= kThreads;
+        const uint4 *xg = reinterpret_cast<const uint4 *>(p.x);
+        uint4 mine = make_uint4(0u, 0u, 0u, 0u);               // a piece past the rotated length (the padding)
+        float ss = __uint_as_float(settled(warm, warm, warm));
+        for (int base = 0; base < nx; base += 4 * kThreads) {
+            uint4 v[4];
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+                const int e = base + i * kThreads + tid;
+                v[i] = e < nx ? __ldcg(xg + e) : make_uint4(0u, 0u, 0u, 0u);
+            }
+            if (base == 0) {
+                for (int b = tid; b < blk_hi - blk_lo; b += kThreads)
+                    asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(smem_addr(xrec) + b * kXRecBytes + 96), "r"(0) : "memory");
+                for (int e = tid; e < tab_entries; e += kThreads) {
+                    const int c = e & 511;
+                    const uint32_t shell = (p.cls_shell_nibbles[c >> 3] >> (4 * (c & 7))) & 15u;
+                    const int odd = (int)((p.cls_odd_bits[c >> 5] >> (c & 31)) & 1u);
+                    const GemvProblemDev &pe = p.prob[e >> 10];
+                    tab[e] = make_float2(p.shell_inv_norm[shell] * ((e & 512) ? pe.gain1 : pe.gain0), __int_as_float(shell ? odd - 16 : 0));
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 4; i++) {
+                const int e = base + i * kThreads + tid;
+                const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[k]));
+                    ss = fmaf(f.x, f.x, ss);
+                    ss = fmaf(f.y, f.y, ss);
+                }
+                if (8 * e >= c_lo && 8 * e < c_hi) {
+                    long long a[8];
+                    const uint32_t flips = p.rot_negate ? (__ldg(p.rot_negate + (e >> 2)) >> (8 * (e & 3))) & 0xffu : 0u;
+                    rot_load8(v[i], flips, a);
+                    rot_butterflies<3>(a);
+#pragma unroll
+                    for (int k = 0; k < 8; k++) rot[8 * e - c_lo + k] = a[k];
+                } else if (e >= e_lo && e < e_hi) {
+                    mine = v[i];
+                }
+            }
+        }
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+        if (lane == 0) warp_max[warp] = __float_as_uint(ss);
+        __syncthreads();                               // publishes the sums of squares, the first stages, the block constants
+        rot_later_passes(rot, p.rot_log2, c_hi - c_lo, tid, kThreads);
+        {
+            // every thread of every CTA adds the sixteen sums in the same order
+            float total = __uint_as_float(warp_max[lane & (kWarps - 1)]);
+#pragma unroll
+            for (int off = kWarps / 2; off >= 1; off >>= 1) total += __shfl_xor_sync(0xffffffffu, total, off);
+            // total * 1.0625 covers the rounding of the sum and of the FP16 results: it is below 2^e2, so
+            // every |x'| is below 2^ceil(e2 / 2)
+            const int e2 = (int)((__float_as_uint(total * 1.0625f) >> 23) & 255u) - 126;
+            xexp[0] = max((e2 + 1) >> 1, -13);
+        }
+        const float scale = pow2f(29 - xexp[0]);
+        for (int e = e_lo + tid; e < e_hi; e += kThreads) {
+            uint4 v;
+            if (8 * e < c_hi) v = rot_round8(rot + (8 * e - c_lo), p.rot_scale);
+            else v = one_each ? mine : __ldcg(xg + e);
+            convert_item(v, e % 3, xs0 + (uint32_t)(e / 3) * kXRecBytes, scale);
+        }
+        if (!NO_WEIGHTS) {
+#pragma unroll
+            for (int s = kEarlySlots; s < kSlots; s++) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
+        }
+        __syncthreads();                               // publishes the x records
+    } else {
         const int nx = p.nb * 3, e_lo = 3 * blk_lo, e_hi = 3 * blk_hi;
         const bool one_each = e_hi - e_lo <= kThreads;         // then no thread meets two of the pieces wanted
         uint4 mine[BATCH];
@@ -1079,16 +1172,25 @@ GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
     }
     // the widest stretch of x a CTA meets: its units lie in consecutive panels
     p.xblocks = 0;
+    p.rot_span = 0;
     for (int c = 0; c < g.grid; c++) {
         const int f0 = p.cta_first[c], f1 = p.cta_first[c + 1];
         const int lo = panel_of_unit(p, f0) * p.panel * kTileCells;
         int hi = (panel_of_unit(p, f1 - 1 > f0 ? f1 - 1 : f0) + 1) * p.panel * kTileCells;
         if (hi > p.nb) hi = p.nb;
         if (hi - lo > p.xblocks) p.xblocks = hi - lo;
+        if (p.rot_log2 > 0) {
+            // the whole rotation blocks that meet the CTA's blocks of x (the kernel computes the same)
+            const int mask = (1 << p.rot_log2) - 1;
+            int c_lo = (24 * lo) & ~mask, c_hi = (24 * hi + mask) & ~mask;
+            if (c_lo > p.rot_n) c_lo = p.rot_n;
+            if (c_hi > p.rot_n) c_hi = p.rot_n;
+            if (c_hi - c_lo > p.rot_span) p.rot_span = c_hi - c_lo;
+        }
     }
     const int vectors = p.batch <= 1 ? 1 : (p.batch == 2 ? 2 : 4);             // the kernel is built for 1, 2 and 4
     const size_t xbytes = ((size_t)p.xblocks * kXRecBytes + 127) / 128 * 128 * vectors;
-    g.smem = (size_t)kWarps * kSlots * kTileBytes + 8192 /* alignment of the tables */ + (size_t)p.nprob * 8192 + xbytes + kWarps * kSlots * 8 + kWarps * 4 * vectors + 16;
+    g.smem = (size_t)kWarps * kSlots * kTileBytes + 8192 /* alignment of the tables */ + (size_t)p.nprob * 8192 + xbytes + kWarps * kSlots * 8 + kWarps * 4 * vectors + 16 + (size_t)p.rot_span * 8;
     return g;
 }
 
@@ -1108,6 +1210,7 @@ int gemv_configure(const llvq_ctx *ctx) {
     if (allow_max_smem(gemv_planes_kernel<true, 1>, bytes)) return -1;
     if (allow_max_smem(gemv_planes_kernel<false, 2>, bytes)) return -1;
     if (allow_max_smem(gemv_planes_kernel<false, 4>, bytes)) return -1;
+    if (allow_max_smem(gemv_planes_kernel<false, 1, true>, bytes)) return -1;
     if (allow_max_smem(gemv_onehot_kernel, bytes)) return -1;
     return 0;
 }
@@ -1125,6 +1228,7 @@ cudaError_t launch_gemv(int layout, const GemvParams &p, const GemvLaunch &g, bo
     cfg.numAttrs = 1;
     if (layout == LLVQ_PLANES) {
         if (no_weights) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<true, 1>, p);
+        if (p.rot_log2 > 0) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 1, true>, p);
         if (p.batch <= 1) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 1>, p);
         if (p.batch == 2) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 2>, p);
         return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 4>, p);

@@ -82,6 +82,12 @@ struct GemvParams {
     uint32_t cls_odd_bits[16];        // bit c & 31 of word c >> 5: odd type
     float shell_inv_norm[16];         // [m] = 1 / (4 sqrt m)
     int *error;               // set when a bounded wait ran out
+    // rotation of x inside the GEMV (llvq_gemv_rotated); rot_log2 = 0 means none
+    int rot_log2;             // log2 of the rotation's block length (3..)
+    int rot_n;                // coordinates rotated: a multiple of the block length, at most 24 nb
+    int rot_span;             // most coordinates any CTA rotates (set by gemv_plan)
+    const uint32_t *rot_negate;   // sign-flip bits, or null
+    double rot_scale;         // 2^-24 / sqrt(block length)
 #ifdef LLVQ_TRACE
     unsigned long long *trace;   // timeline buffer (debug builds only)
     int trace_launch;

@@ -24,42 +24,13 @@
 #include <cuda_runtime.h>
 
 #include "llvq_internal.cuh"
+#include "llvq_rotate.cuh"
 
 namespace llvq {
 namespace {
 
 constexpr int kRotThreads = 512;
 constexpr int kRotMinChunkLog2 = 12;     // a CTA takes at least 4096 coordinates: eight a thread and pass
-
-// R stages of the in-place butterfly on 2^R values: (a, b) -> (a + b, a - b) over every pair that differs in
-// one index bit.  With the values taken at stride 2^s these are stages s .. s + R - 1 of the transform.
-template <int R>
-__device__ __forceinline__ void butterflies(long long (&a)[8]) {
-#pragma unroll
-    for (int h = 1; h < (1 << R); h <<= 1) {
-#pragma unroll
-        for (int i = 0; i < (1 << R); i++) {
-            if ((i & h) == 0) {
-                const long long u = a[i], w = a[i + h];
-                a[i] = u + w;
-                a[i + h] = u - w;
-            }
-        }
-    }
-}
-
-template <int R>
-__device__ __forceinline__ void pass(long long *v, int s, int chunk, int tid) {
-    for (int g = tid; g < (chunk >> R); g += kRotThreads) {
-        const int base = ((g >> s) << (s + R)) | (g & ((1 << s) - 1));
-        long long a[8];
-#pragma unroll
-        for (int j = 0; j < (1 << R); j++) a[j] = v[base + (j << s)];
-        butterflies<R>(a);
-#pragma unroll
-        for (int j = 0; j < (1 << R); j++) v[base + (j << s)] = a[j];
-    }
-}
 
 __global__ void __launch_bounds__(kRotThreads)
 rotate_kernel(const __half *x, __half *y, const uint32_t *__restrict__ negate, long long n, int chunk_log2,
@@ -84,20 +55,13 @@ rotate_kernel(const __half *x, __half *y, const uint32_t *__restrict__ negate, l
             const long long at = first + 8 * g;
             const uint4 raw = *reinterpret_cast<const uint4 *>(x + at);
             const uint32_t flips = negate ? (negate[at >> 5] >> (at & 31)) & 0xffu : 0u;
-            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-            for (int i = 0; i < 4; i++) {
-                const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
-                const long long lo = __float2ll_rn(f.x * 16777216.f), hi = __float2ll_rn(f.y * 16777216.f);
-                a[2 * i] = ((flips >> (2 * i)) & 1u) ? -lo : lo;
-                a[2 * i + 1] = ((flips >> (2 * i + 1)) & 1u) ? -hi : hi;
-            }
-            if (block_log2 >= 3) butterflies<3>(a);
+            rot_load8(raw, flips, a);
+            if (block_log2 >= 3) rot_butterflies<3>(a);
             else if (block_log2 == 2) {
                 // two blocks of four: the butterflies of stages 0 and 1 never pair i with i + 4
                 long long b[8] = {a[0], a[1], a[2], a[3], 0, 0, 0, 0}, c[8] = {a[4], a[5], a[6], a[7], 0, 0, 0, 0};
-                butterflies<2>(b);
-                butterflies<2>(c);
+                rot_butterflies<2>(b);
+                rot_butterflies<2>(c);
 #pragma unroll
                 for (int i = 0; i < 4; i++) { a[i] = b[i]; a[4 + i] = c[i]; }
             } else if (block_log2 == 1) {
@@ -119,24 +83,11 @@ rotate_kernel(const __half *x, __half *y, const uint32_t *__restrict__ negate, l
 
     // Passes over the stages 3.., three at a time: a thread takes the eight (four, two) values that differ in
     // the pass's index bits.
-    for (int s = 3; s < block_log2; s += 3) {
-        const int r = block_log2 - s;
-        if (r >= 3) pass<3>(v, s, chunk, tid);
-        else if (r == 2) pass<2>(v, s, chunk, tid);
-        else pass<1>(v, s, chunk, tid);
-        __syncthreads();
-    }
+    rot_later_passes(v, block_log2, chunk, tid, kRotThreads);
 
     // The one rounding: exact sum -> f64 (exact below 2^53) -> times 2^-24 / sqrt(B) -> FP16, nearest even.
     for (int g = tid; 8 * g < count; g += kRotThreads) {
-        uint32_t out[4];
-#pragma unroll
-        for (int i = 0; i < 4; i++) {
-            const __half lo = __double2half((double)v[8 * g + 2 * i] * scale);
-            const __half hi = __double2half((double)v[8 * g + 2 * i + 1] * scale);
-            out[i] = (uint32_t)__half_as_ushort(lo) | ((uint32_t)__half_as_ushort(hi) << 16);
-        }
-        *reinterpret_cast<uint4 *>(y + first + 8 * g) = make_uint4(out[0], out[1], out[2], out[3]);
+        *reinterpret_cast<uint4 *>(y + first + 8 * g) = rot_round8(v + 8 * g, scale);
     }
 }
 

@@ -135,3 +135,72 @@ def test_rotate_error_codes(B, ctx):
     assert B.rotate_block(4096, 3) == 0 and B.rotate_block(0) == 0
     y = B.rotate(ctx, x)
     assert not y.any()
+
+
+# ---------------------------------------------------------------- the rotation inside the GEMV's launch
+def _rotated_reference(oracle, case, k, block, neg):
+    xr = np.concatenate([oracle.rotate(case.x[:k], block, neg), case.x[k:]])
+    return dataclasses.replace(case, x=xr)
+
+
+@pytest.mark.parametrize("rows,k,block,signs", [
+    (256, 2560, 0, False), (96, 4096, 0, True), (64, 9728, 0, True), (40, 17408, 0, False), (72, 5120, 0, True),
+    (33, 2560, 8, True), (64, 2560, 64, False), (48, 12288, 1024, True), (32, 16384, 0, False), (8, 32768, 8192, True),
+    (1, 24, 0, False), (300, 96, 32, True), (4096, 2560, 0, True)])
+def test_gemv_rotated_matches_oracle_chain_and_the_two_launch_form(B, ctx, oracle, rows, k, block, signs):
+    case = make_case(rows, k, seed=3 * rows + k)
+    kp = case.nb * 24
+    if k == 24:
+        k = 24                                                   # 24 = 8 * 3: blocks of eight
+    neg = np.random.default_rng(k + rows).integers(0, 2, size=k) if signs else None
+    bits = None if neg is None else _bits(neg)
+    buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    y = torch.full((rows,), float("nan"), dtype=torch.float32, device="cuda")
+    B.gemv_rotated(ctx, [(buf, case.d_scale, GAIN, y, rows)], case.d_x, kp, n=k, block=block, negate_bits=bits)
+    torch.cuda.synchronize()
+    ref = _rotated_reference(oracle, case, k, block, neg)
+    err, _ = check_gemv(oracle, ref, y)
+    assert err <= 1e-6
+    # the same through llvq_rotate and llvq_gemv: the two differ only by the fixed-point quantum of the GEMV
+    xr = case.d_x.clone()
+    B.rotate(ctx, case.d_x[:k], block=block, negate_bits=bits, y=xr[:k])
+    _same(xr, ref.x)
+    y2 = B.gemv(ctx, 0, buf, case.d_scale, GAIN, xr, rows, kp)
+    torch.cuda.synchronize()
+    _, wnorm, _ = oracle.matvec(case.codes, rows, case.nb, case.row_scale, GAIN, ref.x, nthreads=8)
+    bound = 1e-6 * wnorm * float(np.linalg.norm(ref.x.astype(np.float64))) + 1e-30
+    assert (np.abs(y.cpu().numpy().astype(np.float64) - y2.cpu().numpy().astype(np.float64)) <= bound).all()
+    assert torch.equal(case.d_x.cpu(), torch.from_numpy(case.x))      # x itself is left alone
+
+
+def test_gemv_rotated_grouped_launch_and_outlier_activation(B, ctx, oracle):
+    """q/k/v-like group sharing one x; x with one huge entry (what the rotation is for): the bound on the
+    rotated magnitudes is then loosest, and the result must still meet the bar with room."""
+    k = 2560
+    cases = [make_case(r, k, seed=50 + i, tensor_id=i) for i, r in enumerate((128, 32, 40))]
+    x = cases[0].x.copy()
+    x[777] = np.float16(30000.0)
+    d_x = torch.from_numpy(x).cuda()
+    kp = cases[0].nb * 24
+    bufs = [B.expand(ctx, 0, c.d_codes, c.rows, c.nb) for c in cases]
+    ys = [torch.empty(c.rows, dtype=torch.float32, device="cuda") for c in cases]
+    B.gemv_rotated(ctx, [(b, c.d_scale, GAIN, y, c.rows) for b, c, y in zip(bufs, cases, ys)], d_x, kp, n=k)
+    torch.cuda.synchronize()
+    xr = np.concatenate([oracle.rotate(x[:k]), x[k:]])
+    for c, y in zip(cases, ys):
+        err, _ = check_gemv(oracle, dataclasses.replace(c, x=xr), y)
+        assert err <= 1e-5
+
+
+def test_gemv_rotated_error_codes(B, ctx):
+    case = make_case(64, 96, seed=1)
+    buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    y = torch.empty(64, dtype=torch.float32, device="cuda")
+    prob = [(buf, case.d_scale, GAIN, y, 64)]
+    for kwargs in ({"n": 96, "block": 4}, {"n": 104}, {"n": 0}, {"n": 92}, {"n": 96, "block": 64}, {"n": 96, "block": 3}):
+        with pytest.raises(B.LlvqError) as e:
+            B.gemv_rotated(ctx, prob, case.d_x, 96, **kwargs)
+        assert e.value.code == -1
+    B.gemv_rotated(ctx, prob, case.d_x, 96, n=96)
+    torch.cuda.synchronize()
+    assert torch.isfinite(y).all()
