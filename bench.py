@@ -477,11 +477,16 @@ def main():
             for ln in copies[i % ncopies].launches:
                 k = ln["mats"][0].k
                 B.rotate(ctx, ln["x"][:k], y=xr[id(ln["x"])][:k])
+        def rot_fused_512(i):
+            for ln in copies[i % ncopies].launches:
+                B.gemv_rotated(ctx, ln["problems"], ln["x"], ln["k_padded"], n=ln["mats"][0].k, block=min(512, int(B.rotate_block(ln["mats"][0].k))))
         t_f = time_arm(rot_fused, ncopies, arm_steps, 3)
+        t_f512 = time_arm(rot_fused_512, ncopies, arm_steps, 3)
         t_2 = time_arm(rot_two, ncopies, arm_steps, 3)
         t_0 = time_arm(rot_only, ncopies, arm_steps, 3)
         n_launch = len(copies[0].launches)
-        arms["rotated"] = {"us_per_gemv_fused": t_f * 1e3 / n_gemv, "us_per_gemv_two_launches": t_2 * 1e3 / n_gemv,
+        arms["rotated"] = {"us_per_gemv_fused": t_f * 1e3 / n_gemv, "us_per_gemv_fused_blocks_of_512_at_most": t_f512 * 1e3 / n_gemv,
+                           "us_per_gemv_two_launches": t_2 * 1e3 / n_gemv,
                            "us_per_rotation_alone": t_0 * 1e3 / n_launch, "rotations_per_step": n_launch,
                            "block_lengths": sorted({int(B.rotate_block(ln["mats"][0].k)) for ln in copies[0].launches})}
         # no-weights control: the same launches without record reads

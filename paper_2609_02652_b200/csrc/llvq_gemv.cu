@@ -648,8 +648,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                     const uint32_t flips = p.rot_negate ? (__ldg(p.rot_negate + (e >> 2)) >> (8 * (e & 3))) & 0xffu : 0u;
                     rot_load8(v[i], flips, a);
                     rot_butterflies<3>(a);
-#pragma unroll
-                    for (int k = 0; k < 8; k++) rot[8 * e - c_lo + k] = a[k];
+                    rot_store8(rot, 8 * e - c_lo, a);
                 } else if (e >= e_lo && e < e_hi) {
                     mine = v[i];
                 }
@@ -673,7 +672,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         const float scale = pow2f(29 - xexp[0]);
         for (int e = e_lo + tid; e < e_hi; e += kThreads) {
             uint4 v;
-            if (8 * e < c_hi) v = rot_round8(rot + (8 * e - c_lo), p.rot_scale);
+            if (8 * e < c_hi) v = rot_round8(rot, 8 * e - c_lo, p.rot_scale);
             else v = one_each ? mine : __ldcg(xg + e);
             convert_item(v, e % 3, xs0 + (uint32_t)(e / 3) * kXRecBytes, scale);
         }

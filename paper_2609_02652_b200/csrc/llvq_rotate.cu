@@ -76,8 +76,7 @@ rotate_kernel(const __half *x, __half *y, const uint32_t *__restrict__ negate, l
 #pragma unroll
             for (int i = 0; i < 8; i++) a[i] = 0;                // past the end of x: never mixed with a block of x
         }
-#pragma unroll
-        for (int i = 0; i < 8; i++) v[8 * g + i] = a[i];
+        rot_store8(v, 8 * g, a);
     }
     __syncthreads();
 
@@ -87,7 +86,7 @@ rotate_kernel(const __half *x, __half *y, const uint32_t *__restrict__ negate, l
 
     // The one rounding: exact sum -> f64 (exact below 2^53) -> times 2^-24 / sqrt(B) -> FP16, nearest even.
     for (int g = tid; 8 * g < count; g += kRotThreads) {
-        *reinterpret_cast<uint4 *>(y + first + 8 * g) = rot_round8(v + 8 * g, scale);
+        *reinterpret_cast<uint4 *>(y + first + 8 * g) = rot_round8(v, 8 * g, scale);
     }
 }
 
