@@ -286,6 +286,8 @@ def main():
     ap.add_argument("--ungrouped", action="store_true", help="one launch a matrix instead of row-concatenated groups")
     ap.add_argument("--profile-batch", type=int, default=0,
                     help="profiling runs: only launch llvq_gemv_batch with this many activation vectors, one launch a matrix, and exit")
+    ap.add_argument("--profile-rotated", action="store_true",
+                    help="profiling runs: only launch llvq_rotate and llvq_gemv_rotated on the workload's launches, and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.lean:
@@ -338,6 +340,19 @@ def main():
         torch.cuda.synchronize()
         B.status(ctx)
         print(json.dumps({"profile": "llvq_gemv_batch", "vectors": nvec, "config": wl.name, "launches": (args.warmup + args.steps) * len(mats)}))
+        return
+
+    if args.profile_rotated:
+        # the rotation as a kernel of its own and inside the GEMV, for a profiler to capture; nothing is measured here
+        for i in range(args.warmup + args.steps):
+            for ln in copies[i % ncopies].launches:
+                k = ln["mats"][0].k
+                B.rotate(ctx, ln["x"][:k])
+                B.gemv_rotated(ctx, ln["problems"], ln["x"], ln["k_padded"], n=k)
+        torch.cuda.synchronize()
+        B.status(ctx)
+        print(json.dumps({"profile": "llvq_rotate + llvq_gemv_rotated", "config": wl.name,
+                          "launches": 2 * (args.warmup + args.steps) * launches_per_step}))
         return
 
     # expander throughput (load-time step, outside the timed region)
