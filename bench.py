@@ -412,28 +412,77 @@ def main():
     gbps = step_bytes / (ms_per_step * 1e-3) / 1e9            # per GPU
     per_shape = None
 
-    # end to end: x from pinned host memory, y back to the host, every step, through the same calls
-    pinned_x = [ln["x"].cpu().pin_memory() for ln in copies[0].launches]
-    pinned_y = [[torch.empty(y.shape, dtype=y.dtype).pin_memory() for y in ln["ys"]] for ln in copies[0].launches]
-    h2d = sum(x.numel() * 2 for x in pinned_x)
-    d2h = sum(y.numel() * 4 for ys in pinned_y for y in ys)
+    # End to end: every step copies that step's activations from pinned host memory to the device, runs the step's
+    # launches through the same C-ABI calls, copies every y back to pinned host memory and waits for it.  The
+    # host buffers are one block of x and one block of y a step (the launches' vectors at 256-byte offsets), so a
+    # step is one copy in, the launches, one copy out; the sequence is captured once per record copy as a CUDA
+    # graph, the way a serving loop would issue it, and replayed and waited for step by step.
+    def _offsets(sizes, align):
+        out, at = [], 0
+        for n in sizes:
+            out.append(at)
+            at += -(-n // align) * align
+        return out, at
+    l0 = copies[0].launches
+    x_off, x_total = _offsets([ln["x"].numel() for ln in l0], 128)
+    y_sizes = [m.rows for ln in l0 for m in ln["mats"]]
+    y_off, y_total = _offsets(y_sizes, 64)
+    host_x = torch.zeros(x_total, dtype=torch.float16).pin_memory()
+    host_y = torch.zeros(y_total, dtype=torch.float32).pin_memory()
+    dev_x = torch.zeros(x_total, dtype=torch.float16, device=device)
+    dev_y = torch.zeros(y_total, dtype=torch.float32, device=device)
+    for ln, off in zip(l0, x_off):
+        host_x[off:off + ln["x"].numel()] = ln["x"].cpu()
+    h2d = host_x.numel() * 2
+    d2h = host_y.numel() * 4
+    e2e_graphs = []
+    e2e_keep = []
+    side = torch.cuda.Stream()
+    for cp in copies:
+        yi = 0
+        plist = []
+        for ln, xo in zip(cp.launches, x_off):
+            ys = []
+            for m in ln["mats"]:
+                ys.append(dev_y[y_off[yi]:y_off[yi] + m.rows])
+                yi += 1
+            plist.append((B.make_problems([(b_, s_, datagen.GAIN, y_, m.rows) for b_, s_, y_, m in zip(ln["bufs"], ln["scales"], ys, ln["mats"])]),
+                          dev_x[xo:xo + ln["x"].numel()], ln["k_padded"]))
+        e2e_keep.append(plist)
+        def issue(plist=plist):
+            dev_x.copy_(host_x, non_blocking=True)
+            for probs, xv, kp in plist:
+                B.gemv_grouped(ctx, B.PLANES, probs, xv, kp)
+            host_y.copy_(dev_y, non_blocking=True)
+        with torch.cuda.stream(side):
+            issue()
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            issue()
+        e2e_graphs.append(g)
 
     def e2e_step(i):
-        cp = copies[i % ncopies]
-        for ln, px, pys in zip(cp.launches, pinned_x, pinned_y):
-            ln["x"].copy_(px, non_blocking=True)
-            B.gemv_grouped(ctx, B.PLANES, ln["problems"], ln["x"], ln["k_padded"])
-            for y, py in zip(ln["ys"], pys):
-                py.copy_(y, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        e2e_graphs[i % ncopies].replay()
+        torch.cuda.synchronize()
 
     e2e_steps = 1 if args.lean else min(args.steps, 300)
-    for i in range(0 if args.lean else 10):
+    for i in range(1 if args.lean else 10):
         e2e_step(i)
+    # the copies back are the results the launches computed: the last step's y against the device arrays
+    yi = 0
+    for ln in copies[(0 if args.lean else 9) % ncopies].launches:
+        for m in ln["mats"]:
+            assert torch.equal(host_y[y_off[yi]:y_off[yi] + m.rows], dev_y[y_off[yi]:y_off[yi] + m.rows].cpu())
+            yi += 1
     t1 = time.perf_counter()
     for i in range(e2e_steps):
         e2e_step(i)
     e2e_us = (time.perf_counter() - t1) / e2e_steps * 1e6 / n_gemv / world
+    # ... and they are the right results: one matrix of the last step against the untimed path's y (same records, same x)
+    run_step(B, ctx, B.PLANES, copies[(e2e_steps - 1) % ncopies])
+    torch.cuda.synchronize()
+    assert torch.equal(host_y[y_off[0]:y_off[0] + l0[0]["mats"][0].rows], copies[(e2e_steps - 1) % ncopies].launches[0]["ys"][0].cpu())
 
     arms = {}
     if len(mats) > 7:
@@ -562,7 +611,7 @@ def main():
                          "how": "algorithmic bytes of a step / CUDA-event time of the step, averaged over its launches"},
             "cpu_baseline": cpu_baseline,
             "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "how": "x from pinned host memory and y back to the host every step, stream synchronised per step"},
+                    "how": "every step: one copy of the step's x vectors from pinned host memory, the launches, one copy of every y back to pinned host memory, issued as a captured CUDA graph of those C-ABI calls and waited for before the next step"},
             "gpu_launches": args.steps * launches_per_step,
             "clocks": clocks, "parity_worst_normalised_error": worst,
             "expand_blocks_per_s": expand_rate, "per_shape": per_shape, "arms": arms,
