@@ -483,6 +483,7 @@ int llvqo_record(uint64_t code, uint32_t *fields, int8_t *x) {
 }
 
 size_t llvqo_planes_bytes(int64_t rows, int64_t nb) { return (size_t)((rows + 31) / 32) * (size_t)nb * 448u; }
+size_t llvqo_planes13_bytes(int64_t rows, int64_t nb) { return (size_t)((rows + 31) / 32) * (size_t)nb * 416u; }
 size_t llvqo_onehot_bytes(int64_t rows, int64_t nb) { return (size_t)((rows + 31) / 32) * (size_t)nb * 640u; }
 
 /*
@@ -514,6 +515,17 @@ size_t llvqo_onehot_bytes(int64_t rows, int64_t nb) { return (size_t)((rows + 31
  *           16 s .. 16 s + 15 of that block (read "row (m,e,g), slot s" above as row (s,e,g));
  *           word w of lane L at 128 w + 4 L; header word of pair P at 384 + 4 P.
  * A row group occupies 448 nb bytes.
+ *
+ * 13-byte layout: the matvec needs of the header only what fixes the block's scale and the
+ * parity of its coordinates, so the 16-bit header shrinks to one byte
+ *     shell (4 bits, 0 for the sentinel) | parity << 4 | gain << 5
+ * and everything else stays: the same code words at the same places, then the header bytes.
+ *   tile, 1664 bytes: header byte of pair P, half-step h, row half e at 1536 + 8 P + 2 h + e;
+ *   pair, 832 bytes: header byte of pair P, half-step m, row half e at 768 + 4 P + 2 m + e;
+ *   single, 416 bytes: header byte of pair P (slot = t >> 1 = the 16-row half), row half e at 384 + 2 P + e.
+ * A row group occupies 416 nb bytes.  Every lattice point of the ball has such a record: the
+ * layout is exact for all blocks at 4.33 bits a weight (the rate the paper reaches with a
+ * 12-byte record plus an exception table for five-level blocks, Sec. 3.3).
  */
 typedef struct { const uint8_t *code; const uint16_t *hdr; int64_t nb; } group_t;   /* code[(r*nb+b)*24+i], hdr[r*nb+b] */
 
@@ -543,7 +555,8 @@ static void hs_words(const group_t *G, int64_t b0, int64_t b1, int m, int g, int
     *hw = hs_header(G, b0, b1, m, 0, g, t >> 1) | hs_header(G, b0, b1, m, 1, g, t >> 1) << 16;
 }
 
-void llvqo_pack_planes(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t *out) {
+static void pack_planes_any(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t *out, int compact) {
+    const size_t cell = compact ? 416u : 448u, words4 = 1536u, words2 = 768u, words1 = 384u;
     int64_t ngroups = (rows + 31) / 32, ntiles = nb / 4, left = nb % 4;
     uint8_t *code = malloc((size_t)32 * nb * 24);
     uint16_t *hdr = malloc((size_t)32 * nb * 2);
@@ -556,10 +569,11 @@ void llvqo_pack_planes(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t 
                 else { memset(&rec, 0, sizeof rec); rec.cls = SENTINEL_CLASS; }
                 int parity = rec.cls == SENTINEL_CLASS ? 0 : (rec.x[0] & 1);
                 for (int i = 0; i < NCOORD; i++) code[((size_t)r * nb + b) * 24 + i] = (uint8_t)(8 + (rec.x[i] - parity) / 2);
-                hdr[(size_t)r * nb + b] = (uint16_t)(rec.cls | (rec.gain << 9));
+                hdr[(size_t)r * nb + b] = compact ? (uint16_t)((rec.cls == SENTINEL_CLASS ? 0 : g_cls[rec.cls].shell) | (parity << 4) | (rec.gain << 5))
+                                                  : (uint16_t)(rec.cls | (rec.gain << 9));
             }
         group_t G = {code, hdr, nb};
-        uint8_t *grp = out + (size_t)rg * (size_t)nb * 448u;
+        uint8_t *grp = out + (size_t)rg * (size_t)nb * cell;
         uint32_t w[3], hw;
         for (int g = 0; g < 8; g++)
             for (int t = 0; t < 4; t++) {
@@ -567,28 +581,33 @@ void llvqo_pack_planes(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t 
                 for (int64_t T = 0; T < ntiles; T++)
                     for (int h = 0; h < 4; h++) {
                         hs_words(&G, 4 * T + 2 * (h >> 1), 4 * T + 2 * (h >> 1) + 1, h & 1, g, t, w, &hw);
-                        uint8_t *tile = grp + (size_t)T * 1792u;
+                        uint8_t *tile = grp + (size_t)T * 4u * cell;
                         for (int q = 0; q < 3; q++) { int k = 3 * h + q; memcpy(tile + 512 * (k >> 2) + 16 * L + 4 * (k & 3), &w[q], 4); }
-                        memcpy(tile + 1536 + 16 * P + 4 * h, &hw, 4);
+                        if (compact) { tile[words4 + 8 * P + 2 * h] = (uint8_t)hw; tile[words4 + 8 * P + 2 * h + 1] = (uint8_t)(hw >> 16); }
+                        else memcpy(tile + words4 + 16 * P + 4 * h, &hw, 4);
                     }
-                uint8_t *rest = grp + (size_t)ntiles * 1792u;
+                uint8_t *rest = grp + (size_t)ntiles * 4u * cell;
                 if (left >= 2) {
                     for (int m = 0; m < 2; m++) {
                         hs_words(&G, 4 * ntiles, 4 * ntiles + 1, m, g, t, w, &hw);
                         for (int q = 0; q < 3; q++) memcpy(rest + 128 * (3 * m + q) + 4 * L, &w[q], 4);
-                        memcpy(rest + 768 + 8 * P + 4 * m, &hw, 4);
+                        if (compact) { rest[words2 + 4 * P + 2 * m] = (uint8_t)hw; rest[words2 + 4 * P + 2 * m + 1] = (uint8_t)(hw >> 16); }
+                        else memcpy(rest + words2 + 8 * P + 4 * m, &hw, 4);
                     }
-                    rest += 896;
+                    rest += 2u * cell;
                 }
                 if (left & 1) {
                     hs_words(&G, nb - 1, -1, 0, g, t, w, &hw);
                     for (int q = 0; q < 3; q++) memcpy(rest + 128 * q + 4 * L, &w[q], 4);
-                    memcpy(rest + 384 + 4 * P, &hw, 4);
+                    if (compact) { rest[words1 + 2 * P] = (uint8_t)hw; rest[words1 + 2 * P + 1] = (uint8_t)(hw >> 16); }
+                    else memcpy(rest + words1 + 4 * P, &hw, 4);
                 }
             }
     }
     free(code); free(hdr);
 }
+void llvqo_pack_planes(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t *out) { pack_planes_any(codes, rows, nb, out, 0); }
+void llvqo_pack_planes13(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t *out) { pack_planes_any(codes, rows, nb, out, 1); }
 
 /*
  * One-hot layout, 20 bytes a block: the cell of (row group, block column) is five arrays of 32

@@ -66,6 +66,10 @@ def lib() -> ctypes.CDLL:
             L.llvqo_pack_planes.argtypes = [vp, i64, i64, vp]
             L.llvqo_pack_planes.restype = None
             L.llvqo_pack_onehot.argtypes = [vp, i64, i64, vp]
+            L.llvqo_pack_planes13.argtypes = [vp, i64, i64, vp]
+            L.llvqo_pack_planes13.restype = None
+            L.llvqo_planes13_bytes.argtypes = [i64, i64]
+            L.llvqo_planes13_bytes.restype = ctypes.c_size_t
             L.llvqo_pack_onehot.restype = None
             L.llvqo_dequant.argtypes = [vp, i64, i64, vp, vp, vp]
             L.llvqo_dequant.restype = None
@@ -168,6 +172,19 @@ def pack_planes(codes: np.ndarray, rows: int, nb: int) -> np.ndarray:
     assert codes.size == rows * nb
     out = np.zeros(planes_bytes(rows, nb), np.uint8)
     lib().llvqo_pack_planes(_ptr(codes), rows, nb, _ptr(out))
+    return out
+
+
+def planes13_bytes(rows: int, nb: int) -> int:
+    return int(lib().llvqo_planes13_bytes(rows, nb))
+
+
+def pack_planes13(codes: np.ndarray, rows: int, nb: int) -> np.ndarray:
+    """Expected bytes of the 13-byte layout: the 14-byte layout's codes with a one-byte header (shell, parity, gain)."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint64).ravel()
+    assert codes.size == rows * nb
+    out = np.zeros(planes13_bytes(rows, nb), np.uint8)
+    lib().llvqo_pack_planes13(_ptr(codes), rows, nb, _ptr(out))
     return out
 
 

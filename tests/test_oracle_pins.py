@@ -329,6 +329,83 @@ def test_planes_layout_round_trip(oracle, rows, nb):
                 assert v == (8 - level - par if (rec["smask"] >> i) & 1 else 8 + level)
 
 
+def _unpack_planes13_cell(buf, nb, row, b):
+    """Reader of the 13-byte layout from its description: (row, block) -> header byte fields and the 24 codes."""
+    rg, r = divmod(row, 32)
+    m, e, g = r // 16, (r // 8) % 2, r % 8
+    grp = rg * nb * 416
+    ntiles, left = divmod(nb, 4)
+
+    def word(off):
+        return int.from_bytes(buf[off: off + 4].tobytes(), "little")
+
+    j = b - 4 * ntiles
+    if j < 0:
+        base = grp + (b // 4) * 1664
+        slot, h = b % 2, 2 * ((b % 4) // 2) + m
+        addr = lambda q, lane: base + 512 * ((3 * h + q) >> 2) + 16 * lane + 4 * ((3 * h + q) & 3)
+        hb = int(buf[base + 1536 + 8 * (2 * g + slot) + 2 * h + e])
+    elif left >= 2 and j < 2:
+        base = grp + ntiles * 1664
+        slot = j
+        addr = lambda q, lane: base + 128 * (3 * m + q) + 4 * lane
+        hb = int(buf[base + 768 + 4 * (2 * g + slot) + 2 * m + e])
+    else:
+        base = grp + ntiles * 1664 + (832 if left == 3 else 0)
+        slot = m
+        addr = lambda q, lane: base + 128 * q + 4 * lane
+        hb = int(buf[base + 384 + 2 * (2 * g + slot) + e])
+    assert hb >> 6 == 0
+    codes = []
+    for i in range(24):
+        kappa = 24 * slot + i
+        if kappa < 32:
+            c, t, ii = kappa // 16, (kappa % 16) // 4, kappa % 4
+            w = word(addr(e, 4 * g + t))
+        else:
+            c, t, ii = e, (kappa - 32) // 4, (kappa - 32) % 4
+            w = word(addr(2, 4 * g + t))
+        codes.append((w >> (4 * (2 * ii + c))) & 15)
+    return hb & 15, (hb >> 4) & 1, (hb >> 5) & 1, codes
+
+
+@pytest.mark.parametrize("rows,nb", [(32, 4), (37, 7), (64, 1), (5, 2), (33, 3), (20, 6), (50, 9)])
+def test_planes13_layout_round_trip(oracle, rows, nb):
+    """The 13-byte layout holds, for every block, the shell, the parity and the gain bit in its header byte and the
+    same 24 codes as the 14-byte layout: enough to rebuild the block's weights exactly."""
+    codes = _codes(oracle, rows, nb, seed=8)
+    buf = oracle.pack_planes13(codes, rows, nb)
+    assert buf.size == ((rows + 31) // 32) * nb * 416 == oracle.planes13_bytes(rows, nb)
+    xs, cls = oracle.decode_batch(codes)
+    seen = np.zeros(buf.size, bool)
+    for row in range(((rows + 31) // 32) * 32):
+        for b in range(nb):
+            shell, par, gain, u = _unpack_planes13_cell(buf, nb, row, b)
+            if row >= rows or cls[row * nb + b] < 0:
+                assert (shell, par, gain) == (0, 0, 0) and u == [8] * 24
+                continue
+            x = xs[row * nb + b]
+            assert shell == int((x.astype(np.int64) ** 2).sum()) // 16 and par == int(x[0]) & 1
+            assert gain == int(codes[row * nb + b]) >> 47
+            assert [2 * (v - 8) + par for v in u] == x.tolist()
+            assert _unpack_planes_cell(oracle.pack_planes(codes, rows, nb), nb, row, b)[2] == u
+    # 13 bytes a block: 12 of codes, one header byte (4.33 bits a weight)
+    assert buf.size * 8 / (((rows + 31) // 32) * 32 * nb * 24) == pytest.approx(13 * 8 / 24)
+
+
+def test_planes13_layout_worked_example_by_hand(oracle):
+    """One row, one block, index 0 = (0^22, 4, 4) in shell 2, even: codes 8 except the last two (10); the single's
+    header bytes sit at 384 + 2 P + e, and row 0 is (g, e, half) = (0, 0, 0): byte 384 = shell 2, no parity, no gain."""
+    buf = oracle.pack_planes13(np.array([0], np.uint64), 1, 1)
+    assert buf.size == 416
+    words = buf[:384].view(np.uint32)
+    assert int(words[1]) == 0xA8A88888                        # as in the 14-byte layout: the same code words
+    assert [int(w) for i, w in enumerate(words) if i != 1] == [0x88888888] * 95
+    assert int(buf[384]) == 2 and not buf[385:].any()
+    buf = oracle.pack_planes13(np.array([1 << 47], np.uint64), 1, 1)
+    assert int(buf[384]) == 2 | (1 << 5)
+
+
 @pytest.mark.parametrize("rows,nb", [(32, 3), (37, 5)])
 def test_onehot_layout_round_trip_and_field_widths(oracle, rows, nb):
     codes = _codes(oracle, rows, nb, seed=6)
