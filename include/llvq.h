@@ -75,6 +75,7 @@ extern "C" {
 
 #define LLVQ_PLANES 0
 #define LLVQ_ONEHOT 1
+#define LLVQ_PLANES13 2
 
 #define LLVQ_OK 0
 #define LLVQ_EINVAL (-1) /* null pointer, bad shape, unknown layout                         */

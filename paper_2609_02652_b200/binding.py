@@ -14,6 +14,7 @@ import torch
 
 PLANES = 0
 ONEHOT = 1
+PLANES13 = 2      # the 14-byte layout's codes with a one-byte header: 13 bytes a block
 MAX_GROUP = 8
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libllvq.so")

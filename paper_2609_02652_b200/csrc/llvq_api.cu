@@ -24,7 +24,7 @@ inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_
 
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
-int layout_cell_bytes(int layout) { return layout == LLVQ_PLANES ? kCellBytes : kOneHotCellBytes; }
+int layout_cell_bytes(int layout) { return layout == LLVQ_PLANES ? kCellBytes : (layout == LLVQ_PLANES13 ? kCell13Bytes : kOneHotCellBytes); }
 
 }  // namespace
 
@@ -159,7 +159,7 @@ uint64_t llvq_class_base(const llvq_ctx *ctx, int c) {
 
 int llvq_layout_bytes(int layout, int64_t rows, int64_t k_padded, size_t *bytes) {
     if (!bytes || rows <= 0 || k_padded <= 0 || k_padded % 24 != 0) return LLVQ_EINVAL;
-    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT) return LLVQ_EINVAL;
+    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT && layout != LLVQ_PLANES13) return LLVQ_EINVAL;
     const size_t groups = (size_t)((rows + kRowsPerGroup - 1) / kRowsPerGroup);
     *bytes = groups * (size_t)(k_padded / 24) * (size_t)layout_cell_bytes(layout);
     return LLVQ_OK;
@@ -214,7 +214,8 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
                     bool no_weights, void *stream, int batch = 1, const llvq_rotation *rot = nullptr) {
     if (!ctx || !problems || !x || n < 1 || n > LLVQ_MAX_GROUP) return LLVQ_EINVAL;
     if (batch < 1 || batch > kVectorsPerPass || (batch > 1 && (n != 1 || layout != LLVQ_PLANES || no_weights))) return LLVQ_EINVAL;
-    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT) return LLVQ_EINVAL;
+    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT && layout != LLVQ_PLANES13) return LLVQ_EINVAL;
+    if (layout == LLVQ_PLANES13 && (no_weights || batch != 1 || rot)) return LLVQ_EINVAL;
     if (k_padded <= 0 || k_padded % 24 != 0) return LLVQ_EINVAL;
     if (k_padded > LLVQ_MAX_K) return LLVQ_ESIZE;
     if (!aligned(x, 16)) return LLVQ_EALIGN;
@@ -370,7 +371,7 @@ int llvq_dequant_fp16(llvq_ctx *ctx, int layout, const void *layout_buf, const v
 int llvq_decode_i8(llvq_ctx *ctx, int layout, const void *layout_buf, int8_t *coords, uint16_t *class_ids, int64_t rows,
                    int64_t nb, void *stream) {
     if (!ctx || !layout_buf || !coords || !class_ids || rows <= 0 || nb <= 0) return LLVQ_EINVAL;
-    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT) return LLVQ_EINVAL;
+    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT && layout != LLVQ_PLANES13) return LLVQ_EINVAL;
     if (!aligned(layout_buf, 128) || !aligned(class_ids, 2)) return LLVQ_EALIGN;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;

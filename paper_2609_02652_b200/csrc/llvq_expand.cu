@@ -132,6 +132,13 @@ __device__ __forceinline__ uint32_t spread4(uint32_t h) {
 // One warp writes one piece of a row group: a tile (four blocks), the pair after the tiles or the
 // single at the end (see include/llvq.h).  First every lane decodes the blocks of its own row into
 // shared memory in coordinate order, then lane 4g+t gathers the words it owns in the layout.
+// two header pairs (each two 16-bit fields of which the low byte counts) -> four bytes
+__device__ __forceinline__ uint32_t bytes4(uint32_t a, uint32_t b) {
+    return (a & 0xffu) | ((a >> 8) & 0xff00u) | ((b & 0xffu) << 16) | ((b << 8) & 0xff000000u);
+}
+
+// COMPACT: the 13-byte layout - the same code words, the header one byte: shell | parity << 4 | gain << 5.
+template <bool COMPACT>
 __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, const uint64_t *__restrict__ codes, int64_t rows, int64_t nb,
                                                             uint8_t *__restrict__ out, uint32_t *bad_count) {
     __shared__ uint32_t nat_all[8][4][4][32];              // [warp][block of the piece][word 0..2, header][row]
@@ -145,7 +152,8 @@ __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, cons
     uint32_t (*nat)[4][32] = nat_all[threadIdx.x >> 5];
     const int64_t rg = piece_id / pieces, u = piece_id % pieces;
     const int64_t row = rg * kRowsPerGroup + lane;
-    uint8_t *grp = out + (size_t)rg * (size_t)nb * kCellBytes;
+    constexpr int kCell = COMPACT ? kCell13Bytes : kCellBytes, kTile = COMPACT ? kTile13Bytes : kTileBytes;
+    uint8_t *grp = out + (size_t)rg * (size_t)nb * kCell;
     const bool is_tile = u < tiles;
     const bool is_pair = !is_tile && left >= 2 && u == tiles;
     const int ncell = is_tile ? 4 : (is_pair ? 2 : 1);
@@ -160,7 +168,8 @@ __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, cons
             d.cls = kEmptyClass; d.gain = 0; d.smask = 0; d.mag[0] = d.mag[1] = d.mag[2] = 0;
         }
         nat[q][0][lane] = code_word(d, 0); nat[q][1][lane] = code_word(d, 1); nat[q][2][lane] = code_word(d, 2);
-        nat[q][3][lane] = (uint32_t)d.cls | ((uint32_t)d.gain << 9);
+        if (COMPACT) nat[q][3][lane] = d.cls == kEmptyClass ? 0u : ((uint32_t)T.desc[d.cls].shell | ((uint32_t)T.desc[d.cls].odd << 4) | ((uint32_t)d.gain << 5));
+        else nat[q][3][lane] = (uint32_t)d.cls | ((uint32_t)d.gain << 9);
     }
     __syncwarp();
     const int g = lane >> 2, t = lane & 3;
@@ -186,28 +195,36 @@ __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, cons
         uint32_t w[12], hw[4];
 #pragma unroll
         for (int h = 0; h < 4; h++) half_step(2 * (h >> 1), h & 1, w + 3 * h, hw[h]);
-        uint8_t *tile = grp + (size_t)u * kTileBytes;
+        uint8_t *tile = grp + (size_t)u * kTile;
 #pragma unroll
         for (int j = 0; j < 3; j++)
             *reinterpret_cast<uint4 *>(tile + 512 * j + 16 * lane) = make_uint4(w[4 * j], w[4 * j + 1], w[4 * j + 2], w[4 * j + 3]);
-        if ((t & 1) == 0) *reinterpret_cast<uint4 *>(tile + 1536 + 16 * (lane >> 1)) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+        if ((t & 1) == 0) {
+            if (COMPACT) *reinterpret_cast<uint2 *>(tile + 1536 + 8 * (lane >> 1)) = make_uint2(bytes4(hw[0], hw[1]), bytes4(hw[2], hw[3]));
+            else *reinterpret_cast<uint4 *>(tile + 1536 + 16 * (lane >> 1)) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+        }
     } else if (is_pair) {
-        uint8_t *pair = grp + (size_t)tiles * kTileBytes;
+        uint8_t *pair = grp + (size_t)tiles * kTile;
+        uint32_t hw[2];
 #pragma unroll
         for (int m = 0; m < 2; m++) {
-            uint32_t w[3], hw;
-            half_step(0, m, w, hw);
+            uint32_t w[3];
+            half_step(0, m, w, hw[m]);
 #pragma unroll
             for (int q = 0; q < 3; q++) *reinterpret_cast<uint32_t *>(pair + 128 * (3 * m + q) + 4 * lane) = w[q];
-            if ((t & 1) == 0) *reinterpret_cast<uint32_t *>(pair + 768 + 8 * (lane >> 1) + 4 * m) = hw;
+            if (!COMPACT && (t & 1) == 0) *reinterpret_cast<uint32_t *>(pair + 768 + 8 * (lane >> 1) + 4 * m) = hw[m];
         }
+        if (COMPACT && (t & 1) == 0) *reinterpret_cast<uint32_t *>(pair + 768 + 4 * (lane >> 1)) = bytes4(hw[0], hw[1]);
     } else {
-        uint8_t *one = grp + (size_t)tiles * kTileBytes + (left == 3 ? 2 * kCellBytes : 0);
+        uint8_t *one = grp + (size_t)tiles * kTile + (left == 3 ? 2 * kCell : 0);
         uint32_t w[3], hw;
         half_step(0, 0, w, hw);
 #pragma unroll
         for (int q = 0; q < 3; q++) *reinterpret_cast<uint32_t *>(one + 128 * q + 4 * lane) = w[q];
-        if ((t & 1) == 0) *reinterpret_cast<uint32_t *>(one + 384 + 4 * (lane >> 1)) = hw;
+        if ((t & 1) == 0) {
+            if (COMPACT) *reinterpret_cast<uint16_t *>(one + 384 + 2 * (lane >> 1)) = (uint16_t)((hw & 0xffu) | ((hw >> 8) & 0xff00u));
+            else *reinterpret_cast<uint32_t *>(one + 384 + 4 * (lane >> 1)) = hw;
+        }
     }
     if (bad && bad_count) atomicAdd(bad_count, (uint32_t)bad);
 }
@@ -253,12 +270,13 @@ __global__ void __launch_bounds__(256) expand_onehot_kernel(DeviceTables T, cons
 cudaError_t launch_expand(const llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, int64_t nb,
                           void *out, uint32_t *bad_count, cudaStream_t s) {
     const int64_t groups = (rows + kRowsPerGroup - 1) / kRowsPerGroup;
-    if (layout == LLVQ_PLANES) {
+    if (layout == LLVQ_PLANES || layout == LLVQ_PLANES13) {
         const int64_t left = nb % kTileCells;
         const int64_t pieces = nb / kTileCells + (left >= 2 ? 1 : 0) + (left & 1);
         const int64_t threads = groups * pieces * 32;
         const int64_t blocks = (threads + 255) / 256;
-        expand_planes_kernel<<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count);
+        if (layout == LLVQ_PLANES13) expand_planes_kernel<true><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count);
+        else expand_planes_kernel<false><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count);
     } else {
         const int64_t threads = groups * nb * 32;
         const int64_t blocks = (threads + 255) / 256;

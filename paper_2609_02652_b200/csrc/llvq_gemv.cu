@@ -228,6 +228,11 @@ __device__ __forceinline__ uint4 lds128(uint32_t a) {
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
     return v;
 }
+__device__ __forceinline__ uint2 lds64(uint32_t a) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a));
+    return v;
+}
 __device__ __forceinline__ uint32_t lds32(uint32_t a) {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
@@ -328,14 +333,22 @@ struct HalfA {
     uint32_t a0, a1, a2, a3, c0, c1;
     float2 k0, k1;
 };
+// COMPACT (13-byte layout): the two headers are the bytes at bit SHIFT and SHIFT + 8 of hw.
+template <bool COMPACT = false, int SHIFT = 0>
 __device__ __forceinline__ HalfA decode_half(uint32_t wa, uint32_t wb, uint32_t wc, uint32_t hw, uint32_t tq) {
     constexpr uint32_t kNib = 0x0f0f0f0fu;
     HalfA h;
     h.a0 = wa & kNib; h.a1 = wb & kNib; h.a2 = (wa >> 4) & kNib; h.a3 = (wb >> 4) & kNib;
     h.c0 = wc & kNib; h.c1 = (wc >> 4) & kNib;
-    // the headers of rows g (low half of hw) and g + 8 (high half), eight bytes an entry; tq is 8 KiB-aligned
-    h.k0 = lds_f2(and_or(hw << 3, 0x1ff8u, tq));
-    h.k1 = lds_f2(and_or(hw >> 13, 0x1ff8u, tq));
+    if (COMPACT) {
+        // one byte a header, eight bytes an entry
+        h.k0 = lds_f2(and_or(SHIFT >= 3 ? hw >> (SHIFT - 3) : hw << (3 - SHIFT), 0x7f8u, tq));
+        h.k1 = lds_f2(and_or(hw >> (SHIFT + 5), 0x7f8u, tq));
+    } else {
+        // the headers of rows g (low half of hw) and g + 8 (high half), eight bytes an entry; tq is 8 KiB-aligned
+        h.k0 = lds_f2(and_or(hw << 3, 0x1ff8u, tq));
+        h.k1 = lds_f2(and_or(hw >> 13, 0x1ff8u, tq));
+    }
     return h;
 }
 template <bool FIRST>
@@ -444,8 +457,11 @@ __device__ __forceinline__ bool advance(const GemvParams &p, Cursor &c, int n) {
 // BATCH sets of total_groups * 32.
 // ROTATE: x is rotated on its way into the records (llvq_gemv_rotated): every CTA rotates the Walsh-Hadamard
 // blocks of x that its share of the matrix touches, exactly as the rotation kernel does, and rounds them to FP16.
-template <bool NO_WEIGHTS, int BATCH, bool ROTATE = false>
+// COMPACT: the 13-byte layout (one header byte a block; the code words are where the 14-byte layout has them).
+template <bool NO_WEIGHTS, int BATCH, bool ROTATE = false, bool COMPACT = false>
 __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
+    constexpr int kSrcCell = COMPACT ? kCell13Bytes : kCellBytes;        // bytes of a block column of a row group
+    constexpr int kSrcTile = COMPACT ? kTile13Bytes : kTileBytes;        // bytes of a tile in memory (a ring slot always has kTileBytes)
     extern __shared__ __align__(128) unsigned char smem[];
     // shared memory: ring | per-matrix block constants (1024 x {gain / (4 sqrt m), parity - 16}) | x records | barriers
     unsigned char *ring = smem;
@@ -511,8 +527,8 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     Cursor cc = locate(p, u0), ic = cc;
     int q = 0;
     const uint8_t *isrc = nullptr;                     // first byte of the issue side's row group
-    if (n_units > 0) isrc = group_base(p, ic.group, kCellBytes, q);
-    const uint32_t tail_bytes = (uint32_t)p.tail_cells * kCellBytes;
+    if (n_units > 0) isrc = group_base(p, ic.group, kSrcCell, q);
+    const uint32_t tail_bytes = (uint32_t)p.tail_cells * kSrcCell;
 
     // The issue side's walk: inext is the next unit's first byte, ileft the units left in its stretch of its
     // row group.  next() hands out the unit's source and size and steps on.
@@ -525,10 +541,10 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     const int n_tiles_total = p.tiles;
     Walk iw;
     iw.c = ic;
-    iw.next = isrc + (size_t)ic.col * kTileBytes;      // the leftover blocks follow the last tile
+    iw.next = isrc + (size_t)ic.col * kSrcTile;      // the leftover blocks follow the last tile
     iw.left = ic.end - ic.col;
     iw.done = 0;
-    iw.bytes = ic.col < n_tiles_total ? (uint32_t)kTileBytes : tail_bytes;
+    iw.bytes = ic.col < n_tiles_total ? (uint32_t)kSrcTile : tail_bytes;
     // the stretch ends or its last unit is the leftover one: the next unit starts elsewhere or has another size
     auto walk_turn = [&](Walk &w) {
         if (w.left == 0) {
@@ -536,17 +552,17 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             advance(p, w.c, 1);
             if (w.done < n_units) {
                 int qi;
-                w.next = group_base(p, w.c.group, kCellBytes, qi) + (size_t)w.c.col * kTileBytes;
+                w.next = group_base(p, w.c.group, kSrcCell, qi) + (size_t)w.c.col * kSrcTile;
             }
             w.left = w.c.end - w.c.col;
         }
-        w.bytes = w.c.col < n_tiles_total ? (uint32_t)kTileBytes : tail_bytes;
+        w.bytes = w.c.col < n_tiles_total ? (uint32_t)kSrcTile : tail_bytes;
     };
     auto walk_next = [&](Walk &w, const uint8_t *&src, uint32_t &bytes) {
         src = w.next;
         bytes = w.bytes;
         w.done++;
-        w.next += kTileBytes;
+        w.next += kSrcTile;
         w.c.col++;
         if (--w.left <= 1) walk_turn(w);               // rare: at most twice a stretch
     };
@@ -707,6 +723,15 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                     }
                     // block constants of every matrix of the launch: (class | gain << 9) -> {gain / (4 sqrt m), parity - 16},
                     // from the class constants in the kernel's parameters
+                    if (COMPACT) {
+                        // 13-byte layout: the header byte is shell | parity << 4 | gain << 5 - 64 entries a matrix
+                        for (int e = tid; e < p.nprob * 64; e += kThreads) {
+                            const uint32_t shell = e & 15u;
+                            const GemvProblemDev &pe = p.prob[e >> 6];
+                            tab[(e >> 6) * 1024 + (e & 63)] = make_float2(p.shell_inv_norm[shell] * ((e & 32) ? pe.gain1 : pe.gain0),
+                                                                         __int_as_float(shell ? ((e >> 4) & 1) - 16 : 0));
+                        }
+                    } else
                     for (int e = tid; e < tab_entries; e += kThreads) {
                         const int c = e & 511;
                         const uint32_t shell = (p.cls_shell_nibbles[c >> 3] >> (4 * (c & 7))) & 15u;
@@ -800,7 +825,10 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             const uint4 a0 = lds128(sbuf + lane16);
             const uint4 a1 = lds128(sbuf + lane16 + 512);
             const uint4 a2 = lds128(sbuf + lane16 + 1024);
-            const uint4 hh = lds128(sbuf + pair16 + 1536);
+            // headers: four words a lane pair (14-byte layout) or two (13-byte layout: hh.x serves half-steps 0, 1, hh.y 2, 3)
+            uint4 hh;
+            if (COMPACT) { const uint2 h2 = lds64(sbuf + (pair16 >> 1) + 1536); hh = make_uint4(h2.x, h2.y, h2.y, h2.x); }
+            else hh = lds128(sbuf + pair16 + 1536);
             // The slot's words are in registers: refill it at once with the unit kSlots ahead, so
             // that every slot but the one just read is in flight while this unit is decoded.  The
             // copy's address is made to depend on the loaded words, which holds the copy back
@@ -821,10 +849,10 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                     const LaneOffsets xj = {xa.b0 + j * xrec_stride, xa.b1 + j * xrec_stride, xa.b2 + j * xrec_stride, xa.xs + j * xrec_stride};
                     sx[j] = load_step<0>(xj);
                 }
-                const HalfA h0 = decode_half(a0.x, a0.y, a0.z, hh.x, tq);
+                const HalfA h0 = decode_half<COMPACT, 0>(a0.x, a0.y, a0.z, hh.x, tq);
 #pragma unroll
                 for (int j = 0; j < BATCH; j++) contract_half<true>(h0, sx[j], acc[j][0], acc[j][1]);
-                const HalfA h1 = decode_half(a0.w, a1.x, a1.y, hh.y, tq);
+                const HalfA h1 = decode_half<COMPACT, 16>(a0.w, a1.x, a1.y, COMPACT ? hh.x : hh.y, tq);
 #pragma unroll
                 for (int j = 0; j < BATCH; j++) contract_half<true>(h1, sx[j], acc[j][2], acc[j][3]);
 #pragma unroll
@@ -832,10 +860,10 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                     const LaneOffsets xj = {xa.b0 + j * xrec_stride, xa.b1 + j * xrec_stride, xa.b2 + j * xrec_stride, xa.xs + j * xrec_stride};
                     sx[j] = load_step<2 * kXRecBytes>(xj);
                 }
-                const HalfA h2 = decode_half(a1.z, a1.w, a2.x, hh.z, tq);
+                const HalfA h2 = decode_half<COMPACT, 0>(a1.z, a1.w, a2.x, COMPACT ? hh.y : hh.z, tq);
 #pragma unroll
                 for (int j = 0; j < BATCH; j++) contract_half<false>(h2, sx[j], acc[j][0], acc[j][1]);
-                const HalfA h3 = decode_half(a2.y, a2.z, a2.w, hh.w, tq);
+                const HalfA h3 = decode_half<COMPACT, 16>(a2.y, a2.z, a2.w, COMPACT ? hh.y : hh.w, tq);
 #pragma unroll
                 for (int j = 0; j < BATCH; j++) contract_half<false>(h3, sx[j], acc[j][2], acc[j][3]);
             }
@@ -864,9 +892,10 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
 #pragma unroll
                 for (int m = 0; m < 2; m++) {
                     const uint32_t wa = lds32(piece + 128 * (3 * m) + lane4), wb = lds32(piece + 128 * (3 * m + 1) + lane4);
-                    const uint32_t wc = lds32(piece + 128 * (3 * m + 2) + lane4), hw = lds32(piece + 768 + 8 * (lane >> 1) + 4 * m);
+                    const uint32_t wc = lds32(piece + 128 * (3 * m + 2) + lane4);
+                    const uint32_t hw = COMPACT ? lds32(piece + 768 + 4 * (lane >> 1)) : lds32(piece + 768 + 8 * (lane >> 1) + 4 * m);
                     guard |= settled(wa, wb, wc) | settled(hw, wa, wb);
-                    const HalfA h = decode_half(wa, wb, wc, hw, tq);
+                    const HalfA h = m == 0 ? decode_half<COMPACT, 0>(wa, wb, wc, hw, tq) : decode_half<COMPACT, 16>(wa, wb, wc, hw, tq);
 #pragma unroll
                     for (int j = 0; j < BATCH; j++) {
                         const uint32_t xj = xt + j * xrec_stride;
@@ -874,16 +903,18 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                         contract_half<false>(h, load_step<0>(ta), acc[j][2 * m], acc[j][2 * m + 1]);
                     }
                 }
-                piece += 2 * kCellBytes;
+                piece += 2 * kSrcCell;
             }
             if (p.tail_cells & 1) {
                 // one block: the slots of this half-step are the two halves of the row group
                 const uint32_t xl = xs0 + (uint32_t)(p.nb - 1) * kXRecBytes;
                 const LaneOffsets l1 = lane_offsets(lane, true);
                 const uint32_t wa = lds32(piece + lane4), wb = lds32(piece + 128 + lane4);
-                const uint32_t wc = lds32(piece + 256 + lane4), hw = lds32(piece + 384 + 4 * (lane >> 1));
+                const uint32_t wc = lds32(piece + 256 + lane4);
+                // 13-byte layout: two bytes a lane pair, the pairs two to a word
+                const uint32_t hw = COMPACT ? lds32(piece + 384 + 4 * (lane >> 2)) >> (8 * (lane & 2)) : lds32(piece + 384 + 4 * (lane >> 1));
                 guard |= settled(wa, wb, wc) | settled(hw, wa, wb);
-                const HalfA h = decode_half(wa, wb, wc, hw, tq);
+                const HalfA h = decode_half<COMPACT, 0>(wa, wb, wc, hw, tq);
 #pragma unroll
                 for (int j = 0; j < BATCH; j++) {
                     const uint32_t xj = xl + j * xrec_stride;
@@ -1031,21 +1062,23 @@ __global__ void __launch_bounds__(256) gemv_fp16_kernel(const __half *__restrict
 // ---- helpers reading a record back: thread = (row group, block column, row of the group)
 // The 24 codes (c[j] = codes of coordinates 8j..8j+7, a nibble each) and the header of one block of one row,
 // found from the layout's description in include/llvq.h: which piece, half-step, lane, word and nibble.
+template <bool COMPACT>
 __device__ __forceinline__ void read_planes_record(const uint8_t *buf, int64_t nb, int64_t rg, int64_t b, int r,
                                                    uint32_t c[3], uint32_t &hdr) {
     const int64_t tiles = nb / kTileCells, left = nb % kTileCells;
-    const uint8_t *grp = buf + (size_t)rg * (size_t)nb * kCellBytes;
+    constexpr int kCell = COMPACT ? kCell13Bytes : kCellBytes, kTile = COMPACT ? kTile13Bytes : kTileBytes;
+    const uint8_t *grp = buf + (size_t)rg * (size_t)nb * kCell;
     const int m = r >> 4, e = (r >> 3) & 1, g = r & 7;
     const int64_t j = b - tiles * kTileCells;
     const uint8_t *base;
     int slot, kind, h = 0;                         // kind 0 tile, 1 pair, 2 single
     if (j < 0) {
-        base = grp + (size_t)(b / kTileCells) * kTileBytes;
+        base = grp + (size_t)(b / kTileCells) * kTile;
         slot = (int)(b & 1); h = 2 * (int)((b % kTileCells) >> 1) + m; kind = 0;
     } else if (left >= 2 && j < 2) {
-        base = grp + (size_t)tiles * kTileBytes; slot = (int)j; kind = 1;
+        base = grp + (size_t)tiles * kTile; slot = (int)j; kind = 1;
     } else {
-        base = grp + (size_t)tiles * kTileBytes + (left == 3 ? 2 * kCellBytes : 0); slot = m; kind = 2;
+        base = grp + (size_t)tiles * kTile + (left == 3 ? 2 * kCell : 0); slot = m; kind = 2;
     }
     auto word = [&](int q, int lane) -> uint32_t {
         const int k = 3 * h + q;
@@ -1055,10 +1088,14 @@ __device__ __forceinline__ void read_planes_record(const uint8_t *buf, int64_t n
         return *reinterpret_cast<const uint32_t *>(a);
     };
     const int pair = 2 * g + slot;
-    const uint32_t hw = *reinterpret_cast<const uint32_t *>(kind == 0 ? base + 1536 + 16 * pair + 4 * h
-                                                            : kind == 1 ? base + 768 + 8 * pair + 4 * m
-                                                                        : base + 384 + 4 * pair);
-    hdr = (hw >> (16 * e)) & 0xffffu;
+    if (COMPACT) {
+        hdr = kind == 0 ? base[1536 + 8 * pair + 2 * h + e] : kind == 1 ? base[768 + 4 * pair + 2 * m + e] : base[384 + 2 * pair + e];
+    } else {
+        const uint32_t hw = *reinterpret_cast<const uint32_t *>(kind == 0 ? base + 1536 + 16 * pair + 4 * h
+                                                                : kind == 1 ? base + 768 + 8 * pair + 4 * m
+                                                                            : base + 384 + 4 * pair);
+        hdr = (hw >> (16 * e)) & 0xffffu;
+    }
     c[0] = c[1] = c[2] = 0;
     for (int i = 0; i < 24; i++) {
         const int kappa = 24 * slot + i;
@@ -1074,9 +1111,16 @@ __device__ __forceinline__ void record_coords(int layout, const uint8_t *buf, in
                                               const uint32_t *cls_parity, const uint8_t *cls_dist, int &cls, int &gain, int x[24]) {
     if (layout == LLVQ_PLANES) {
         uint32_t c[3], hdr;
-        read_planes_record(buf, nb, rg, b, lane, c, hdr);
+        read_planes_record<false>(buf, nb, rg, b, lane, c, hdr);
         cls = (int)(hdr & 511u); gain = (int)((hdr >> 9) & 1u);
         const int par = cls_parity[cls] ? 1 : 0;
+        for (int i = 0; i < 24; i++) x[i] = 2 * ((int)((c[i >> 3] >> (4 * (i & 7))) & 15u) - 8) + par;
+    } else if (layout == LLVQ_PLANES13) {
+        // no class id in this layout: `cls` returns the header byte (shell | parity << 4 | gain << 5)
+        uint32_t c[3], hdr;
+        read_planes_record<true>(buf, nb, rg, b, lane, c, hdr);
+        cls = (int)hdr; gain = (int)((hdr >> 5) & 1u);
+        const int par = (int)((hdr >> 4) & 1u);
         for (int i = 0; i < 24; i++) x[i] = 2 * ((int)((c[i >> 3] >> (4 * (i & 7))) & 15u) - 8) + par;
     } else {
         const uint32_t *cell = reinterpret_cast<const uint32_t *>(buf + ((size_t)rg * (size_t)nb + (size_t)b) * kOneHotCellBytes);
@@ -1134,7 +1178,7 @@ GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
     g.grid = p.total_units < sm_count ? p.total_units : sm_count;
     p.units_base = p.total_units / (g.grid * kWarps);
     p.units_rem = p.total_units % (g.grid * kWarps);
-    if (layout != LLVQ_PLANES) {
+    if (layout == LLVQ_ONEHOT) {
         g.smem = ((size_t)p.nb * 48 + 127) / 128 * 128;
         return g;
     }
@@ -1210,6 +1254,7 @@ int gemv_configure(const llvq_ctx *ctx) {
     if (allow_max_smem(gemv_planes_kernel<false, 2>, bytes)) return -1;
     if (allow_max_smem(gemv_planes_kernel<false, 4>, bytes)) return -1;
     if (allow_max_smem(gemv_planes_kernel<false, 1, true>, bytes)) return -1;
+    if (allow_max_smem(gemv_planes_kernel<false, 1, false, true>, bytes)) return -1;
     if (allow_max_smem(gemv_onehot_kernel, bytes)) return -1;
     return 0;
 }
@@ -1225,6 +1270,7 @@ cudaError_t launch_gemv(int layout, const GemvParams &p, const GemvLaunch &g, bo
     attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (layout == LLVQ_PLANES13) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 1, false, true>, p);
     if (layout == LLVQ_PLANES) {
         if (no_weights) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<true, 1>, p);
         if (p.rot_log2 > 0) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 1, true>, p);

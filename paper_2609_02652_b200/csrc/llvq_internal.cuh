@@ -16,6 +16,8 @@ constexpr int kCellBytes = 448;        // 32 rows x 14 bytes
 constexpr int kTileCells = 4;
 constexpr int kTileBytes = 1792;
 constexpr int kOneHotCellBytes = 640;  // 32 rows x 20 bytes
+constexpr int kCell13Bytes = 416;      // 13-byte layout: 32 rows x 13 bytes
+constexpr int kTile13Bytes = 1664;
 constexpr int kMaxGridCtas = 256;      // the GEMV launches one CTA a multiprocessor; more multiprocessors than this share the work of 256
 
 struct DeviceTables {
