@@ -560,6 +560,18 @@ def main():
                     B.gemv_noweights(ctx, ln["scales"][mi], ln["x"], m.rows, ln["k_padded"], y=ln["ys"][mi])
         t = time_arm(nw, ncopies, arm_steps, 3)
         arms["noweights"] = {"us_per_gemv": t * 1e3 / n_gemv, "launches_per_step": n_gemv}
+        # the 13-byte layout: the same codes and arithmetic, a one-byte header (exact for every block)
+        p13_copies = make_copies(B, ctx, mats, B.PLANES13, ncopies, device, grouped=not args.ungrouped)
+        run_step(B, ctx, B.PLANES13, p13_copies[0])
+        torch.cuda.synchronize()
+        if not args.no_verify:
+            from oracle import oracle as O
+            verify(O, p13_copies, cores, 4 if len(mats) > 7 and not args.ungrouped else None)
+        t = time_arm(lambda i: run_step(B, ctx, B.PLANES13, p13_copies[i % len(p13_copies)]), len(p13_copies), arm_steps, 3)
+        pb = sum(gemv_bytes(e["m"].rows, e["m"].nb, 13) for e in mats)
+        arms["planes13"] = {"us_per_gemv": t * 1e3 / n_gemv, "gbps": pb / (t * 1e-3) / 1e9, "frac": pb / (t * 1e-3) / 1e9 / peak,
+                            "bytes_per_block": 13, "bits_per_weight": 13 * 8 / 24}
+        del p13_copies
         # one-hot layout
         oh_copies = make_copies(B, ctx, mats, B.ONEHOT, max(2, ncopies * 14 // 20 + 1), device, grouped=not args.ungrouped)
         run_step(B, ctx, B.ONEHOT, oh_copies[0])

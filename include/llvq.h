@@ -28,7 +28,7 @@
  *   - Return value: 0 on success, a negative LLVQ_E* code otherwise.  No call aborts, throws or
  *     traps; a failed call enqueues nothing.
  *
- * Layouts (both written by llvq_expand, read by the GEMV; rows are taken 32 at a time, a "row
+ * Layouts (all written by llvq_expand, read by the GEMV; rows are taken 32 at a time, a "row
  * group", rows past the end are filled with the empty record, class id 511):
  *   LLVQ_PLANES  14 bytes a block [Sec. 3.2 "Planes14": class id 9 b, gain 1 b, sign mask 24 b,
  *                three binary planes of the per-coordinate level 3 x 24 b = 106 bits in 112].
@@ -62,6 +62,20 @@
  *                distinct magnitudes.  Per cell five arrays of 32 words (word t of row l at
  *                128t+4l): V0 = smask | class[7:0]<<24, V1 = mask1 | class[8]<<24 | gain<<25,
  *                V2..V4 = mask2..mask4.  A row group takes 640*nb bytes.
+ *   LLVQ_PLANES13 13 bytes a block, exact for every block [Sec. 3.3 reaches this rate, 4.34 bits a
+ *                weight, with "Planes12x": a 12-byte two-plane record, an exception table holding the
+ *                exact record of every five-level block, and extra CTAs that add the correction].
+ *                Here the rate comes from the header instead of the levels: the matvec needs of the
+ *                class only what fixes the block's scale and the parity of its coordinates, so the
+ *                16-bit header becomes one byte = shell (4 bits, 0 for the empty record) | parity << 4
+ *                | gain << 5, and the 24 four-bit codes stay as they are - no level cap, no exception
+ *                table, no second stream.  The code words sit where LLVQ_PLANES has them; the header
+ *                bytes follow them: tile 1664 bytes, byte of pair P, half-step h, row half e at
+ *                1536 + 8 P + 2 h + e; pair 832 bytes, byte at 768 + 4 P + 2 m + e; single 416 bytes,
+ *                byte at 384 + 2 P + e.  A row group takes 416*nb bytes.
+ *                Accepted by llvq_layout_bytes, llvq_expand, llvq_gemv, llvq_gemv_grouped and
+ *                llvq_decode_i8 (which returns the header byte in place of a class id); the other
+ *                calls return LLVQ_EINVAL for it.  y is bit for bit what LLVQ_PLANES gives.
  */
 #ifndef LLVQ_H
 #define LLVQ_H
@@ -75,7 +89,7 @@ extern "C" {
 
 #define LLVQ_PLANES 0
 #define LLVQ_ONEHOT 1
-#define LLVQ_PLANES13 2
+#define LLVQ_PLANES13 2   /* no counterpart record in the paper: see above */
 
 #define LLVQ_OK 0
 #define LLVQ_EINVAL (-1) /* null pointer, bad shape, unknown layout                         */
