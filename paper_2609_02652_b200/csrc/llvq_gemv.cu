@@ -629,7 +629,8 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         const int nx = p.nb * 3, e_lo = 3 * blk_lo, e_hi = 3 * blk_hi;
         const bool one_each = e_hi - e_lo <= kThreads;
         const uint4 *xg = reinterpret_cast<const uint4 *>(p.x);
-        uint4 mine = make_uint4(0u, 0u, 0u, 0u);               // a piece past the rotated length (the padding)
+        uint4 mine = make_uint4(0u, 0u, 0u, 0u);               // a piece of this CTA's share past the rotated length
+        int mine_e = -1;
         float ss = __uint_as_float(settled(warm, warm, warm));
         for (int base = 0; base < nx; base += 4 * kThreads) {
             uint4 v[4];
@@ -667,6 +668,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                     rot_store8(rot, 8 * e - c_lo, a);
                 } else if (e >= e_lo && e < e_hi) {
                     mine = v[i];
+                    mine_e = e;
                 }
             }
         }
@@ -686,12 +688,13 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             xexp[0] = max((e2 + 1) >> 1, -13);
         }
         const float scale = pow2f(29 - xexp[0]);
+        // rotated pieces: from the exact sums; pieces past the rotated length: as they are (the one this thread
+        // met in the scan, or read again when the share is too wide for that)
         for (int e = e_lo + tid; e < e_hi; e += kThreads) {
-            uint4 v;
-            if (8 * e < c_hi) v = rot_round8(rot, 8 * e - c_lo, p.rot_scale);
-            else v = one_each ? mine : __ldcg(xg + e);
-            convert_item(v, e % 3, xs0 + (uint32_t)(e / 3) * kXRecBytes, scale);
+            if (8 * e < c_hi) convert_item(rot_round8(rot, 8 * e - c_lo, p.rot_scale), e % 3, xs0 + (uint32_t)(e / 3) * kXRecBytes, scale);
+            else if (!one_each) convert_item(__ldcg(xg + e), e % 3, xs0 + (uint32_t)(e / 3) * kXRecBytes, scale);
         }
+        if (one_each && mine_e >= 0) convert_item(mine, mine_e % 3, xs0 + (uint32_t)(mine_e / 3) * kXRecBytes, scale);
         if (!NO_WEIGHTS) {
 #pragma unroll
             for (int s = kEarlySlots; s < kSlots; s++) issue(my_bar + 8 * s, my_ring + s * kTileBytes);

@@ -204,3 +204,37 @@ def test_gemv_rotated_error_codes(B, ctx):
     B.gemv_rotated(ctx, prob, case.d_x, 96, n=96)
     torch.cuda.synchronize()
     assert torch.isfinite(y).all()
+
+
+def test_gemv_rotated_partial_length_passes_the_rest_through(B, ctx, oracle):
+    """Only the first n entries are rotated; the entries after them - here real values, not padding - enter the
+    matvec as they are."""
+    rows, k = 96, 2560
+    case = make_case(rows, k, seed=77)
+    kp = case.nb * 24
+    buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    for n, block in ((2048, 0), (1024, 256), (2560 - 512, 512), (8, 8)):
+        y = torch.empty(rows, dtype=torch.float32, device="cuda")
+        B.gemv_rotated(ctx, [(buf, case.d_scale, GAIN, y, rows)], case.d_x, kp, n=n, block=block)
+        torch.cuda.synchronize()
+        ref = _rotated_reference(oracle, case, n, block, None)
+        assert np.array_equal(ref.x[n:], case.x[n:]) and np.abs(case.x[n:k].astype(np.float64)).max() > 0
+        err, _ = check_gemv(oracle, ref, y)
+        assert err <= 1e-6
+
+
+def test_gemv_rotated_refuses_a_block_that_does_not_fit_shared_memory(B, ctx):
+    """A CTA rotates whole blocks: with three matrices' block-constant tables beside a 16384-coordinate block the
+    shared memory of a multiprocessor is exceeded, and the call says so instead of launching."""
+    k = 16384
+    cases = [make_case(32, k, seed=5, tensor_id=i) for i in range(8)]
+    kp = cases[0].nb * 24
+    bufs = [B.expand(ctx, 0, c.d_codes, c.rows, c.nb) for c in cases]
+    ys = [torch.empty(c.rows, dtype=torch.float32, device="cuda") for c in cases]
+    probs = [(b, c.d_scale, GAIN, y, c.rows) for b, c, y in zip(bufs, cases, ys)]
+    with pytest.raises(B.LlvqError) as e:
+        B.gemv_rotated(ctx, probs, cases[0].d_x, kp, n=k)
+    assert e.value.code == -3
+    B.gemv_rotated(ctx, probs, cases[0].d_x, kp, n=k, block=1024)       # a shorter block fits
+    torch.cuda.synchronize()
+    assert all(torch.isfinite(y).all() for y in ys)
