@@ -126,3 +126,28 @@ def test_what_the_layout_does_not_take(B, ctx):
     assert e.value.code == -3
     B.gemv(ctx, L13, buf, case.d_scale, GAIN, case.d_x, 64, 96, y=y)
     assert torch.isfinite(y).all()
+
+
+def test_gemv_random_shapes_grouped(B, ctx, oracle):
+    """Seeded random shapes and groupings in the 13-byte layout: the oracle's bar on every row, and bit for bit the
+    14-byte layout's result."""
+    rng = np.random.default_rng(13)
+    for it in range(25):
+        k = int(rng.integers(1, 300)) * 24 - int(rng.integers(0, 24))
+        k = max(k, 1)
+        nmat = int(rng.integers(1, 5))
+        rows = [int(rng.integers(1, 300)) for _ in range(nmat)]
+        cases = [make_case(r, k, seed=500 + it, tensor_id=i) for i, r in enumerate(rows)]
+        kp = cases[0].nb * 24
+        x = cases[0].d_x
+        ys = {}
+        for layout in (L13, 0):
+            bufs = [B.expand(ctx, layout, c.d_codes, c.rows, c.nb) for c in cases]
+            ys[layout] = [torch.full((c.rows,), float("nan"), dtype=torch.float32, device="cuda") for c in cases]
+            B.gemv_grouped(ctx, layout, [(b_, c.d_scale, GAIN, y, c.rows) for b_, c, y in zip(bufs, cases, ys[layout])], x, kp)
+        torch.cuda.synchronize()
+        B.status(ctx)
+        for i, c in enumerate(cases):
+            c.x = cases[0].x
+            check_gemv(oracle, c, ys[L13][i])
+            assert torch.equal(ys[L13][i], ys[0][i]), (it, k, rows)

@@ -238,3 +238,30 @@ def test_gemv_rotated_refuses_a_block_that_does_not_fit_shared_memory(B, ctx):
     B.gemv_rotated(ctx, probs, cases[0].d_x, kp, n=k, block=1024)       # a shorter block fits
     torch.cuda.synchronize()
     assert all(torch.isfinite(y).all() for y in ys)
+
+
+def test_gemv_rotated_random_shapes(B, ctx, oracle):
+    """Seeded random shapes, rotated lengths, block lengths, sign vectors and groupings, each against the oracle chain."""
+    rng = np.random.default_rng(2026)
+    for it in range(30):
+        k = int(rng.integers(1, 260)) * 24 if it % 3 else int(rng.choice([2560, 4096, 5120, 1536, 9728, 3072]))
+        kp = (k + 23) // 24 * 24
+        nmat = int(rng.integers(1, 4))
+        rows = [int(rng.integers(1, 200)) for _ in range(nmat)]
+        cases = [make_case(r, k, seed=1000 + it, tensor_id=i) for i, r in enumerate(rows)]
+        x = cases[0].x
+        # the rotated length: a multiple of 8, anywhere up to k_padded; the block: any power of two >= 8 dividing it
+        n = int(rng.integers(1, kp // 8 + 1)) * 8
+        divisors = [b for b in (8, 16, 32, 64, 128, 256, 512, 1024, 2048, 4096) if n % b == 0]
+        block = int(rng.choice(divisors + [0]))
+        neg = rng.integers(0, 2, size=n) if rng.random() < 0.5 else None
+        bufs = [B.expand(ctx, 0, c.d_codes, c.rows, c.nb) for c in cases]
+        ys = [torch.full((c.rows,), float("nan"), dtype=torch.float32, device="cuda") for c in cases]
+        B.gemv_rotated(ctx, [(b_, c.d_scale, GAIN, y, c.rows) for b_, c, y in zip(bufs, cases, ys)], cases[0].d_x, kp, n=n, block=block,
+                       negate_bits=None if neg is None else _bits(neg))
+        torch.cuda.synchronize()
+        B.status(ctx)
+        xr = np.concatenate([oracle.rotate(x[:n], block, neg), x[n:]])
+        for c, y in zip(cases, ys):
+            err, _ = check_gemv(oracle, dataclasses.replace(c, x=xr), y)
+            assert err <= 1e-5, (it, k, n, block, rows)
