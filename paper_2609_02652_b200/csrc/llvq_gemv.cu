@@ -566,19 +566,20 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         w.c.col++;
         if (--w.left <= 1) walk_turn(w);               // rare: at most twice a stretch
     };
-    // issue the copy of the next unit (lane 0 alone, by predicate) onto barrier `b` and buffer `dst`
-    const int my_issues = lane == 0 ? n_units : 0;     // lanes other than 0 never issue
+    // issue the copy of the next unit (one elected lane) onto barrier `b` and buffer `dst`
     auto issue = [&](uint32_t b, uint32_t dst) {
         const int done = iw.done;
         const uint8_t *src;
         uint32_t bytes;
         walk_next(iw, src, bytes);
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.lt.s32 p, %0, %1;\n\t"
-            "@p mbarrier.arrive.expect_tx.shared::cta.b64 _, [%2], %3;\n\t"
-            "@p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%4], [%5], %3, [%2];\n\t}"
-            ::"r"(done), "r"(my_issues), "r"(b), "r"(bytes), "r"(dst), "l"(src));
+        if (done < n_units) {                          // the same for every lane of the warp
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "elect.sync _|p, 0xffffffff;\n\t"
+                "@p mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t"
+                "@p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%2], [%3], %1, [%0];\n\t}"
+                ::"r"(b), "r"(bytes), "r"(dst), "l"(src));
+        }
         // No "memory" clobber: the only memory the copy writes is the slot, whose last reads feed
         // `dst` through settled() and whose next reads follow the next wait on `b`; a clobber here
         // would pin every shared-memory read of the decode behind the copy.
