@@ -46,6 +46,24 @@ def test_layout_bytes_and_argument_checks(lib):
     assert lib.llvq_gemv_fp16(None, None, None, 8, 8, None) == -1
     assert lib.llvq_gemv(None, 0, None, None, None, None, None, 1, 24, None) == -1
     assert b"aligned" in lib.llvq_strerror(-2)
+    # the 13-byte layout: 13/14 of the 14-byte layout's size, for any shape
+    assert binding.layout_bytes(binding.PLANES13, 3072, 3072) == 3072 * 128 * 13
+    assert binding.layout_bytes(binding.PLANES13, 33, 48) == 2 * 2 * 416
+    assert lib.llvq_layout_bytes(3, 32, 24, ctypes.byref(n)) == -1
+
+
+def test_rotation_block_rule_and_argument_checks(lib):
+    """The host query of the rotation, against the oracle's rule (largest power of two dividing n, at most 16384)."""
+    from oracle import oracle as O
+    from paper_2609_02652_b200 import binding
+
+    for n in (8, 24, 2560, 4096, 5120, 9728, 12288, 17408, 25600, 98304, 7, 1, 3 * 16384, 5 * 32768):
+        assert binding.rotate_block(n) == O.rotate_block(n), n
+        for b in (1, 2, 8, 64, 512, 4096, 16384, 32768, 3, 0):
+            assert binding.rotate_block(n, b) == O.rotate_block(n, b), (n, b)
+    assert binding.rotate_block(0) == 0 and binding.rotate_block(-8) == 0
+    assert lib.llvq_rotate(None, None, None, None, 8, 0, None) == -1
+    assert lib.llvq_gemv_rotated(None, None, 1, None, 24, None, None) == -1
 
 
 def test_missing_library_fails_loudly(monkeypatch):
