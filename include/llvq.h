@@ -63,8 +63,8 @@
  *                128t+4l): V0 = smask | class[7:0]<<24, V1 = mask1 | class[8]<<24 | gain<<25,
  *                V2..V4 = mask2..mask4.  A row group takes 640*nb bytes.
  *   LLVQ_PLANES13 13 bytes a block, exact for every block [Sec. 3.3 reaches this rate, 4.34 bits a
- *                weight, with "Planes12x": a 12-byte two-plane record, an exception table holding the
- *                exact record of every five-level block, and extra CTAs that add the correction].
+ *                weight, with its "Planes12x" layout: 12 bytes for blocks of up to four levels, the
+ *                five-level blocks kept exactly in a side table and applied by further thread blocks].
  *                Here the rate comes from the header instead of the levels: the matvec needs of the
  *                class only what fixes the block's scale and the parity of its coordinates, so the
  *                16-bit header becomes one byte = shell (4 bits, 0 for the empty record) | parity << 4
@@ -269,7 +269,8 @@ int llvq_dequant_fp16(llvq_ctx *ctx, int layout, const void *layout_buf, const v
                       const float *gain, void *W, int64_t rows, int64_t k_padded, void *stream);
 
 /* Test hook: the integer coordinates (coords[(row*nb + b)*24 + i]) and class id
- * (class_ids[row*nb + b]) a layout buffer decodes to, for the bit-exact check of Sec. 2.4. */
+ * (class_ids[row*nb + b]) a layout buffer decodes to, for the bit-exact check of Sec. 2.4.
+ * LLVQ_PLANES13 keeps no class id: class_ids receives the header byte (shell | parity << 4 | gain << 5). */
 int llvq_decode_i8(llvq_ctx *ctx, int layout, const void *layout_buf, int8_t *coords,
                    uint16_t *class_ids, int64_t rows, int64_t nb, void *stream);
 
