@@ -3,8 +3,9 @@
 
 A step is one pass over the workload's per-token sequence of lattice GEMVs (for the default
 workload, the seven projections of a 4B-like decoder layer, issued as four row-concatenated
-launches).  Inputs are synthetic and seeded; every row of every arm is checked against the f64
-CPU oracle before anything is timed.  Weights rotate through enough distinct copies that no
+launches).  Inputs are synthetic and seeded; every row of the timed path is checked against the f64
+CPU oracle before anything is timed (that check is also the cpu_baseline leg: the oracle's time on the
+host cores); the comparison arms are then checked against the timed path's outputs.  Weights rotate through enough distinct copies that no
 launch finds its records in L2.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
@@ -177,6 +178,19 @@ def verify(oracle, copies, threads, max_launches=None):
             worst = max(worst, float(ratio.max()))
             gemvs += 1
     return worst, secs, blocks, gemvs
+
+
+def same_outputs(ref_copies, arm_copies, exact: bool) -> None:
+    """An arm's outputs against those of the main arm, which the oracle checked row by row: bit for bit where the
+    arithmetic is the same, else to 1e-4 of the output's scale (the GPU tests hold every arm to the oracle itself)."""
+    for lr, la in zip(ref_copies[0].launches, arm_copies[0].launches):
+        for m, yr, ya in zip(lr["mats"], lr["ys"], la["ys"]):
+            if exact:
+                ok = torch.equal(yr, ya)
+            else:
+                ok = bool(torch.isfinite(ya).all()) and float((yr - ya).abs().max()) <= 1e-4 * float(yr.abs().max()) + 1e-30
+            if not ok:
+                raise SystemExit(f"arm output differs from the checked one on {m.name}")
 
 
 def capture_graphs(B, ctx, layout, copies, total_steps, first_step=0, chunk=512):
@@ -564,9 +578,9 @@ def main():
         p13_copies = make_copies(B, ctx, mats, B.PLANES13, ncopies, device, grouped=not args.ungrouped)
         run_step(B, ctx, B.PLANES13, p13_copies[0])
         torch.cuda.synchronize()
-        if not args.no_verify:
-            from oracle import oracle as O
-            verify(O, p13_copies, cores, 4 if len(mats) > 7 and not args.ungrouped else None)
+        run_step(B, ctx, B.PLANES, copies[0])
+        torch.cuda.synchronize()
+        same_outputs(copies, p13_copies, exact=True)
         t = time_arm(lambda i: run_step(B, ctx, B.PLANES13, p13_copies[i % len(p13_copies)]), len(p13_copies), arm_steps, 3)
         pb = sum(gemv_bytes(e["m"].rows, e["m"].nb, 13) for e in mats)
         arms["planes13"] = {"us_per_gemv": t * 1e3 / n_gemv, "gbps": pb / (t * 1e-3) / 1e9, "frac": pb / (t * 1e-3) / 1e9 / peak,
@@ -576,9 +590,9 @@ def main():
         oh_copies = make_copies(B, ctx, mats, B.ONEHOT, max(2, ncopies * 14 // 20 + 1), device, grouped=not args.ungrouped)
         run_step(B, ctx, B.ONEHOT, oh_copies[0])
         torch.cuda.synchronize()
-        if not args.no_verify:
-            from oracle import oracle as O
-            verify(O, oh_copies, cores, 4 if len(mats) > 7 and not args.ungrouped else None)
+        run_step(B, ctx, B.PLANES, copies[0])
+        torch.cuda.synchronize()
+        same_outputs(copies, oh_copies, exact=False)
         t = time_arm(lambda i: run_step(B, ctx, B.ONEHOT, oh_copies[i % len(oh_copies)]), len(oh_copies), arm_steps, 3)
         ob = sum(gemv_bytes(e["m"].rows, e["m"].nb, 20) for e in mats)
         arms["onehot"] = {"us_per_gemv": t * 1e3 / n_gemv, "gbps": ob / (t * 1e-3) / 1e9, "frac": ob / (t * 1e-3) / 1e9 / peak, "bytes_per_block": 20}
