@@ -566,13 +566,23 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         w.c.col++;
         if (--w.left <= 1) walk_turn(w);               // rare: at most twice a stretch
     };
-    // issue the copy of the next unit (one elected lane) onto barrier `b` and buffer `dst`
+    // issue the copy of the next unit onto barrier `b` and buffer `dst`: by one elected lane under a condition that
+    // is the same for the whole warp, or (the four-vector build, where that form costs a register too many) by
+    // lane 0 under its own predicate
+    const int my_issues = lane == 0 ? n_units : 0;
     auto issue = [&](uint32_t b, uint32_t dst) {
         const int done = iw.done;
         const uint8_t *src;
         uint32_t bytes;
         walk_next(iw, src, bytes);
-        if (done < n_units) {                          // the same for every lane of the warp
+        if constexpr (BATCH >= 4) {
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "setp.lt.s32 p, %0, %1;\n\t"
+                "@p mbarrier.arrive.expect_tx.shared::cta.b64 _, [%2], %3;\n\t"
+                "@p cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%4], [%5], %3, [%2];\n\t}"
+                ::"r"(done), "r"(my_issues), "r"(b), "r"(bytes), "r"(dst), "l"(src));
+        } else if (done < n_units) {
             asm volatile(
                 "{\n\t.reg .pred p;\n\t"
                 "elect.sync _|p, 0xffffffff;\n\t"
@@ -846,7 +856,33 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                 acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
             }
 #else
-            {
+            if constexpr (BATCH == 1) {
+                // one vector: every shared-memory load first, then the eight contractions back to back (four independent
+                // accumulator tiles in the tensor pipe at once), then the eight scale steps
+                const StepX s1 = load_step<0>(xa), s2 = load_step<2 * kXRecBytes>(xa);
+                const HalfA h0 = decode_half<COMPACT, 0>(a0.x, a0.y, a0.z, hh.x, tq);
+                const HalfA h1 = decode_half<COMPACT, 16>(a0.w, a1.x, a1.y, COMPACT ? hh.x : hh.y, tq);
+                const HalfA h2 = decode_half<COMPACT, 0>(a1.z, a1.w, a2.x, COMPACT ? hh.y : hh.z, tq);
+                const HalfA h3 = decode_half<COMPACT, 16>(a2.y, a2.z, a2.w, COMPACT ? hh.y : hh.w, tq);
+                int d0[4], d1[4], d2[4], d3[4];
+                mma_k32(d0, h0.a0, h0.a1, h0.a2, h0.a3, s1.b0, s1.b1);
+                mma_k32(d1, h1.a0, h1.a1, h1.a2, h1.a3, s1.b0, s1.b1);
+                mma_k32(d2, h2.a0, h2.a1, h2.a2, h2.a3, s2.b0, s2.b1);
+                mma_k32(d3, h3.a0, h3.a1, h3.a2, h3.a3, s2.b0, s2.b1);
+                mma_k16(d0, h0.c0, h0.c1, s1.b2);
+                mma_k16(d1, h1.c0, h1.c1, s1.b2);
+                mma_k16(d2, h2.c0, h2.c1, s2.b2);
+                mma_k16(d3, h3.c0, h3.c1, s2.b2);
+                auto e = [](const int (&d)[4], float ky, int xsum, int r) { return __float_as_int(ky) * xsum + (d[2 * r] + 256 * d[2 * r + 1]); };
+                acc[0][0] = (float)e(d0, h0.k0.y, s1.xsum, 0) * h0.k0.x;
+                acc[0][1] = (float)e(d0, h0.k1.y, s1.xsum, 1) * h0.k1.x;
+                acc[0][2] = (float)e(d1, h1.k0.y, s1.xsum, 0) * h1.k0.x;
+                acc[0][3] = (float)e(d1, h1.k1.y, s1.xsum, 1) * h1.k1.x;
+                acc[0][0] = fmaf((float)e(d2, h2.k0.y, s2.xsum, 0), h2.k0.x, acc[0][0]);
+                acc[0][1] = fmaf((float)e(d2, h2.k1.y, s2.xsum, 1), h2.k1.x, acc[0][1]);
+                acc[0][2] = fmaf((float)e(d3, h3.k0.y, s2.xsum, 0), h3.k0.x, acc[0][2]);
+                acc[0][3] = fmaf((float)e(d3, h3.k1.y, s2.xsum, 1), h3.k1.x, acc[0][3]);
+            } else {
                 StepX sx[BATCH];
 #pragma unroll
                 for (int j = 0; j < BATCH; j++) {
