@@ -34,11 +34,11 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) per algorithmic byte of gemv_planes_kernel, from one ncu capture of the
 # 8192 x 8192 launch (profiles/gemv_planes_kernel_config4_8192x8192.txt: 39.365 MB against 39.289 MB);
 # traffic grows in proportion to the records streamed, so a launch's traffic is its bytes times this.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 39.3651 / 39.2888
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 39.3580 / 39.2888
 # from the same capture: 5 847 216 warp instructions for 87 552 block columns (32 rows x 24 weights each), and the share
 # of issue slots busy over the launch
-NCU_WARP_INSTR_PER_CELL = 5847216 / 87552
-NCU_ISSUE_BUSY_PCT = 56.5
+NCU_WARP_INSTR_PER_CELL = 5826348 / 87552
+NCU_ISSUE_BUSY_PCT = 56.6
 METRIC = "us_per_lattice_gemv"
 
 
