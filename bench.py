@@ -1,16 +1,20 @@
 #!/usr/bin/env python
 """Benchmark of the batch-1 lattice GEMV path (one JSON line on stdout, rank 0).
 
-A step is one pass over the workload's per-token sequence of lattice GEMVs (for the default
-workload, the seven projections of a 4B-like decoder layer, issued as four row-concatenated
-launches).  Inputs are synthetic and seeded; every row of the timed path is checked against the f64
-CPU oracle before anything is timed (that check is also the cpu_baseline leg: the oracle's time on the
-host cores); the comparison arms are then checked against the timed path's outputs.  Weights rotate through enough distinct copies that no
-launch finds its records in L2.
+A step is one pass over the workload's per-token sequence of lattice GEMVs: for the default workload, the
+14B-like stack, the 280 projections of 40 decoder layers issued as 160 row-concatenated launches (q/k/v and
+gate/up share a launch).  Inputs are synthetic and seeded.  Every row of the first layer of the timed path is
+checked against the f64 CPU oracle before anything is timed (that check is also the cpu_baseline leg: the
+oracle's time on the host cores).  The records are larger than L2 (or rotate through enough distinct copies),
+so no launch finds its records there.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+Protocol: W untimed warm-up steps, then `--rounds` rounds (seven unless told otherwise) of exactly K steps each,
+each round bracketed by a barrier and a device synchronisation and timed with CUDA events on the launching
+stream; the first two rounds are discarded, `value` is the median of the rest, `min` / `max` its range.
 
-With --impl reference the CPU oracle itself is timed on the host cores (a bounded sample a step).
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--rounds R] [--impl reference]
+
+With --impl reference the CPU oracle itself is timed on the host cores (one whole GEMV of the workload a step).
 """
 from __future__ import annotations
 
@@ -32,14 +36,15 @@ from paper_2609_02652_b200 import datagen  # noqa: E402
 
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) per algorithmic byte of gemv_planes_kernel, from one ncu capture of the
-# 8192 x 8192 launch (profiles/gemv_planes_kernel_config4_8192x8192.txt: 39.365 MB against 39.289 MB);
-# traffic grows in proportion to the records streamed, so a launch's traffic is its bytes times this.
+# 8192 x 8192 launch (profiles/gemv_planes_kernel_config4_8192x8192.txt); traffic grows in proportion
+# to the records streamed, so a launch's traffic is its bytes times this.
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 39.3580 / 39.2888
-# from the same capture: 5 847 216 warp instructions for 87 552 block columns (32 rows x 24 weights each), and the share
-# of issue slots busy over the launch
+# from the same capture: warp instructions per block column (32 rows x 24 weights), and the share of issue
+# slots busy over the launch
 NCU_WARP_INSTR_PER_CELL = 5826348 / 87552
 NCU_ISSUE_BUSY_PCT = 56.6
 METRIC = "us_per_lattice_gemv"
+DISCARD_ROUNDS = 2
 
 
 def measured_peaks():
@@ -108,7 +113,7 @@ class Copy:
 
 
 def build_inputs(wl, device):
-    """Host-side codes/scales/x for every matrix; x is shared inside a launch group."""
+    """Codes (on the device), scales and x (on the host) for every matrix; x is shared inside a launch group."""
     mats = []
     group_x = {}
     for m in wl.matrices:
@@ -120,11 +125,15 @@ def build_inputs(wl, device):
     return mats
 
 
-def make_copies(B, ctx, mats, layout, ncopies, device, grouped=True):
+def make_copies(B, ctx, mats, layout, ncopies, device, grouped=True, keep_codes=None):
+    """Expands every matrix once and clones the records ncopies - 1 times.  Codes of matrices outside
+    `keep_codes` (a set of tensor ids, None = all) are dropped once expanded: they are needed only by the oracle."""
     first = {}
     for e in mats:
         m = e["m"]
         first[m.tensor_id] = B.expand(ctx, layout, e["codes"], m.rows, m.nb)
+        if keep_codes is not None and m.tensor_id not in keep_codes:
+            e["codes"] = None
     torch.cuda.synchronize()
     copies = []
     for c in range(ncopies):
@@ -151,6 +160,11 @@ def make_copies(B, ctx, mats, layout, ncopies, device, grouped=True):
     return copies
 
 
+def copies_needed(layout_bytes: int) -> int:
+    """Distinct copies of the records so that a launch never finds its records in L2: three times L2 in rotation."""
+    return max(2, -(-3 * L2_BYTES // layout_bytes)) if layout_bytes < 3 * L2_BYTES else 1
+
+
 def run_step(B, ctx, layout, cp):
     for ln in cp.launches:
         B.gemv_grouped(ctx, layout, ln["problems"], ln["x"], ln["k_padded"])
@@ -158,8 +172,8 @@ def run_step(B, ctx, layout, cp):
 
 def verify(oracle, copies, threads, max_launches=None):
     """Every row of copy 0 (of its first max_launches launches) against the f64 oracle.
-    Returns (worst normalised error, oracle seconds, blocks, GEMVs checked)."""
-    worst, secs, blocks, gemvs = 0.0, 0.0, 0, 0
+    Returns (worst normalised error, oracle seconds, blocks, GEMVs checked, seconds of index decode alone on one core)."""
+    worst, secs, blocks, gemvs, decode_secs = 0.0, 0.0, 0, 0, 0.0
     for ln in copies[0].launches[:max_launches]:
         xh = ln["x"].cpu().numpy()
         for e, y in zip(ln["members"], ln["ys"]):
@@ -168,6 +182,11 @@ def verify(oracle, copies, threads, max_launches=None):
             t0 = time.perf_counter()
             y_ref, wn, ab = oracle.matvec(codes, m.rows, m.nb, e["scale"].numpy(), datagen.GAIN, xh, nthreads=threads)
             secs += time.perf_counter() - t0
+            # the decode alone, on a bounded sample of the same codes (one core), scaled to the matrix by blocks
+            sample = codes.reshape(-1)[:min(codes.size, 1 << 18)]
+            t0 = time.perf_counter()
+            oracle.decode_batch(sample)
+            decode_secs += (time.perf_counter() - t0) * (m.blocks / sample.size)
             blocks += m.blocks
             yv = y.cpu().numpy().astype(np.float64)
             denom = wn * float(np.linalg.norm(xh.astype(np.float64)))
@@ -177,7 +196,7 @@ def verify(oracle, copies, threads, max_launches=None):
                 raise SystemExit(f"parity failure on {m.name}: normalised error {ratio.max():.3e}")
             worst = max(worst, float(ratio.max()))
             gemvs += 1
-    return worst, secs, blocks, gemvs
+    return worst, secs, blocks, gemvs, decode_secs
 
 
 def same_outputs(ref_copies, arm_copies, exact: bool) -> None:
@@ -193,8 +212,8 @@ def same_outputs(ref_copies, arm_copies, exact: bool) -> None:
                 raise SystemExit(f"arm output differs from the checked one on {m.name}")
 
 
-def capture_graphs(B, ctx, layout, copies, total_steps, first_step=0, chunk=512):
-    """CUDA graphs that run steps first_step .. first_step+total_steps-1 (copy = step mod copies)."""
+def capture_graphs(fn_step, total_steps, first_step=0, chunk=512):
+    """CUDA graphs that run fn_step(first_step) .. fn_step(first_step + total_steps - 1)."""
     graphs, done = [], 0
     stream = torch.cuda.Stream()
     while done < total_steps:
@@ -202,7 +221,7 @@ def capture_graphs(B, ctx, layout, copies, total_steps, first_step=0, chunk=512)
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=stream):
             for i in range(n):
-                run_step(B, ctx, layout, copies[(first_step + done + i) % len(copies)])
+                fn_step(first_step + done + i)
         graphs.append(g)
         done += n
     return graphs
@@ -216,26 +235,6 @@ def time_graphs(graphs):
     e1.record()
     e1.synchronize()
     return e0.elapsed_time(e1)
-
-
-def time_arm(fn_step, ncopies, steps, warmup):
-    """Times an arm whose step is fn_step(copy_index) through one CUDA graph of `steps` steps."""
-    stream = torch.cuda.Stream()
-    for i in range(max(3, warmup)):
-        fn_step(i % ncopies)
-    torch.cuda.synchronize()
-    g = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(g, stream=stream):
-        for i in range(steps):
-            fn_step(i % ncopies)
-    g.replay()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    g.replay()
-    e1.record()
-    e1.synchronize()
-    return e0.elapsed_time(e1) / steps
 
 
 def max_over_ranks(ms: float, dist, device) -> float:
@@ -252,60 +251,253 @@ def us_per_gemv_of_job(ms_per_step: float, n_gemv: int, world: int) -> float:
     return ms_per_step * 1e3 / (n_gemv * world)
 
 
+def summarise_rounds(ms_rounds):
+    """Median and range of the rounds kept (the first DISCARD_ROUNDS are dropped when enough rounds were run)."""
+    kept = ms_rounds[DISCARD_ROUNDS:] if len(ms_rounds) > DISCARD_ROUNDS else ms_rounds
+    return statistics.median(kept), min(kept), max(kept), len(kept)
+
+
+def time_rounds(fn_step, steps, warmup, rounds, dist=None, device=None):
+    """The protocol: warm-up steps, one untimed replay of the timed graphs (a graph's first launch uploads it,
+    which is not a step), then `rounds` timed replays of exactly `steps` steps, each between a barrier and a
+    synchronisation; a multi-rank round counts as its slowest rank's.  Returns the list of ms per round."""
+    warm = capture_graphs(fn_step, max(3, warmup))
+    graphs = capture_graphs(fn_step, steps, first_step=max(3, warmup))
+    torch.cuda.synchronize()
+    time_graphs(warm)
+    time_graphs(graphs)
+    out = []
+    for _ in range(rounds):
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ms = time_graphs(graphs)
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        out.append(max_over_ranks(ms, dist, device))
+    return out
+
+
+def time_arm(fn_step, ncopies, steps, warmup, rounds=5):
+    """Median ms per step of an arm whose step is fn_step(copy_index)."""
+    med, _, _, _ = summarise_rounds([ms / steps for ms in time_rounds(lambda i: fn_step(i % ncopies), steps, warmup, rounds)])
+    return med
+
+
 def reference_arm(args, wl):
-    """Times the CPU oracle as it stands: each step decodes and multiplies a bounded sample."""
+    """Times the CPU oracle as it stands: each step decodes and multiplies one whole GEMV of the workload (its
+    smallest matrix, so that a step stays bounded); value and ms_per_step are that GEMV's measured time."""
     from oracle import oracle as O
 
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     cores = os.cpu_count() or 1
-    m = wl.matrices[0]
-    sample_rows = min(m.rows, 512)
-    codes = datagen.make_codes(m.rows, m.nb, wl.seed, m.tensor_id, count=sample_rows * m.nb).numpy().astype(np.uint64)
-    scale = datagen.make_row_scale(m.rows, wl.seed, m.tensor_id).numpy()[:sample_rows]
+    m = min(wl.matrices, key=lambda mm: mm.blocks)
+    codes = datagen.make_codes(m.rows, m.nb, wl.seed, m.tensor_id).numpy().astype(np.uint64)
+    scale = datagen.make_row_scale(m.rows, wl.seed, m.tensor_id).numpy()
     x = datagen.make_x(m.k, m.k_padded, wl.seed, m.tensor_id).numpy()
     for _ in range(args.warmup):
-        O.matvec(codes, sample_rows, m.nb, scale, datagen.GAIN, x, nthreads=cores)
+        O.matvec(codes, m.rows, m.nb, scale, datagen.GAIN, x, nthreads=cores)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        O.matvec(codes, sample_rows, m.nb, scale, datagen.GAIN, x, nthreads=cores)
+        O.matvec(codes, m.rows, m.nb, scale, datagen.GAIN, x, nthreads=cores)
     dt = (time.perf_counter() - t0) / args.steps
-    blocks_per_s = sample_rows * m.nb / dt
-    # scale the sample to the whole workload: seconds per block x blocks of a step / GEMVs of a step
-    us_per_gemv = wl.blocks / blocks_per_s / len(wl.matrices) * 1e6
-    sample = f"{sample_rows} rows of {m.name} ({sample_rows * m.nb} blocks) per step, scaled by blocks to the whole workload"
-    line = {"impl": "reference", "metric": METRIC, "value": us_per_gemv, "unit": "us", "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": wl.blocks / blocks_per_s * 1e3, "higher_is_better": False, "scaling": "weak",
+    sample = f"one GEMV a step: {m.name} ({m.rows} x {m.k}, {m.blocks} blocks) of {wl.name}, index decode + f64 matvec"
+    line = {"impl": "reference", "metric": METRIC, "value": dt * 1e6, "unit": "us", "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": False, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"config {wl.config}: {wl.name}", "gemvs_per_step": len(wl.matrices)},
-            "cpu_baseline": {"value": us_per_gemv, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample,
-                             "blocks_per_s": blocks_per_s},
-            "e2e": {"value": us_per_gemv, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+            "config": {"workload": f"config {wl.config}: {wl.name}", "sample": sample, "gemvs_per_step": 1},
+            "cpu_baseline": {"value": dt * 1e6, "unit": "us", "cores": cores, "kind": "oracle", "sample": sample,
+                             "blocks_per_s": m.blocks / dt},
+            "e2e": {"value": dt * 1e6, "unit": "us", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
+
+
+def figures(ms_per_step, n_gemv, step_bytes, peak):
+    gbps = step_bytes / (ms_per_step * 1e-3) / 1e9
+    return {"us": ms_per_step * 1e3 / n_gemv, "gbps": gbps, "frac": gbps / peak}
+
+
+def side_workload(B, ctx, config, device, peak, steps_target=3000, rounds=7):
+    """Another configuration through the same protocol (no oracle run here: the GPU tests check these workloads)."""
+    wl = datagen.workload(config)
+    mats = build_inputs(wl, device)
+    step_bytes = sum(gemv_bytes(e["m"].rows, e["m"].nb) for e in mats)
+    layout_bytes = sum(14 * e["m"].blocks for e in mats)
+    ncopies = copies_needed(layout_bytes)
+    copies = make_copies(B, ctx, mats, B.PLANES, ncopies, device, keep_codes=set())
+    launches = len(copies[0].launches)
+    steps = max(3, min(400, steps_target // launches))
+    med, lo, hi, kept = summarise_rounds([ms / steps for ms in time_rounds(lambda i: run_step(B, ctx, B.PLANES, copies[i % ncopies]),
+                                                                           steps, 3, rounds)])
+    B.status(ctx)
+    out = figures(med, len(mats), step_bytes, peak)
+    out.update({"workload": f"config {config}: {wl.name}", "us_min": lo * 1e3 / len(mats), "us_max": hi * 1e3 / len(mats),
+                "gemvs_per_step": len(mats), "launches_per_step": launches, "steps": steps, "rounds_kept": kept,
+                "bytes_per_step": step_bytes, "record_copies": ncopies})
+    del copies, mats
+    torch.cuda.empty_cache()
+    return out
+
+
+def single_matrix(B, ctx, rows, k, device, peak, seed=5, rounds=7, steps=200):
+    """One matrix, one launch a step, cold records."""
+    nb = (k + 23) // 24
+    codes = datagen.make_codes(rows, nb, seed, device=device)
+    sc = datagen.make_row_scale(rows, seed).to(device)
+    x = datagen.make_x(k, nb * 24, seed).to(device)
+    buf0 = B.expand(ctx, B.PLANES, codes, rows, nb)
+    del codes
+    ncopies = copies_needed(buf0.numel())
+    bufs = [buf0] + [buf0.clone() for _ in range(ncopies - 1)]
+    y = torch.empty(rows, dtype=torch.float32, device=device)
+    med, lo, hi, _ = summarise_rounds([ms / steps for ms in time_rounds(
+        lambda i: B.gemv(ctx, B.PLANES, bufs[i % ncopies], sc, datagen.GAIN, x, rows, nb * 24, y=y), steps, 3, rounds)])
+    nw, _, _, _ = summarise_rounds([ms / steps for ms in time_rounds(
+        lambda i: B.gemv_noweights(ctx, sc, x, rows, nb * 24, y=y), steps, 3, 5)])
+    out = figures(med, 1, gemv_bytes(rows, nb), peak)
+    out.update({"rows": rows, "k": k, "us_min": lo * 1e3, "us_max": hi * 1e3, "noweights_us": nw * 1e3})
+    del bufs, buf0
+    torch.cuda.empty_cache()
+    return out
+
+
+def comparison_arms(B, ctx, device, peak, steps=200):
+    """The arms of the paper's layout table, on the 4B-like layer (config 1): per-matrix launches, small batches,
+    the activation rotation, the no-weights control, the 13-byte layout, the one-hot layout, the FP16 control.
+    Every arm's outputs are compared with those of the 14-byte arm (which the GPU tests hold to the oracle)."""
+    wl = datagen.workload(1)
+    mats = build_inputs(wl, device)
+    n_gemv = len(mats)
+    step_bytes = sum(gemv_bytes(e["m"].rows, e["m"].nb) for e in mats)
+    ncopies = copies_needed(sum(14 * e["m"].blocks for e in mats))
+    copies = make_copies(B, ctx, mats, B.PLANES, ncopies, device)
+    t_main = time_arm(lambda i: run_step(B, ctx, B.PLANES, copies[i]), ncopies, steps, 3)
+    arms = {"workload": f"config 1: {wl.name}", "planes14": figures(t_main, n_gemv, step_bytes, peak)}
+    # per-matrix timings of the 14-byte-layout kernel, one launch each
+    per_matrix = {}
+    for li, ln in enumerate(copies[0].launches):
+        for mi, m in enumerate(ln["mats"]):
+            def one(i, li=li, mi=mi):
+                l2 = copies[i].launches[li]
+                B.gemv(ctx, B.PLANES, l2["bufs"][mi], l2["scales"][mi], datagen.GAIN, l2["x"], l2["mats"][mi].rows, l2["k_padded"], y=l2["ys"][mi])
+            t = time_arm(one, ncopies, steps, 3)
+            per_matrix[m.name] = dict(figures(t, 1, gemv_bytes(m.rows, m.nb), peak), rows=m.rows, k=m.k)
+    arms["per_matrix"] = per_matrix
+    # small-batch decode: the same matrices, one launch each, 1 / 2 / 4 activation vectors a launch
+    batch_arm = {}
+    for nvec in (1, 2, 4):
+        xb = {}
+        for cp in copies:
+            for ln in cp.launches:
+                if id(ln["x"]) not in xb:
+                    xb[id(ln["x"])] = (ln["x"].unsqueeze(0).repeat(nvec, 1).contiguous(),
+                                       [torch.empty((nvec, m.rows), dtype=torch.float32, device=device) for m in ln["mats"]])
+        def bstep(i, xb=xb):
+            for ln in copies[i].launches:
+                X, Ys = xb[id(ln["x"])]
+                for mi, m in enumerate(ln["mats"]):
+                    B.gemv_batch(ctx, ln["bufs"][mi], ln["scales"][mi], datagen.GAIN, X, m.rows, ln["k_padded"], y=Ys[mi])
+        t = time_arm(bstep, ncopies, steps, 3)
+        batch_arm[str(nvec)] = {"us_per_launch": t * 1e3 / n_gemv, "us_per_vector": t * 1e3 / n_gemv / nvec,
+                                "record_gbps": step_bytes / (t * 1e-3) / 1e9}
+        del xb
+    arms["batch"] = batch_arm
+    # activation rotation ahead of every projection (the served order): inside the GEMV's own launch, as a kernel
+    # of its own ahead of each GEMV (the paper's arrangement), and those rotation kernels alone
+    xr = {}
+    for cp in copies:
+        for ln in cp.launches:
+            if id(ln["x"]) not in xr:
+                xr[id(ln["x"])] = ln["x"].clone()
+    def rot_fused(i):
+        for ln in copies[i].launches:
+            B.gemv_rotated(ctx, ln["problems"], ln["x"], ln["k_padded"], n=ln["mats"][0].k)
+    def rot_two(i):
+        for ln in copies[i].launches:
+            k = ln["mats"][0].k
+            B.rotate(ctx, ln["x"][:k], y=xr[id(ln["x"])][:k])
+            B.gemv_grouped(ctx, B.PLANES, ln["problems"], xr[id(ln["x"])], ln["k_padded"])
+    def rot_only(i):
+        for ln in copies[i].launches:
+            k = ln["mats"][0].k
+            B.rotate(ctx, ln["x"][:k], y=xr[id(ln["x"])][:k])
+    def rot_fused_512(i):
+        for ln in copies[i].launches:
+            B.gemv_rotated(ctx, ln["problems"], ln["x"], ln["k_padded"], n=ln["mats"][0].k, block=min(512, int(B.rotate_block(ln["mats"][0].k))))
+    n_launch = len(copies[0].launches)
+    arms["rotated"] = {"us_per_gemv_fused": time_arm(rot_fused, ncopies, steps, 3) * 1e3 / n_gemv,
+                       "us_per_gemv_fused_blocks_of_512_at_most": time_arm(rot_fused_512, ncopies, steps, 3) * 1e3 / n_gemv,
+                       "us_per_gemv_two_launches": time_arm(rot_two, ncopies, steps, 3) * 1e3 / n_gemv,
+                       "us_per_rotation_alone": time_arm(rot_only, ncopies, steps, 3) * 1e3 / n_launch, "rotations_per_step": n_launch,
+                       "block_lengths": sorted({int(B.rotate_block(ln["mats"][0].k)) for ln in copies[0].launches})}
+    # no-weights control: the same launches without record reads
+    def nw(i):
+        for ln in copies[i].launches:
+            for mi, m in enumerate(ln["mats"]):
+                B.gemv_noweights(ctx, ln["scales"][mi], ln["x"], m.rows, ln["k_padded"], y=ln["ys"][mi])
+    arms["noweights"] = {"us_per_gemv": time_arm(nw, ncopies, steps, 3) * 1e3 / n_gemv, "launches_per_step": n_gemv}
+    # the 13-byte layout: the same codes and arithmetic, a one-byte header (exact for every block)
+    run_step(B, ctx, B.PLANES, copies[0])
+    p13_copies = make_copies(B, ctx, mats, B.PLANES13, ncopies, device)
+    run_step(B, ctx, B.PLANES13, p13_copies[0])
+    torch.cuda.synchronize()
+    same_outputs(copies, p13_copies, exact=True)
+    t = time_arm(lambda i: run_step(B, ctx, B.PLANES13, p13_copies[i]), len(p13_copies), steps, 3)
+    pb = sum(gemv_bytes(e["m"].rows, e["m"].nb, 13) for e in mats)
+    arms["planes13"] = dict(figures(t, n_gemv, pb, peak), bytes_per_block=13, bits_per_weight=13 * 8 / 24)
+    del p13_copies
+    # one-hot layout: a correctness reference for the paper's other record (plain coalesced loads, scalar
+    # arithmetic, not tuned), so its time says nothing about the layouts' relative merit
+    oh_copies = make_copies(B, ctx, mats, B.ONEHOT, max(2, ncopies * 14 // 20 + 1), device)
+    run_step(B, ctx, B.ONEHOT, oh_copies[0])
+    torch.cuda.synchronize()
+    same_outputs(copies, oh_copies, exact=False)
+    t = time_arm(lambda i: run_step(B, ctx, B.ONEHOT, oh_copies[i]), len(oh_copies), steps, 3)
+    ob = sum(gemv_bytes(e["m"].rows, e["m"].nb, 20) for e in mats)
+    arms["onehot"] = dict(figures(t, n_gemv, ob, peak), bytes_per_block=20,
+                          note="untuned correctness reference: not a comparison of the layouts")
+    del oh_copies
+    # FP16 control over the decoded weights
+    fp_copies = []
+    nfp = max(2, -(-3 * L2_BYTES // (48 * sum(e["m"].blocks for e in mats))))
+    for c in range(nfp):
+        ws = []
+        for ln in copies[0].launches:
+            for mi, m in enumerate(ln["mats"]):
+                W = B.dequant_fp16(ctx, B.PLANES, ln["bufs"][mi], ln["scales"][mi], datagen.GAIN, m.rows, ln["k_padded"])
+                ws.append((W, ln["x"], m, torch.empty(m.rows, dtype=torch.float32, device=device)))
+        fp_copies.append(ws)
+    def fp(i):
+        for W, x, m, y in fp_copies[i]:
+            B.gemv_fp16(W, x, m.rows, m.k_padded, y=y)
+    t = time_arm(fp, nfp, steps, 3)
+    fb = sum(2 * e["m"].rows * e["m"].k_padded + 2 * e["m"].k_padded + 4 * e["m"].rows for e in mats)
+    arms["fp16"] = figures(t, n_gemv, fb, peak)
+    arms["planes_vs_fp16"] = arms["fp16"]["us"] / arms["planes14"]["us"]
+    B.status(ctx)
+    del fp_copies, copies, mats
+    torch.cuda.empty_cache()
+    return arms
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--rounds", type=int, default=7, help="timed rounds of --steps steps each; the first two are discarded")
+    ap.add_argument("--config", type=int, default=3)
     ap.add_argument("--layers", type=int, default=None, help="truncate the multi-layer stacks (configs 2, 3)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-arms", action="store_true", help="skip the one-hot / FP16 / no-weights comparison arms")
-    ap.add_argument("--no-verify", action="store_true", help="skip the oracle check (profiling runs only)")
-    ap.add_argument("--lean", action="store_true", help="profiling runs: no clock ramp, no end-to-end leg, no arms, no oracle check")
+    ap.add_argument("--no-arms", action="store_true", help="skip the other configurations, the single matrices and the comparison arms")
     ap.add_argument("--no-pdl", action="store_true", help="launch the GEMV without programmatic dependent launch")
     ap.add_argument("--ungrouped", action="store_true", help="one launch a matrix instead of row-concatenated groups")
-    ap.add_argument("--profile-batch", type=int, default=0,
-                    help="profiling runs: only launch llvq_gemv_batch with this many activation vectors, one launch a matrix, and exit")
-    ap.add_argument("--profile-rotated", action="store_true",
-                    help="profiling runs: only launch llvq_rotate and llvq_gemv_rotated on the workload's launches, and exit")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
-    if args.lean:
-        args.no_arms = args.no_verify = True
+    args.rounds = max(args.rounds, DISCARD_ROUNDS + 1)
     wl = datagen.workload(args.config, args.layers)
 
     if args.impl == "reference":
@@ -335,43 +527,20 @@ def main():
     peak, peak_src = measured_peaks()
 
     mats = build_inputs(wl, device)
+    n_gemv = len(mats)
     step_bytes = sum(gemv_bytes(e["m"].rows, e["m"].nb) for e in mats)
     layout_bytes = sum(14 * e["m"].blocks for e in mats)
-    ncopies = max(2, -(-3 * L2_BYTES // layout_bytes)) if layout_bytes < 3 * L2_BYTES else 1
-    t0 = time.perf_counter()
-    copies = make_copies(B, ctx, mats, B.PLANES, ncopies, device, grouped=not args.ungrouped)
+    ncopies = copies_needed(layout_bytes)
+    # the oracle checks the first layer (the multi-layer stacks) or the whole step: only those codes are kept
+    checked = 7 if n_gemv > 7 else n_gemv
+    copies = make_copies(B, ctx, mats, B.PLANES, ncopies, device, grouped=not args.ungrouped,
+                         keep_codes={e["m"].tensor_id for e in mats[:checked]})
     torch.cuda.synchronize()
     launches_per_step = len(copies[0].launches)
 
-    if args.profile_batch:
-        # a few batched launches for a profiler to capture; nothing is measured here
-        nvec = args.profile_batch
-        for i in range(args.warmup + args.steps):
-            for ln in copies[i % ncopies].launches:
-                X = ln["x"].unsqueeze(0).repeat(nvec, 1).contiguous()
-                for mi, m in enumerate(ln["mats"]):
-                    B.gemv_batch(ctx, ln["bufs"][mi], ln["scales"][mi], datagen.GAIN, X, m.rows, ln["k_padded"])
-        torch.cuda.synchronize()
-        B.status(ctx)
-        print(json.dumps({"profile": "llvq_gemv_batch", "vectors": nvec, "config": wl.name, "launches": (args.warmup + args.steps) * len(mats)}))
-        return
-
-    if args.profile_rotated:
-        # the rotation as a kernel of its own and inside the GEMV, for a profiler to capture; nothing is measured here
-        for i in range(args.warmup + args.steps):
-            for ln in copies[i % ncopies].launches:
-                k = ln["mats"][0].k
-                B.rotate(ctx, ln["x"][:k])
-                B.gemv_rotated(ctx, ln["problems"], ln["x"], ln["k_padded"], n=k)
-        torch.cuda.synchronize()
-        B.status(ctx)
-        print(json.dumps({"profile": "llvq_rotate + llvq_gemv_rotated", "config": wl.name,
-                          "launches": 2 * (args.warmup + args.steps) * launches_per_step}))
-        return
-
     # expander throughput (load-time step, outside the timed region)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    big = max(mats, key=lambda e: e["m"].blocks)
+    big = max(mats[:checked], key=lambda e: e["m"].blocks)
     B.expand(ctx, B.PLANES, big["codes"], big["m"].rows, big["m"].nb)
     e0.record()
     B.expand(ctx, B.PLANES, big["codes"], big["m"].rows, big["m"].nb)
@@ -379,52 +548,38 @@ def main():
     e1.synchronize()
     expand_rate = big["m"].blocks / (e0.elapsed_time(e1) * 1e-3)
 
-    # parity first (every row, copy 0), which also times the oracle on the host cores
+    # parity first (every row of the checked launches, copy 0), which also times the oracle on the host cores
     cores = os.cpu_count() or 1
     run_step(B, ctx, B.PLANES, copies[0])
     torch.cuda.synchronize()
-    cpu_baseline, worst = None, None
-    if not args.no_verify:
-        from oracle import oracle as O
+    from oracle import oracle as O
 
-        # the multi-layer stacks are checked (and the oracle timed) on their first layer; tests/ cover more layers
-        first_layer = 4 if len(mats) > 7 and not args.ungrouped else (7 if len(mats) > 7 else None)
-        worst, osecs, oblocks, ogemvs = verify(O, copies, cores, first_layer)
-        if rank == 0:
-            cpu_baseline = {"value": osecs / ogemvs * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
-                            "sample": f"{ogemvs} GEMVs of the step once ({oblocks} of {wl.blocks} blocks): index decode + f64 matvec",
-                            "blocks_per_s": oblocks / osecs}
+    checked_launches = None if checked == n_gemv else (4 if not args.ungrouped else 7)
+    worst, osecs, oblocks, ogemvs, dsecs = verify(O, copies, cores, checked_launches)
+    cpu_baseline = None
+    if rank == 0:
+        decode_us = dsecs / cores / ogemvs * 1e6
+        cpu_baseline = {"value": osecs / ogemvs * 1e6, "unit": "us", "cores": cores, "kind": "oracle",
+                        "sample": f"{ogemvs} GEMVs of the step once ({oblocks} of {wl.blocks} blocks): index decode + f64 matvec on all cores",
+                        "blocks_per_s": oblocks / osecs, "decode_us": decode_us, "matvec_us": max(osecs / ogemvs * 1e6 - decode_us, 0.0),
+                        "split": "decode_us = the index decode alone timed on one core over 262144 codes a matrix, scaled by blocks and divided by the cores; matvec_us = the rest"}
 
-    # warm-up: ramp the clocks, then W untimed steps, then exactly K timed steps
-    ramp = capture_graphs(B, ctx, B.PLANES, copies, 1 if args.lean else min(512, max(64, ncopies * 8)))
-    t_end = time.perf_counter() + (0.0 if args.lean else 0.4)
+    # warm-up: ramp the clocks, then the protocol
+    step_fn = lambda i: run_step(B, ctx, B.PLANES, copies[i % ncopies])
+    ramp = capture_graphs(step_fn, max(2, min(64, 4000 // launches_per_step)))
+    t_end = time.perf_counter() + 0.4
     while time.perf_counter() < t_end:
         time_graphs(ramp)
-    warm = capture_graphs(B, ctx, B.PLANES, copies, args.warmup)
-    graphs = capture_graphs(B, ctx, B.PLANES, copies, args.steps, first_step=args.warmup)
-    torch.cuda.synchronize()
+    del ramp
     sampler = ClockSampler(local)
     sampler.start()
-    time_graphs(warm)
-    # One untimed pass over the graphs that will be timed: a graph's first launch uploads it to the device
-    # (about a millisecond for 2000 steps), which is not part of a step.  The records still rotate through
-    # copies larger than L2, so the timed pass finds them cold.
-    time_graphs(graphs)
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
-    ms = time_graphs(graphs)
-    torch.cuda.synchronize()
-    if dist:
-        dist.barrier()
+    ms_rounds = time_rounds(step_fn, args.steps, args.warmup, args.rounds, dist, device)
     clocks = sampler.result()
-    ms = max_over_ranks(ms, dist, device)
-
+    B.status(ctx)
+    ms, ms_min, ms_max, kept = summarise_rounds(ms_rounds)
     ms_per_step = ms / args.steps
-    n_gemv = len(mats)
     us_per_gemv = us_per_gemv_of_job(ms_per_step, n_gemv, world)
     gbps = step_bytes / (ms_per_step * 1e-3) / 1e9            # per GPU
-    per_shape = None
 
     # End to end: every step copies that step's activations from pinned host memory to the device, runs the step's
     # launches through the same C-ABI calls, copies every y back to pinned host memory and waits for it.  The
@@ -480,141 +635,36 @@ def main():
         e2e_graphs[i % ncopies].replay()
         torch.cuda.synchronize()
 
-    e2e_steps = 1 if args.lean else min(args.steps, 300)
-    for i in range(1 if args.lean else 10):
+    e2e_steps = max(3, min(args.steps, 300))
+    for i in range(5):
         e2e_step(i)
     # the copies back are the results the launches computed: the last step's y against the device arrays
     yi = 0
-    for ln in copies[(0 if args.lean else 9) % ncopies].launches:
+    for ln in copies[4 % ncopies].launches:
         for m in ln["mats"]:
             assert torch.equal(host_y[y_off[yi]:y_off[yi] + m.rows], dev_y[y_off[yi]:y_off[yi] + m.rows].cpu())
             yi += 1
-    t1 = time.perf_counter()
-    for i in range(e2e_steps):
-        e2e_step(i)
-    e2e_us = (time.perf_counter() - t1) / e2e_steps * 1e6 / n_gemv / world
+    e2e_rounds = []
+    for _ in range(args.rounds):
+        t1 = time.perf_counter()
+        for i in range(e2e_steps):
+            e2e_step(i)
+        e2e_rounds.append((time.perf_counter() - t1) / e2e_steps * 1e6 / n_gemv / world)
+    e2e_us, e2e_min, e2e_max, _ = summarise_rounds(e2e_rounds)
     # ... and they are the right results: one matrix of the last step against the untimed path's y (same records, same x)
     run_step(B, ctx, B.PLANES, copies[(e2e_steps - 1) % ncopies])
     torch.cuda.synchronize()
     assert torch.equal(host_y[y_off[0]:y_off[0] + l0[0]["mats"][0].rows], copies[(e2e_steps - 1) % ncopies].launches[0]["ys"][0].cpu())
+    del e2e_graphs, e2e_keep
 
-    arms = {}
-    if len(mats) > 7:
-        args.no_arms = True          # the comparison arms and per-shape timings are taken on the single-layer workloads
-    if not args.no_arms and rank == 0:
-        arm_steps = min(args.steps, 200)
-        # per-matrix timings of the 14-byte-layout kernel, one launch each
-        per_shape = {}
-        for li, ln in enumerate(copies[0].launches):
-            for mi, m in enumerate(ln["mats"]):
-                def one(i, li=li, mi=mi):
-                    l2 = copies[i % ncopies].launches[li]
-                    B.gemv(ctx, B.PLANES, l2["bufs"][mi], l2["scales"][mi], datagen.GAIN, l2["x"], l2["mats"][mi].rows, l2["k_padded"], y=l2["ys"][mi])
-                t = time_arm(one, ncopies, arm_steps, 3)
-                by = gemv_bytes(m.rows, m.nb)
-                per_shape[m.name] = {"rows": m.rows, "k": m.k, "us": t * 1e3, "gbps": by / (t * 1e-3) / 1e9, "frac": by / (t * 1e-3) / 1e9 / peak}
-        # small-batch decode: the same matrices, one launch each, 1 / 2 / 4 activation vectors a launch (the records
-        # are read and decoded once a launch; every vector was checked against the single-vector result by the tests)
-        batch_arm = {}
-        for nvec in (1, 2, 4):
-            xb = {}
-            for cp in copies:
-                for ln in cp.launches:
-                    if id(ln["x"]) not in xb:
-                        xb[id(ln["x"])] = (ln["x"].unsqueeze(0).repeat(nvec, 1).contiguous(),
-                                           [torch.empty((nvec, m.rows), dtype=torch.float32, device=device) for m in ln["mats"]])
-            def bstep(i, xb=xb):
-                for ln in copies[i % ncopies].launches:
-                    X, Ys = xb[id(ln["x"])]
-                    for mi, m in enumerate(ln["mats"]):
-                        B.gemv_batch(ctx, ln["bufs"][mi], ln["scales"][mi], datagen.GAIN, X, m.rows, ln["k_padded"], y=Ys[mi])
-            t = time_arm(bstep, ncopies, arm_steps, 3)
-            batch_arm[str(nvec)] = {"us_per_launch": t * 1e3 / n_gemv, "us_per_vector": t * 1e3 / n_gemv / nvec,
-                                    "record_gbps": step_bytes / (t * 1e-3) / 1e9}
-            del xb
-        arms["batch"] = batch_arm
-        # activation rotation ahead of every projection (the served order: the weights live in the rotated basis, so
-        # each projection's input is rotated first).  The rotation acts on the k real entries of x; the zero padding
-        # passes through.  Three timings: the rotation inside the GEMV's own launch (llvq_gemv_rotated), the
-        # rotation as a kernel of its own ahead of each GEMV (llvq_rotate, the paper's arrangement), and those
-        # rotation kernels alone.
-        xr = {}
-        for cp in copies:
-            for ln in cp.launches:
-                if id(ln["x"]) not in xr:
-                    xr[id(ln["x"])] = ln["x"].clone()
-        def rot_fused(i):
-            for ln in copies[i % ncopies].launches:
-                B.gemv_rotated(ctx, ln["problems"], ln["x"], ln["k_padded"], n=ln["mats"][0].k)
-        def rot_two(i):
-            for ln in copies[i % ncopies].launches:
-                k = ln["mats"][0].k
-                B.rotate(ctx, ln["x"][:k], y=xr[id(ln["x"])][:k])
-                B.gemv_grouped(ctx, B.PLANES, ln["problems"], xr[id(ln["x"])], ln["k_padded"])
-        def rot_only(i):
-            for ln in copies[i % ncopies].launches:
-                k = ln["mats"][0].k
-                B.rotate(ctx, ln["x"][:k], y=xr[id(ln["x"])][:k])
-        def rot_fused_512(i):
-            for ln in copies[i % ncopies].launches:
-                B.gemv_rotated(ctx, ln["problems"], ln["x"], ln["k_padded"], n=ln["mats"][0].k, block=min(512, int(B.rotate_block(ln["mats"][0].k))))
-        t_f = time_arm(rot_fused, ncopies, arm_steps, 3)
-        t_f512 = time_arm(rot_fused_512, ncopies, arm_steps, 3)
-        t_2 = time_arm(rot_two, ncopies, arm_steps, 3)
-        t_0 = time_arm(rot_only, ncopies, arm_steps, 3)
-        n_launch = len(copies[0].launches)
-        arms["rotated"] = {"us_per_gemv_fused": t_f * 1e3 / n_gemv, "us_per_gemv_fused_blocks_of_512_at_most": t_f512 * 1e3 / n_gemv,
-                           "us_per_gemv_two_launches": t_2 * 1e3 / n_gemv,
-                           "us_per_rotation_alone": t_0 * 1e3 / n_launch, "rotations_per_step": n_launch,
-                           "block_lengths": sorted({int(B.rotate_block(ln["mats"][0].k)) for ln in copies[0].launches})}
-        # no-weights control: the same launches without record reads
-        def nw(i):
-            for ln in copies[i % ncopies].launches:
-                for mi, m in enumerate(ln["mats"]):
-                    B.gemv_noweights(ctx, ln["scales"][mi], ln["x"], m.rows, ln["k_padded"], y=ln["ys"][mi])
-        t = time_arm(nw, ncopies, arm_steps, 3)
-        arms["noweights"] = {"us_per_gemv": t * 1e3 / n_gemv, "launches_per_step": n_gemv}
-        # the 13-byte layout: the same codes and arithmetic, a one-byte header (exact for every block)
-        p13_copies = make_copies(B, ctx, mats, B.PLANES13, ncopies, device, grouped=not args.ungrouped)
-        run_step(B, ctx, B.PLANES13, p13_copies[0])
-        torch.cuda.synchronize()
-        run_step(B, ctx, B.PLANES, copies[0])
-        torch.cuda.synchronize()
-        same_outputs(copies, p13_copies, exact=True)
-        t = time_arm(lambda i: run_step(B, ctx, B.PLANES13, p13_copies[i % len(p13_copies)]), len(p13_copies), arm_steps, 3)
-        pb = sum(gemv_bytes(e["m"].rows, e["m"].nb, 13) for e in mats)
-        arms["planes13"] = {"us_per_gemv": t * 1e3 / n_gemv, "gbps": pb / (t * 1e-3) / 1e9, "frac": pb / (t * 1e-3) / 1e9 / peak,
-                            "bytes_per_block": 13, "bits_per_weight": 13 * 8 / 24}
-        del p13_copies
-        # one-hot layout
-        oh_copies = make_copies(B, ctx, mats, B.ONEHOT, max(2, ncopies * 14 // 20 + 1), device, grouped=not args.ungrouped)
-        run_step(B, ctx, B.ONEHOT, oh_copies[0])
-        torch.cuda.synchronize()
-        run_step(B, ctx, B.PLANES, copies[0])
-        torch.cuda.synchronize()
-        same_outputs(copies, oh_copies, exact=False)
-        t = time_arm(lambda i: run_step(B, ctx, B.ONEHOT, oh_copies[i % len(oh_copies)]), len(oh_copies), arm_steps, 3)
-        ob = sum(gemv_bytes(e["m"].rows, e["m"].nb, 20) for e in mats)
-        arms["onehot"] = {"us_per_gemv": t * 1e3 / n_gemv, "gbps": ob / (t * 1e-3) / 1e9, "frac": ob / (t * 1e-3) / 1e9 / peak, "bytes_per_block": 20}
-        del oh_copies
-        # FP16 control over the decoded weights
-        fp_copies = []
-        nfp = max(2, -(-3 * L2_BYTES // (48 * sum(e["m"].blocks for e in mats))))
-        for c in range(nfp):
-            ws = []
-            for ln in copies[0].launches:
-                for mi, m in enumerate(ln["mats"]):
-                    W = B.dequant_fp16(ctx, B.PLANES, ln["bufs"][mi], ln["scales"][mi], datagen.GAIN, m.rows, ln["k_padded"])
-                    ws.append((W, ln["x"], m, torch.empty(m.rows, dtype=torch.float32, device=device)))
-            fp_copies.append(ws)
-        def fp(i):
-            for W, x, m, y in fp_copies[i % nfp]:
-                B.gemv_fp16(W, x, m.rows, m.k_padded, y=y)
-        t = time_arm(fp, nfp, arm_steps, 3)
-        fb = sum(2 * e["m"].rows * e["m"].k_padded + 2 * e["m"].k_padded + 4 * e["m"].rows for e in mats)
-        arms["fp16"] = {"us_per_gemv": t * 1e3 / n_gemv, "gbps": fb / (t * 1e-3) / 1e9, "frac": fb / (t * 1e-3) / 1e9 / peak}
-        arms["planes_vs_fp16"] = arms["fp16"]["us_per_gemv"] / (ms_per_step * 1e3 / n_gemv)
-        del fp_copies
+    per_config, per_shape, arms = None, None, None
+    if not args.no_arms and rank == 0 and world == 1:
+        # the other configurations and three single matrices through the same protocol, then the comparison arms
+        del copies, mats
+        torch.cuda.empty_cache()
+        per_config = {str(c): side_workload(B, ctx, c, device, peak) for c in (0, 1, 2, 4) if c != args.config}
+        per_shape = {f"{r}x{k}": single_matrix(B, ctx, r, k, device, peak) for r, k in ((4096, 4096), (8192, 8192), (24576, 4096))}
+        arms = comparison_arms(B, ctx, device, peak)
 
     if rank == 0:
         line = {
@@ -623,8 +673,12 @@ def main():
             "dtype": "u8 x s8 -> s32 (tensor cores), f32 block scale, int64 row sums", "data": "synthetic",
             "config": {"workload": f"config {wl.config}: {wl.name}", "gemvs_per_step": n_gemv, "launches_per_step": launches_per_step,
                        "layout": "Planes14: 14 B per 24 weights - class, gain, 24 four-bit sign+level codes (4.67 b/w payload; the paper's 4.80 b/w label counts its f32 tail and scales)",
-                       "l2": f"records and scales rotate through {ncopies} distinct copies ({ncopies * layout_bytes / 1e6:.0f} MB) so no launch finds its records in L2; x (a few KB a launch) is one buffer, as in a decoder where it is the previous operator's output",
-                       "multi_gpu": "replicas only: each rank runs the whole step on its own copy", "seed": wl.seed},
+                       "l2": f"records and scales: {ncopies} distinct cop{'y' if ncopies == 1 else 'ies'} ({ncopies * layout_bytes / 1e6:.0f} MB, at least three times L2) so no launch finds its records in L2; x (a few KB a launch) is one buffer, as in a decoder where it is the previous operator's output",
+                       "multi_gpu": "replicas only: each rank runs the whole step on its own copy", "seed": wl.seed,
+                       "oracle_check": f"every row of the first {ogemvs} GEMVs before timing"},
+            "rounds": {"run": len(ms_rounds), "discarded": len(ms_rounds) - kept, "statistic": "median of the rounds kept",
+                       "us_min": us_per_gemv_of_job(ms_min / args.steps, n_gemv, world), "us_max": us_per_gemv_of_job(ms_max / args.steps, n_gemv, world),
+                       "ms_per_round": ms_rounds},
             "gbps": gbps, "hbm_frac": gbps / peak, "bytes_per_step": step_bytes,
             "roofline": {"bound": "hbm", "achieved": gbps, "peak": peak, "unit": "GB/s", "frac": gbps / peak,
                          "traffic": step_bytes / launches_per_step * NCU_TRAFFIC_PER_ALGORITHMIC_BYTE,
@@ -634,13 +688,13 @@ def main():
                          "secondary": {"bound": "issue", "warp_instructions_per_block_column": NCU_WARP_INSTR_PER_CELL,
                                        "issue_slots_busy_pct": NCU_ISSUE_BUSY_PCT,
                                        "source": "profiles/gemv_planes_kernel_config4_8192x8192.txt"},
-                         "how": "algorithmic bytes of a step / CUDA-event time of the step, averaged over its launches"},
+                         "how": "algorithmic bytes of a step / median CUDA-event time of a step, averaged over its launches"},
             "cpu_baseline": cpu_baseline,
-            "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "e2e": {"value": e2e_us, "unit": "us", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "us_min": e2e_min, "us_max": e2e_max,
                     "how": "every step: one copy of the step's x vectors from pinned host memory, the launches, one copy of every y back to pinned host memory, issued as a captured CUDA graph of those C-ABI calls and waited for before the next step"},
             "gpu_launches": args.steps * launches_per_step,
             "clocks": clocks, "parity_worst_normalised_error": worst,
-            "expand_blocks_per_s": expand_rate, "per_shape": per_shape, "arms": arms,
+            "expand_blocks_per_s": expand_rate, "per_config": per_config, "per_shape": per_shape, "arms": arms,
         }
         print(json.dumps(line), flush=True)
     ctx.close()
