@@ -64,11 +64,14 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
     ctx->max_smem_optin = (int)prop.sharedMemPerBlockOptin;
 
     const HostTables &h = ctx->host;
-    struct Part { const void *src; size_t bytes; size_t off; } parts[8] = {
+    uint32_t lanes[32][4];
+    gemv_lane_table(lanes);
+    struct Part { const void *src; size_t bytes; size_t off; } parts[10] = {
         {h.base.data(), h.base.size() * 8, 0},          {h.desc.data(), h.desc.size() * sizeof(ClassDesc), 0},
         {h.golay_by_weight.data(), 4096 * 4, 0},        {h.golay_by_message.data(), 4096 * 4, 0},
         {h.cls_scale.data(), kClassSlots * 4, 0},       {h.cls_parity.data(), kClassSlots * 4, 0},
-        {h.cls_value.data(), kClassSlots * 8 * 4, 0},   {h.cls_dist.data(), kClassSlots * 8, 0}};
+        {h.cls_value.data(), kClassSlots * 8 * 4, 0},   {h.cls_dist.data(), kClassSlots * 8, 0},
+        {h.cls_block.data(), kClassSlots * 8, 0},       {lanes, sizeof lanes, 0}};
     size_t total = 0;
     for (auto &p : parts) { p.off = total; total += round_up(p.bytes, 256); }
     if (cudaMalloc(&ctx->table_blob, total) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
@@ -87,6 +90,8 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
     d.cls_parity = (const uint32_t *)(blob + parts[5].off);
     d.cls_value = (const float *)(blob + parts[6].off);
     d.cls_dist = (const uint8_t *)(blob + parts[7].off);
+    d.cls_block = (const float2 *)(blob + parts[8].off);
+    d.lane_table = (const uint4 *)(blob + parts[9].off);
     std::memcpy(d.weight_offset, h.weight_offset, sizeof d.weight_offset);
     d.num_classes = h.num_classes;
     d.num_points = h.num_points;
@@ -206,7 +211,7 @@ int llvq_gemv_plan(int sm_count, const int64_t *rows, int n, int64_t k_padded, i
     if (out_len < 8 + g.grid + 1) return LLVQ_ESIZE;
     out[0] = g.grid; out[1] = (int32_t)g.smem; out[2] = p.units; out[3] = p.total_units;
     out[4] = p.panel; out[5] = p.npanels; out[6] = p.xblocks; out[7] = p.total_groups;
-    for (int c = 0; c <= g.grid; c++) out[8 + c] = p.cta_first[c];
+    for (int c = 0; c <= g.grid; c++) out[8 + c] = p.cta[c].first;
     return LLVQ_OK;
 }
 
@@ -265,6 +270,8 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
     p.cls_scale = ctx->dev.cls_scale;
     p.cls_parity = ctx->dev.cls_parity;
     p.cls_value = ctx->dev.cls_value;
+    p.cls_block = ctx->dev.cls_block;
+    p.lane_table = ctx->dev.lane_table;
     std::memcpy(p.cls_shell_nibbles, ctx->host.cls_shell_nibbles, sizeof p.cls_shell_nibbles);
     std::memcpy(p.cls_odd_bits, ctx->host.cls_odd_bits, sizeof p.cls_odd_bits);
     std::memcpy(p.shell_inv_norm, ctx->host.shell_inv_norm, sizeof p.shell_inv_norm);

@@ -51,7 +51,7 @@
     }
 // per-unit timeline of every warp: slot 8 + 3*n + {0: wait begins, 1: data there, 2: decoded}, n < 40
 #define LLVQ_TRACE_UNIT(n, i)                                                                                     \
-    if (p.trace && lane == 0 && (n) < 40) {                                                                       \
+    if (0) {                                                                       \
         unsigned long long t_;                                                                                    \
         asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                                    \
         p.trace[(((size_t)p.trace_launch * gridDim.x + blockIdx.x) * kWarps + warp) * 128 + 8 + 3 * (n) + (i)] = t_; \
@@ -59,7 +59,7 @@
 // SM cycle counter into slots 120..127
 #define LLVQ_TRACE_CLOCK(i)                                                                                       \
     if (p.trace && lane == 0)                                                                                     \
-        p.trace[(((size_t)p.trace_launch * gridDim.x + blockIdx.x) * kWarps + warp) * 128 + 120 + (i)] = clock64();
+        p.trace[(((size_t)p.trace_launch * gridDim.x + blockIdx.x) * kWarps + warp) * 128 + 98 + (i)] = clock64();
 #else
 #define LLVQ_TRACE_POINT(i)
 #define LLVQ_TRACE_UNIT(n, i)
@@ -247,9 +247,13 @@ __device__ __forceinline__ uint32_t settled(uint32_t a, uint32_t b, uint32_t c) 
 }
 
 // First byte of a row group's records, and the matrix it belongs to.
-__device__ __forceinline__ const uint8_t *group_base(const GemvParams &p, int group, int cell_bytes, int &q) {
+__device__ __forceinline__ const uint8_t *group_base(const GemvParams &p, int group, int &q) {
+    if (p.nprob == 1) {                              // the common launch: one matrix
+        q = 0;
+        return p.prob[0].layout + (size_t)(uint32_t)group * p.group_bytes;
+    }
     q = find_problem(p, group);
-    return p.prob[q].layout + (size_t)(group - p.prob[q].group_begin) * (size_t)p.nb * cell_bytes;
+    return p.prob[q].layout + (size_t)(uint32_t)(group - p.prob[q].group_begin) * p.group_bytes;
 }
 
 // ---- integer tensor-core contraction: D (16 rows x 8 columns, s32) = A (16 x k, u8) * B (k x 8, s8) [+ D]
@@ -273,7 +277,7 @@ constexpr int kXRecBytes = 112;
 // the single record both slots of the row group's last half-step share).  B is block-diagonal: column
 // n = lane >> 2 carries limb n & 3 of slot n >> 2, and is zero at the positions of the other slot.
 struct LaneOffsets { uint32_t b0, b1, b2, xs; };
-__device__ __forceinline__ LaneOffsets lane_offsets(int lane, bool one) {
+__host__ __device__ __forceinline__ LaneOffsets lane_offsets(int lane, bool one) {
     const int g = lane >> 2, t = lane & 3, l = g & 3;
     const uint32_t zero = 96, second = one ? 0 : kXRecBytes;
     LaneOffsets o;
@@ -480,6 +484,18 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
 
     LLVQ_TRACE_POINT(0)
     LLVQ_TRACE_CLOCK(7)
+    // The parameters the start of a CTA needs are read up front, all at once: a parameter line's first read by a
+    // multiprocessor costs some two hundred cycles, and the chain below would otherwise meet them one by one.
+    const CtaShare me = p.cta[blockIdx.x];
+    const int next_first = p.cta[blockIdx.x + 1].first;
+    const int h_nprob = p.nprob, h_units = p.units, h_groups = p.total_groups, h_panel = p.panel, h_npanels = p.npanels, h_tiles = p.tiles;
+    const FastDiv h_div_panel = p.div_panel, h_div_last = p.div_last;
+    const uint32_t h_group_bytes = p.group_bytes, h_tail_cells = (uint32_t)p.tail_cells;
+    const uint8_t *h_layout0 = p.prob[0].layout;
+    const float2 *h_cls_block = p.cls_block;
+    const uint4 *h_lane_table = p.lane_table;
+    asm volatile("" ::"r"(me.first), "r"(next_first), "r"(h_nprob), "r"(h_units), "r"(h_groups), "r"(h_panel), "r"(h_npanels), "r"(h_tiles),
+                 "r"(h_div_panel.mul), "r"(h_div_last.mul), "r"(h_group_bytes), "r"(h_tail_cells), "l"(h_layout0), "l"(h_cls_block), "l"(h_lane_table));
     // a warp's barriers are used by that warp alone: no block-wide synchronisation is needed for them; they
     // are set up before any load is in flight, so that the fence has nothing to wait for
     if (lane == 0) {
@@ -489,46 +505,35 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     }
     __syncwarp();
 
-    LLVQ_TRACE_CLOCK(3)
-    // x on its way into L2 (its values are read only after the wait below, through L2, which is where the
-    // previous kernel's writes to x land)
-    const int tab_entries = p.nprob * 1024;
-    uint32_t warm = 0;
-    for (int e = tid * 128; e < p.nb * 48 * p.batch; e += kThreads * 128) {
-        // a load whose value is not used: it brings the line into L2 and the translation into this
-        // multiprocessor's TLB, which a prefetch hint does not promise.  The register stays claimed until
-        // after the wait (settled() below), so nothing stalls on the load's return before then.
-        uint32_t w;
-        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(w) : "l"(reinterpret_cast<const char *>(p.x) + e));
-        warm |= w;
-    }
     // The CTA's units come from the host's plan; its warps share them evenly (the odd ones spread over the
-    // warps).  The blocks of x the CTA's units touch are those of the panels its range lies in.
-    const int cta_u0 = p.cta_first[blockIdx.x], cta_u1 = p.cta_first[blockIdx.x + 1];
-    const int cta_n = cta_u1 - cta_u0;
+    // warps).  The blocks of x the CTA's units touch, [blk_lo, blk_hi), are those of the panels its range lies in.
+    const int cta_u0 = me.first, cta_n = next_first - cta_u0;
     const int u0 = cta_u0 + (warp * cta_n + kWarps - 1) / kWarps;
     const int n_units = cta_u0 + ((warp + 1) * cta_n + kWarps - 1) / kWarps - u0;
-    const int blk_lo = panel_of_unit(p, cta_u0) * p.panel * kTileCells;
-    const int blk_hi = min(p.nb, (panel_of_unit(p, max(cta_u1 - 1, cta_u0)) + 1) * p.panel * kTileCells);
+    const int blk_lo = me.blk_lo, blk_hi = me.blk_hi;
     const uint32_t xs0 = smem_addr(xrec) - (uint32_t)blk_lo * kXRecBytes;     // address of block 0's record, were it there
 
-    // ROTATE: the coordinates [c_lo, c_hi) this CTA rotates are the whole rotation blocks that meet its blocks of x
-    int c_lo = 0, c_hi = 0;
-    if (ROTATE) {
-        const int mask = (1 << p.rot_log2) - 1;
-        c_lo = min(p.rot_n, (24 * blk_lo) & ~mask);
-        c_hi = min(p.rot_n, (24 * blk_hi + mask) & ~mask);
-        if (p.rot_negate)       // the sign flips are the caller's constants: on their way before the wait
-            for (int w = (c_lo >> 5) + tid; w < ((c_hi + 31) >> 5); w += kThreads) warm |= __ldg(p.rot_negate + w);
+    // consume side and issue side walk the same sequence of units.  The warp's first unit lies in the panel of
+    // the CTA's first unit (the plan names it) or, seldom, in a later one.
+    Cursor cc;
+    {
+        int panel = me.panel, first = panel * h_panel, w = min(h_panel, h_units - first), r = u0 - me.panel_first;
+        while (r >= h_groups * w && panel < h_npanels - 1) {
+            r -= h_groups * w;
+            panel++;
+            first += h_panel;
+            w = min(h_panel, h_units - first);
+        }
+        cc.panel = panel;
+        cc.end = first + w;
+        cc.group = panel == h_npanels - 1 ? fast_div(r, h_div_last, w) : fast_div(r, h_div_panel, w);
+        cc.col = first + (r - cc.group * w);
     }
-
-    LLVQ_TRACE_CLOCK(4)
-    // consume side and issue side walk the same sequence of units
-    Cursor cc = locate(p, u0), ic = cc;
+    Cursor ic = cc;
     int q = 0;
     const uint8_t *isrc = nullptr;                     // first byte of the issue side's row group
-    if (n_units > 0) isrc = group_base(p, ic.group, kSrcCell, q);
-    const uint32_t tail_bytes = (uint32_t)p.tail_cells * kSrcCell;
+    if (n_units > 0) isrc = h_nprob == 1 ? h_layout0 + (size_t)(uint32_t)ic.group * h_group_bytes : group_base(p, ic.group, q);
+    const uint32_t tail_bytes = h_tail_cells * kSrcCell;
 
     // The issue side's walk: inext is the next unit's first byte, ileft the units left in its stretch of its
     // row group.  next() hands out the unit's source and size and steps on.
@@ -538,7 +543,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         int left, done;
         uint32_t bytes;       // size of the next unit
     };
-    const int n_tiles_total = p.tiles;
+    const int n_tiles_total = h_tiles;
     Walk iw;
     iw.c = ic;
     iw.next = isrc + (size_t)ic.col * kSrcTile;      // the leftover blocks follow the last tile
@@ -552,7 +557,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             advance(p, w.c, 1);
             if (w.done < n_units) {
                 int qi;
-                w.next = group_base(p, w.c.group, kSrcCell, qi) + (size_t)w.c.col * kSrcTile;
+                w.next = group_base(p, w.c.group, qi) + (size_t)w.c.col * kSrcTile;
             }
             w.left = w.c.end - w.c.col;
         }
@@ -595,27 +600,66 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         // would pin every shared-memory read of the decode behind the copy.
     };
 
+    // Loads of the caller's constants and of the library's tables go out now and are used after the wait: this
+    // thread's class constants {1 / (4 sqrt m), parity - 16} (class = thread index), this lane's operand offsets,
+    // the first run's row scale, the rotation's sign flips; and x on its way into L2 with its translation into
+    // this multiprocessor's TLB (its values are read only after the wait, through L2, which is where the previous
+    // kernel's writes to x land).
+    static_assert(kThreads == 512, "one thread a class slot");
+    float2 my_class = make_float2(0.f, 0.f);
+    if (!COMPACT) asm volatile("ld.global.nc.v2.f32 {%0, %1}, [%2];" : "=f"(my_class.x), "=f"(my_class.y) : "l"(h_cls_block + tid));
+    uint4 lane_consts;
+    asm volatile("ld.global.nc.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(lane_consts.x), "=r"(lane_consts.y), "=r"(lane_consts.z), "=r"(lane_consts.w) : "l"(h_lane_table + lane));
+    const int my_row = (lane >> 2) + 8 * (lane & 3);       // the row of the group this lane ends up with
+    uint16_t first_scale_bits = 0;
+    if (n_units > 0) {
+        const GemvProblemDev &p0 = p.prob[q];
+        const int row0 = (cc.group - p0.group_begin) * kRowsPerGroup + my_row;
+        if (row0 < p0.rows) asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(first_scale_bits) : "l"(p0.row_scale + row0));
+    }
+    uint32_t warm = 0;
+    for (int e = tid * 128; e < p.nb * 48 * p.batch; e += kThreads * 128) {
+        // a load whose value is not used: the register stays claimed until after the wait (settled() below), so
+        // nothing stalls on the load's return before then
+        uint32_t w;
+        asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(w) : "l"(reinterpret_cast<const char *>(p.x) + e));
+        warm |= w;
+    }
+    // ROTATE: the coordinates [c_lo, c_hi) this CTA rotates are the whole rotation blocks that meet its blocks of x
+    int c_lo = 0, c_hi = 0;
+    if (ROTATE) {
+        const int mask = (1 << p.rot_log2) - 1;
+        c_lo = min(p.rot_n, (24 * blk_lo) & ~mask);
+        c_hi = min(p.rot_n, (24 * blk_hi + mask) & ~mask);
+        if (p.rot_negate)       // the sign flips are the caller's constants: on their way before the wait
+            for (int w = (c_lo >> 5) + tid; w < ((c_hi + 31) >> 5); w += kThreads) warm |= __ldg(p.rot_negate + w);
+    }
     if (!NO_WEIGHTS) {
 #pragma unroll
         for (int s = 0; s < kEarlySlots; s++) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
     }
-    LLVQ_TRACE_CLOCK(5)
-    // what the loop needs that does not depend on the previous kernel: this lane's constants, and the scale of
-    // its row in the first run (the scales, like the records, are the caller's weights)
     const uint32_t lane16 = 16 * lane, lane4 = 4 * lane, pair16 = 16 * (lane >> 1);
     const int tiles = p.tiles;
-    const LaneOffsets lo = lane_offsets(lane, false);
     const bool odd_lane = lane & 1, high_lane = lane & 2;
     const float limb_scale = odd_lane ? 65536.f : 1.f;     // this lane's limb pair: 256^0,1 or 256^2,3
-    const int my_row = (lane >> 2) + 8 * (lane & 3);       // the row of the group this lane ends up with
     const uint32_t tab0 = smem_addr(tab);
-    q = n_units > 0 ? find_problem(p, cc.group) : 0;
-    float first_row_scale = 0.f;
-    if (n_units > 0) {
-        const GemvProblemDev &p0 = p.prob[q];
-        const int row0 = (cc.group - p0.group_begin) * kRowsPerGroup + my_row;
-        if (row0 < p0.rows) first_row_scale = __half2float(p0.row_scale[row0]);
-    }
+    // the block constants of every matrix of the launch: (class | gain << 9) -> {gain / (4 sqrt m), parity - 16}
+    // (13-byte layout: the header byte is shell | parity << 4 | gain << 5 - 64 entries a matrix)
+    auto build_tables = [&]() {
+        if (COMPACT) {
+            for (int e = tid; e < p.nprob * 64; e += kThreads) {
+                const uint32_t shell = e & 15u;
+                const GemvProblemDev &pe = p.prob[e >> 6];
+                tab[(e >> 6) * 1024 + (e & 63)] = make_float2(p.shell_inv_norm[shell] * ((e & 32) ? pe.gain1 : pe.gain0),
+                                                             __int_as_float(shell ? ((e >> 4) & 1) - 16 : 0));
+            }
+        } else {
+            for (int m = 0; m < p.nprob; m++) {
+                tab[m * 1024 + tid] = make_float2(my_class.x * p.prob[m].gain0, my_class.y);
+                tab[m * 1024 + 512 + tid] = make_float2(my_class.x * p.prob[m].gain1, my_class.y);
+            }
+        }
+    };
     LLVQ_TRACE_CLOCK(6)
     // let the next kernel in the stream start its own prefetch, then wait for the previous one:
     // x, y and the reduction scratch may still be in use by it
@@ -653,13 +697,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             if (base == 0) {
                 for (int b = tid; b < blk_hi - blk_lo; b += kThreads)
                     asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(smem_addr(xrec) + b * kXRecBytes + 96), "r"(0) : "memory");
-                for (int e = tid; e < tab_entries; e += kThreads) {
-                    const int c = e & 511;
-                    const uint32_t shell = (p.cls_shell_nibbles[c >> 3] >> (4 * (c & 7))) & 15u;
-                    const int odd = (int)((p.cls_odd_bits[c >> 5] >> (c & 31)) & 1u);
-                    const GemvProblemDev &pe = p.prob[e >> 10];
-                    tab[e] = make_float2(p.shell_inv_norm[shell] * ((e & 512) ? pe.gain1 : pe.gain0), __int_as_float(shell ? odd - 16 : 0));
-                }
+                build_tables();
             }
 #pragma unroll
             for (int i = 0; i < 4; i++) {
@@ -735,24 +773,7 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                         const int jj = BATCH == 1 ? 0 : b / (blk_hi - blk_lo), bb = b - jj * (blk_hi - blk_lo);
                         asm volatile("st.shared.v4.u32 [%0], {%1, %1, %1, %1};" ::"r"(smem_addr(xrec) + jj * xrec_stride + bb * kXRecBytes + 96), "r"(0) : "memory");
                     }
-                    // block constants of every matrix of the launch: (class | gain << 9) -> {gain / (4 sqrt m), parity - 16},
-                    // from the class constants in the kernel's parameters
-                    if (COMPACT) {
-                        // 13-byte layout: the header byte is shell | parity << 4 | gain << 5 - 64 entries a matrix
-                        for (int e = tid; e < p.nprob * 64; e += kThreads) {
-                            const uint32_t shell = e & 15u;
-                            const GemvProblemDev &pe = p.prob[e >> 6];
-                            tab[(e >> 6) * 1024 + (e & 63)] = make_float2(p.shell_inv_norm[shell] * ((e & 32) ? pe.gain1 : pe.gain0),
-                                                                         __int_as_float(shell ? ((e >> 4) & 1) - 16 : 0));
-                        }
-                    } else
-                    for (int e = tid; e < tab_entries; e += kThreads) {
-                        const int c = e & 511;
-                        const uint32_t shell = (p.cls_shell_nibbles[c >> 3] >> (4 * (c & 7))) & 15u;
-                        const int odd = (int)((p.cls_odd_bits[c >> 5] >> (c & 31)) & 1u);
-                        const GemvProblemDev &pe = p.prob[e >> 10];
-                        tab[e] = make_float2(p.shell_inv_norm[shell] * ((e & 512) ? pe.gain1 : pe.gain0), __int_as_float(shell ? odd - 16 : 0));
-                    }
+                    build_tables();
                 }
 #pragma unroll
                 for (int i = 0; i < 4; i++) {
@@ -787,6 +808,9 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         }
         __syncthreads();                               // publishes the x records
     }
+    const LaneOffsets lo = {lane_consts.x, lane_consts.y, lane_consts.z, lane_consts.w};
+    float first_row_scale;
+    asm volatile("cvt.f32.f16 %0, %1;" : "=f"(first_row_scale) : "h"(first_scale_bits));
     LLVQ_TRACE_POINT(3)
     LLVQ_TRACE_CLOCK(2)
 
@@ -991,7 +1015,9 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         }
         if (advance(p, cc, run) && cc.panel < p.npanels) q = find_problem(p, cc.group);
     }
+    LLVQ_TRACE_CLOCK(14)
     settle(p, handed);
+    LLVQ_TRACE_CLOCK(15)
 
     LLVQ_TRACE_POINT(5)
     if (failed) {
@@ -1039,7 +1065,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_onehot_kernel(const __grid_c
     int u0, n_units;
     warp_range(p, warp, u0, n_units);
     int group = u0 / p.units, k = u0 - group * p.units, q = 0;
-    const uint8_t *grp = n_units > 0 ? group_base(p, group, kOneHotCellBytes, q) : nullptr;
+    const uint8_t *grp = n_units > 0 ? group_base(p, group, q) : nullptr;
     long long sum = 0;
     int count = 0;
     for (int n = 0; n < n_units; n++) {
@@ -1069,7 +1095,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_onehot_kernel(const __grid_c
             if (k == p.units) {
                 k = 0;
                 group++;
-                if (group < p.total_groups) grp = group_base(p, group, kOneHotCellBytes, q);
+                if (group < p.total_groups) grp = group_base(p, group, q);
             }
         }
     }
@@ -1212,12 +1238,20 @@ __global__ void __launch_bounds__(256) dequant_kernel(int layout, const uint8_t 
 
 }  // namespace
 
+void gemv_lane_table(uint32_t (*out)[4]) {
+    for (int lane = 0; lane < 32; lane++) {
+        const LaneOffsets o = lane_offsets(lane, false);
+        out[lane][0] = o.b0; out[lane][1] = o.b1; out[lane][2] = o.b2; out[lane][3] = o.xs;
+    }
+}
+
 GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
     GemvLaunch g;
     // one CTA a multiprocessor
     g.grid = p.total_units < sm_count ? p.total_units : sm_count;
     p.units_base = p.total_units / (g.grid * kWarps);
     p.units_rem = p.total_units % (g.grid * kWarps);
+    p.group_bytes = (uint32_t)p.nb * (uint32_t)(layout == LLVQ_ONEHOT ? kOneHotCellBytes : (layout == LLVQ_PLANES13 ? kCell13Bytes : kCellBytes));
     if (layout == LLVQ_ONEHOT) {
         g.smem = ((size_t)p.nb * 48 + 127) / 128 * 128;
         return g;
@@ -1242,25 +1276,31 @@ GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
         if (lead > 0.6 * mean) lead = 0.6 * mean;
         const double skew = mean > 0 ? lead / mean : 0.0;
         double acc = 0.0;
-        p.cta_first[0] = 0;
+        p.cta[0].first = 0;
         for (int c = 0; c < g.grid; c++) {
             const double w = g.grid > 1 ? 1.0 + skew * (1.0 - 2.0 * c / (g.grid - 1)) : 1.0;
             acc += mean * w;
             int f = (int)(acc + 0.5);
-            if (f < p.cta_first[c]) f = p.cta_first[c];
+            if (f < p.cta[c].first) f = p.cta[c].first;
             if (f > p.total_units) f = p.total_units;
-            p.cta_first[c + 1] = f;
+            p.cta[c + 1].first = f;
         }
-        p.cta_first[g.grid] = p.total_units;
+        p.cta[g.grid].first = p.total_units;
+        p.cta[g.grid].blk_lo = p.cta[g.grid].blk_hi = p.cta[g.grid].panel = 0;
+        p.cta[g.grid].panel_first = 0;
     }
-    // the widest stretch of x a CTA meets: its units lie in consecutive panels
+    // the stretch of x a CTA meets: the whole panels its units lie in (consecutive ones)
     p.xblocks = 0;
     p.rot_span = 0;
     for (int c = 0; c < g.grid; c++) {
-        const int f0 = p.cta_first[c], f1 = p.cta_first[c + 1];
+        const int f0 = p.cta[c].first, f1 = p.cta[c + 1].first;
         const int lo = panel_of_unit(p, f0) * p.panel * kTileCells;
         int hi = (panel_of_unit(p, f1 - 1 > f0 ? f1 - 1 : f0) + 1) * p.panel * kTileCells;
         if (hi > p.nb) hi = p.nb;
+        p.cta[c].blk_lo = (uint16_t)lo;
+        p.cta[c].blk_hi = (uint16_t)hi;
+        p.cta[c].panel = (uint16_t)panel_of_unit(p, f0);
+        p.cta[c].panel_first = p.cta[c].panel * (p.total_groups * p.panel);
         if (hi - lo > p.xblocks) p.xblocks = hi - lo;
         if (p.rot_log2 > 0) {
             // the whole rotation blocks that meet the CTA's blocks of x (the kernel computes the same)
@@ -1379,10 +1419,14 @@ constexpr int kStaticMaxDevices = 64;
 
 static __device__ __align__(256) unsigned long long g_static_accum[kStaticMaxRows];   // 512 KiB of scratch
 static __device__ __align__(256) int g_static_error[64];
+static __device__ __align__(256) float2 g_static_cls_block[llvq::kClassSlots];   // {1 / (4 sqrt m), parity - 16} of every class slot
+static __device__ __align__(256) uint4 g_static_lane_table[32];                  // a lane's operand offsets
 
 struct StaticDevice {
     bool ready = false;
     unsigned long long *accum = nullptr;
+    float2 *cls_block = nullptr;
+    uint4 *lane_table = nullptr;
     uint32_t cls_shell_nibbles[64], cls_odd_bits[16];      // class constants (host copies, handed to every launch)
     float shell_inv_norm[16];
     int *error = nullptr;
@@ -1400,6 +1444,12 @@ int static_setup(int device, StaticDevice &d) {
     memcpy(d.cls_shell_nibbles, host.cls_shell_nibbles, sizeof d.cls_shell_nibbles);
     memcpy(d.cls_odd_bits, host.cls_odd_bits, sizeof d.cls_odd_bits);
     memcpy(d.shell_inv_norm, host.shell_inv_norm, sizeof d.shell_inv_norm);
+    uint32_t lanes[32][4];
+    llvq::gemv_lane_table(lanes);
+    if (cudaGetSymbolAddress((void **)&d.cls_block, g_static_cls_block) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaGetSymbolAddress((void **)&d.lane_table, g_static_lane_table) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaMemcpy(d.cls_block, host.cls_block.data(), sizeof(float2) * llvq::kClassSlots, cudaMemcpyHostToDevice) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaMemcpy(d.lane_table, lanes, sizeof lanes, cudaMemcpyHostToDevice) != cudaSuccess) return LLVQ_ECUDA;
     if (cudaMemset(d.accum, 0, sizeof(unsigned long long) * kStaticMaxRows) != cudaSuccess) return LLVQ_ECUDA;
     if (cudaMemset(d.error, 0, sizeof(int) * 64) != cudaSuccess) return LLVQ_ECUDA;
     if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return LLVQ_ECUDA;
@@ -1462,6 +1512,8 @@ extern "C" int llvq_gemv_static(const void *layout_buf, const void *row_scale, c
     memcpy(p.cls_odd_bits, d.cls_odd_bits, sizeof p.cls_odd_bits);
     memcpy(p.shell_inv_norm, d.shell_inv_norm, sizeof p.shell_inv_norm);
     p.error = d.error;
+    p.cls_block = d.cls_block;
+    p.lane_table = d.lane_table;
     const llvq::GemvLaunch g = llvq::gemv_plan(LLVQ_PLANES, p, d.sm_count);
     if (g.smem + 1024 > (size_t)d.max_smem_optin) return LLVQ_ESIZE;
     return llvq::launch_gemv(LLVQ_PLANES, p, g, false, true, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;

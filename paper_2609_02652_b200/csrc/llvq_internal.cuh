@@ -29,6 +29,8 @@ struct DeviceTables {
     const uint32_t *cls_parity;      // 512
     const float *cls_value;          // 512 x 8
     const uint8_t *cls_dist;         // 512 x 8
+    const float2 *cls_block;         // 512 x {1 / (4 sqrt m), parity - 16}
+    const uint4 *lane_table;         // 32 x {b0, b1, b2, xs}: a lane's operand offsets in two consecutive x records
     int weight_offset[25];
     int num_classes;
     uint64_t num_points;
@@ -59,6 +61,15 @@ struct GemvProblemDev {
     int qexp_base;     // log2 of this matrix's fixed-point quantum, before the exponent of max |x| is added
 };
 
+// A CTA's share of a launch, planned on the host: its first unit, the panel that unit lies in and the panel's first
+// unit, and the blocks of x [blk_lo, blk_hi) its units touch (the whole panels its range of units meets).
+struct CtaShare {
+    int first;
+    int panel_first;
+    uint16_t blk_lo, blk_hi;
+    uint16_t panel, pad;
+};
+
 struct GemvParams {
     GemvProblemDev prob[LLVQ_MAX_GROUP];
     int nprob;
@@ -73,11 +84,14 @@ struct GemvParams {
     int panel, npanels;          // unit columns a panel, panels (set by gemv_plan; the 14-byte layout's order of work)
     FastDiv div_panel_units, div_panel, div_last;   // by total_groups * panel, by panel, by the last panel's width
     int xblocks;                 // most blocks of x any CTA needs (set by gemv_plan)
-    int cta_first[kMaxGridCtas + 1];   // first unit of every CTA of the grid, and the total (set by gemv_plan)
+    uint32_t group_bytes;        // bytes of a row group's records (set by gemv_plan)
+    CtaShare cta[kMaxGridCtas + 1];    // the share of every CTA of the grid; [grid].first is the total (set by gemv_plan)
     unsigned long long *accum;   // total_groups x 32 fixed-point row accumulators (context scratch, zero between launches)
     const float *cls_scale;
     const uint32_t *cls_parity;
     const float *cls_value;
+    const float2 *cls_block;     // 512 x {1 / (4 sqrt m), parity - 16 as an integer's bits}; zeros for an unused class slot
+    const uint4 *lane_table;     // 32 x this lane's offsets of its operand words in the x records of a half-step
     // the class constants the 14-byte GEMV needs, in the parameters themselves (no load from global memory
     // stands between a CTA's start and its block-constant table)
     uint32_t cls_shell_nibbles[64];   // nibble c & 7 of word c >> 3: shell of class c, 0 if unused
@@ -124,6 +138,7 @@ struct GemvLaunch {
 };
 // Completes the launch geometry in `p` (order of work, shares of x) and returns grid and dynamic shared memory.
 GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count);
+void gemv_lane_table(uint32_t (*out)[4]);      // fills the 32 entries of DeviceTables::lane_table (host)
 cudaError_t launch_gemv(int layout, const GemvParams &p, const GemvLaunch &g, bool no_weights, bool pdl, cudaStream_t s);
 cudaError_t launch_wait_limit_selftest(const llvq_ctx *ctx, cudaStream_t s);
 cudaError_t launch_gemv_fp16(const __half *W, const __half *x, float *y, int64_t rows, int64_t k, cudaStream_t s);

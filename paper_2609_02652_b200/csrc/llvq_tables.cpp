@@ -175,9 +175,11 @@ bool build_tables(HostTables &t) {
     std::memset(t.cls_shell_nibbles, 0, sizeof t.cls_shell_nibbles);
     std::memset(t.cls_odd_bits, 0, sizeof t.cls_odd_bits);
     for (int m = 0; m < 16; m++) t.shell_inv_norm[m] = (m >= 2 && m <= 12) ? (float)(1.0 / (4.0 * std::sqrt((double)m))) : 0.f;
+    t.cls_block.assign(kClassSlots, HostTables::BlockConst{0.f, 0});
     for (size_t c = 0; c < all.size(); c++) {
         t.cls_shell_nibbles[c >> 3] |= (uint32_t)all[c].shell << (4 * (c & 7));
         if (all[c].odd) t.cls_odd_bits[c >> 5] |= 1u << (c & 31);
+        t.cls_block[c] = HostTables::BlockConst{t.shell_inv_norm[all[c].shell], (all[c].odd ? 1 : 0) - 16};
     }
     t.base[all.size()] = running;
     t.num_points = running;

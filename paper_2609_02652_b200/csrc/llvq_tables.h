@@ -40,6 +40,8 @@ struct HostTables {
     uint32_t cls_shell_nibbles[64];        // nibble c & 7 of word c >> 3: shell of class c (2..12), 0 if unused
     uint32_t cls_odd_bits[16];             // bit c & 31 of word c >> 5: class c is of the odd type
     float shell_inv_norm[16];              // [m] = 1 / (4 sqrt(m)) for m = 2..12, else 0
+    struct BlockConst { float inv_norm; int32_t offset; };
+    std::vector<BlockConst> cls_block;     // kClassSlots: {1 / (4 sqrt(shell)), parity - 16}; zeros if unused
     std::vector<float> cls_value;          // kClassSlots * 8: dist[l] / (4 sqrt(shell)), l < 5
     std::vector<uint8_t> cls_dist;         // kClassSlots * 8: dist[l]
 };
