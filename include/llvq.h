@@ -96,7 +96,8 @@ extern "C" {
 #define LLVQ_EALIGN (-2) /* a device pointer is not aligned as documented                   */
 #define LLVQ_ESIZE (-3)  /* a buffer or the context's scratch is too small for the request  */
 #define LLVQ_ECUDA (-4)  /* a CUDA runtime call failed                                      */
-#define LLVQ_ETIMEOUT (-5) /* a bounded wait inside a kernel ran out (llvq_status only)         */
+#define LLVQ_ETIMEOUT (-5) /* a bounded wait inside a kernel ran out (llvq_status, llvq_static_status) */
+#define LLVQ_EINDEX (-6) /* an expanded code word named no point of the ball (llvq_status only) */
 
 #define LLVQ_MAX_GROUP 8       /* matrices in one grouped launch                             */
 #define LLVQ_MAX_K 98304       /* largest k_padded the GEMV accepts                          */
@@ -123,15 +124,20 @@ typedef struct llvq_rotation {
 
 /* Builds the class, index-base and Golay tables on the host, uploads them to `device`, and
  * allocates the context's reduction scratch (scratch_bytes; 0 = default 8 MiB, eight bytes a row
- * of the largest launch, rows rounded up to 32 per matrix).  Synchronous. */
+ * of the largest launch, rows rounded up to 32 per matrix).  Synchronous.  (The third argument is
+ * this library's addition to the call the paper's statement of the problem implies: the scratch is
+ * the one thing whose size depends on the caller's largest launch.) */
 int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes);
 void llvq_destroy(llvq_ctx *ctx);
 const char *llvq_strerror(int code);
 
 /* Synchronises `stream` and reports whether any GEMV launched on this context since the last
  * call gave up on one of its bounded waits (LLVQ_ETIMEOUT; the flag and the scratch are then
- * reset).  Every wait inside the kernels on an asynchronous copy has a time limit of about a second;
- * none can spin forever, and none traps. */
+ * reset), else whether any llvq_expand on this context since the last call met a code word that
+ * names no point (LLVQ_EINDEX; the count is then reset - the 512-slot class table exists so that
+ * such a code can never index out of bounds [Sec. 2.3], and this is how a caller that passed no
+ * bad_count learns of it).  Every wait inside the kernels on an asynchronous copy has a time limit
+ * of about a second; none can spin forever, and none traps. */
 int llvq_status(llvq_ctx *ctx, void *stream);
 
 /* Enqueues a one-warp kernel that waits, with a limit of about a millisecond, on a barrier nothing
@@ -142,7 +148,12 @@ int llvq_selftest_wait_limit(llvq_ctx *ctx, void *stream);
 
 /* The GEMV is launched with programmatic dependent launch (on by default): its record prefetch
  * starts while the previous kernel of the stream drains, and it waits for that kernel before it
- * touches x, y or the scratch.  enabled = 0 launches it as an ordinary kernel. */
+ * touches x, y or the scratch.  What it reads AHEAD of that wait are the caller's weights: the layout
+ * buffer, the row scales and a rotation's negate_bits.  They must therefore be complete before the
+ * kernel that precedes the GEMV on the stream starts (weights loaded once satisfy this trivially);
+ * llvq_expand takes care of it by itself (the next GEMV on the context is launched as an ordinary
+ * kernel); a caller whose own kernel writes scales or records right before a GEMV disables the
+ * feature.  enabled = 0 launches every GEMV as an ordinary kernel. */
 int llvq_set_pdl(llvq_ctx *ctx, int enabled);
 
 /* Host queries.  Number of classes (301), points in the ball, and first index of class c
@@ -157,12 +168,17 @@ int llvq_layout_bytes(int layout, int64_t rows, int64_t k_padded, size_t *bytes)
  * (128-byte aligned, at least llvq_layout_bytes).  A code that names no point (index not below
  * the number of points, or bits above bit 47 set) becomes the empty record (class 511, all
  * fields zero) and, if bad_count is not null, adds one to *bad_count (device uint32, which the
- * caller zeroes).  Bit-exact by construction: integer arithmetic only. */
+ * caller zeroes).  The context counts such codes as well, whether or not bad_count is given: the next
+ * llvq_status returns LLVQ_EINDEX if any expansion since the last one met one.  Bit-exact by construction:
+ * integer arithmetic only.  The GEMV enqueued next on this context is launched without programmatic dependent
+ * launch, so that it cannot read records ahead of this expansion (see llvq_set_pdl). */
 int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, int64_t nb,
                 void *layout_out, size_t out_bytes, uint32_t *bad_count, void *stream);
 
 /* [Sec. 2.3] y[row] = row_scale[row] * sum_b gain[g_b] / (4 sqrt(m_b)) * sum_i x_b,i * x[24b+i],
- * m_b the shell of block b's class.  gain is a HOST pointer to two floats.  x is fp16, 16-byte
+ * m_b the shell of block b's class.  gain is a HOST pointer to two floats; the larger of their magnitudes
+ * must be zero or lie in [2^-60, 2^60) (LLVQ_EINVAL otherwise: the fixed-point quantum is a power of two
+ * formed from its exponent).  x is fp16, 16-byte
  * aligned; y is f32; x must be finite.  LLVQ_PLANES: x is taken as fixed point on a scale set by
  * the largest |x| (X_i = rint(x_i 2^F), |X_i| < 2^29; exact for every x_i within 2^-18 of the
  * largest, rounded to within 2^-29 of the largest below that), the inner sums over a block are integer and
@@ -227,6 +243,16 @@ int llvq_gemv_rotated(llvq_ctx *ctx, const llvq_problem *problems, int n, const 
  * It calls no cudaMalloc, cudaFree or other allocating routine. */
 int llvq_gemv_static(const void *layout_buf, const void *row_scale, const float *gain, const void *x, float *y,
                      int64_t rows, int64_t k_padded, void *stream);
+
+/* llvq_status for llvq_gemv_static (which has no context to ask): synchronises `stream` and reports whether a
+ * llvq_gemv_static launch on the CURRENT device gave up on one of its bounded waits since the last call
+ * (LLVQ_ETIMEOUT).  The flag and the built-in scratch are then cleared (two memsets, no allocation), so the
+ * calls that follow start clean; without this call such a time-out would go unseen and leave partial sums in
+ * the shared scratch.  llvq_static_selftest_wait_limit enqueues the one-warp kernel of
+ * llvq_selftest_wait_limit against that flag: the next llvq_static_status returns LLVQ_ETIMEOUT, the one after
+ * LLVQ_OK. */
+int llvq_static_status(void *stream);
+int llvq_static_selftest_wait_limit(void *stream);
 
 /* [Table "layout scale", FP16 control] y = W x, W fp16 row-major rows x k (k a multiple of 8,
  * W and x 16-byte aligned), f32 accumulation, f32 y. */

@@ -23,7 +23,7 @@ _lib = None
 SYMBOLS = (
     "llvq_create", "llvq_destroy", "llvq_strerror", "llvq_status", "llvq_selftest_wait_limit", "llvq_set_pdl", "llvq_num_classes", "llvq_class_base", "llvq_layout_bytes",
     "llvq_expand", "llvq_gemv", "llvq_gemv_batch", "llvq_gemv_plan", "llvq_gemv_grouped", "llvq_gemv_static", "llvq_gemv_fp16", "llvq_gemv_noweights", "llvq_dequant_fp16",
-    "llvq_decode_i8", "llvq_rotate", "llvq_rotate_block", "llvq_gemv_rotated",
+    "llvq_decode_i8", "llvq_rotate", "llvq_rotate_block", "llvq_gemv_rotated", "llvq_static_status", "llvq_static_selftest_wait_limit",
 )
 
 
@@ -76,6 +76,8 @@ def load() -> ctypes.CDLL:
         L.llvq_decode_i8.argtypes = [vp, ci, vp, vp, vp, i64, i64, vp]
         L.llvq_rotate.argtypes = [vp, vp, vp, vp, i64, i64, vp]
         L.llvq_gemv_rotated.argtypes = [vp, ctypes.POINTER(Problem), ci, vp, i64, ctypes.POINTER(Rotation), vp]
+        L.llvq_static_status.argtypes = [vp]
+        L.llvq_static_selftest_wait_limit.argtypes = [vp]
         L.llvq_rotate_block.argtypes = [i64, i64]
         L.llvq_rotate_block.restype = i64
         for name in SYMBOLS:
@@ -139,7 +141,8 @@ def destroy(ctx: Context) -> None:
 
 
 def status(ctx: Context, stream=None) -> None:
-    """Synchronises the stream; raises if a kernel on this context gave up on a bounded wait."""
+    """Synchronises the stream; raises LlvqError(-5) if a kernel on this context gave up on a bounded wait, else
+    LlvqError(-6) if an expansion since the last call met a code word that names no point."""
     _check(load().llvq_status(ctx.ptr, _stream(stream)), "llvq_status")
 
 
@@ -220,6 +223,17 @@ def gemv_static(layout_buf: torch.Tensor, row_scale: torch.Tensor, gain, x: torc
                                    _gain(gain), _dev(x, torch.float16, "x"), _dev(y, torch.float32, "y"), int(rows),
                                    int(k_padded), _stream(stream)), "llvq_gemv_static")
     return y
+
+
+def static_status(stream=None) -> None:
+    """llvq_static_status: synchronises the stream; raises LlvqError(-5) if a llvq_gemv_static launch on the current
+    device gave up on a bounded wait (the built-in flag and scratch are then cleared)."""
+    _check(load().llvq_static_status(_stream(stream)), "llvq_static_status")
+
+
+def static_selftest_wait_limit(stream=None) -> None:
+    """Enqueues the bounded-wait self-test against the static entry point's flag; the next static_status() raises."""
+    _check(load().llvq_static_selftest_wait_limit(_stream(stream)), "llvq_static_selftest_wait_limit")
 
 
 def make_problems(problems) -> ctypes.Array:

@@ -24,6 +24,13 @@ inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_
 
 size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// The fixed-point quantum is a power of two formed from the exponent of the larger gain: gains whose larger
+// magnitude lies outside [2^-60, 2^60) (zero excepted: a matrix of zero gain is all zeros) are refused.
+bool gain_in_range(const float *gain) {
+    const float gm = std::fmax(std::fabs(gain[0]), std::fabs(gain[1]));
+    return gm == 0.f || (gm >= 8.673617379884035e-19f && gm < 1.152921504606847e18f);
+}
+
 int layout_cell_bytes(int layout) { return layout == LLVQ_PLANES ? kCellBytes : (layout == LLVQ_PLANES13 ? kCell13Bytes : kOneHotCellBytes); }
 
 }  // namespace
@@ -38,6 +45,7 @@ const char *llvq_strerror(int code) {
         case LLVQ_ESIZE: return "buffer or context scratch too small";
         case LLVQ_ECUDA: return "CUDA runtime error";
         case LLVQ_ETIMEOUT: return "a bounded wait inside a kernel ran out; the affected outputs are incomplete";
+        case LLVQ_EINDEX: return "a code word named no point of the ball (index out of range or bits above bit 47 set); its record is empty";
         default: return "unknown error";
     }
 }
@@ -53,10 +61,7 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
     llvq_ctx *ctx = new (std::nothrow) llvq_ctx();
     if (!ctx) return LLVQ_ECUDA;
     ctx->device = device;
-    ctx->table_blob = nullptr; ctx->accum = nullptr; ctx->error = nullptr; ctx->use_pdl = 1;
-#ifdef LLVQ_TRACE
-    ctx->trace = nullptr; ctx->trace_launch = 0;
-#endif
+    ctx->table_blob = nullptr; ctx->accum = nullptr; ctx->error = nullptr; ctx->bad_codes = nullptr; ctx->use_pdl = 1; ctx->weights_dirty = 0;
     if (!build_tables(ctx->host)) { delete ctx; return LLVQ_EINVAL; }
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return LLVQ_ECUDA; }
@@ -100,10 +105,11 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
     ctx->accum_slots = scratch_bytes / 8;
     if (cudaMalloc(&ctx->accum, ctx->accum_slots * 8) != cudaSuccess ||
         cudaMemset(ctx->accum, 0, ctx->accum_slots * 8) != cudaSuccess ||
-        cudaMalloc(&ctx->error, 4) != cudaSuccess || cudaMemset(ctx->error, 0, 4) != cudaSuccess) {
+        cudaMalloc(&ctx->error, 8) != cudaSuccess || cudaMemset(ctx->error, 0, 8) != cudaSuccess) {
         llvq_destroy(ctx);
         return LLVQ_ECUDA;
     }
+    ctx->bad_codes = reinterpret_cast<uint32_t *>(ctx->error + 1);
     if (gemv_configure(ctx) != 0 || rotate_configure() != 0 || cudaDeviceSynchronize() != cudaSuccess) { llvq_destroy(ctx); return LLVQ_ECUDA; }
     *out = ctx;
     return LLVQ_OK;
@@ -122,13 +128,17 @@ int llvq_status(llvq_ctx *ctx, void *stream) {
     if (!ctx) return LLVQ_EINVAL;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
-    int flag = 0;
+    int flags[2] = {0, 0};                             // {a wait ran out, codes that named no point}
     if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return LLVQ_ECUDA;
-    if (cudaMemcpy(&flag, ctx->error, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return LLVQ_ECUDA;
-    if (flag) {
+    if (cudaMemcpy(flags, ctx->error, 8, cudaMemcpyDeviceToHost) != cudaSuccess) return LLVQ_ECUDA;
+    if (flags[0]) {
         cudaMemset(ctx->error, 0, 4);
         cudaMemset(ctx->accum, 0, ctx->accum_slots * 8);   // an abandoned reduction leaves sums behind
         return LLVQ_ETIMEOUT;
+    }
+    if (flags[1]) {
+        cudaMemset(ctx->bad_codes, 0, 4);
+        return LLVQ_EINDEX;
     }
     return LLVQ_OK;
 }
@@ -145,15 +155,6 @@ int llvq_set_pdl(llvq_ctx *ctx, int enabled) {
     ctx->use_pdl = enabled ? 1 : 0;
     return LLVQ_OK;
 }
-
-#ifdef LLVQ_TRACE
-// debug builds only: eight 64-bit timestamps a warp a launch are stored at `buf`
-int llvq_trace_set(llvq_ctx *ctx, unsigned long long *buf) {
-    ctx->trace = buf;
-    ctx->trace_launch = 0;
-    return LLVQ_OK;
-}
-#endif
 
 int llvq_num_classes(const llvq_ctx *ctx) { return ctx ? ctx->host.num_classes : LLVQ_EINVAL; }
 
@@ -180,6 +181,9 @@ int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, 
     if (rows * nb > ((int64_t)1 << 36)) return LLVQ_ESIZE;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
+    // the GEMV reads records ahead of its wait for the previous kernel of the stream: the next one on this context
+    // is launched as an ordinary kernel, so that it cannot overtake this expansion
+    ctx->weights_dirty = 1;
     return launch_expand(ctx, layout, codes, rows, nb, layout_out, bad_count, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
 }
 
@@ -254,6 +258,8 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
     if (groups > ((int64_t)1 << 26) || p.units > 2047 || groups * p.units > 0x7fffffffll) return LLVQ_ESIZE;
     if ((size_t)groups * 32 * (size_t)batch > ctx->accum_slots) return LLVQ_ESIZE;
     if (!(gain_max < 3.0e38f)) return LLVQ_EINVAL;
+    for (int i = 0; i < n; i++)
+        if (!gain_in_range(problems[i].gain)) return LLVQ_EINVAL;
     // quantum of the fixed-point row accumulators, per matrix so that grouping does not change it:
     // a unit sums at most four blocks, each bounded by max|gain| * sqrt(24) * max|x| < 2^ge * 5 * 2^xe;
     // 4 * 5 < 2^5, and the unit value is kept under 2^39 quanta (see deliver() in llvq_gemv.cu), which
@@ -287,15 +293,13 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
         p.rot_negate = rot->negate_bits;
         p.rot_scale = std::ldexp(1.0 / std::sqrt((double)((int64_t)1 << l)), -24);
     }
-#ifdef LLVQ_TRACE
-    p.trace = ctx->trace;
-    p.trace_launch = ctx->trace ? ctx->trace_launch++ : 0;
-#endif
     const GemvLaunch g = gemv_plan(layout, p, ctx->sm_count);
     if (g.smem + 1024 > (size_t)ctx->max_smem_optin) return LLVQ_ESIZE;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
-    return launch_gemv(layout, p, g, no_weights, ctx->use_pdl != 0, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+    const bool pdl = ctx->use_pdl != 0 && !ctx->weights_dirty;
+    ctx->weights_dirty = 0;
+    return launch_gemv(layout, p, g, no_weights, pdl, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
 }
 
 int llvq_gemv(llvq_ctx *ctx, int layout, const void *layout_buf, const void *row_scale, const float *gain, const void *x,

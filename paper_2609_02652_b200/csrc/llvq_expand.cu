@@ -140,7 +140,7 @@ __device__ __forceinline__ uint32_t bytes4(uint32_t a, uint32_t b) {
 // COMPACT: the 13-byte layout - the same code words, the header one byte: shell | parity << 4 | gain << 5.
 template <bool COMPACT>
 __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, const uint64_t *__restrict__ codes, int64_t rows, int64_t nb,
-                                                            uint8_t *__restrict__ out, uint32_t *bad_count) {
+                                                            uint8_t *__restrict__ out, uint32_t *bad_count, uint32_t *ctx_bad) {
     __shared__ uint32_t nat_all[8][4][4][32];              // [warp][block of the piece][word 0..2, header][row]
     const int64_t tiles = nb / kTileCells, left = nb % kTileCells;
     const int64_t pieces = tiles + (left >= 2 ? 1 : 0) + (left & 1);
@@ -226,11 +226,14 @@ __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, cons
             else *reinterpret_cast<uint32_t *>(one + 384 + 4 * (lane >> 1)) = hw;
         }
     }
-    if (bad && bad_count) atomicAdd(bad_count, (uint32_t)bad);
+    if (bad) {
+        atomicAdd(ctx_bad, (uint32_t)bad);               // the context's own count: llvq_status reports it
+        if (bad_count) atomicAdd(bad_count, (uint32_t)bad);
+    }
 }
 
 __global__ void __launch_bounds__(256) expand_onehot_kernel(DeviceTables T, const uint64_t *__restrict__ codes, int64_t rows, int64_t nb,
-                                                            uint8_t *__restrict__ out, uint32_t *bad_count) {
+                                                            uint8_t *__restrict__ out, uint32_t *bad_count, uint32_t *ctx_bad) {
     const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int lane = (int)(gid & 31);
     const int64_t cell_id = gid >> 5;
@@ -262,7 +265,10 @@ __global__ void __launch_bounds__(256) expand_onehot_kernel(DeviceTables T, cons
     cell[2 * 32 + lane] = mask[1];
     cell[3 * 32 + lane] = mask[2];
     cell[4 * 32 + lane] = mask[3];
-    if (!ok && bad_count) atomicAdd(bad_count, 1u);
+    if (!ok) {
+        atomicAdd(ctx_bad, 1u);
+        if (bad_count) atomicAdd(bad_count, 1u);
+    }
 }
 
 }  // namespace
@@ -275,12 +281,12 @@ cudaError_t launch_expand(const llvq_ctx *ctx, int layout, const uint64_t *codes
         const int64_t pieces = nb / kTileCells + (left >= 2 ? 1 : 0) + (left & 1);
         const int64_t threads = groups * pieces * 32;
         const int64_t blocks = (threads + 255) / 256;
-        if (layout == LLVQ_PLANES13) expand_planes_kernel<true><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count);
-        else expand_planes_kernel<false><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count);
+        if (layout == LLVQ_PLANES13) expand_planes_kernel<true><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count, ctx->bad_codes);
+        else expand_planes_kernel<false><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count, ctx->bad_codes);
     } else {
         const int64_t threads = groups * nb * 32;
         const int64_t blocks = (threads + 255) / 256;
-        expand_onehot_kernel<<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count);
+        expand_onehot_kernel<<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count, ctx->bad_codes);
     }
     return cudaGetLastError();
 }

@@ -36,55 +36,18 @@
 // bounded.
 #include <cmath>
 #include <cstring>
+#include <mutex>
 
 #include "llvq_internal.cuh"
 #include "llvq_rotate.cuh"
 
-// Optional timeline (compiled in only with -DLLVQ_TRACE, never in the shipped library): lane 0 of
-// every warp stores the global timer at a few points of the kernel.
-#ifdef LLVQ_TRACE
-#define LLVQ_TRACE_POINT(i)                                                                                       \
-    if (p.trace && lane == 0) {                                                                                   \
-        unsigned long long t_;                                                                                    \
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                                    \
-        p.trace[(((size_t)p.trace_launch * gridDim.x + blockIdx.x) * kWarps + warp) * 128 + (i)] = t_;            \
-    }
-// per-unit timeline of every warp: slot 8 + 3*n + {0: wait begins, 1: data there, 2: decoded}, n < 40
-#define LLVQ_TRACE_UNIT(n, i)                                                                                     \
-    if (0) {                                                                       \
-        unsigned long long t_;                                                                                    \
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_));                                                    \
-        p.trace[(((size_t)p.trace_launch * gridDim.x + blockIdx.x) * kWarps + warp) * 128 + 8 + 3 * (n) + (i)] = t_; \
-    }
-// SM cycle counter into slots 120..127
-#define LLVQ_TRACE_CLOCK(i)                                                                                       \
-    if (p.trace && lane == 0)                                                                                     \
-        p.trace[(((size_t)p.trace_launch * gridDim.x + blockIdx.x) * kWarps + warp) * 128 + 98 + (i)] = clock64();
-#else
-#define LLVQ_TRACE_POINT(i)
-#define LLVQ_TRACE_UNIT(n, i)
-#define LLVQ_TRACE_CLOCK(i)
-#endif
-
 namespace llvq {
 namespace {
 
-#ifndef LLVQ_WARPS
-#define LLVQ_WARPS 16
-#endif
-#ifndef LLVQ_SLOTS
-#define LLVQ_SLOTS 2
-#endif
-#ifndef LLVQ_MINB
-#define LLVQ_MINB 1
-#endif
-constexpr int kWarps = LLVQ_WARPS;         // warps per CTA
+constexpr int kWarps = 16;                 // warps per CTA
 constexpr int kThreads = kWarps * 32;
-constexpr int kSlots = LLVQ_SLOTS;         // ring slots per warp
-#ifndef LLVQ_EARLY
-#define LLVQ_EARLY 1
-#endif
-constexpr int kEarlySlots = LLVQ_EARLY;    // slots filled before the wait for the previous kernel; the rest once x is being prepared
+constexpr int kSlots = 2;                  // ring slots per warp
+constexpr int kEarlySlots = 1;             // slots filled before the wait for the previous kernel; the rest once x is being prepared
 
 // fixed-point accumulator word: bits 53..63 count units, bits 0..52 sum the biased unit values
 constexpr int kCountShift = 53;
@@ -432,16 +395,6 @@ __host__ __device__ inline int panel_of_unit(const GemvParams &p, int f) {
     const int j = fast_div(f, p.div_panel_units, p.total_groups * p.panel);
     return j < p.npanels ? j : p.npanels - 1;
 }
-__device__ __forceinline__ Cursor locate(const GemvParams &p, int f) {
-    Cursor c;
-    c.panel = panel_of_unit(p, f);
-    const int first = c.panel * p.panel;
-    c.end = min(first + p.panel, p.units);
-    const int r = f - c.panel * (p.total_groups * p.panel), w = c.end - first;
-    c.group = c.panel == p.npanels - 1 ? fast_div(r, p.div_last, w) : fast_div(r, p.div_panel, w);
-    c.col = first + (r - c.group * w);
-    return c;
-}
 // steps over n units of the current row group's stretch; true if the row group changed
 __device__ __forceinline__ bool advance(const GemvParams &p, Cursor &c, int n) {
     c.col += n;
@@ -463,7 +416,7 @@ __device__ __forceinline__ bool advance(const GemvParams &p, Cursor &c, int n) {
 // blocks of x that its share of the matrix touches, exactly as the rotation kernel does, and rounds them to FP16.
 // COMPACT: the 13-byte layout (one header byte a block; the code words are where the 14-byte layout has them).
 template <bool NO_WEIGHTS, int BATCH, bool ROTATE = false, bool COMPACT = false>
-__global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
+__global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
     constexpr int kSrcCell = COMPACT ? kCell13Bytes : kCellBytes;        // bytes of a block column of a row group
     constexpr int kSrcTile = COMPACT ? kTile13Bytes : kTileBytes;        // bytes of a tile in memory (a ring slot always has kTileBytes)
     extern __shared__ __align__(128) unsigned char smem[];
@@ -482,8 +435,6 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
     const uint32_t my_ring = smem_addr(ring + warp * kSlots * kTileBytes);
     const uint32_t my_bar = smem_addr(bars + warp * kSlots);
 
-    LLVQ_TRACE_POINT(0)
-    LLVQ_TRACE_CLOCK(7)
     // The parameters the start of a CTA needs are read up front, all at once: a parameter line's first read by a
     // multiprocessor costs some two hundred cycles, and the chain below would otherwise meet them one by one.
     const CtaShare me = p.cta[blockIdx.x];
@@ -660,14 +611,10 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             }
         }
     };
-    LLVQ_TRACE_CLOCK(6)
     // let the next kernel in the stream start its own prefetch, then wait for the previous one:
     // x, y and the reduction scratch may still be in use by it
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    LLVQ_TRACE_POINT(1)
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    LLVQ_TRACE_POINT(2)
-    LLVQ_TRACE_CLOCK(0)
     // One pass over x finds the largest |x| (fp16 bit patterns of non-negative values order like integers):
     // every |x| is below 2^xexp, xexp = e - 14 with e the biased exponent of the largest magnitude.  The
     // pieces of x this CTA needs stay in registers meanwhile and then become fixed-point records on the scale
@@ -786,8 +733,12 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             if (lane == 0) warp_max[j * kWarps + warp] = m;    // plain stores: atomics on one word would serialise the warps
         }
         __syncthreads();                               // publishes the maxima, the block constants and the zeroed sums
-        LLVQ_TRACE_POINT(4)
-        LLVQ_TRACE_CLOCK(1)
+        // the second copy of records goes out now that the loads of x have returned: ahead of the conversion, whose
+        // arithmetic hides its issue
+        if (!NO_WEIGHTS) {
+#pragma unroll
+            for (int s = kEarlySlots; s < kSlots; s++) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
+        }
 #pragma unroll
         for (int j = 0; j < BATCH; j++) {
             const uint32_t m = warp_max[j * kWarps + (lane < kWarps ? lane : 0)];
@@ -802,17 +753,11 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
                     convert_item(j < p.batch ? __ldcg(xg + e) : make_uint4(0u, 0u, 0u, 0u), e % 3, xsj + (uint32_t)(e / 3) * kXRecBytes, scale);
             }
         }
-        if (!NO_WEIGHTS) {
-#pragma unroll
-            for (int s = kEarlySlots; s < kSlots; s++) issue(my_bar + 8 * s, my_ring + s * kTileBytes);
-        }
         __syncthreads();                               // publishes the x records
     }
     const LaneOffsets lo = {lane_consts.x, lane_consts.y, lane_consts.z, lane_consts.w};
     float first_row_scale;
     asm volatile("cvt.f32.f16 %0, %1;" : "=f"(first_row_scale) : "h"(first_scale_bits));
-    LLVQ_TRACE_POINT(3)
-    LLVQ_TRACE_CLOCK(2)
 
     int n = 0;
     uint32_t parity = 0;                               // every slot completes once a round of kSlots units
@@ -855,11 +800,9 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
 
 #pragma unroll 1
         for (int t = 0; t < run_tiles; t++) {
-            LLVQ_TRACE_UNIT(n + t, 0)
             if (!mbar_try(bar, parity)) {
                 if (!mbar_wait(bar, parity)) { failed = true; break; }
             }
-            LLVQ_TRACE_UNIT(n + t, 1)
             const uint4 a0 = lds128(sbuf + lane16);
             const uint4 a1 = lds128(sbuf + lane16 + 512);
             const uint4 a2 = lds128(sbuf + lane16 + 1024);
@@ -873,13 +816,6 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
             // until the four shared-memory reads of the whole warp have completed.
             issue(bar, sbuf + (settled(a0.w, a1.w, a2.w) | settled(hh.w, hh.x, a0.x)));
             float acc[BATCH][4];
-#ifdef LLVQ_STREAM_ONLY
-#pragma unroll
-            for (int j = 0; j < BATCH; j++) {
-                acc[j][0] = __uint_as_float((a0.x ^ a1.y ^ a2.z ^ hh.w) & 0x007fffffu);   // debug: bytes only, no decode
-                acc[j][1] = acc[j][2] = acc[j][3] = 0.f;
-            }
-#else
             if constexpr (BATCH == 1) {
                 // one vector: every shared-memory load first, then the eight contractions back to back (four independent
                 // accumulator tiles in the tensor pipe at once), then the eight scale steps
@@ -931,10 +867,8 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
 #pragma unroll
                 for (int j = 0; j < BATCH; j++) contract_half<false>(h3, sx[j], acc[j][2], acc[j][3]);
             }
-#endif
 #pragma unroll
             for (int j = 0; j < BATCH; j++) sum[j] += __float2ll_rn(quad_sum(acc[j]) * inv_q);
-            LLVQ_TRACE_UNIT(n + t, 2)
             xa.b0 += 4 * kXRecBytes; xa.b1 += 4 * kXRecBytes; xa.b2 += 4 * kXRecBytes; xa.xs += 4 * kXRecBytes;
             bar += 8;
             sbuf += kTileBytes;
@@ -998,7 +932,6 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         }
         // with no records read (the control launch) every unit contributes zero
         n += run;
-        if (n == n_units) { LLVQ_TRACE_POINT(6) }
         if (BATCH == 1) {
             hand_over(p, pr, p.accum, pr.y, cc.group, my_row, sum[0], run, xexp[0] + pr.qexp_base, row_scale, handed);
         } else {
@@ -1015,11 +948,8 @@ __global__ void __launch_bounds__(kThreads, LLVQ_MINB) gemv_planes_kernel(const 
         }
         if (advance(p, cc, run) && cc.panel < p.npanels) q = find_problem(p, cc.group);
     }
-    LLVQ_TRACE_CLOCK(14)
     settle(p, handed);
-    LLVQ_TRACE_CLOCK(15)
 
-    LLVQ_TRACE_POINT(5)
     if (failed) {
         // a wait ran out: report it, then give the copies still in flight a bounded chance to land
         // (a slot that is not pending returns at once or runs into the same bound)
@@ -1257,10 +1187,8 @@ GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
         return g;
     }
     // panels of about sixteen unit columns, as equal as they come
-#ifndef LLVQ_PANEL
-#define LLVQ_PANEL 16
-#endif
-    const int want = (p.units + LLVQ_PANEL / 2) / LLVQ_PANEL > 1 ? (p.units + LLVQ_PANEL / 2) / LLVQ_PANEL : 1;
+    constexpr int kPanelColumns = 16;
+    const int want = (p.units + kPanelColumns / 2) / kPanelColumns > 1 ? (p.units + kPanelColumns / 2) / kPanelColumns : 1;
     p.panel = (p.units + want - 1) / want;
     p.npanels = (p.units + p.panel - 1) / p.panel;
     p.div_panel_units = make_fastdiv((uint32_t)(p.total_groups * p.panel));
@@ -1433,6 +1361,7 @@ struct StaticDevice {
     int sm_count = 0, max_smem_optin = 0;
 };
 StaticDevice g_static_dev[kStaticMaxDevices];
+std::mutex g_static_mutex;                 // guards the first call's set-up on a device
 
 // Once per device, with that device current: resolve the arrays' device addresses, build the class
 // constants on the host, zero the accumulators, raise the kernel's shared-memory limit.  Allocates no device memory.
@@ -1476,9 +1405,13 @@ extern "C" int llvq_gemv_static(const void *layout_buf, const void *row_scale, c
     if (cudaGetDevice(&device) != cudaSuccess) return LLVQ_ECUDA;
     if (device < 0 || device >= kStaticMaxDevices) return LLVQ_EINVAL;
     StaticDevice &d = g_static_dev[device];
-    if (!d.ready) {
-        const int rc = static_setup(device, d);
-        if (rc != LLVQ_OK) return rc;
+    {
+        // two host threads may make the first call on a device at once: one of them sets up, the other waits
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!d.ready) {
+            const int rc = static_setup(device, d);
+            if (rc != LLVQ_OK) return rc;
+        }
     }
     GemvParams p;
     memset(&p, 0, sizeof p);
@@ -1494,7 +1427,7 @@ extern "C" int llvq_gemv_static(const void *layout_buf, const void *row_scale, c
     p.prob[0].gain1 = gain[1];
     {
         const float gm = fmaxf(fabsf(gain[0]), fabsf(gain[1]));
-        if (!(gm < 3.0e38f)) return LLVQ_EINVAL;
+        if (!(gm == 0.f || (gm >= 8.673617379884035e-19f && gm < 1.152921504606847e18f))) return LLVQ_EINVAL;   // as llvq_gemv
         int ge = 0;
         frexpf(gm > 0.f ? gm : 1.f, &ge);
         p.prob[0].qexp_base = ge + 5 - 39;               // same quantum as llvq_gemv
@@ -1519,3 +1452,43 @@ extern "C" int llvq_gemv_static(const void *layout_buf, const void *row_scale, c
     return llvq::launch_gemv(LLVQ_PLANES, p, g, false, true, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
 }
 
+
+// Reports and repairs what a llvq_gemv_static launch that gave up on a bounded wait leaves behind.  Without a
+// context there is no llvq_status to do it: the flag such a launch raises and the partial sums it abandons live in
+// the library's own arrays, and an unreported time-out would spoil every later call on the device.
+extern "C" int llvq_static_status(void *stream) {
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return LLVQ_ECUDA;
+    if (device < 0 || device >= kStaticMaxDevices) return LLVQ_EINVAL;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return LLVQ_ECUDA;
+    StaticDevice &d = g_static_dev[device];
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!d.ready) return LLVQ_OK;                  // no call was made on this device yet
+    }
+    int flag = 0;
+    if (cudaMemcpy(&flag, d.error, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) return LLVQ_ECUDA;
+    if (!flag) return LLVQ_OK;
+    // no allocation here either: both arrays are the library's own
+    if (cudaMemset(d.error, 0, sizeof(int) * 64) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaMemset(d.accum, 0, sizeof(unsigned long long) * kStaticMaxRows) != cudaSuccess) return LLVQ_ECUDA;
+    return LLVQ_ETIMEOUT;
+}
+
+// Points the wait-limit self-test at the static entry point's error flag, so that the path above can be exercised
+// without any fault on the GPU.
+extern "C" int llvq_static_selftest_wait_limit(void *stream) {
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess) return LLVQ_ECUDA;
+    if (device < 0 || device >= kStaticMaxDevices) return LLVQ_EINVAL;
+    StaticDevice &d = g_static_dev[device];
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!d.ready) {
+            const int rc = static_setup(device, d);
+            if (rc != LLVQ_OK) return rc;
+        }
+    }
+    llvq::wait_limit_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(d.error);
+    return cudaGetLastError() == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+}

@@ -104,10 +104,6 @@ struct GemvParams {
     int rot_span;             // most coordinates any CTA rotates (set by gemv_plan)
     const uint32_t *rot_negate;   // sign-flip bits, or null
     double rot_scale;         // 2^-24 / sqrt(block length)
-#ifdef LLVQ_TRACE
-    unsigned long long *trace;   // timeline buffer (debug builds only)
-    int trace_launch;
-#endif
 };
 
 }  // namespace llvq
@@ -120,11 +116,9 @@ struct llvq_ctx {
     unsigned long long *accum;   // reduction scratch: one 64-bit accumulator a row of the largest launch
     size_t accum_slots;
     int *error;              // device flag: a kernel's bounded wait ran out
+    uint32_t *bad_codes;     // device count: codes that named no point, over the expansions since the last llvq_status
     int use_pdl;             // launch the GEMV with programmatic stream serialization
-#ifdef LLVQ_TRACE
-    unsigned long long *trace;
-    int trace_launch;
-#endif
+    int weights_dirty;       // an expansion was enqueued since the last GEMV: that GEMV must not read records ahead of it
     int sm_count;
     int max_smem_optin;
 };

@@ -46,6 +46,9 @@ def test_layout_bytes_and_argument_checks(lib):
     assert lib.llvq_gemv_fp16(None, None, None, 8, 8, None) == -1
     assert lib.llvq_gemv(None, 0, None, None, None, None, None, 1, 24, None) == -1
     assert b"aligned" in lib.llvq_strerror(-2)
+    # the code for an expanded code word that names no point is declared and named
+    assert "#define LLVQ_EINDEX (-6)" in open(os.path.join(ROOT, "include", "llvq.h")).read()
+    assert b"no point" in lib.llvq_strerror(-6)
     # the 13-byte layout: 13/14 of the 14-byte layout's size, for any shape
     assert binding.layout_bytes(binding.PLANES13, 3072, 3072) == 3072 * 128 * 13
     assert binding.layout_bytes(binding.PLANES13, 33, 48) == 2 * 2 * 416

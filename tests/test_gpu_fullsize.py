@@ -36,6 +36,33 @@ def test_config4_in_full(B, ctx, oracle):
         del buf
 
 
+def test_config1_in_full(B, ctx, oracle):
+    """The 4B-like layer in full: every record of its seven matrices byte for byte against the oracle, and every
+    row of the row-concatenated launches the bench times against the f64 matvec."""
+    from paper_2609_02652_b200 import datagen
+
+    wl = datagen.workload(1)
+    groups = {}
+    for m in wl.matrices:
+        groups.setdefault(m.group, []).append(m)
+    for members in groups.values():
+        probs, keep = [], []
+        for m in members:
+            case = make_case(m.rows, m.k, seed=wl.seed, tensor_id=m.tensor_id)
+            buf = B.expand(ctx, B.PLANES, case.d_codes, m.rows, m.nb)
+            assert np.array_equal(buf.cpu().numpy(), oracle.pack_planes(case.codes, m.rows, m.nb)), m.name
+            y = torch.full((m.rows,), float("nan"), dtype=torch.float32, device="cuda")
+            probs.append((buf, case.d_scale, GAIN, y, m.rows))
+            keep.append((m, case, y))
+        # members of a group share x (the first member's)
+        x = keep[0][1]
+        B.gemv_grouped(ctx, B.PLANES, probs, x.d_x, members[0].k_padded)
+        B.status(ctx)
+        for m, case, y in keep:
+            case.x = x.x
+            check_gemv(oracle, case, y, nthreads=16)
+
+
 @pytest.mark.parametrize("config,layers", [(2, (0, 17, 35)), (3, (0, 39))])
 def test_stacks_sampled(B, ctx, oracle, config, layers):
     """Every matrix of the sampled layers runs as the bench runs it (row-concatenated groups); 96 rows

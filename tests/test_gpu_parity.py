@@ -83,6 +83,9 @@ def test_expand_whole_first_shell_class_edges_and_bad_codes(B, ctx, oracle, layo
     out = B.expand(ctx, layout, torch.from_numpy(codes.view(np.int64)).cuda(), 131, 7, bad_count=cnt)
     assert np.array_equal(out.cpu().numpy(), _expected(oracle, layout, case))
     assert int(cnt.item()) == len(bad)
+    with pytest.raises(B.LlvqError) as e:                     # the context counted them too
+        B.status(ctx)
+    assert e.value.code == -6
 
 
 @pytest.mark.parametrize("layout", [0, 1])
@@ -116,6 +119,9 @@ def test_gemv_special_cases(B, ctx, oracle):
     case.d_scale = torch.from_numpy(case.row_scale).cuda()
     case.d_codes = torch.from_numpy(case.codes.view(np.int64)).cuda()
     buf = B.expand(ctx, 0, case.d_codes, case.rows, case.nb)
+    with pytest.raises(B.LlvqError) as e:                     # the one code that names no point is reported
+        B.status(ctx)
+    assert e.value.code == -6
     y = B.gemv(ctx, 0, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
     check_gemv(oracle, case, y)
     assert y[5].item() == 0.0
@@ -383,3 +389,52 @@ def test_gemv_without_programmatic_dependent_launch(B, oracle):
         check_gemv(oracle, case, y2)
     finally:
         ctx.close()
+
+
+def test_invalid_codes_surface_through_status(B, ctx):
+    """A caller that passes no bad_count still learns that codes named no point: llvq_status returns LLVQ_EINDEX
+    once, then LLVQ_OK; a clean expansion in between does not raise."""
+    case = make_case(64, 96, seed=7)
+    B.expand(ctx, B.PLANES, case.d_codes, case.rows, case.nb)
+    B.status(ctx)
+    bad = case.d_codes.clone()
+    bad[5] = (1 << 47) - 1                                  # index 2^47 - 1 >= number of points
+    bad[70] = 1 << 60                                       # bits above bit 47
+    for layout in (B.PLANES, B.ONEHOT, B.PLANES13):
+        B.expand(ctx, layout, bad, case.rows, case.nb)      # bad_count = None
+        with pytest.raises(B.LlvqError) as e:
+            B.status(ctx)
+        assert e.value.code == -6 and "no point" in str(e.value)
+        B.status(ctx)
+
+
+def test_expand_then_gemv_back_to_back_on_fresh_buffers(B, ctx, oracle):
+    """llvq_expand followed at once by llvq_gemv on the same stream, programmatic dependent launch on: the GEMV
+    reads records ahead of its dependency wait, so the library launches this one as an ordinary kernel.  Fresh
+    buffers every round (filled with the pattern a stale read would show)."""
+    case = make_case(2048, 3072, seed=9)
+    y_ref = None
+    for it in range(20):
+        buf = torch.full((B.layout_bytes(B.PLANES, case.rows, case.nb * 24),), 0x88, dtype=torch.uint8, device="cuda")
+        B.expand(ctx, B.PLANES, case.d_codes, case.rows, case.nb, out=buf)
+        y = B.gemv(ctx, B.PLANES, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
+        if y_ref is None:
+            check_gemv(oracle, case, y)
+            y_ref = y.clone()
+        assert torch.equal(y, y_ref), it
+    B.status(ctx)
+
+
+def test_gain_range(B, ctx):
+    case = make_case(64, 96, seed=11)
+    buf = B.expand(ctx, B.PLANES, case.d_codes, case.rows, case.nb)
+    for gain in ((1e-30, 1e-31), (3e18, 1.0), (float("inf"), 1.0)):
+        with pytest.raises(B.LlvqError) as e:
+            B.gemv(ctx, B.PLANES, buf, case.d_scale, gain, case.d_x, case.rows, 96)
+        assert e.value.code == -1
+    y = B.gemv(ctx, B.PLANES, buf, case.d_scale, (0.0, 0.0), case.d_x, case.rows, 96)
+    assert (y == 0).all()
+    y = B.gemv(ctx, B.PLANES, buf, case.d_scale, (2.0 ** -59, 2.0 ** -59), case.d_x, case.rows, 96)
+    assert torch.isfinite(y).all()
+    y1 = B.gemv(ctx, B.PLANES, buf, case.d_scale, (1.0, 1.0), case.d_x, case.rows, 96)
+    assert torch.allclose(y.double() * 2.0 ** 59, y1.double(), rtol=1e-6, atol=0)

@@ -50,6 +50,9 @@ def test_expand_invalid_codes_and_full_first_shell(B, ctx, oracle):
     out = B.expand(ctx, L13, torch.from_numpy(bad.view(np.int64)).cuda(), 2, 3, bad_count=cnt)
     assert np.array_equal(out.cpu().numpy(), oracle.pack_planes13(bad, 2, 3))
     assert cnt.item() == 4
+    with pytest.raises(B.LlvqError) as e:                     # the context counted them too
+        B.status(ctx)
+    assert e.value.code == -6
 
 
 @pytest.mark.parametrize("rows,k", [(40, 24 * 7), (257, 24 * 21), (3072, 3072), (33, 24 * 2), (5, 24)])
@@ -89,6 +92,9 @@ def test_gemv_special_cases_and_grouped(B, ctx, oracle):
     case.d_scale = torch.from_numpy(case.row_scale).cuda()
     case.d_codes = torch.from_numpy(case.codes.view(np.int64)).cuda()
     buf = B.expand(ctx, L13, case.d_codes, case.rows, case.nb)
+    with pytest.raises(B.LlvqError) as e:                     # the one code that names no point is reported
+        B.status(ctx)
+    assert e.value.code == -6
     y = B.gemv(ctx, L13, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
     check_gemv(oracle, case, y)
     assert y[5].item() == 0.0

@@ -225,12 +225,40 @@ def test_shell2_is_enumerated_exactly_once(oracle):
     assert all(is_leech_point(x) for x in xs[::97])
 
 
-@pytest.mark.parametrize("lo,hi", [(196_560, 196_560 + 2_000_000), (16_969_680 - 1_500_000, 16_969_680)])
-def test_shell3_ranges_are_injective(oracle, lo, hi):
-    xs, _ = oracle.decode_batch(np.arange(lo, hi, dtype=np.uint64))
-    packed = np.ascontiguousarray(xs).view([("a", "u8"), ("b", "u8"), ("c", "u8")]).ravel()
+def test_shell3_is_enumerated_exactly_once(oracle):
+    """All 16 773 120 indices of the second non-empty shell decode to distinct points of norm 48: the decode is
+    injective there, and since the count is the theta coefficient it is onto as well."""
+    lo, hi = KISSING, 16_969_680
+    parts = []
+    for a in range(lo, hi, 1 << 21):
+        b = min(a + (1 << 21), hi)
+        xs, _ = oracle.decode_batch(np.arange(a, b, dtype=np.uint64))
+        assert ((xs.astype(np.int32) ** 2).sum(1) == 48).all()
+        parts.append(np.ascontiguousarray(xs).view([("a", "u8"), ("b", "u8"), ("c", "u8")]).ravel().copy())
+    packed = np.concatenate(parts)
+    del parts
+    assert packed.size == hi - lo == 16_773_120
     assert np.unique(packed).size == hi - lo
-    assert ((xs.astype(int) ** 2).sum(1) == 48).all()
+
+
+def test_worked_values_of_the_index_order(oracle):
+    """Index -> (class, point) for indices spread over the ball, worked out independently of this oracle (a separate
+    program written from the same readings before the oracle existed: class order = shell, even before odd, codeword
+    weight, magnitude tuples; order inside a class = codeword rank, arrangement ranks, sign bits, the last support
+    sign repairing the sum; odd classes = arrangement rank * 4096 + message bits).  A change to any of those readings
+    moves these points."""
+    expect = {
+        196_559: (2, [3, -1, 1, 1, -1, 1, -1, -1, -1, -1, 1, -1, 1, 1, -1, -1, 1, -1, 1, 1, 1, 1, -1, 1]),
+        196_560: (3, [2, 2, 2, 2, 2, 0, 0, 2, 0, 0, 2, 0, -2] + [0] * 10 + [4]),
+        16_969_680: (7, [0] * 23 + [8]),
+        40_556_880_458_640: (222, [0] * 21 + [8, 8, 8]),
+        12_345_678_901_234: (163, [5, -1, 1, -5, 5, 1, 1, -3, -1, 3, -1, 1, 3, -1, -1, 3, 1, -3, 1, -3, 3, -3, -1, -1]),
+        N_PAPER - 1: (300, [3, 3, -3, -3, 3, -3, 3, 3, 3, 3, -3, 3, -3, -3, 3, 3, -3, 3, -3, -3, -3, 1, -1, 1]),
+    }
+    for idx, (cls, x) in expect.items():
+        c, got = oracle.decode(idx)
+        assert c == cls and got.tolist() == x, idx
+        assert oracle.encode(np.array(x, dtype=np.int8)) == idx
 
 
 def test_worked_examples_derived_by_hand(oracle):

@@ -47,5 +47,43 @@ def test_static_entry_point_matches_context_entry_point_twice_in_a_row():
         B.gemv_static(dummy[: B.layout_bytes(B.PLANES, rows, 24)], sc[:rows], GAIN, xx, rows, 24, yy[:rows])
         torch.cuda.synchronize()
         assert (yy[:rows] == 0).all()
+        # none of those launches gave up on a wait: the built-in flag is clear
+        B.static_status()
+        # ... and the calls after the first allocated nothing on the device: the free memory is what it was
+        case = make_case(1000, 2560, seed=31)
+        buf = B.expand(ctx, B.PLANES, case.d_codes, 1000, case.nb)
+        y = torch.empty(1000, dtype=torch.float32, device="cuda")
+        B.gemv_static(buf, case.d_scale, GAIN, case.d_x, 1000, case.nb * 24, y)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        for _ in range(3):
+            B.gemv_static(buf, case.d_scale, GAIN, case.d_x, 1000, case.nb * 24, y)
+        B.static_status()
+        assert torch.cuda.mem_get_info()[0] == free_before
+    finally:
+        ctx.close()
+
+
+def test_static_time_out_is_reported_and_repaired():
+    """A wait that runs out (the one-warp self-test kernel: nothing faults) raises the static entry point's flag;
+    llvq_static_status reports it once, clears flag and scratch, and the next launch is right again."""
+    from paper_2609_02652_b200 import binding as B
+
+    B.load()
+    torch.cuda.set_device(0)
+    ctx = B.create(0)
+    try:
+        case = make_case(257, 960, seed=33)
+        buf = B.expand(ctx, B.PLANES, case.d_codes, case.rows, case.nb)
+        ref = B.gemv(ctx, B.PLANES, buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24)
+        B.static_selftest_wait_limit()
+        with pytest.raises(B.LlvqError) as e:
+            B.static_status()
+        assert e.value.code == -5
+        B.static_status()                               # reported once, then clear
+        y = torch.empty(case.rows, dtype=torch.float32, device="cuda")
+        B.gemv_static(buf, case.d_scale, GAIN, case.d_x, case.rows, case.nb * 24, y)
+        B.static_status()
+        assert torch.equal(y, ref)
     finally:
         ctx.close()
