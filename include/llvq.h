@@ -62,9 +62,11 @@
  *                distinct magnitudes.  Per cell five arrays of 32 words (word t of row l at
  *                128t+4l): V0 = smask | class[7:0]<<24, V1 = mask1 | class[8]<<24 | gain<<25,
  *                V2..V4 = mask2..mask4.  A row group takes 640*nb bytes.
- *   LLVQ_PLANES13 13 bytes a block, exact for every block [Sec. 3.3 reaches this rate, 4.34 bits a
- *                weight, with its "Planes12x" layout: 12 bytes for blocks of up to four levels, the
- *                five-level blocks kept exactly in a side table and applied by further thread blocks].
+ *   LLVQ_PLANES13 13 bytes a block, exact for every block.  Not the paper's next rate point: its "Planes12x" layout
+ *                [Sec. 3.3: 12 bytes for blocks of up to four levels, the five-level blocks kept exactly in a side table
+ *                and applied by further thread blocks] is smaller (about 12.1 bytes a block of payload on this library's
+ *                synthetic data against 13; 4.342 against about 4.47 bits a weight on the paper's accounting) and is not
+ *                built here.
  *                Here the rate comes from the header instead of the levels: the matvec needs of the
  *                class only what fixes the block's scale and the parity of its coordinates, so the
  *                16-bit header becomes one byte = shell (4 bits, 0 for the empty record) | parity << 4
