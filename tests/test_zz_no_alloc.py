@@ -87,3 +87,47 @@ def test_static_time_out_is_reported_and_repaired():
         assert torch.equal(y, ref)
     finally:
         ctx.close()
+
+
+_FIRST_CALL_FROM_TWO_THREADS = r"""
+import sys, threading
+import numpy as np, torch
+sys.path.insert(0, sys.argv[1]); sys.path.insert(0, sys.argv[1] + "/tests")
+from helpers import GAIN, make_case
+from paper_2609_02652_b200 import binding as B
+B.load(); torch.cuda.set_device(0)
+ctx = B.create(0)
+cases = [make_case(513, 1200, seed=41 + i) for i in range(2)]
+bufs = [B.expand(ctx, B.PLANES, c.d_codes, c.rows, c.nb) for c in cases]
+refs = [B.gemv(ctx, B.PLANES, b, c.d_scale, GAIN, c.d_x, c.rows, c.nb * 24) for b, c in zip(bufs, cases)]
+ys = [torch.empty(c.rows, dtype=torch.float32, device="cuda") for c in cases]
+torch.cuda.synchronize()
+gate, rcs = threading.Barrier(2), [None, None]
+def first_call(i):
+    # the process's first llvq_gemv_static calls, from two host threads at once: one sets the device up, the other
+    # waits for it; the launches themselves are serialised on one stream (they share the built-in scratch)
+    gate.wait()
+    try:
+        B.gemv_static(bufs[i], cases[i].d_scale, GAIN, cases[i].d_x, cases[i].rows, cases[i].nb * 24, ys[i], stream=torch.cuda.default_stream())
+        rcs[i] = 0
+    except Exception as e:
+        rcs[i] = repr(e)
+ts = [threading.Thread(target=first_call, args=(i,)) for i in range(2)]
+[t.start() for t in ts]; [t.join() for t in ts]
+B.static_status()
+assert rcs == [0, 0], rcs
+assert all(torch.equal(y, r) for y, r in zip(ys, refs))
+print("ok")
+"""
+
+
+def test_first_call_from_two_host_threads_at_once():
+    """The set-up the first call on a device does is guarded: two threads that make that first call together both
+    succeed and both get llvq_gemv's results.  Needs a process that has not called the entry point yet: a child."""
+    import os
+    import subprocess
+    import sys
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", _FIRST_CALL_FROM_TWO_THREADS, root], capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0 and r.stdout.strip().endswith("ok"), r.stdout + r.stderr
