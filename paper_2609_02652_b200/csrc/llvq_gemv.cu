@@ -486,41 +486,69 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
     if (n_units > 0) isrc = h_nprob == 1 ? h_layout0 + (size_t)(uint32_t)ic.group * h_group_bytes : group_base(p, ic.group, q);
     const uint32_t tail_bytes = h_tail_cells * kSrcCell;
 
-    // The issue side's walk: inext is the next unit's first byte, ileft the units left in its stretch of its
-    // row group.  next() hands out the unit's source and size and steps on.
+    // The issue side's walk.  A stretch is a row group's columns inside one panel; its units are consecutive in memory.
+    // `next` is the next unit's first byte, `left` the units left in the stretch; next() hands out the unit's source and
+    // size and steps on.  At the end of a stretch the same columns of the next row group follow, group_bytes further on,
+    // as long as that row group belongs to the same matrix and panel (`spans` counts those stretches down); at the end of
+    // a span the next matrix's first row group follows, or the next panel's first stretch.
     struct Walk {
-        Cursor c;
         const uint8_t *next;
         int left, done;
+        int first, width;     // the current panel's first unit column, and the units of a stretch in it
+        int spans;            // stretches the short step still reaches, this one included
+        int span_end;         // first row group past the span
+        int q;                // the span's matrix
+        int turn_at;          // 1 while the stretch ends with the leftover blocks (a unit of another size), else 0
         uint32_t bytes;       // size of the next unit
     };
     const int n_tiles_total = h_tiles;
     Walk iw;
-    iw.c = ic;
     iw.next = isrc + (size_t)ic.col * kSrcTile;      // the leftover blocks follow the last tile
     iw.left = ic.end - ic.col;
     iw.done = 0;
+    iw.first = ic.panel * h_panel;
+    iw.width = ic.end - iw.first;
+    iw.q = q;
+    iw.span_end = (h_nprob == 1 || q + 1 == h_nprob) ? h_groups : p.prob[q + 1].group_begin;
+    iw.spans = iw.span_end - ic.group;
+    iw.turn_at = (h_tail_cells != 0 && ic.end == h_units) ? 1 : 0;
     iw.bytes = ic.col < n_tiles_total ? (uint32_t)kSrcTile : tail_bytes;
-    // the stretch ends or its last unit is the leftover one: the next unit starts elsewhere or has another size
-    auto walk_turn = [&](Walk &w) {
-        if (w.left == 0) {
-            w.c.col--;
-            advance(p, w.c, 1);
-            if (w.done < n_units) {
-                int qi;
-                w.next = group_base(p, w.c.group, qi) + (size_t)w.c.col * kSrcTile;
-            }
-            w.left = w.c.end - w.c.col;
-        }
-        w.bytes = w.c.col < n_tiles_total ? (uint32_t)kSrcTile : tail_bytes;
-    };
     auto walk_next = [&](Walk &w, const uint8_t *&src, uint32_t &bytes) {
         src = w.next;
         bytes = w.bytes;
         w.done++;
         w.next += kSrcTile;
-        w.c.col++;
-        if (--w.left <= 1) walk_turn(w);               // rare: at most twice a stretch
+        if (--w.left <= w.turn_at && w.done < n_units) {     // once a stretch (twice where it ends with the leftover unit)
+            if (w.left == 0) {
+                if (--w.spans > 0) {
+                    // from the end of this stretch (counted in whole tiles) to the same columns of the next row group:
+                    // negative where a row group is shorter than its units counted as whole tiles
+                    w.next += (long long)h_group_bytes - (long long)w.width * kSrcTile;
+                } else {
+                    int g = w.span_end;
+                    if (g == h_groups) {               // the panel is done: the next one's first stretch
+                        g = 0;
+                        w.q = -1;
+                        w.first += h_panel;
+                        w.width = min(h_panel, h_units - w.first);
+                        w.turn_at = (h_tail_cells != 0 && w.first + w.width == h_units) ? 1 : 0;
+                    }
+                    const uint8_t *base = h_layout0;
+                    w.span_end = h_groups;
+                    if (h_nprob != 1) {                // the next matrix (they follow each other in the order of row groups)
+                        w.q++;
+                        base = p.prob[w.q].layout - (size_t)(uint32_t)p.prob[w.q].group_begin * h_group_bytes;
+                        if (w.q + 1 < h_nprob) w.span_end = p.prob[w.q + 1].group_begin;
+                    }
+                    w.spans = w.span_end - g;
+                    w.next = base + (size_t)(uint32_t)g * h_group_bytes + (size_t)w.first * kSrcTile;
+                }
+                w.left = w.width;
+                w.bytes = (w.turn_at && w.left == 1) ? tail_bytes : (uint32_t)kSrcTile;
+            } else {
+                w.bytes = tail_bytes;                  // one unit left, and it is the leftover one
+            }
+        }
     };
     // issue the copy of the next unit onto barrier `b` and buffer `dst`: by one elected lane under a condition that
     // is the same for the whole warp, or (the four-vector build, where that form costs a register too many) by
