@@ -38,10 +38,10 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes (read + write) per algorithmic byte of gemv_planes_kernel, from one ncu capture of the
 # 8192 x 8192 launch (profiles/gemv_planes_kernel_config4_8192x8192.txt); traffic grows in proportion
 # to the records streamed, so a launch's traffic is its bytes times this.
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 39.362048 / 39.288864
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 39.362304 / 39.288864
 # from the same capture: warp instructions per block column (32 rows x 24 weights), and the share of issue
 # slots busy over the launch
-NCU_WARP_INSTR_PER_CELL = 5676863 / 87552
+NCU_WARP_INSTR_PER_CELL = 5668779 / 87552
 NCU_ISSUE_BUSY_PCT = 54.4
 METRIC = "us_per_lattice_gemv"
 DISCARD_ROUNDS = 2
