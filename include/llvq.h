@@ -78,6 +78,51 @@
  *                Accepted by llvq_layout_bytes, llvq_expand, llvq_gemv, llvq_gemv_grouped and
  *                llvq_decode_i8 (which returns the header byte in place of a class id); the other
  *                calls return LLVQ_EINVAL for it.  y is bit for bit what LLVQ_PLANES gives.
+ *   LLVQ_PLANES10X 10 bytes a block plus a sparse table of exact records: this library's form of the paper's
+ *                "Planes12x" overlay [Sec. 3.3: a short record for most blocks, the exact record of the others in
+ *                a per-matrix exception table, the correction applied in the same launch, reconstruction
+ *                bit-exact].  The paper's short record keeps a two-bit level and a sign a coordinate, which a
+ *                class table turns into a value; the tensor-core contraction used here wants a code the value
+ *                is affine in, so the short record keeps a three-bit WINDOW code instead, and the header
+ *                byte of LLVQ_PLANES13 in place of the class:
+ *                  v_i = u_i - o, u_i the four-bit code of LLVQ_PLANES, o the block's window base: the
+ *                  smallest o in {3, 4, 5, 6} with o <= min u_i and max u_i <= o + 7;
+ *                  header byte = shell | parity << 4 | gain << 5 | (o - 3) << 6;  x_i = 2 (v_i + o - 8) + parity.
+ *                A block with no such o (its codes span more than eight consecutive values, or reach below 3)
+ *                is an EXCEPTION: its short record is all zero - the empty record, which adds nothing - and
+ *                its exact record goes to the table.  Rows past the end and codes that name no point also
+ *                get the all-zero record (and no table entry).
+ *                  Tile = blocks 4T..4T+3 of a row group, 1280 bytes; rows, lanes, half-steps and positions
+ *                  as in LLVQ_PLANES.  Group(h, e, c) of lane L = 4g + t is the four codes of row (m, e, g)
+ *                  of half-step h = 2s + m at positions 16c + 4t + i (c = 0, 1) or 32 + 4t + i (c = 2),
+ *                  i = 0..3.  The lane owns nine words V0..V8; byte i of a word carries code i of two
+ *                  groups, in bits 0..2 and 3..5:
+ *                    V(2h + e), h = 0..3, e = 0, 1:  Group(h, e, 0), Group(h, e, 1)
+ *                    V8:                             Group(0, 0, 2), Group(1, 0, 2)
+ *                  and bits 6, 7 of the bytes carry the six groups left, X0..X5 = Group(0, 1, 2),
+ *                  Group(1, 1, 2), Group(2, 0, 2), Group(2, 1, 2), Group(3, 0, 2), Group(3, 1, 2): bits
+ *                  0, 1 of code i of Xk are bits 6, 7 of byte i of Vk; bit 2 of code i of Xk is bit
+ *                  6 + (k & 1) of byte i of V(6 + (k >> 1)).
+ *                  Vk of lane L at byte 16 L + 4 k (k < 4), 512 + 16 L + 4 (k - 4) (k < 8), 1024 + 4 L
+ *                  (k = 8); header byte of pair P, half-step h, row half e at 1152 + 8 P + 2 h + e.
+ *                  The nb mod 4 blocks left over follow the tiles exactly as in LLVQ_PLANES13 (four-bit
+ *                  codes, bits 6, 7 of the header byte zero: a pair of 832 bytes, a single of 416): they
+ *                  hold every block exactly and never make an exception.  A row group takes
+ *                  1280 (nb / 4) + 416 (nb mod 4) bytes.
+ *                  After the last row group, at the next multiple of 128 bytes: the index, one uint32 a
+ *                  row group and one more - entry g = table entries of the row groups before g.  After
+ *                  the index, at the next multiple of 128 bytes: the table, 16 bytes an entry, ordered by
+ *                  row group, tile, block, row:  word 0 = shell | parity << 4 | gain << 5 | (row of the
+ *                  group) << 8 | (block column) << 13;  words 1..3 = the 24 four-bit codes, coordinate
+ *                  8 j + n in nibble n of word 1 + j.  Bytes between the parts are zero.
+ *                The table's size depends on the data: llvq_overlay_count counts the exceptions of a matrix,
+ *                llvq_overlay_bytes sizes the buffer for a given number, llvq_layout_bytes sizes it for one
+ *                exception in 32 blocks.  llvq_expand takes the room for entries from out_bytes; entries that
+ *                do not fit are dropped, the index stops at the capacity, and the next llvq_status returns
+ *                LLVQ_ESIZE.  k_padded / 24 must be below 2^19.
+ *                Accepted by the calls that accept LLVQ_PLANES13.  With no exception in a matrix y is bit for
+ *                bit what LLVQ_PLANES gives; an exception's product is rounded to the accumulator's quantum
+ *                by itself instead of together with its tile's.
  */
 #ifndef LLVQ_H
 #define LLVQ_H
@@ -92,11 +137,13 @@ extern "C" {
 #define LLVQ_PLANES 0
 #define LLVQ_ONEHOT 1
 #define LLVQ_PLANES13 2   /* no counterpart record in the paper: see above */
+#define LLVQ_PLANES10X 3  /* the paper's sparse overlay ("Planes12x") with a window code: see above */
 
 #define LLVQ_OK 0
 #define LLVQ_EINVAL (-1) /* null pointer, bad shape, unknown layout                         */
 #define LLVQ_EALIGN (-2) /* a device pointer is not aligned as documented                   */
-#define LLVQ_ESIZE (-3)  /* a buffer or the context's scratch is too small for the request  */
+#define LLVQ_ESIZE (-3)  /* a buffer or the context's scratch is too small for the request; from llvq_status:
+                            an LLVQ_PLANES10X expansion had more exceptions than its buffer had room for */
 #define LLVQ_ECUDA (-4)  /* a CUDA runtime call failed                                      */
 #define LLVQ_ETIMEOUT (-5) /* a bounded wait inside a kernel ran out (llvq_status, llvq_static_status) */
 #define LLVQ_EINDEX (-6) /* an expanded code word named no point of the ball (llvq_status only) */
@@ -135,7 +182,8 @@ const char *llvq_strerror(int code);
 
 /* Synchronises `stream` and reports whether any GEMV launched on this context since the last
  * call gave up on one of its bounded waits (LLVQ_ETIMEOUT; the flag and the scratch are then
- * reset), else whether any llvq_expand on this context since the last call met a code word that
+ * reset), else whether an LLVQ_PLANES10X expansion ran out of room for its exception table (LLVQ_ESIZE;
+ * expand again into a larger buffer), else whether any llvq_expand on this context since the last call met a code word that
  * names no point (LLVQ_EINDEX; the count is then reset - the 512-slot class table exists so that
  * such a code can never index out of bounds [Sec. 2.3], and this is how a caller that passed no
  * bad_count learns of it).  Every wait inside the kernels on an asynchronous copy has a time limit
@@ -165,6 +213,13 @@ uint64_t llvq_class_base(const llvq_ctx *ctx, int c);
 
 /* Bytes of a layout buffer for a rows x (k_padded/24) matrix. Host query. */
 int llvq_layout_bytes(int layout, int64_t rows, int64_t k_padded, size_t *bytes);
+
+/* [Sec. 3.3, the exception table of the sparse overlay] Host queries and a counting pass for LLVQ_PLANES10X.
+ * llvq_overlay_count decodes the rows*nb code words and writes to *count (HOST) how many blocks the layout keeps
+ * in its exception table; it synchronises `stream`.  llvq_overlay_bytes gives the bytes of a layout buffer with
+ * room for `exceptions` table entries. */
+int llvq_overlay_count(llvq_ctx *ctx, const uint64_t *codes, int64_t rows, int64_t nb, uint64_t *count, void *stream);
+int llvq_overlay_bytes(int64_t rows, int64_t k_padded, uint64_t exceptions, size_t *bytes);
 
 /* [Sec. 2.2] Unfolds rows*nb code words (row-major, codes[row*nb + b]) into `layout_out`
  * (128-byte aligned, at least llvq_layout_bytes).  A code that names no point (index not below

@@ -610,6 +610,156 @@ void llvqo_pack_planes(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t 
 void llvqo_pack_planes13(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t *out) { pack_planes_any(codes, rows, nb, out, 1); }
 
 /*
+ * 10-byte layout with an exception table (the sparse overlay of Sec. 3.3, with a window code in place of the
+ * paper's level code).  For a block with four-bit codes u_0..u_23 (u_i = 8 + floor(x_i / 2)) the window base o
+ * is the smallest of 3, 4, 5, 6 with o <= min u and max u <= o + 7; the short record keeps v_i = u_i - o in three
+ * bits and the header byte shell | parity << 4 | gain << 5 | (o - 3) << 6.  A block with no such o is an
+ * exception: all-zero short record, exact record in the table.  Rows past the end and codes that name no point:
+ * all-zero short record, no table entry.
+ *
+ * Tile (blocks 4T..4T+3 of a row group), 1280 bytes.  Rows, lanes, half-steps, positions as in the 14-byte layout.
+ * Group(h, e, c) of lane (g, t): the codes of row (m, e, g), m = h & 1, at positions 16 c + 4 t + i (c < 2) or
+ * 32 + 4 t + i (c = 2), i = 0..3, of half-step h.  Nine words V0..V8 a lane; byte i of a word holds code i of two
+ * groups (bits 0..2 and 3..5): V(2h+e) = Group(h,e,0), Group(h,e,1); V8 = Group(0,0,2), Group(1,0,2).  The other six
+ * groups X0..X5 = Group(0,1,2), Group(1,1,2), Group(2,0,2), Group(2,1,2), Group(3,0,2), Group(3,1,2) live in bits 6, 7:
+ * bits 0, 1 of code i of Xk are bits 6, 7 of byte i of Vk; bit 2 of it is bit 6 + (k & 1) of byte i of V(6 + (k >> 1)).
+ * Vk of lane L at 16 L + 4 k (k < 4), 512 + 16 L + 4 (k - 4) (k < 8), 1024 + 4 L (k = 8); header byte of pair P,
+ * half-step h, row half e at 1152 + 8 P + 2 h + e.
+ * The nb mod 4 last blocks follow in the 13-byte layout's pair and single (four-bit codes, exact).
+ * After the row groups, at the next multiple of 128: the index (row groups + 1 uint32; entry g = exceptions of the
+ * row groups before g, never above the capacity); after it, at the next multiple of 128: the table, 16 bytes an
+ * entry, in the order row group, tile, block, row: word 0 = shell | parity << 4 | gain << 5 | row of the group << 8 |
+ * block column << 13, words 1..3 the four-bit codes (coordinate 8 j + n in nibble n of word 1 + j).
+ */
+static size_t up128(size_t v) { return (v + 127u) & ~(size_t)127u; }
+static size_t p10_group_bytes(int64_t nb) { return (size_t)(nb / 4) * 1280u + (size_t)(nb % 4) * 416u; }
+static size_t p10_index_offset(int64_t rows, int64_t nb) { return up128((size_t)((rows + 31) / 32) * p10_group_bytes(nb)); }
+static size_t p10_table_offset(int64_t rows, int64_t nb) { return p10_index_offset(rows, nb) + up128((size_t)((rows + 31) / 32 + 1) * 4u); }
+size_t llvqo_planes10x_bytes(int64_t rows, int64_t nb, uint64_t exceptions) { return p10_table_offset(rows, nb) + (size_t)exceptions * 16u; }
+
+/* window base of a block's codes, 0 if none fits */
+static int window_base(const uint8_t *u) {
+    int lo = 15, hi = 0;
+    for (int i = 0; i < NCOORD; i++) { if (u[i] < lo) lo = u[i]; if (u[i] > hi) hi = u[i]; }
+    for (int o = 3; o <= 6; o++) if (o <= lo && hi <= o + 7) return o;
+    return 0;
+}
+
+/* returns the number of exceptions met (all of them, also those past `capacity`, which are not stored) */
+int64_t llvqo_pack_planes10x(const uint64_t *codes, int64_t rows, int64_t nb, uint8_t *out, uint64_t capacity) {
+    const int64_t ngroups = (rows + 31) / 32, ntiles = nb / 4, left = nb % 4;
+    const size_t gbytes = p10_group_bytes(nb);
+    memset(out, 0, llvqo_planes10x_bytes(rows, nb, capacity));
+    uint32_t *index = (uint32_t *)(out + p10_index_offset(rows, nb));
+    uint8_t *table = out + p10_table_offset(rows, nb);
+    uint8_t *u = malloc((size_t)32 * nb * 24);        /* four-bit codes */
+    uint8_t *v = malloc((size_t)32 * nb * 24);        /* what the short record stores */
+    uint8_t *hb = malloc((size_t)32 * nb);            /* header byte of the exact record (no window bits) */
+    uint8_t *hs = malloc((size_t)32 * nb);            /* header byte of the short record */
+    uint8_t *exc = malloc((size_t)32 * nb);
+    uint64_t count = 0;
+    for (int64_t rg = 0; rg < ngroups; rg++) {
+        index[rg] = (uint32_t)(count < capacity ? count : capacity);
+        for (int r = 0; r < 32; r++)
+            for (int64_t b = 0; b < nb; b++) {
+                record_t rec;
+                int64_t row = rg * 32 + r;
+                size_t at = (size_t)r * nb + b;
+                if (row < rows) make_record(codes[row * nb + b], &rec);
+                else { memset(&rec, 0, sizeof rec); rec.cls = SENTINEL_CLASS; }
+                int empty = rec.cls == SENTINEL_CLASS;
+                int parity = empty ? 0 : (rec.x[0] & 1);
+                for (int i = 0; i < NCOORD; i++) u[at * 24 + i] = (uint8_t)(8 + (rec.x[i] - parity) / 2);
+                hb[at] = empty ? 0 : (uint8_t)(g_cls[rec.cls].shell | (parity << 4) | (rec.gain << 5));
+                int o = empty ? 0 : window_base(u + at * 24);
+                exc[at] = !empty && o == 0;
+                hs[at] = o ? (uint8_t)(hb[at] | ((o - 3) << 6)) : 0;
+                for (int i = 0; i < NCOORD; i++) v[at * 24 + i] = o ? (uint8_t)(u[at * 24 + i] - o) : 0;
+            }
+        uint8_t *grp = out + (size_t)rg * gbytes;
+        /* the tiles: three-bit codes */
+        for (int64_t T = 0; T < ntiles; T++) {
+            uint8_t *tile = grp + (size_t)T * 1280u;
+            for (int g = 0; g < 8; g++)
+                for (int t = 0; t < 4; t++) {
+                    int L = 4 * g + t, P = 2 * g + (t >> 1);
+                    uint32_t grpw[4][2][3];              /* [h][e][c]: byte i = code i of Group(h, e, c) */
+                    for (int h = 0; h < 4; h++)
+                        for (int e = 0; e < 2; e++)
+                            for (int c = 0; c < 3; c++) {
+                                uint32_t w = 0;
+                                for (int i = 0; i < 4; i++) {
+                                    int kappa = (c < 2 ? 16 * c : 32) + 4 * t + i;
+                                    int64_t b = 4 * T + 2 * (h >> 1) + kappa / 24;
+                                    int row = 16 * (h & 1) + 8 * e + g;
+                                    w |= (uint32_t)v[((size_t)row * nb + b) * 24 + kappa % 24] << (8 * i);
+                                }
+                                grpw[h][e][c] = w;
+                            }
+                    uint32_t V[9];
+                    for (int k = 0; k < 8; k++) V[k] = grpw[k >> 1][k & 1][0] | grpw[k >> 1][k & 1][1] << 3;
+                    V[8] = grpw[0][0][2] | grpw[1][0][2] << 3;
+                    const uint32_t X[6] = {grpw[0][1][2], grpw[1][1][2], grpw[2][0][2], grpw[2][1][2], grpw[3][0][2], grpw[3][1][2]};
+                    for (int k = 0; k < 6; k++) {
+                        V[k] |= (X[k] & 0x03030303u) << 6;
+                        V[6 + (k >> 1)] |= ((X[k] >> 2) & 0x01010101u) << (6 + (k & 1));
+                    }
+                    for (int k = 0; k < 9; k++) {
+                        size_t at = k < 4 ? 16u * L + 4u * k : (k < 8 ? 512u + 16u * L + 4u * (k - 4) : 1024u + 4u * L);
+                        memcpy(tile + at, &V[k], 4);
+                    }
+                    for (int h = 0; h < 4; h++)
+                        for (int e = 0; e < 2; e++) {
+                            int row = 16 * (h & 1) + 8 * e + g;
+                            int64_t b = 4 * T + 2 * (h >> 1) + (t >> 1);
+                            tile[1152 + 8 * P + 2 * h + e] = hs[(size_t)row * nb + b];
+                        }
+                }
+            /* the tile's exceptions: block by block, row by row */
+            for (int q = 0; q < 4; q++)
+                for (int r = 0; r < 32; r++) {
+                    size_t at = (size_t)r * nb + 4 * T + q;
+                    if (!exc[at]) continue;
+                    if (count < capacity) {
+                        uint32_t e4[4] = {(uint32_t)hb[at] | (uint32_t)r << 8 | (uint32_t)(4 * T + q) << 13, 0, 0, 0};
+                        for (int i = 0; i < NCOORD; i++) e4[1 + i / 8] |= (uint32_t)u[at * 24 + i] << (4 * (i % 8));
+                        memcpy(table + (size_t)count * 16u, e4, 16);
+                    }
+                    count++;
+                }
+        }
+        /* the blocks left over: the 13-byte layout's pair and single */
+        uint16_t *hdr16 = malloc((size_t)32 * nb * 2);
+        for (size_t at = 0; at < (size_t)32 * nb; at++) hdr16[at] = hb[at];
+        group_t G = {u, hdr16, nb};
+        uint8_t *rest0 = grp + (size_t)ntiles * 1280u;
+        uint32_t w[3], hw;
+        for (int g = 0; g < 8; g++)
+            for (int t = 0; t < 4; t++) {
+                int L = 4 * g + t, P = 2 * g + (t >> 1);
+                uint8_t *rest = rest0;
+                if (left >= 2) {
+                    for (int m = 0; m < 2; m++) {
+                        hs_words(&G, 4 * ntiles, 4 * ntiles + 1, m, g, t, w, &hw);
+                        for (int q = 0; q < 3; q++) memcpy(rest + 128 * (3 * m + q) + 4 * L, &w[q], 4);
+                        rest[768 + 4 * P + 2 * m] = (uint8_t)hw; rest[768 + 4 * P + 2 * m + 1] = (uint8_t)(hw >> 16);
+                    }
+                    rest += 832;
+                }
+                if (left & 1) {
+                    hs_words(&G, nb - 1, -1, 0, g, t, w, &hw);
+                    for (int q = 0; q < 3; q++) memcpy(rest + 128 * q + 4 * L, &w[q], 4);
+                    rest[384 + 2 * P] = (uint8_t)hw; rest[384 + 2 * P + 1] = (uint8_t)(hw >> 16);
+                }
+            }
+        free(hdr16);
+    }
+    index[ngroups] = (uint32_t)(count < capacity ? count : capacity);
+    free(u); free(v); free(hb); free(hs); free(exc);
+    return (int64_t)count;
+}
+
+/*
  * One-hot layout, 20 bytes a block: the cell of (row group, block column) is five arrays of 32
  * words, one entry a row: V0 = smask | class[7:0] << 24, V1 = mask1 | class[8] << 24 | gain << 25,
  * V2 = mask2, V3 = mask3, V4 = mask4.  Word t of row l sits at 128 t + 4 l; a row group occupies

@@ -71,6 +71,10 @@ def lib() -> ctypes.CDLL:
             L.llvqo_planes13_bytes.argtypes = [i64, i64]
             L.llvqo_planes13_bytes.restype = ctypes.c_size_t
             L.llvqo_pack_onehot.restype = None
+            L.llvqo_planes10x_bytes.argtypes = [i64, i64, u64]
+            L.llvqo_planes10x_bytes.restype = ctypes.c_size_t
+            L.llvqo_pack_planes10x.argtypes = [vp, i64, i64, vp, u64]
+            L.llvqo_pack_planes10x.restype = i64
             L.llvqo_dequant.argtypes = [vp, i64, i64, vp, vp, vp]
             L.llvqo_dequant.restype = None
             L.llvqo_matvec.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, vp, ci]
@@ -186,6 +190,23 @@ def pack_planes13(codes: np.ndarray, rows: int, nb: int) -> np.ndarray:
     out = np.zeros(planes13_bytes(rows, nb), np.uint8)
     lib().llvqo_pack_planes13(_ptr(codes), rows, nb, _ptr(out))
     return out
+
+
+def planes10x_bytes(rows: int, nb: int, exceptions: int) -> int:
+    return int(lib().llvqo_planes10x_bytes(rows, nb, exceptions))
+
+
+def pack_planes10x(codes: np.ndarray, rows: int, nb: int, capacity: int | None = None) -> tuple[np.ndarray, int]:
+    """The 10-byte layout with its exception table (Sec. 3.3, the sparse overlay): the buffer with room for
+    `capacity` table entries (default: exactly as many as the matrix has) and the number of exceptions met."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint64)
+    assert codes.size == rows * nb
+    if capacity is None:
+        scratch = np.zeros(planes10x_bytes(rows, nb, 0), np.uint8)
+        capacity = int(lib().llvqo_pack_planes10x(_ptr(codes), rows, nb, _ptr(scratch), 0))
+    out = np.zeros(planes10x_bytes(rows, nb, capacity), np.uint8)
+    n = int(lib().llvqo_pack_planes10x(_ptr(codes), rows, nb, _ptr(out), capacity))
+    return out, n
 
 
 def pack_onehot(codes: np.ndarray, rows: int, nb: int) -> np.ndarray:

@@ -434,6 +434,171 @@ def test_planes13_layout_worked_example_by_hand(oracle):
     assert int(buf[384]) == 2 | (1 << 5)
 
 
+def _p10_offsets(rows, nb):
+    groups = (rows + 31) // 32
+    gbytes = (nb // 4) * 1280 + (nb % 4) * 416
+    idx = -(-groups * gbytes // 128) * 128
+    return groups, gbytes, idx, idx + -(-(groups + 1) * 4 // 128) * 128
+
+
+def _unpack_planes10x_cell(buf, rows, nb, row, b):
+    """Reader of the 10-byte layout's short record from its description: (row, block) -> header byte, window base
+    (None for a block past the tiles, whose codes are four-bit) and the 24 stored codes."""
+    rg, r = divmod(row, 32)
+    m, e, g = r // 16, (r // 8) % 2, r % 8
+    _, gbytes, _, _ = _p10_offsets(rows, nb)
+    grp = rg * gbytes
+    ntiles, left = divmod(nb, 4)
+
+    def word(off):
+        return int.from_bytes(buf[off: off + 4].tobytes(), "little")
+
+    j = b - 4 * ntiles
+    if j >= 0:                                   # pair or single, as in the 13-byte layout
+        if left >= 2 and j < 2:
+            base, slot = grp + ntiles * 1280, j
+            addr = lambda q, lane: base + 128 * (3 * m + q) + 4 * lane
+            hb = int(buf[base + 768 + 4 * (2 * g + slot) + 2 * m + e])
+        else:
+            base, slot = grp + ntiles * 1280 + (832 if left == 3 else 0), m
+            addr = lambda q, lane: base + 128 * q + 4 * lane
+            hb = int(buf[base + 384 + 2 * (2 * g + slot) + e])
+        codes = []
+        for i in range(24):
+            kappa = 24 * slot + i
+            if kappa < 32:
+                c, t, ii = kappa // 16, (kappa % 16) // 4, kappa % 4
+                w = word(addr(e, 4 * g + t))
+            else:
+                c, t, ii = e, (kappa - 32) // 4, (kappa - 32) % 4
+                w = word(addr(2, 4 * g + t))
+            codes.append((w >> (4 * (2 * ii + c))) & 15)
+        assert hb >> 6 == 0
+        return hb, None, codes
+    base = grp + (b // 4) * 1280
+    slot, h = b % 2, 2 * ((b % 4) // 2) + m
+
+    def V(k, lane):
+        return word(base + (16 * lane + 4 * k if k < 4 else (512 + 16 * lane + 4 * (k - 4) if k < 8 else 1024 + 4 * lane)))
+
+    left_over = [(0, 1), (1, 1), (2, 0), (2, 1), (3, 0), (3, 1)]       # the groups X0..X5 as (h, e)
+    codes = []
+    for i in range(24):
+        kappa = 24 * slot + i
+        if kappa < 32:
+            c, t, ii = kappa // 16, (kappa % 16) // 4, kappa % 4
+            codes.append((V(2 * h + e, 4 * g + t) >> (8 * ii + 3 * c)) & 7)
+            continue
+        t, ii = (kappa - 32) // 4, (kappa - 32) % 4
+        lane = 4 * g + t
+        if (h, e) == (0, 0):
+            codes.append((V(8, lane) >> (8 * ii)) & 7)
+        elif (h, e) == (1, 0):
+            codes.append((V(8, lane) >> (8 * ii + 3)) & 7)
+        else:
+            k = left_over.index((h, e))
+            low = (V(k, lane) >> (8 * ii + 6)) & 3
+            high = (V(6 + (k >> 1), lane) >> (8 * ii + 6 + (k & 1))) & 1
+            codes.append(low | high << 2)
+    hb = int(buf[base + 1152 + 8 * (2 * g + slot) + 2 * h + e])
+    return hb, 3 + (hb >> 6), codes
+
+
+@pytest.mark.parametrize("rows,nb,rate", [(32, 4, 0.0), (37, 7, 0.3), (64, 1, 0.5), (5, 2, 0.5), (33, 3, 0.2), (20, 6, 0.1), (50, 9, 0.25),
+                                          (70, 12, 1.0), (96, 8, 0.02)])
+def test_planes10x_layout_round_trip(oracle, rows, nb, rate):
+    """Short records plus exception table rebuild every block exactly; the window base is the smallest that fits; the
+    table is ordered row group, tile, block, row; the index counts it; everything else in the buffer is zero."""
+    from helpers import make_overlay_case, window_base
+
+    codes = make_overlay_case(oracle, rows, 24 * nb, seed=8, rate=rate, device=None).codes
+    codes[min(3, codes.size - 1)] = N_PAPER                      # a code that names no point
+    buf, n = oracle.pack_planes10x(codes, rows, nb)
+    groups, gbytes, idx_off, tab_off = _p10_offsets(rows, nb)
+    assert buf.size == tab_off + 16 * n == oracle.planes10x_bytes(rows, nb, n)
+    xs, cls = oracle.decode_batch(codes)
+    want_o = window_base(xs)
+    index = buf[idx_off: idx_off + 4 * (groups + 1)].view(np.uint32)
+    table = buf[tab_off:].view(np.uint32).reshape(-1, 4)
+    assert index[0] == 0 and index[-1] == n and (np.diff(index.astype(np.int64)) >= 0).all()
+    assert not buf[groups * gbytes: idx_off].any() and not buf[idx_off + 4 * (groups + 1): tab_off].any()
+    expected_entries = []
+    for rg in range(groups):
+        per_group = []
+        for row in range(32 * rg, 32 * rg + 32):
+            for b in range(nb):
+                hb, o, v = _unpack_planes10x_cell(buf, rows, nb, row, b)
+                at = row * nb + b
+                if row >= rows or cls[at] < 0:
+                    assert hb == 0 and (v == [0] * 24 if o is not None else v == [8] * 24)
+                    continue
+                x = xs[at]
+                shell, par, gain = int((x.astype(np.int64) ** 2).sum()) // 16, int(x[0]) & 1, int(codes[at]) >> 47
+                u = [8 + (int(c) - par) // 2 for c in x]
+                if o is None:                        # past the tiles: four-bit codes, always exact
+                    assert hb == shell | par << 4 | gain << 5 and v == u
+                elif want_o[at] == 0:                # an exception: nothing in the short record, everything in the table
+                    assert hb == 0 and v == [0] * 24
+                    per_group.append((b // 4, b % 4, row % 32, shell | par << 4 | gain << 5, u))
+                else:
+                    assert o == want_o[at] and hb == shell | par << 4 | gain << 5 | (o - 3) << 6
+                    assert [c + o for c in v] == u and [2 * (c + o - 8) + par for c in v] == x.tolist()
+        per_group.sort(key=lambda t: t[:3])
+        assert index[rg + 1] - index[rg] == len(per_group)
+        expected_entries += per_group
+    assert len(expected_entries) == n
+    for ent, (tile, q, r, hb, u) in zip(table, expected_entries):
+        assert int(ent[0]) == hb | r << 8 | (4 * tile + q) << 13
+        assert [(int(ent[1 + i // 8]) >> (4 * (i % 8))) & 15 for i in range(24)] == u
+    # a table with less room keeps the first entries, and the index stops at the capacity
+    if n > 1:
+        small, n2 = oracle.pack_planes10x(codes, rows, nb, capacity=n // 2)
+        assert n2 == n and small.size == tab_off + 16 * (n // 2)
+        assert np.array_equal(small[:idx_off], buf[:idx_off]) and np.array_equal(small[tab_off:], buf[tab_off: tab_off + 16 * (n // 2)])
+        assert np.array_equal(small[idx_off: idx_off + 4 * (groups + 1)].view(np.uint32), np.minimum(index, n // 2))
+
+
+def test_planes10x_layout_worked_example_by_hand(oracle):
+    """One row, four blocks: index 0 = (0^22, 4, 4) (shell 2: codes 8 and 10, window base 3, stored 5 and 7), a code
+    that names no point, index 0 with the gain bit, and (8, -8, 0^22) (shell 8: codes 12, 4, 8 - no window)."""
+    x = np.zeros(24, np.int8)
+    x[0], x[1] = 8, -8
+    wide = oracle.encode(x)
+    buf, n = oracle.pack_planes10x(np.array([0, N_PAPER, 1 << 47, wide], np.uint64), 1, 4)
+    assert n == 1 and buf.size == 1280 + 128 + 16
+    words = buf[:1152].view(np.uint32)
+    # row 0 is (m, e, g) = (0, 0, 0): lanes 0..3.  Block 0 is slot 0 of half-step 0: V0 of lane t holds its coordinates
+    # 4t.. in bits 0..2 and, for t < 2, 16 + 4t.. in bits 3..5 (for t >= 2 those are block 1's: zero)
+    assert [int(words[4 * t]) for t in range(4)] == [0x2D2D2D2D, 0x3D3D2D2D, 0x05050505, 0x05050505]
+    # positions 32.. belong to slot 1 (block 1, empty), so V8 is zero; block 2 is slot 0 of half-step 2: V4 of the
+    # same lanes, at byte 512 + 16 t
+    assert [int(words[128 + 4 * t]) for t in range(4)] == [0x2D2D2D2D, 0x3D3D2D2D, 0x05050505, 0x05050505]
+    assert not words[256:].any()                             # V8 of every lane
+    rest = np.ones(1152 // 4, bool)
+    rest[[0, 4, 8, 12, 128, 132, 136, 140]] = False
+    assert not words[rest].any()
+    hdr = buf[1152:1280]
+    assert int(hdr[0]) == 2 and int(hdr[4]) == (2 | 1 << 5) and int(hdr.astype(np.int64).sum()) == 2 + 34
+    assert buf[1280:1288].view(np.uint32).tolist() == [0, 1]
+    assert buf[1408:1424].view(np.uint32).tolist() == [8 | 0 << 8 | 3 << 13, 0x8888884C, 0x88888888, 0x88888888]
+
+
+def test_planes10x_rate_on_the_synthetic_stream(oracle):
+    """About one block in eight thousand of the synthetic stream is an exception; the paper's rule (five levels)
+    would send about one in 160 to the table."""
+    from helpers import window_base
+    from paper_2609_02652_b200 import datagen
+
+    codes = datagen.make_codes(1024, 128, 21).numpy().astype(np.uint64).ravel()
+    xs, _ = oracle.decode_batch(codes)
+    rate = float((window_base(xs) == 0).mean())
+    assert 0.00005 < rate < 0.0004
+    levels = np.array([len(set(np.abs(r).tolist())) for r in xs[:20000]])
+    assert 0.004 < float((levels >= 5).mean()) < 0.009
+    _, n = oracle.pack_planes10x(codes, 1024, 128)
+    assert n == int((window_base(xs) == 0).sum())
+
+
 @pytest.mark.parametrize("rows,nb", [(32, 3), (37, 5)])
 def test_onehot_layout_round_trip_and_field_widths(oracle, rows, nb):
     codes = _codes(oracle, rows, nb, seed=6)
