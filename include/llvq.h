@@ -87,7 +87,10 @@
  *                byte of LLVQ_PLANES13 in place of the class:
  *                  v_i = u_i - o, u_i the four-bit code of LLVQ_PLANES, o the block's window base: the
  *                  smallest o in {3, 4, 5, 6} with o <= min u_i and max u_i <= o + 7;
- *                  header byte = shell | parity << 4 | gain << 5 | (o - 3) << 6;  x_i = 2 (v_i + o - 8) + parity.
+ *                  header byte = (f ^ shell) | shell << 4 with f = (o - 3) | parity << 2 | gain << 3;
+ *                  x_i = 2 (v_i + o - 8) + parity.  (The byte indexes a table in shared memory whose bank is
+ *                  chosen by the low four bits: with the shell mixed into them, the headers that occur
+ *                  together in a tile - a few shells, either parity, either gain - fall into different banks.)
  *                A block with no such o (its codes span more than eight consecutive values, or reach below 3)
  *                is an EXCEPTION: its short record is all zero - the empty record, which adds nothing - and
  *                its exact record goes to the table.  Rows past the end and codes that name no point also
@@ -106,7 +109,7 @@
  *                  Vk of lane L at byte 16 L + 4 k (k < 4), 512 + 16 L + 4 (k - 4) (k < 8), 1024 + 4 L
  *                  (k = 8); header byte of pair P, half-step h, row half e at 1152 + 8 P + 2 h + e.
  *                  The nb mod 4 blocks left over follow the tiles exactly as in LLVQ_PLANES13 (four-bit
- *                  codes, bits 6, 7 of the header byte zero: a pair of 832 bytes, a single of 416): they
+ *                  codes, that layout's header byte: a pair of 832 bytes, a single of 416): they
  *                  hold every block exactly and never make an exception.  A row group takes
  *                  1280 (nb / 4) + 416 (nb mod 4) bytes.
  *                  After the last row group, at the next multiple of 128 bytes: the index, one uint32 a
@@ -120,9 +123,11 @@
  *                exception in 32 blocks.  llvq_expand takes the room for entries from out_bytes; entries that
  *                do not fit are dropped, the index stops at the capacity, and the next llvq_status returns
  *                LLVQ_ESIZE.  k_padded / 24 must be below 2^19.
- *                Accepted by the calls that accept LLVQ_PLANES13.  With no exception in a matrix y is bit for
- *                bit what LLVQ_PLANES gives; an exception's product is rounded to the accumulator's quantum
- *                by itself instead of together with its tile's.
+ *                Accepted by the calls that accept LLVQ_PLANES13.  y is reproducible (the same bits for the
+ *                same buffer whatever the launch) and agrees with LLVQ_PLANES to within a few accumulator
+ *                quanta a tile, not bit for bit: a block's integer sum is the same, but its two halves (low
+ *                and high limbs of x) split differently for a shifted code before each is rounded to f32, and
+ *                an exception's product is rounded to the quantum by itself instead of with its tile's.
  */
 #ifndef LLVQ_H
 #define LLVQ_H

@@ -613,7 +613,7 @@ void llvqo_pack_planes13(const uint64_t *codes, int64_t rows, int64_t nb, uint8_
  * 10-byte layout with an exception table (the sparse overlay of Sec. 3.3, with a window code in place of the
  * paper's level code).  For a block with four-bit codes u_0..u_23 (u_i = 8 + floor(x_i / 2)) the window base o
  * is the smallest of 3, 4, 5, 6 with o <= min u and max u <= o + 7; the short record keeps v_i = u_i - o in three
- * bits and the header byte shell | parity << 4 | gain << 5 | (o - 3) << 6.  A block with no such o is an
+ * bits and the header byte (f ^ shell) | shell << 4, f = (o - 3) | parity << 2 | gain << 3.  A block with no such o is an
  * exception: all-zero short record, exact record in the table.  Rows past the end and codes that name no point:
  * all-zero short record, no table entry.
  *
@@ -625,7 +625,7 @@ void llvqo_pack_planes13(const uint64_t *codes, int64_t rows, int64_t nb, uint8_
  * bits 0, 1 of code i of Xk are bits 6, 7 of byte i of Vk; bit 2 of it is bit 6 + (k & 1) of byte i of V(6 + (k >> 1)).
  * Vk of lane L at 16 L + 4 k (k < 4), 512 + 16 L + 4 (k - 4) (k < 8), 1024 + 4 L (k = 8); header byte of pair P,
  * half-step h, row half e at 1152 + 8 P + 2 h + e.
- * The nb mod 4 last blocks follow in the 13-byte layout's pair and single (four-bit codes, exact).
+ * The nb mod 4 last blocks follow in the 13-byte layout's pair and single (four-bit codes, that layout's header byte, exact).
  * After the row groups, at the next multiple of 128: the index (row groups + 1 uint32; entry g = exceptions of the
  * row groups before g, never above the capacity); after it, at the next multiple of 128: the table, 16 bytes an
  * entry, in the order row group, tile, block, row: word 0 = shell | parity << 4 | gain << 5 | row of the group << 8 |
@@ -673,7 +673,7 @@ int64_t llvqo_pack_planes10x(const uint64_t *codes, int64_t rows, int64_t nb, ui
                 hb[at] = empty ? 0 : (uint8_t)(g_cls[rec.cls].shell | (parity << 4) | (rec.gain << 5));
                 int o = empty ? 0 : window_base(u + at * 24);
                 exc[at] = !empty && o == 0;
-                hs[at] = o ? (uint8_t)(hb[at] | ((o - 3) << 6)) : 0;
+                hs[at] = o ? (uint8_t)((((o - 3) | (parity << 2) | (rec.gain << 3)) ^ g_cls[rec.cls].shell) | (g_cls[rec.cls].shell << 4)) : 0;
                 for (int i = 0; i < NCOORD; i++) v[at * 24 + i] = o ? (uint8_t)(u[at * 24 + i] - o) : 0;
             }
         uint8_t *grp = out + (size_t)rg * gbytes;

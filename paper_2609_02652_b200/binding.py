@@ -15,6 +15,7 @@ import torch
 PLANES = 0
 ONEHOT = 1
 PLANES13 = 2      # the 14-byte layout's codes with a one-byte header: 13 bytes a block
+PLANES10X = 3     # three-bit window codes, 10 bytes a block, plus a table of the blocks no window holds
 MAX_GROUP = 8
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libllvq.so")
@@ -24,6 +25,7 @@ SYMBOLS = (
     "llvq_create", "llvq_destroy", "llvq_strerror", "llvq_status", "llvq_selftest_wait_limit", "llvq_set_pdl", "llvq_num_classes", "llvq_class_base", "llvq_layout_bytes",
     "llvq_expand", "llvq_gemv", "llvq_gemv_batch", "llvq_gemv_plan", "llvq_gemv_grouped", "llvq_gemv_static", "llvq_gemv_fp16", "llvq_gemv_noweights", "llvq_dequant_fp16",
     "llvq_decode_i8", "llvq_rotate", "llvq_rotate_block", "llvq_gemv_rotated", "llvq_static_status", "llvq_static_selftest_wait_limit",
+    "llvq_overlay_count", "llvq_overlay_bytes",
 )
 
 
@@ -78,6 +80,8 @@ def load() -> ctypes.CDLL:
         L.llvq_gemv_rotated.argtypes = [vp, ctypes.POINTER(Problem), ci, vp, i64, ctypes.POINTER(Rotation), vp]
         L.llvq_static_status.argtypes = [vp]
         L.llvq_static_selftest_wait_limit.argtypes = [vp]
+        L.llvq_overlay_count.argtypes = [vp, vp, i64, i64, ctypes.POINTER(ctypes.c_uint64), vp]
+        L.llvq_overlay_bytes.argtypes = [i64, i64, ctypes.c_uint64, ctypes.POINTER(sz)]
         L.llvq_rotate_block.argtypes = [i64, i64]
         L.llvq_rotate_block.restype = i64
         for name in SYMBOLS:
@@ -142,7 +146,8 @@ def destroy(ctx: Context) -> None:
 
 def status(ctx: Context, stream=None) -> None:
     """Synchronises the stream; raises LlvqError(-5) if a kernel on this context gave up on a bounded wait, else
-    LlvqError(-6) if an expansion since the last call met a code word that names no point."""
+    LlvqError(-3) if a PLANES10X expansion had more exceptions than its buffer had room for, else LlvqError(-6) if an
+    expansion since the last call met a code word that names no point."""
     _check(load().llvq_status(ctx.ptr, _stream(stream)), "llvq_status")
 
 
@@ -169,9 +174,25 @@ def layout_bytes(layout: int, rows: int, k_padded: int) -> int:
     return int(n.value)
 
 
+def overlay_bytes(rows: int, k_padded: int, exceptions: int) -> int:
+    """Bytes of a PLANES10X buffer with room for `exceptions` entries in its exception table."""
+    n = ctypes.c_size_t()
+    _check(load().llvq_overlay_bytes(int(rows), int(k_padded), int(exceptions), ctypes.byref(n)), "llvq_overlay_bytes")
+    return int(n.value)
+
+
+def overlay_count(ctx: Context, codes: torch.Tensor, rows: int, nb: int, stream=None) -> int:
+    """Blocks of the matrix that PLANES10X keeps in its exception table (synchronises the stream)."""
+    n = ctypes.c_uint64()
+    _check(load().llvq_overlay_count(ctx.ptr, _dev(codes, torch.int64, "codes"), int(rows), int(nb), ctypes.byref(n), _stream(stream)),
+           "llvq_overlay_count")
+    return int(n.value)
+
+
 def expand(ctx: Context, layout: int, codes: torch.Tensor, rows: int, nb: int, out: torch.Tensor | None = None,
            bad_count: torch.Tensor | None = None, stream=None) -> torch.Tensor:
-    """codes: int64 CUDA tensor of rows*nb code words -> uint8 layout buffer."""
+    """codes: int64 CUDA tensor of rows*nb code words -> uint8 layout buffer (PLANES10X: sized by llvq_layout_bytes,
+    i.e. with room for one exception in 32 blocks, unless `out` is given)."""
     if out is None:
         out = torch.empty(layout_bytes(layout, rows, nb * 24), dtype=torch.uint8, device=codes.device)
     bc = _dev(bad_count, torch.int32, "bad_count") if bad_count is not None else None

@@ -42,7 +42,7 @@ const char *llvq_strerror(int code) {
         case LLVQ_OK: return "ok";
         case LLVQ_EINVAL: return "invalid argument (null pointer, bad shape or unknown layout)";
         case LLVQ_EALIGN: return "device pointer not aligned as documented";
-        case LLVQ_ESIZE: return "buffer or context scratch too small";
+        case LLVQ_ESIZE: return "buffer or context scratch too small (from llvq_status: an exception table had no room for some of its entries)";
         case LLVQ_ECUDA: return "CUDA runtime error";
         case LLVQ_ETIMEOUT: return "a bounded wait inside a kernel ran out; the affected outputs are incomplete";
         case LLVQ_EINDEX: return "a code word named no point of the ball (index out of range or bits above bit 47 set); its record is empty";
@@ -105,11 +105,14 @@ int llvq_create(llvq_ctx **out, int device, size_t scratch_bytes) {
     ctx->accum_slots = scratch_bytes / 8;
     if (cudaMalloc(&ctx->accum, ctx->accum_slots * 8) != cudaSuccess ||
         cudaMemset(ctx->accum, 0, ctx->accum_slots * 8) != cudaSuccess ||
-        cudaMalloc(&ctx->error, 8) != cudaSuccess || cudaMemset(ctx->error, 0, 8) != cudaSuccess) {
+        cudaMalloc(&ctx->error, 32) != cudaSuccess || cudaMemset(ctx->error, 0, 32) != cudaSuccess) {
         llvq_destroy(ctx);
         return LLVQ_ECUDA;
     }
+    // one small block: the error flag, the two counts llvq_status reports, and the scratch of llvq_overlay_count
     ctx->bad_codes = reinterpret_cast<uint32_t *>(ctx->error + 1);
+    ctx->overflow = reinterpret_cast<uint32_t *>(ctx->error + 2);
+    ctx->counter = reinterpret_cast<unsigned long long *>(ctx->error + 4);
     if (gemv_configure(ctx) != 0 || rotate_configure() != 0 || cudaDeviceSynchronize() != cudaSuccess) { llvq_destroy(ctx); return LLVQ_ECUDA; }
     *out = ctx;
     return LLVQ_OK;
@@ -128,13 +131,17 @@ int llvq_status(llvq_ctx *ctx, void *stream) {
     if (!ctx) return LLVQ_EINVAL;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;
-    int flags[2] = {0, 0};                             // {a wait ran out, codes that named no point}
+    int flags[3] = {0, 0, 0};                          // {a wait ran out, codes that named no point, table entries without room}
     if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return LLVQ_ECUDA;
-    if (cudaMemcpy(flags, ctx->error, 8, cudaMemcpyDeviceToHost) != cudaSuccess) return LLVQ_ECUDA;
+    if (cudaMemcpy(flags, ctx->error, 12, cudaMemcpyDeviceToHost) != cudaSuccess) return LLVQ_ECUDA;
     if (flags[0]) {
         cudaMemset(ctx->error, 0, 4);
         cudaMemset(ctx->accum, 0, ctx->accum_slots * 8);   // an abandoned reduction leaves sums behind
         return LLVQ_ETIMEOUT;
+    }
+    if (flags[2]) {
+        cudaMemset(ctx->overflow, 0, 4);
+        return LLVQ_ESIZE;
     }
     if (flags[1]) {
         cudaMemset(ctx->bad_codes, 0, 4);
@@ -163,8 +170,31 @@ uint64_t llvq_class_base(const llvq_ctx *ctx, int c) {
     return ctx->host.base[(size_t)c];
 }
 
+int llvq_overlay_bytes(int64_t rows, int64_t k_padded, uint64_t exceptions, size_t *bytes) {
+    if (!bytes || rows <= 0 || k_padded <= 0 || k_padded % 24 != 0 || k_padded / 24 >= ((int64_t)1 << 19)) return LLVQ_EINVAL;
+    *bytes = overlay_table_offset(rows, k_padded / 24) + (size_t)exceptions * 16;
+    return LLVQ_OK;
+}
+
+int llvq_overlay_count(llvq_ctx *ctx, const uint64_t *codes, int64_t rows, int64_t nb, uint64_t *count, void *stream) {
+    if (!ctx || !codes || !count || rows <= 0 || nb <= 0 || nb >= ((int64_t)1 << 19)) return LLVQ_EINVAL;
+    if (!aligned(codes, 8)) return LLVQ_EALIGN;
+    if (rows * nb > ((int64_t)1 << 36)) return LLVQ_ESIZE;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return LLVQ_ECUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    unsigned long long n = 0;
+    if (cudaMemsetAsync(ctx->counter, 0, 8, s) != cudaSuccess || launch_overlay_count(ctx, codes, rows, nb, ctx->counter, s) != cudaSuccess ||
+        cudaMemcpyAsync(&n, ctx->counter, 8, cudaMemcpyDeviceToHost, s) != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess)
+        return LLVQ_ECUDA;
+    *count = n;
+    return LLVQ_OK;
+}
+
 int llvq_layout_bytes(int layout, int64_t rows, int64_t k_padded, size_t *bytes) {
     if (!bytes || rows <= 0 || k_padded <= 0 || k_padded % 24 != 0) return LLVQ_EINVAL;
+    if (layout == LLVQ_PLANES10X)       // room for one exception in 32 blocks
+        return llvq_overlay_bytes(rows, k_padded, (uint64_t)((rows * (k_padded / 24) + 31) / 32), bytes);
     if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT && layout != LLVQ_PLANES13) return LLVQ_EINVAL;
     const size_t groups = (size_t)((rows + kRowsPerGroup - 1) / kRowsPerGroup);
     *bytes = groups * (size_t)(k_padded / 24) * (size_t)layout_cell_bytes(layout);
@@ -175,7 +205,8 @@ int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, 
                 size_t out_bytes, uint32_t *bad_count, void *stream) {
     if (!ctx || !codes || !layout_out || rows <= 0 || nb <= 0) return LLVQ_EINVAL;
     size_t need = 0;
-    if (llvq_layout_bytes(layout, rows, nb * 24, &need) != LLVQ_OK) return LLVQ_EINVAL;
+    // the 10-byte layout takes whatever room the buffer has past its fixed part for the exception table
+    if ((layout == LLVQ_PLANES10X ? llvq_overlay_bytes(rows, nb * 24, 0, &need) : llvq_layout_bytes(layout, rows, nb * 24, &need)) != LLVQ_OK) return LLVQ_EINVAL;
     if (out_bytes < need) return LLVQ_ESIZE;
     if (!aligned(layout_out, 128) || !aligned(codes, 8) || (bad_count && !aligned(bad_count, 4))) return LLVQ_EALIGN;
     if (rows * nb > ((int64_t)1 << 36)) return LLVQ_ESIZE;
@@ -184,7 +215,7 @@ int llvq_expand(llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, 
     // the GEMV reads records ahead of its wait for the previous kernel of the stream: the next one on this context
     // is launched as an ordinary kernel, so that it cannot overtake this expansion
     ctx->weights_dirty = 1;
-    return launch_expand(ctx, layout, codes, rows, nb, layout_out, bad_count, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
+    return launch_expand(ctx, layout, codes, rows, nb, layout_out, out_bytes, bad_count, (cudaStream_t)stream) == cudaSuccess ? LLVQ_OK : LLVQ_ECUDA;
 }
 
 constexpr int kVectorsPerPass = 4;      // activation vectors one launch of the GEMV kernel carries
@@ -223,8 +254,9 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
                     bool no_weights, void *stream, int batch = 1, const llvq_rotation *rot = nullptr) {
     if (!ctx || !problems || !x || n < 1 || n > LLVQ_MAX_GROUP) return LLVQ_EINVAL;
     if (batch < 1 || batch > kVectorsPerPass || (batch > 1 && (n != 1 || layout != LLVQ_PLANES || no_weights))) return LLVQ_EINVAL;
-    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT && layout != LLVQ_PLANES13) return LLVQ_EINVAL;
-    if (layout == LLVQ_PLANES13 && (no_weights || batch != 1 || rot)) return LLVQ_EINVAL;
+    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT && layout != LLVQ_PLANES13 && layout != LLVQ_PLANES10X) return LLVQ_EINVAL;
+    if ((layout == LLVQ_PLANES13 || layout == LLVQ_PLANES10X) && (no_weights || batch != 1 || rot)) return LLVQ_EINVAL;
+    if (layout == LLVQ_PLANES10X && k_padded / 24 >= ((int64_t)1 << 19)) return LLVQ_EINVAL;
     if (k_padded <= 0 || k_padded % 24 != 0) return LLVQ_EINVAL;
     if (k_padded > LLVQ_MAX_K) return LLVQ_ESIZE;
     if (!aligned(x, 16)) return LLVQ_EALIGN;
@@ -251,6 +283,10 @@ static int run_gemv(llvq_ctx *ctx, int layout, const llvq_problem *problems, int
         p.prob[i].group_begin = (int)groups;
         p.prob[i].gain0 = q.gain[0];
         p.prob[i].gain1 = q.gain[1];
+        if (layout == LLVQ_PLANES10X) {
+            p.prob[i].exc_index = reinterpret_cast<const uint32_t *>(p.prob[i].layout + overlay_index_offset(q.rows, p.nb));
+            p.prob[i].exc_table = reinterpret_cast<const uint4 *>(p.prob[i].layout + overlay_table_offset(q.rows, p.nb));
+        }
         gain_max = std::fmax(gain_max, std::fmax(std::fabs(q.gain[0]), std::fabs(q.gain[1])));
         if (q.rows > ((int64_t)1 << 30)) return LLVQ_ESIZE;
         groups += (q.rows + kRowsPerGroup - 1) / kRowsPerGroup;
@@ -382,7 +418,7 @@ int llvq_dequant_fp16(llvq_ctx *ctx, int layout, const void *layout_buf, const v
 int llvq_decode_i8(llvq_ctx *ctx, int layout, const void *layout_buf, int8_t *coords, uint16_t *class_ids, int64_t rows,
                    int64_t nb, void *stream) {
     if (!ctx || !layout_buf || !coords || !class_ids || rows <= 0 || nb <= 0) return LLVQ_EINVAL;
-    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT && layout != LLVQ_PLANES13) return LLVQ_EINVAL;
+    if (layout != LLVQ_PLANES && layout != LLVQ_ONEHOT && layout != LLVQ_PLANES13 && layout != LLVQ_PLANES10X) return LLVQ_EINVAL;
     if (!aligned(layout_buf, 128) || !aligned(class_ids, 2)) return LLVQ_EALIGN;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return LLVQ_ECUDA;

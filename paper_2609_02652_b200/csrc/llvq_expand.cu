@@ -137,10 +137,37 @@ __device__ __forceinline__ uint32_t bytes4(uint32_t a, uint32_t b) {
     return (a & 0xffu) | ((a >> 8) & 0xff00u) | ((b & 0xffu) << 16) | ((b << 8) & 0xff000000u);
 }
 
-// COMPACT: the 13-byte layout - the same code words, the header one byte: shell | parity << 4 | gain << 5.
-template <bool COMPACT>
+// The window base of the 10-byte layout for a block's 24 four-bit codes (three words of eight nibbles): the
+// smallest o in 3..6 with o <= the smallest code and the largest code <= o + 7; 0 if there is none.
+__device__ __forceinline__ uint32_t window_base(const uint32_t cw[3]) {
+    uint32_t lo = 15u, hi = 0u;
+#pragma unroll
+    for (int j = 0; j < 3; j++)
+#pragma unroll
+        for (int n = 0; n < 8; n++) {
+            const uint32_t u = (cw[j] >> (4 * n)) & 15u;
+            lo = min(lo, u);
+            hi = max(hi, u);
+        }
+    const uint32_t o = max(3u, hi > 7u ? hi - 7u : 0u);
+    return o <= min(6u, lo) ? o : 0u;
+}
+
+// header byte of the 13-byte layout: shell | parity << 4 | gain << 5 (0 for the empty record)
+__device__ __forceinline__ uint32_t header_byte(const DeviceTables &T, const Decoded &d) {
+    return d.cls == kEmptyClass ? 0u : ((uint32_t)T.desc[d.cls].shell | ((uint32_t)T.desc[d.cls].odd << 4) | ((uint32_t)d.gain << 5));
+}
+
+// LAYOUT = LLVQ_PLANES, LLVQ_PLANES13 (the same code words, the header one byte) or LLVQ_PLANES10X (tiles of
+// three-bit window codes, the blocks a window cannot hold listed in the exception table; the leftover blocks as in
+// LLVQ_PLANES13).  For LLVQ_PLANES10X the first word of every tile holds, on entry, the tile's first entry in its row
+// group's part of the table (overlay_offsets_kernel), `index` the row groups' first entries, and `capacity` the
+// entries the table has room for.
+template <int LAYOUT>
 __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, const uint64_t *__restrict__ codes, int64_t rows, int64_t nb,
-                                                            uint8_t *__restrict__ out, uint32_t *bad_count, uint32_t *ctx_bad) {
+                                                            uint8_t *__restrict__ out, uint32_t *bad_count, uint32_t *ctx_bad,
+                                                            const uint32_t *index, uint4 *table, uint32_t capacity) {
+    constexpr bool COMPACT = LAYOUT != LLVQ_PLANES, OVERLAY = LAYOUT == LLVQ_PLANES10X;
     __shared__ uint32_t nat_all[8][4][4][32];              // [warp][block of the piece][word 0..2, header][row]
     const int64_t tiles = nb / kTileCells, left = nb % kTileCells;
     const int64_t pieces = tiles + (left >= 2 ? 1 : 0) + (left & 1);
@@ -152,12 +179,17 @@ __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, cons
     uint32_t (*nat)[4][32] = nat_all[threadIdx.x >> 5];
     const int64_t rg = piece_id / pieces, u = piece_id % pieces;
     const int64_t row = rg * kRowsPerGroup + lane;
-    constexpr int kCell = COMPACT ? kCell13Bytes : kCellBytes, kTile = COMPACT ? kTile13Bytes : kTileBytes;
-    uint8_t *grp = out + (size_t)rg * (size_t)nb * kCell;
+    constexpr int kCell = COMPACT ? kCell13Bytes : kCellBytes, kTile = OVERLAY ? kTile10Bytes : (COMPACT ? kTile13Bytes : kTileBytes);
+    uint8_t *grp = out + (size_t)rg * ((size_t)tiles * kTile + (size_t)left * kCell);
     const bool is_tile = u < tiles;
     const bool is_pair = !is_tile && left >= 2 && u == tiles;
     const int ncell = is_tile ? 4 : (is_pair ? 2 : 1);
     const int64_t b0 = is_tile ? u * kTileCells : (is_pair ? tiles * kTileCells : nb - 1);
+    uint32_t next_entry = 0;                               // OVERLAY: where this tile's next exception goes
+    if (OVERLAY && is_tile) {
+        next_entry = index[rg] + *reinterpret_cast<const uint32_t *>(grp + (size_t)u * kTile);
+        __syncwarp();                                      // every lane has read the word before any lane overwrites it
+    }
     int bad = 0;
 #pragma unroll 1
     for (int q = 0; q < ncell; q++) {
@@ -167,9 +199,26 @@ __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, cons
         } else {
             d.cls = kEmptyClass; d.gain = 0; d.smask = 0; d.mag[0] = d.mag[1] = d.mag[2] = 0;
         }
-        nat[q][0][lane] = code_word(d, 0); nat[q][1][lane] = code_word(d, 1); nat[q][2][lane] = code_word(d, 2);
-        if (COMPACT) nat[q][3][lane] = d.cls == kEmptyClass ? 0u : ((uint32_t)T.desc[d.cls].shell | ((uint32_t)T.desc[d.cls].odd << 4) | ((uint32_t)d.gain << 5));
-        else nat[q][3][lane] = (uint32_t)d.cls | ((uint32_t)d.gain << 9);
+        uint32_t cw[3] = {code_word(d, 0), code_word(d, 1), code_word(d, 2)};
+        uint32_t hdr = COMPACT ? header_byte(T, d) : ((uint32_t)d.cls | ((uint32_t)d.gain << 9));
+        if (OVERLAY && is_tile) {
+            const uint32_t o = d.cls == kEmptyClass ? 0u : window_base(cw);
+            const bool exception = d.cls != kEmptyClass && o == 0u;
+            // the tile's exceptions in the order block, row: this block's follow those of the blocks before
+            const uint32_t votes = __ballot_sync(0xffffffffu, exception);
+            if (exception) {
+                const uint32_t at = next_entry + __popc(votes & ((1u << lane) - 1u));
+                if (at < capacity) table[at] = make_uint4(hdr | (uint32_t)lane << 8 | (uint32_t)(b0 + q) << 13, cw[0], cw[1], cw[2]);
+            }
+            next_entry += __popc(votes);
+            // no borrow between nibbles: every code is at least o
+#pragma unroll
+            for (int j = 0; j < 3; j++) cw[j] = o ? cw[j] - o * 0x11111111u : 0u;
+            // the short record's header byte: the shell above, and below it window, parity and gain mixed with the shell
+            hdr = o ? (((o - 3u) | ((hdr >> 4) & 3u) << 2) ^ (hdr & 15u)) | (hdr & 15u) << 4 : 0u;
+        }
+        nat[q][0][lane] = cw[0]; nat[q][1][lane] = cw[1]; nat[q][2][lane] = cw[2];
+        nat[q][3][lane] = hdr;
     }
     __syncwarp();
     const int g = lane >> 2, t = lane & 3;
@@ -191,7 +240,28 @@ __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, cons
         w[2] = spread4(quad(q0, m, 0, 32 + 4 * t)) | spread4(quad(q0, m, 1, 32 + 4 * t)) << 4;
         hw = header(q0, m, 0, t >> 1) | header(q0, m, 1, t >> 1) << 16;
     };
-    if (is_tile) {
+    if (OVERLAY && is_tile) {
+        // Group(h, e, c): byte i = code i of row (m, e, g) at positions 16c + 4t + i (c < 2) or 32 + 4t + i of half-step h
+        auto group = [&](int h, int e, int c) -> uint32_t { return spread4(quad(2 * (h >> 1), h & 1, e, (c < 2 ? 16 * c : 32) + 4 * t)); };
+        uint32_t V[9], hw[4];
+#pragma unroll
+        for (int k = 0; k < 8; k++) V[k] = group(k >> 1, k & 1, 0) | group(k >> 1, k & 1, 1) << 3;
+        V[8] = group(0, 0, 2) | group(1, 0, 2) << 3;
+        // the six groups left go to bits 6, 7: the low two bits of Xk to Vk, its third bit to V(6 + k / 2)
+        const uint32_t X[6] = {group(0, 1, 2), group(1, 1, 2), group(2, 0, 2), group(2, 1, 2), group(3, 0, 2), group(3, 1, 2)};
+#pragma unroll
+        for (int k = 0; k < 6; k++) {
+            V[k] |= (X[k] & 0x03030303u) << 6;
+            V[6 + (k >> 1)] |= ((X[k] >> 2) & 0x01010101u) << (6 + (k & 1));
+        }
+#pragma unroll
+        for (int h = 0; h < 4; h++) hw[h] = header(2 * (h >> 1), h & 1, 0, t >> 1) | header(2 * (h >> 1), h & 1, 1, t >> 1) << 16;
+        uint8_t *tile = grp + (size_t)u * kTile;
+        *reinterpret_cast<uint4 *>(tile + 16 * lane) = make_uint4(V[0], V[1], V[2], V[3]);
+        *reinterpret_cast<uint4 *>(tile + 512 + 16 * lane) = make_uint4(V[4], V[5], V[6], V[7]);
+        *reinterpret_cast<uint32_t *>(tile + 1024 + 4 * lane) = V[8];
+        if ((t & 1) == 0) *reinterpret_cast<uint2 *>(tile + 1152 + 8 * (lane >> 1)) = make_uint2(bytes4(hw[0], hw[1]), bytes4(hw[2], hw[3]));
+    } else if (is_tile) {
         uint32_t w[12], hw[4];
 #pragma unroll
         for (int h = 0; h < 4; h++) half_step(2 * (h >> 1), h & 1, w + 3 * h, hw[h]);
@@ -271,18 +341,143 @@ __global__ void __launch_bounds__(256) expand_onehot_kernel(DeviceTables T, cons
     }
 }
 
+
+// ---- the exception table of the 10-byte layout is filled in a fixed order, so its entries' places are known before
+// they are written.  One warp a tile counts the tile's exceptions (lane = row).  WRITE: the count goes to the tile's
+// first word (the tile itself is written later); else the counts are added up in *total.
+template <bool WRITE>
+__global__ void __launch_bounds__(256) overlay_count_kernel(DeviceTables T, const uint64_t *__restrict__ codes, int64_t rows, int64_t nb,
+                                                            uint8_t *out, unsigned long long *total) {
+    const int64_t tiles = nb / kTileCells;
+    const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = (int)(gid & 31);
+    const int64_t tile_id = gid >> 5;
+    const int64_t groups = (rows + kRowsPerGroup - 1) / kRowsPerGroup;
+    if (tile_id >= groups * tiles) return;
+    const int64_t rg = tile_id / tiles, u = tile_id % tiles, row = rg * kRowsPerGroup + lane;
+    uint32_t count = 0;
+#pragma unroll 1
+    for (int q = 0; q < kTileCells; q++) {
+        Decoded d;
+        bool exception = false;
+        if (row < rows && decode_code(codes[row * nb + u * kTileCells + q], T, d)) {
+            const uint32_t cw[3] = {code_word(d, 0), code_word(d, 1), code_word(d, 2)};
+            exception = window_base(cw) == 0u;
+        }
+        count += __popc(__ballot_sync(0xffffffffu, exception));
+    }
+    if (lane == 0) {
+        if (WRITE) *reinterpret_cast<uint32_t *>(out + (size_t)rg * overlay_group_bytes(nb) + (size_t)u * kTile10Bytes) = count;
+        else if (count) atomicAdd(total, (unsigned long long)count);
+    }
+}
+
+// One warp a row group: the tiles' counts become their first entries inside the row group's part of the table
+// (an exclusive running sum, left in the same words), and the row group's total goes to index[g + 1].
+__global__ void __launch_bounds__(256) overlay_offsets_kernel(uint8_t *out, int64_t groups, int64_t nb, uint32_t *index) {
+    const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = (int)(gid & 31);
+    const int64_t rg = gid >> 5, tiles = nb / kTileCells;
+    if (rg >= groups) return;
+    uint8_t *grp = out + (size_t)rg * overlay_group_bytes(nb);
+    uint32_t running = 0;
+    for (int64_t base = 0; base < tiles; base += 32) {
+        const int64_t u = base + lane;
+        uint32_t *word = reinterpret_cast<uint32_t *>(grp + (size_t)u * kTile10Bytes);
+        const uint32_t c = u < tiles ? *word : 0u;
+        uint32_t incl = c;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += v;
+        }
+        if (u < tiles) *word = running + incl - c;
+        running += __shfl_sync(0xffffffffu, incl, 31);
+    }
+    if (lane == 0) index[rg + 1] = running;
+}
+
+// One CTA: index[g + 1] = totals of the row groups up to g (index[0] = 0), in place.
+__global__ void __launch_bounds__(1024) overlay_index_kernel(uint32_t *index, int64_t groups) {
+    __shared__ uint32_t warp_sum[32];
+    __shared__ uint32_t carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) { carry_s = 0; index[0] = 0; }
+    __syncthreads();
+    for (int64_t base = 0; base < groups; base += 1024) {
+        const int64_t g = base + tid;
+        const uint32_t c = g < groups ? index[g + 1] : 0u;
+        uint32_t incl = c;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, off);
+            if (lane >= off) incl += v;
+        }
+        if (lane == 31) warp_sum[warp] = incl;
+        __syncthreads();
+        uint32_t before = carry_s;
+        for (int w = 0; w < warp; w++) before += warp_sum[w];
+        if (g < groups) index[g + 1] = before + incl;
+        __syncthreads();
+        if (tid == 1023) carry_s = before + incl;
+        __syncthreads();
+    }
+}
+
+// After the table is filled (one CTA): the index stops at the capacity (so that no reader looks past the table), the
+// entries that found no room are counted, and the bytes between the parts of the buffer are zeroed.
+__global__ void __launch_bounds__(256) overlay_finish_kernel(uint8_t *out, size_t records_end, size_t index_offset, size_t table_offset,
+                                                             int64_t groups, uint32_t capacity, uint32_t *overflow) {
+    uint32_t *index = reinterpret_cast<uint32_t *>(out + index_offset);
+    const int tid = threadIdx.x;
+    if (tid == 0 && index[groups] > capacity) atomicAdd(overflow, index[groups] - capacity);
+    __syncthreads();                                       // the total is read before it is clamped
+    for (int64_t i = tid; i <= groups; i += blockDim.x) index[i] = min(index[i], capacity);
+    for (size_t i = records_end + tid; i < index_offset; i += blockDim.x) out[i] = 0;
+    for (size_t i = index_offset + (size_t)(groups + 1) * 4 + tid; i < table_offset; i += blockDim.x) out[i] = 0;
+}
+
 }  // namespace
 
+cudaError_t launch_overlay_count(const llvq_ctx *ctx, const uint64_t *codes, int64_t rows, int64_t nb, unsigned long long *counter,
+                                 cudaStream_t s) {
+    const int64_t groups = (rows + kRowsPerGroup - 1) / kRowsPerGroup, tiles = nb / kTileCells;
+    if (tiles == 0) return cudaSuccess;
+    const int64_t blocks = (groups * tiles * 32 + 255) / 256;
+    overlay_count_kernel<false><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, nullptr, counter);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_expand(const llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, int64_t nb,
-                          void *out, uint32_t *bad_count, cudaStream_t s) {
+                          void *out, size_t out_bytes, uint32_t *bad_count, cudaStream_t s) {
     const int64_t groups = (rows + kRowsPerGroup - 1) / kRowsPerGroup;
-    if (layout == LLVQ_PLANES || layout == LLVQ_PLANES13) {
-        const int64_t left = nb % kTileCells;
-        const int64_t pieces = nb / kTileCells + (left >= 2 ? 1 : 0) + (left & 1);
+    if (layout == LLVQ_PLANES || layout == LLVQ_PLANES13 || layout == LLVQ_PLANES10X) {
+        const int64_t left = nb % kTileCells, tiles = nb / kTileCells;
+        const int64_t pieces = tiles + (left >= 2 ? 1 : 0) + (left & 1);
         const int64_t threads = groups * pieces * 32;
         const int64_t blocks = (threads + 255) / 256;
-        if (layout == LLVQ_PLANES13) expand_planes_kernel<true><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count, ctx->bad_codes);
-        else expand_planes_kernel<false><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count, ctx->bad_codes);
+        if (layout == LLVQ_PLANES10X) {
+            uint8_t *o8 = (uint8_t *)out;
+            const size_t index_offset = overlay_index_offset(rows, nb), table_offset = overlay_table_offset(rows, nb);
+            uint32_t *index = reinterpret_cast<uint32_t *>(o8 + index_offset);
+            uint4 *table = reinterpret_cast<uint4 *>(o8 + table_offset);
+            const size_t room = (out_bytes - table_offset) / 16;
+            const uint32_t capacity = room > 0xffffffffull ? 0xffffffffu : (uint32_t)room;
+            if (tiles > 0) {
+                overlay_count_kernel<true><<<(unsigned)((groups * tiles * 32 + 255) / 256), 256, 0, s>>>(ctx->dev, codes, rows, nb, o8, nullptr);
+                overlay_offsets_kernel<<<(unsigned)((groups * 32 + 255) / 256), 256, 0, s>>>(o8, groups, nb, index);
+            } else {
+                cudaMemsetAsync(index, 0, (size_t)(groups + 1) * 4, s);
+            }
+            overlay_index_kernel<<<1, 1024, 0, s>>>(index, groups);
+            expand_planes_kernel<LLVQ_PLANES10X><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, o8, bad_count, ctx->bad_codes, index, table, capacity);
+            overlay_finish_kernel<<<1, 256, 0, s>>>(o8, (size_t)groups * overlay_group_bytes(nb), index_offset, table_offset, groups, capacity,
+                                                    ctx->overflow);
+        } else if (layout == LLVQ_PLANES13) {
+            expand_planes_kernel<LLVQ_PLANES13><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count, ctx->bad_codes, nullptr, nullptr, 0);
+        } else {
+            expand_planes_kernel<LLVQ_PLANES><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count, ctx->bad_codes, nullptr, nullptr, 0);
+        }
     } else {
         const int64_t threads = groups * nb * 32;
         const int64_t blocks = (threads + 255) / 256;

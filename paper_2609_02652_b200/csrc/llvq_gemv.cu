@@ -318,6 +318,67 @@ __device__ __forceinline__ HalfA decode_half(uint32_t wa, uint32_t wb, uint32_t 
     }
     return h;
 }
+// The 10-byte layout's tile: nine words a lane (va = V0..V3, vb = V4..V7, v8), three bits a code.  Byte i of a word
+// carries code i of two operand words in bits 0..2 and 3..5; bits 6, 7 carry the six operand words left over: the low
+// two bits of Xk in Vk, its third bit in bit 6 + (k & 1) of V(6 + k / 2).  Two shifts and two ANDs a word pair as in the
+// 14-byte layout, four instructions for each of the six.  hb = the eight header bytes of the lane's rows.
+template <int K>
+__device__ __forceinline__ uint32_t overlay_left_over(uint32_t vk, uint32_t vhigh) {
+    // (vk >> 6 & 0x03030303) | (vhigh >> (4 + (K & 1)) & 0x04040404)
+    return and_or(vhigh >> (4 + (K & 1)), 0x04040404u, (vk >> 6) & 0x03030303u);
+}
+template <int SHIFT>
+__device__ __forceinline__ void header_consts(uint32_t hw, uint32_t tq, float2 &k0, float2 &k1) {
+    k0 = lds_f2(and_or(SHIFT >= 3 ? hw >> (SHIFT - 3) : hw << (3 - SHIFT), 0x7f8u, tq));
+    k1 = lds_f2(and_or(hw >> (SHIFT + 5), 0x7f8u, tq));
+}
+__device__ __forceinline__ void decode_overlay_tile(const uint4 &va, const uint4 &vb, uint32_t v8, const uint2 &hb, uint32_t tq,
+                                                    HalfA &h0, HalfA &h1, HalfA &h2, HalfA &h3) {
+    constexpr uint32_t k7 = 0x07070707u;
+    h0.a0 = va.x & k7; h0.a2 = (va.x >> 3) & k7; h0.a1 = va.y & k7; h0.a3 = (va.y >> 3) & k7;
+    h1.a0 = va.z & k7; h1.a2 = (va.z >> 3) & k7; h1.a1 = va.w & k7; h1.a3 = (va.w >> 3) & k7;
+    h2.a0 = vb.x & k7; h2.a2 = (vb.x >> 3) & k7; h2.a1 = vb.y & k7; h2.a3 = (vb.y >> 3) & k7;
+    h3.a0 = vb.z & k7; h3.a2 = (vb.z >> 3) & k7; h3.a1 = vb.w & k7; h3.a3 = (vb.w >> 3) & k7;
+    h0.c0 = v8 & k7; h1.c0 = (v8 >> 3) & k7;
+    h0.c1 = overlay_left_over<0>(va.x, vb.z);            // X0 = Group(0, 1, 2): low bits in V0, third bit in V6
+    h1.c1 = overlay_left_over<1>(va.y, vb.z);            // X1 = Group(1, 1, 2)
+    h2.c0 = overlay_left_over<2>(va.z, vb.w);            // X2 = Group(2, 0, 2): V2 and V7
+    h2.c1 = overlay_left_over<3>(va.w, vb.w);            // X3 = Group(2, 1, 2)
+    h3.c0 = overlay_left_over<4>(vb.x, v8);              // X4 = Group(3, 0, 2): V4 and V8
+    h3.c1 = overlay_left_over<5>(vb.y, v8);              // X5 = Group(3, 1, 2)
+    header_consts<0>(hb.x, tq, h0.k0, h0.k1);
+    header_consts<16>(hb.x, tq, h1.k0, h1.k1);
+    header_consts<0>(hb.y, tq, h2.k0, h2.k1);
+    header_consts<16>(hb.y, tq, h3.k0, h3.k1);
+}
+// nibbles 0..3 of h to the low nibbles of bytes 0..3
+__device__ __forceinline__ uint32_t spread_nibbles(uint32_t h) {
+    h &= 0xffffu;
+    h = (h | (h << 8)) & 0x00ff00ffu;
+    return (h | (h << 4)) & 0x0f0f0f0fu;
+}
+// One entry of the exception table against the x record of its block (`rec`): the block's whole product, in the
+// accumulator's quanta.  The arithmetic of the tile path for one block: integer sums limb pair by limb pair, the
+// block's scale in f32.  `tail_tab` is the table of the four-bit records' headers (the entry's header byte indexes it).
+__device__ __forceinline__ long long exception_value(const uint4 &ent, uint32_t rec, uint32_t tail_tab, float inv_q) {
+    const float2 k = lds_f2(tail_tab + 8 * (ent.x & 63u));
+    const uint32_t cw[3] = {ent.y, ent.z, ent.w};
+    int d[4] = {0, 0, 0, 0};
+#pragma unroll
+    for (int j = 0; j < 3; j++) {
+        const uint32_t lo4 = spread_nibbles(cw[j]), hi4 = spread_nibbles(cw[j] >> 16);
+#pragma unroll
+        for (int l = 0; l < 4; l++) {
+            d[l] = __dp4a((int)lo4, (int)lds32(rec + 24 * l + 8 * j), d[l]);
+            d[l] = __dp4a((int)hi4, (int)lds32(rec + 24 * l + 8 * j + 4), d[l]);
+        }
+    }
+    const int off = __float_as_int(k.y);
+    const int e_lo = off * (int)lds32(rec + 100) + (d[0] + 256 * d[1]);
+    const int e_hi = off * (int)lds32(rec + 104) + (d[2] + 256 * d[3]);
+    return __float2ll_rn(((float)e_lo * k.x + ((float)e_hi * k.x) * 65536.f) * inv_q);
+}
+
 template <bool FIRST>
 __device__ __forceinline__ void contract_half(const HalfA &h, const StepX &sx, float &r0, float &r1) {
     int d[4];
@@ -414,11 +475,15 @@ __device__ __forceinline__ bool advance(const GemvParams &p, Cursor &c, int n) {
 // BATCH sets of total_groups * 32.
 // ROTATE: x is rotated on its way into the records (llvq_gemv_rotated): every CTA rotates the Walsh-Hadamard
 // blocks of x that its share of the matrix touches, exactly as the rotation kernel does, and rounds them to FP16.
-// COMPACT: the 13-byte layout (one header byte a block; the code words are where the 14-byte layout has them).
-template <bool NO_WEIGHTS, int BATCH, bool ROTATE = false, bool COMPACT = false>
+// LAYOUT: LLVQ_PLANES; LLVQ_PLANES13 (one header byte a block; the code words are where the 14-byte layout has them);
+// LLVQ_PLANES10X (tiles of three-bit codes, leftover blocks as in the 13-byte layout, and after each run the exact
+// records of the run's exception blocks, whose short records are empty and add nothing).
+template <bool NO_WEIGHTS, int BATCH, bool ROTATE = false, int LAYOUT = LLVQ_PLANES>
 __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_constant__ GemvParams p) {
-    constexpr int kSrcCell = COMPACT ? kCell13Bytes : kCellBytes;        // bytes of a block column of a row group
-    constexpr int kSrcTile = COMPACT ? kTile13Bytes : kTileBytes;        // bytes of a tile in memory (a ring slot always has kTileBytes)
+    constexpr bool COMPACT = LAYOUT != LLVQ_PLANES, OVERLAY = LAYOUT == LLVQ_PLANES10X;
+    static_assert(!OVERLAY || (BATCH == 1 && !ROTATE && !NO_WEIGHTS), "the 10-byte layout: one vector, as it is");
+    constexpr int kSrcCell = COMPACT ? kCell13Bytes : kCellBytes;        // bytes of a leftover block column of a row group
+    constexpr int kSrcTile = OVERLAY ? kTile10Bytes : (COMPACT ? kTile13Bytes : kTileBytes);   // bytes of a tile in memory (a ring slot always has kTileBytes)
     extern __shared__ __align__(128) unsigned char smem[];
     // shared memory: ring | per-matrix block constants (1024 x {gain / (4 sqrt m), parity - 16}) | x records | barriers
     unsigned char *ring = smem;
@@ -596,6 +661,20 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
         const int row0 = (cc.group - p0.group_begin) * kRowsPerGroup + my_row;
         if (row0 < p0.rows) asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(first_scale_bits) : "l"(p0.row_scale + row0));
     }
+    // 10-byte layout: the first run's range of the exception table, and the index entry after it (see the run loop)
+    uint32_t exc_first0 = 0, exc_first1 = 0, exc_ahead = 0;
+    int exc_q = 0, exc_lg = 0;
+    if constexpr (OVERLAY) {
+        if (n_units > 0) {
+            const GemvProblemDev &p0 = p.prob[q];
+            exc_lg = cc.group - p0.group_begin;
+            const uint32_t *ix = p0.exc_index + exc_lg;
+            asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_first0) : "l"(ix));
+            asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_first1) : "l"(ix + 1));
+            if (exc_lg + 2 <= ((p0.rows + kRowsPerGroup - 1) >> 5)) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_ahead) : "l"(ix + 2));
+            exc_q = q;
+        }
+    }
     uint32_t warm = 0;
     for (int e = tid * 128; e < p.nb * 48 * p.batch; e += kThreads * 128) {
         // a load whose value is not used: the register stays claimed until after the wait (settled() below), so
@@ -626,11 +705,18 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
     // (13-byte layout: the header byte is shell | parity << 4 | gain << 5 - 64 entries a matrix)
     auto build_tables = [&]() {
         if (COMPACT) {
-            for (int e = tid; e < p.nprob * 64; e += kThreads) {
-                const uint32_t shell = e & 15u;
-                const GemvProblemDev &pe = p.prob[e >> 6];
-                tab[(e >> 6) * 1024 + (e & 63)] = make_float2(p.shell_inv_norm[shell] * ((e & 32) ? pe.gain1 : pe.gain0),
-                                                             __int_as_float(shell ? ((e >> 4) & 1) - 16 : 0));
+            // 10-byte layout: 256 entries for the short records' header bytes ((f ^ shell) | shell << 4, f = window base - 3 |
+            // parity << 2 | gain << 3; the base shifts the codes: x = 2 (v + base - 8) + parity), then the 64 of the four-bit records
+            constexpr int kEntries = OVERLAY ? 320 : 64;
+            for (int e = tid; e < p.nprob * kEntries; e += kThreads) {
+                const int m = e / kEntries, h = e - m * kEntries;
+                const bool window = OVERLAY && h < 256;
+                const uint32_t shell = window ? h >> 4 : h & 15;
+                const int f = (h ^ (h >> 4)) & 15;
+                const int parity = window ? (f >> 2) & 1 : (h >> 4) & 1, gain = window ? (f >> 3) & 1 : (h >> 5) & 1;
+                const int base = window ? 2 * (3 + (f & 3)) : 0;
+                const GemvProblemDev &pe = p.prob[m];
+                tab[m * 1024 + h] = make_float2(p.shell_inv_norm[shell] * (gain ? pe.gain1 : pe.gain0), __int_as_float(shell ? parity - 16 + base : 0));
             }
         } else {
             for (int m = 0; m < p.nprob; m++) {
@@ -813,7 +899,31 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
         // a lane's sums are in units of 2^(xexp - 29)
         const float inv_q = pow2f(-29 - pr.qexp_base);
         const uint32_t tq = tab0 + q * 8192;
+        const uint32_t tq_tail = OVERLAY ? tq + 2048 : tq;          // the table the four-bit records' header bytes index
         const int run = min(cc.end - cc.col, n_units - n);
+        // 10-byte layout: the row group's range of the exception table, on its way while the run is summed
+        // 10-byte layout: the row group's range [exc_begin, exc_end) of the exception table.  The first run's was loaded
+        // at the start of the CTA; a run on the next row group of the same matrix takes it from what the run before
+        // loaded ahead; and this lane's entry of the range goes out now, to be used when the run's tiles are summed.
+        uint32_t exc_begin = exc_first0, exc_end = exc_first1;
+        uint4 exc_entry = make_uint4(~0u, 0u, 0u, 0u);          // a block column no run contains
+        if constexpr (OVERLAY) {
+            const int lg = cc.group - pr.group_begin;
+            const uint32_t *ix = pr.exc_index + lg;
+            if (n != 0) {
+                if (q == exc_q && lg == exc_lg + 1) {
+                    exc_begin = exc_first1;
+                    exc_end = exc_ahead;
+                } else {
+                    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_begin) : "l"(ix));
+                    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_end) : "l"(ix + 1));
+                }
+                exc_first0 = exc_begin; exc_first1 = exc_end;
+                exc_q = q; exc_lg = lg;
+                if (lg + 2 <= ((pr.rows + kRowsPerGroup - 1) >> 5)) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_ahead) : "l"(ix + 2));
+            }
+            if (exc_begin + lane < exc_end) exc_entry = __ldg(pr.exc_table + exc_begin + lane);
+        }
         const int run_tiles = NO_WEIGHTS ? 0 : max(0, min(run, tiles - cc.col));
         // the row's scale is needed only by the arrival that finishes the row, but loading it now
         // keeps a cold read off the tail of the kernel
@@ -831,27 +941,33 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
             if (!mbar_try(bar, parity)) {
                 if (!mbar_wait(bar, parity)) { failed = true; break; }
             }
+            // 10-byte layout: nine words a lane (two 128-bit reads and one word) and the eight header bytes of its pair
             const uint4 a0 = lds128(sbuf + lane16);
             const uint4 a1 = lds128(sbuf + lane16 + 512);
-            const uint4 a2 = lds128(sbuf + lane16 + 1024);
-            // headers: four words a lane pair (14-byte layout) or two (13-byte layout: hh.x serves half-steps 0, 1, hh.y 2, 3)
+            const uint4 a2 = OVERLAY ? make_uint4(lds32(sbuf + lane4 + 1024), 0u, 0u, 0u) : lds128(sbuf + lane16 + 1024);
+            // headers: four words a lane pair (14-byte layout) or two (one byte a header: hh.x serves half-steps 0, 1, hh.y 2, 3)
             uint4 hh;
-            if (COMPACT) { const uint2 h2 = lds64(sbuf + (pair16 >> 1) + 1536); hh = make_uint4(h2.x, h2.y, h2.y, h2.x); }
+            if (COMPACT) { const uint2 h2 = lds64(sbuf + (pair16 >> 1) + (OVERLAY ? 1152 : 1536)); hh = make_uint4(h2.x, h2.y, h2.y, h2.x); }
             else hh = lds128(sbuf + pair16 + 1536);
             // The slot's words are in registers: refill it at once with the unit kSlots ahead, so
             // that every slot but the one just read is in flight while this unit is decoded.  The
             // copy's address is made to depend on the loaded words, which holds the copy back
             // until the four shared-memory reads of the whole warp have completed.
-            issue(bar, sbuf + (settled(a0.w, a1.w, a2.w) | settled(hh.w, hh.x, a0.x)));
+            issue(bar, sbuf + (settled(a0.w, a1.w, OVERLAY ? a2.x : a2.w) | settled(hh.w, hh.x, a0.x)));
             float acc[BATCH][4];
             if constexpr (BATCH == 1) {
                 // one vector: every shared-memory load first, then the eight contractions back to back (four independent
                 // accumulator tiles in the tensor pipe at once), then the eight scale steps
                 const StepX s1 = load_step<0>(xa), s2 = load_step<2 * kXRecBytes>(xa);
-                const HalfA h0 = decode_half<COMPACT, 0>(a0.x, a0.y, a0.z, hh.x, tq);
-                const HalfA h1 = decode_half<COMPACT, 16>(a0.w, a1.x, a1.y, COMPACT ? hh.x : hh.y, tq);
-                const HalfA h2 = decode_half<COMPACT, 0>(a1.z, a1.w, a2.x, COMPACT ? hh.y : hh.z, tq);
-                const HalfA h3 = decode_half<COMPACT, 16>(a2.y, a2.z, a2.w, COMPACT ? hh.y : hh.w, tq);
+                HalfA h0, h1, h2, h3;
+                if constexpr (OVERLAY) {
+                    decode_overlay_tile(a0, a1, a2.x, make_uint2(hh.x, hh.y), tq, h0, h1, h2, h3);
+                } else {
+                    h0 = decode_half<COMPACT, 0>(a0.x, a0.y, a0.z, hh.x, tq);
+                    h1 = decode_half<COMPACT, 16>(a0.w, a1.x, a1.y, COMPACT ? hh.x : hh.y, tq);
+                    h2 = decode_half<COMPACT, 0>(a1.z, a1.w, a2.x, COMPACT ? hh.y : hh.z, tq);
+                    h3 = decode_half<COMPACT, 16>(a2.y, a2.z, a2.w, COMPACT ? hh.y : hh.w, tq);
+                }
                 int d0[4], d1[4], d2[4], d3[4];
                 mma_k32(d0, h0.a0, h0.a1, h0.a2, h0.a3, s1.b0, s1.b1);
                 mma_k32(d1, h1.a0, h1.a1, h1.a2, h1.a3, s1.b0, s1.b1);
@@ -921,7 +1037,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
                     const uint32_t wc = lds32(piece + 128 * (3 * m + 2) + lane4);
                     const uint32_t hw = COMPACT ? lds32(piece + 768 + 4 * (lane >> 1)) : lds32(piece + 768 + 8 * (lane >> 1) + 4 * m);
                     guard |= settled(wa, wb, wc) | settled(hw, wa, wb);
-                    const HalfA h = m == 0 ? decode_half<COMPACT, 0>(wa, wb, wc, hw, tq) : decode_half<COMPACT, 16>(wa, wb, wc, hw, tq);
+                    const HalfA h = m == 0 ? decode_half<COMPACT, 0>(wa, wb, wc, hw, tq_tail) : decode_half<COMPACT, 16>(wa, wb, wc, hw, tq_tail);
 #pragma unroll
                     for (int j = 0; j < BATCH; j++) {
                         const uint32_t xj = xt + j * xrec_stride;
@@ -940,7 +1056,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
                 // 13-byte layout: two bytes a lane pair, the pairs two to a word
                 const uint32_t hw = COMPACT ? lds32(piece + 384 + 4 * (lane >> 2)) >> (8 * (lane & 2)) : lds32(piece + 384 + 4 * (lane >> 1));
                 guard |= settled(wa, wb, wc) | settled(hw, wa, wb);
-                const HalfA h = decode_half<COMPACT, 0>(wa, wb, wc, hw, tq);
+                const HalfA h = decode_half<COMPACT, 0>(wa, wb, wc, hw, tq_tail);
 #pragma unroll
                 for (int j = 0; j < BATCH; j++) {
                     const uint32_t xj = xl + j * xrec_stride;
@@ -957,6 +1073,29 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
             bar += 8;
             sbuf += kTileBytes;
             if (sbuf == sbuf_end) { sbuf = my_ring; bar = my_bar; parity ^= 1u; }
+        }
+        if constexpr (OVERLAY) {
+            // The exact records of this run's exception blocks: every lane takes an entry of the row group's range,
+            // keeps those whose tile lies in the run, and hands the product to the lane that owns the entry's row.
+            // Integer additions in a fixed order: the result does not depend on the launch.
+            for (uint32_t e0 = exc_begin; e0 < exc_end; e0 += 32) {
+                if (e0 != exc_begin) exc_entry = e0 + lane < exc_end ? __ldg(pr.exc_table + e0 + lane) : make_uint4(~0u, 0u, 0u, 0u);
+                long long v = 0;
+                int r = -1;
+                const int b = (int)(exc_entry.x >> 13), unit = b >> 2;
+                if (unit >= cc.col && unit < cc.col + run) {
+                    r = (int)((exc_entry.x >> 8) & 31u);
+                    v = exception_value(exc_entry, xs0 + (uint32_t)b * kXRecBytes, tq_tail, inv_q);
+                }
+                uint32_t votes = __ballot_sync(0xffffffffu, r >= 0);
+                while (votes) {
+                    const int src = __ffs(votes) - 1;
+                    votes &= votes - 1;
+                    const int rr = __shfl_sync(0xffffffffu, r, src);
+                    const long long vv = __shfl_sync(0xffffffffu, v, src);
+                    if (rr == my_row) sum[0] += vv;
+                }
+            }
         }
         // with no records read (the control launch) every unit contributes zero
         n += run;
@@ -1086,12 +1225,13 @@ __global__ void __launch_bounds__(256) gemv_fp16_kernel(const __half *__restrict
 // ---- helpers reading a record back: thread = (row group, block column, row of the group)
 // The 24 codes (c[j] = codes of coordinates 8j..8j+7, a nibble each) and the header of one block of one row,
 // found from the layout's description in include/llvq.h: which piece, half-step, lane, word and nibble.
-template <bool COMPACT>
+// kTile: bytes of a tile in this buffer (the 10-byte layout's leftover blocks are read with COMPACT and its own tile size)
+template <bool COMPACT, int kTile = COMPACT ? kTile13Bytes : kTileBytes>
 __device__ __forceinline__ void read_planes_record(const uint8_t *buf, int64_t nb, int64_t rg, int64_t b, int r,
                                                    uint32_t c[3], uint32_t &hdr) {
     const int64_t tiles = nb / kTileCells, left = nb % kTileCells;
-    constexpr int kCell = COMPACT ? kCell13Bytes : kCellBytes, kTile = COMPACT ? kTile13Bytes : kTileBytes;
-    const uint8_t *grp = buf + (size_t)rg * (size_t)nb * kCell;
+    constexpr int kCell = COMPACT ? kCell13Bytes : kCellBytes;
+    const uint8_t *grp = buf + (size_t)rg * ((size_t)tiles * kTile + (size_t)left * kCell);
     const int m = r >> 4, e = (r >> 3) & 1, g = r & 7;
     const int64_t j = b - tiles * kTileCells;
     const uint8_t *base;
@@ -1130,8 +1270,58 @@ __device__ __forceinline__ void read_planes_record(const uint8_t *buf, int64_t n
     }
 }
 
-// integer coordinates of one record, either layout
-__device__ __forceinline__ void record_coords(int layout, const uint8_t *buf, int64_t nb, int64_t rg, int64_t b, int lane,
+// 10-byte layout: the four-bit codes and the header byte (shell | parity << 4 | gain << 5) of one block of one row -
+// from the short record (three-bit codes plus the window base), from the exception table when the short record is
+// empty and the table lists the block, else the empty record.
+__device__ __forceinline__ void read_overlay_record(const uint8_t *buf, int64_t rows, int64_t nb, int64_t rg, int64_t b, int r,
+                                                    uint32_t c[3], uint32_t &hdr) {
+    const int64_t tiles = nb / kTileCells;
+    if (b >= tiles * kTileCells) {                 // a leftover block: a four-bit record
+        read_planes_record<true, kTile10Bytes>(buf, nb, rg, b, r, c, hdr);
+        return;
+    }
+    const uint8_t *tile = buf + (size_t)rg * overlay_group_bytes(nb) + (size_t)(b / kTileCells) * kTile10Bytes;
+    const int m = r >> 4, e = (r >> 3) & 1, g = r & 7;
+    const int slot = (int)(b & 1), h = 2 * (int)((b % kTileCells) >> 1) + m;
+    auto V = [&](int k, int lane) -> uint32_t {
+        return *reinterpret_cast<const uint32_t *>(tile + (k < 4 ? 16 * lane + 4 * k : (k < 8 ? 512 + 16 * lane + 4 * (k - 4) : 1024 + 4 * lane)));
+    };
+    const uint32_t hb = tile[1152 + 8 * (2 * g + slot) + 2 * h + e];
+    if (hb == 0) {
+        // empty: an exception (then the table has the block), a row past the end or a code that named no point
+        const uint32_t *index = reinterpret_cast<const uint32_t *>(buf + overlay_index_offset(rows, nb));
+        const uint4 *table = reinterpret_cast<const uint4 *>(buf + overlay_table_offset(rows, nb));
+        hdr = 0; c[0] = c[1] = c[2] = 0x88888888u;
+        for (uint32_t i = index[rg]; i < index[rg + 1]; i++) {
+            const uint4 ent = table[i];
+            if ((ent.x >> 13) == (uint32_t)b && ((ent.x >> 8) & 31u) == (uint32_t)r) { hdr = ent.x & 63u; c[0] = ent.y; c[1] = ent.z; c[2] = ent.w; }
+        }
+        return;
+    }
+    const uint32_t f = (hb ^ (hb >> 4)) & 15u;         // window base - 3 | parity << 2 | gain << 3
+    hdr = (hb >> 4) | (f >> 2) << 4;                   // as the 13-byte layout writes it: shell | parity << 4 | gain << 5
+    const uint32_t base = 3u + (f & 3u);
+    c[0] = c[1] = c[2] = 0;
+    for (int i = 0; i < 24; i++) {
+        const int kappa = 24 * slot + i;
+        uint32_t v;
+        if (kappa < 32) {
+            v = (V(2 * h + e, 4 * g + ((kappa & 15) >> 2)) >> (8 * (kappa & 3) + 3 * (kappa >> 4))) & 7u;
+        } else {
+            const int lane = 4 * g + ((kappa - 32) >> 2), sh = 8 * (kappa & 3);
+            if (e == 0 && h < 2) {
+                v = (V(8, lane) >> (sh + 3 * h)) & 7u;
+            } else {
+                const int k = h == 0 ? 0 : (h == 1 ? 1 : 2 * h - 2 + e);          // X0..X5 = (0,1) (1,1) (2,0) (2,1) (3,0) (3,1)
+                v = ((V(k, lane) >> (sh + 6)) & 3u) | (((V(6 + (k >> 1), lane) >> (sh + 6 + (k & 1))) & 1u) << 2);
+            }
+        }
+        c[i >> 3] |= (v + base) << (4 * (i & 7));
+    }
+}
+
+// integer coordinates of one record, any layout
+__device__ __forceinline__ void record_coords(int layout, const uint8_t *buf, int64_t rows, int64_t nb, int64_t rg, int64_t b, int lane,
                                               const uint32_t *cls_parity, const uint8_t *cls_dist, int &cls, int &gain, int x[24]) {
     if (layout == LLVQ_PLANES) {
         uint32_t c[3], hdr;
@@ -1139,10 +1329,11 @@ __device__ __forceinline__ void record_coords(int layout, const uint8_t *buf, in
         cls = (int)(hdr & 511u); gain = (int)((hdr >> 9) & 1u);
         const int par = cls_parity[cls] ? 1 : 0;
         for (int i = 0; i < 24; i++) x[i] = 2 * ((int)((c[i >> 3] >> (4 * (i & 7))) & 15u) - 8) + par;
-    } else if (layout == LLVQ_PLANES13) {
-        // no class id in this layout: `cls` returns the header byte (shell | parity << 4 | gain << 5)
+    } else if (layout == LLVQ_PLANES13 || layout == LLVQ_PLANES10X) {
+        // no class id in these layouts: `cls` returns the header byte (shell | parity << 4 | gain << 5)
         uint32_t c[3], hdr;
-        read_planes_record<true>(buf, nb, rg, b, lane, c, hdr);
+        if (layout == LLVQ_PLANES13) read_planes_record<true>(buf, nb, rg, b, lane, c, hdr);
+        else read_overlay_record(buf, rows, nb, rg, b, lane, c, hdr);
         cls = (int)hdr; gain = (int)((hdr >> 5) & 1u);
         const int par = (int)((hdr >> 4) & 1u);
         for (int i = 0; i < 24; i++) x[i] = 2 * ((int)((c[i >> 3] >> (4 * (i & 7))) & 15u) - 8) + par;
@@ -1172,7 +1363,7 @@ __global__ void __launch_bounds__(256) decode_i8_kernel(int layout, const uint8_
     const int64_t rg = cell_id / nb, b = cell_id % nb, row = rg * kRowsPerGroup + lane;
     if (row >= rows) return;
     int cls, gain, x[24];
-    record_coords(layout, buf, nb, rg, b, lane, cls_parity, cls_dist, cls, gain, x);
+    record_coords(layout, buf, rows, nb, rg, b, lane, cls_parity, cls_dist, cls, gain, x);
     for (int i = 0; i < 24; i++) coords[(row * nb + b) * 24 + i] = (int8_t)x[i];
     class_ids[row * nb + b] = (uint16_t)cls;
 }
@@ -1187,7 +1378,7 @@ __global__ void __launch_bounds__(256) dequant_kernel(int layout, const uint8_t 
     const int64_t rg = cell_id / nb, b = cell_id % nb, row = rg * kRowsPerGroup + lane;
     if (row >= rows) return;
     int cls, gain, x[24];
-    record_coords(layout, buf, nb, rg, b, lane, cls_parity, cls_dist, cls, gain, x);
+    record_coords(layout, buf, rows, nb, rg, b, lane, cls_parity, cls_dist, cls, gain, x);
     // r * gain / (4 sqrt m): cls_scale carries 2^21 / (4 sqrt m)
     const float s = __half2float(row_scale[row]) * ((gain ? g1 : g0) * (cls_scale[cls] * (1.0f / 2097152.0f)));
     __half *dst = W + (row * nb + b) * 24;
@@ -1209,7 +1400,8 @@ GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
     g.grid = p.total_units < sm_count ? p.total_units : sm_count;
     p.units_base = p.total_units / (g.grid * kWarps);
     p.units_rem = p.total_units % (g.grid * kWarps);
-    p.group_bytes = (uint32_t)p.nb * (uint32_t)(layout == LLVQ_ONEHOT ? kOneHotCellBytes : (layout == LLVQ_PLANES13 ? kCell13Bytes : kCellBytes));
+    p.group_bytes = layout == LLVQ_PLANES10X ? (uint32_t)overlay_group_bytes(p.nb)
+                                             : (uint32_t)p.nb * (uint32_t)(layout == LLVQ_ONEHOT ? kOneHotCellBytes : (layout == LLVQ_PLANES13 ? kCell13Bytes : kCellBytes));
     if (layout == LLVQ_ONEHOT) {
         g.smem = ((size_t)p.nb * 48 + 127) / 128 * 128;
         return g;
@@ -1290,7 +1482,8 @@ int gemv_configure(const llvq_ctx *ctx) {
     if (allow_max_smem(gemv_planes_kernel<false, 2>, bytes)) return -1;
     if (allow_max_smem(gemv_planes_kernel<false, 4>, bytes)) return -1;
     if (allow_max_smem(gemv_planes_kernel<false, 1, true>, bytes)) return -1;
-    if (allow_max_smem(gemv_planes_kernel<false, 1, false, true>, bytes)) return -1;
+    if (allow_max_smem(gemv_planes_kernel<false, 1, false, LLVQ_PLANES13>, bytes)) return -1;
+    if (allow_max_smem(gemv_planes_kernel<false, 1, false, LLVQ_PLANES10X>, bytes)) return -1;
     if (allow_max_smem(gemv_onehot_kernel, bytes)) return -1;
     return 0;
 }
@@ -1306,7 +1499,8 @@ cudaError_t launch_gemv(int layout, const GemvParams &p, const GemvLaunch &g, bo
     attr[0].val.programmaticStreamSerializationAllowed = pdl ? 1 : 0;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (layout == LLVQ_PLANES13) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 1, false, true>, p);
+    if (layout == LLVQ_PLANES13) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 1, false, LLVQ_PLANES13>, p);
+    if (layout == LLVQ_PLANES10X) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 1, false, LLVQ_PLANES10X>, p);
     if (layout == LLVQ_PLANES) {
         if (no_weights) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<true, 1>, p);
         if (p.rot_log2 > 0) return cudaLaunchKernelEx(&cfg, gemv_planes_kernel<false, 1, true>, p);

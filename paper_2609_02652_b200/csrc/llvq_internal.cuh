@@ -18,7 +18,17 @@ constexpr int kTileBytes = 1792;
 constexpr int kOneHotCellBytes = 640;  // 32 rows x 20 bytes
 constexpr int kCell13Bytes = 416;      // 13-byte layout: 32 rows x 13 bytes
 constexpr int kTile13Bytes = 1664;
+constexpr int kTile10Bytes = 1280;     // 10-byte layout: 9 words a lane and 128 header bytes a tile; its leftover blocks are 13-byte cells
 constexpr int kMaxGridCtas = 256;      // the GEMV launches one CTA a multiprocessor; more multiprocessors than this share the work of 256
+
+// The 10-byte layout's buffer: row groups, then (128-byte aligned) the index, then (128-byte aligned) the exception table.
+__host__ __device__ inline size_t overlay_group_bytes(int64_t nb) { return (size_t)(nb / kTileCells) * kTile10Bytes + (size_t)(nb % kTileCells) * kCell13Bytes; }
+__host__ __device__ inline size_t overlay_index_offset(int64_t rows, int64_t nb) {
+    return ((size_t)((rows + kRowsPerGroup - 1) / kRowsPerGroup) * overlay_group_bytes(nb) + 127) / 128 * 128;
+}
+__host__ __device__ inline size_t overlay_table_offset(int64_t rows, int64_t nb) {
+    return overlay_index_offset(rows, nb) + ((size_t)((rows + kRowsPerGroup - 1) / kRowsPerGroup + 1) * 4 + 127) / 128 * 128;
+}
 
 struct DeviceTables {
     const uint64_t *base;            // num_classes + 1
@@ -59,6 +69,8 @@ struct GemvProblemDev {
     int group_begin;   // index of this matrix's first row group in the concatenation
     float gain0, gain1;
     int qexp_base;     // log2 of this matrix's fixed-point quantum, before the exponent of max |x| is added
+    const uint32_t *exc_index;   // 10-byte layout: entry g = exception-table entries of this matrix's row groups before g
+    const uint4 *exc_table;      // 10-byte layout: the exact records the short records leave out
 };
 
 // A CTA's share of a launch, planned on the host: its first unit, the panel that unit lies in and the panel's first
@@ -117,6 +129,8 @@ struct llvq_ctx {
     size_t accum_slots;
     int *error;              // device flag: a kernel's bounded wait ran out
     uint32_t *bad_codes;     // device count: codes that named no point, over the expansions since the last llvq_status
+    uint32_t *overflow;      // device count: exception-table entries that found no room, since the last llvq_status
+    unsigned long long *counter;   // device scratch of llvq_overlay_count
     int use_pdl;             // launch the GEMV with programmatic stream serialization
     int weights_dirty;       // an expansion was enqueued since the last GEMV: that GEMV must not read records ahead of it
     int sm_count;
@@ -125,7 +139,10 @@ struct llvq_ctx {
 
 namespace llvq {
 cudaError_t launch_expand(const llvq_ctx *ctx, int layout, const uint64_t *codes, int64_t rows, int64_t nb,
-                          void *out, uint32_t *bad_count, cudaStream_t s);
+                          void *out, size_t out_bytes, uint32_t *bad_count, cudaStream_t s);
+// adds the number of blocks the 10-byte layout would keep in its exception table to *counter (device)
+cudaError_t launch_overlay_count(const llvq_ctx *ctx, const uint64_t *codes, int64_t rows, int64_t nb, unsigned long long *counter,
+                                 cudaStream_t s);
 struct GemvLaunch {
     int grid;
     size_t smem;

@@ -52,7 +52,15 @@ def test_layout_bytes_and_argument_checks(lib):
     # the 13-byte layout: 13/14 of the 14-byte layout's size, for any shape
     assert binding.layout_bytes(binding.PLANES13, 3072, 3072) == 3072 * 128 * 13
     assert binding.layout_bytes(binding.PLANES13, 33, 48) == 2 * 2 * 416
-    assert lib.llvq_layout_bytes(3, 32, 24, ctypes.byref(n)) == -1
+    assert lib.llvq_layout_bytes(4, 32, 24, ctypes.byref(n)) == -1
+    # the 10-byte layout: tiles of 1280 bytes, leftover blocks of 416, then (128-byte aligned) the index and the table
+    from oracle import oracle as O
+    for rows, nb, exc in ((32, 4, 0), (33, 7, 5), (3072, 128, 100), (70, 1, 0), (64, 9, 3)):
+        assert binding.overlay_bytes(rows, 24 * nb, exc) == O.planes10x_bytes(rows, nb, exc)
+        assert binding.layout_bytes(binding.PLANES10X, rows, 24 * nb) == O.planes10x_bytes(rows, nb, (rows * nb + 31) // 32)
+    assert binding.overlay_bytes(32, 96, 0) == 1280 + 128
+    assert lib.llvq_overlay_bytes(32, 24 << 19, 0, ctypes.byref(n)) == -1          # block columns must stay below 2^19
+    assert lib.llvq_overlay_count(None, None, 1, 1, None, None) == -1
 
 
 def test_rotation_block_rule_and_argument_checks(lib):

@@ -122,7 +122,7 @@ def test_what_the_layout_does_not_take(B, ctx):
         B.dequant_fp16(ctx, L13, buf, case.d_scale, GAIN, 64, 96)
     assert e.value.code == -1
     with pytest.raises(B.LlvqError) as e:
-        B.gemv(ctx, 3, buf, case.d_scale, GAIN, case.d_x, 64, 96)
+        B.gemv(ctx, 4, buf, case.d_scale, GAIN, case.d_x, 64, 96)
     assert e.value.code == -1
     with pytest.raises(B.LlvqError) as e:
         B.gemv(ctx, L13, buf[16:], case.d_scale, GAIN, case.d_x, 64, 96)

@@ -501,7 +501,7 @@ def _unpack_planes10x_cell(buf, rows, nb, row, b):
             high = (V(6 + (k >> 1), lane) >> (8 * ii + 6 + (k & 1))) & 1
             codes.append(low | high << 2)
     hb = int(buf[base + 1152 + 8 * (2 * g + slot) + 2 * h + e])
-    return hb, 3 + (hb >> 6), codes
+    return hb, 3 + ((hb ^ (hb >> 4)) & 3), codes
 
 
 @pytest.mark.parametrize("rows,nb,rate", [(32, 4, 0.0), (37, 7, 0.3), (64, 1, 0.5), (5, 2, 0.5), (33, 3, 0.2), (20, 6, 0.1), (50, 9, 0.25),
@@ -541,7 +541,7 @@ def test_planes10x_layout_round_trip(oracle, rows, nb, rate):
                     assert hb == 0 and v == [0] * 24
                     per_group.append((b // 4, b % 4, row % 32, shell | par << 4 | gain << 5, u))
                 else:
-                    assert o == want_o[at] and hb == shell | par << 4 | gain << 5 | (o - 3) << 6
+                    assert o == want_o[at] and hb == (((o - 3) | par << 2 | gain << 3) ^ shell) | shell << 4
                     assert [c + o for c in v] == u and [2 * (c + o - 8) + par for c in v] == x.tolist()
         per_group.sort(key=lambda t: t[:3])
         assert index[rg + 1] - index[rg] == len(per_group)
@@ -578,7 +578,7 @@ def test_planes10x_layout_worked_example_by_hand(oracle):
     rest[[0, 4, 8, 12, 128, 132, 136, 140]] = False
     assert not words[rest].any()
     hdr = buf[1152:1280]
-    assert int(hdr[0]) == 2 and int(hdr[4]) == (2 | 1 << 5) and int(hdr.astype(np.int64).sum()) == 2 + 34
+    assert int(hdr[0]) == (2 << 4 | 2) and int(hdr[4]) == (2 << 4 | (8 ^ 2)) and int(hdr.astype(np.int64).sum()) == 34 + 42
     assert buf[1280:1288].view(np.uint32).tolist() == [0, 1]
     assert buf[1408:1424].view(np.uint32).tolist() == [8 | 0 << 8 | 3 << 13, 0x8888884C, 0x88888888, 0x88888888]
 
