@@ -131,7 +131,10 @@ def make_copies(B, ctx, mats, layout, ncopies, device, grouped=True, keep_codes=
     first = {}
     for e in mats:
         m = e["m"]
-        first[m.tensor_id] = B.expand(ctx, layout, e["codes"], m.rows, m.nb)
+        out = None
+        if layout == B.PLANES10X:      # a buffer with room for exactly the matrix's exceptions
+            out = torch.empty(B.overlay_bytes(m.rows, m.k_padded, B.overlay_count(ctx, e["codes"], m.rows, m.nb)), dtype=torch.uint8, device=device)
+        first[m.tensor_id] = B.expand(ctx, layout, e["codes"], m.rows, m.nb, out=out)
         if keep_codes is not None and m.tensor_id not in keep_codes:
             e["codes"] = None
     torch.cuda.synchronize()
@@ -364,9 +367,66 @@ def single_matrix(B, ctx, rows, k, device, peak, seed=5, rounds=7, steps=200):
     return out
 
 
+def overlay_used_bytes(B, ctx, mats):
+    """Bytes a step reads in the 10-byte layout (short records, index, the table entries in use, scales, x, y), the
+    blocks it covers and how many of them are in the exception tables."""
+    used, blocks, exc = 0, 0, 0
+    for e in mats:
+        m = e["m"]
+        n = B.overlay_count(ctx, e["codes"], m.rows, m.nb)
+        used += B.overlay_bytes(m.rows, m.k_padded, n) + gemv_bytes(m.rows, m.nb, 0)
+        blocks += m.blocks
+        exc += n
+    return used, blocks, exc
+
+
+def with_exceptions(B, ctx, e, share, seed):
+    """The matrix's code words with a share of the blocks replaced by exception blocks of the 10-byte layout, drawn from
+    those the matrix itself contains (found by decoding it with the library and applying the layout's window rule)."""
+    m, codes = e["m"], e["codes"]
+    co, _ = B.decode_i8(ctx, B.PLANES, B.expand(ctx, B.PLANES, codes, m.rows, m.nb), m.rows, m.nb)
+    u = 8 + torch.div(co.reshape(-1, 24).to(torch.int32), 2, rounding_mode="floor")
+    lo, hi = u.min(1).values, u.max(1).values
+    pool = codes.reshape(-1)[torch.clamp(hi - 7, min=3) > torch.clamp(lo, max=6)]
+    if pool.numel() == 0:
+        return codes
+    g = torch.Generator(device=codes.device)
+    g.manual_seed(seed)
+    hit = torch.rand(codes.numel(), device=codes.device, generator=g) < share
+    pick = pool[torch.randint(0, pool.numel(), (codes.numel(),), device=codes.device, generator=g)]
+    return torch.where(hit, pick, codes.reshape(-1)).reshape(codes.shape)
+
+
+def overlay_arm(B, ctx, mats, copies, ncopies, device, peak, steps):
+    """The 10-byte layout with its exception table on the synthetic stream (about one block in eight thousand is an
+    exception) and on the same matrices with 3.38 % of the blocks made exceptions (the share the paper reports for
+    its own overlay on its artifact)."""
+    n_gemv = len(mats)
+    out = {}
+    for label, share in (("synthetic_stream", None), ("exceptions_3_38_pct", 0.0338)):
+        if share is None:
+            ms, ref = mats, copies
+        else:
+            ms = [dict(e, codes=with_exceptions(B, ctx, e, share, 1000 + e["m"].tensor_id)) for e in mats]
+            ref = make_copies(B, ctx, ms, B.PLANES, 1, device)
+            run_step(B, ctx, B.PLANES, ref[0])
+        c10 = make_copies(B, ctx, ms, B.PLANES10X, ncopies, device)
+        run_step(B, ctx, B.PLANES10X, c10[0])
+        torch.cuda.synchronize()
+        B.status(ctx)
+        same_outputs(ref, c10, exact=False)
+        t = time_arm(lambda i: run_step(B, ctx, B.PLANES10X, c10[i]), len(c10), steps, 3)
+        used, blocks, exc = overlay_used_bytes(B, ctx, ms)
+        out[label] = dict(figures(t, n_gemv, used, peak), bytes_per_block=(used - sum(gemv_bytes(e["m"].rows, e["m"].nb, 0) for e in ms)) / blocks,
+                          exception_blocks=exc, exception_share=exc / blocks)
+        out[label]["bits_per_weight"] = out[label]["bytes_per_block"] * 8 / 24
+        del c10, ref
+    return out
+
+
 def comparison_arms(B, ctx, device, peak, steps=200):
     """The arms of the paper's layout table, on the 4B-like layer (config 1): per-matrix launches, small batches,
-    the activation rotation, the no-weights control, the 13-byte layout, the one-hot layout, the FP16 control.
+    the activation rotation, the no-weights control, the 13-byte and the 10-byte layout, the one-hot layout, the FP16 control.
     Every arm's outputs are compared with those of the 14-byte arm (which the GPU tests hold to the oracle)."""
     wl = datagen.workload(1)
     mats = build_inputs(wl, device)
@@ -449,6 +509,8 @@ def comparison_arms(B, ctx, device, peak, steps=200):
     pb = sum(gemv_bytes(e["m"].rows, e["m"].nb, 13) for e in mats)
     arms["planes13"] = dict(figures(t, n_gemv, pb, peak), bytes_per_block=13, bits_per_weight=13 * 8 / 24)
     del p13_copies
+    # the 10-byte layout: three-bit window codes, the blocks no window holds kept exactly in a table (the sparse overlay)
+    arms["planes10x"] = overlay_arm(B, ctx, mats, copies, ncopies, device, peak, steps)
     # one-hot layout: a correctness reference for the paper's other record (plain coalesced loads, scalar
     # arithmetic, not tuned), so its time says nothing about the layouts' relative merit
     oh_copies = make_copies(B, ctx, mats, B.ONEHOT, max(2, ncopies * 14 // 20 + 1), device)
@@ -495,6 +557,7 @@ def main():
     ap.add_argument("--no-arms", action="store_true", help="skip the other configurations, the single matrices and the comparison arms")
     ap.add_argument("--no-pdl", action="store_true", help="launch the GEMV without programmatic dependent launch")
     ap.add_argument("--ungrouped", action="store_true", help="one launch a matrix instead of row-concatenated groups")
+    ap.add_argument("--layout", default="planes14", choices=["planes14", "planes10x"], help="record layout of the timed step (the headline is planes14)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     args.rounds = max(args.rounds, DISCARD_ROUNDS + 1)
@@ -528,12 +591,17 @@ def main():
 
     mats = build_inputs(wl, device)
     n_gemv = len(mats)
-    step_bytes = sum(gemv_bytes(e["m"].rows, e["m"].nb) for e in mats)
-    layout_bytes = sum(14 * e["m"].blocks for e in mats)
+    L = B.PLANES10X if args.layout == "planes10x" else B.PLANES
+    if L == B.PLANES:
+        step_bytes = sum(gemv_bytes(e["m"].rows, e["m"].nb) for e in mats)
+        layout_bytes = sum(14 * e["m"].blocks for e in mats)
+    else:
+        step_bytes, _, _ = overlay_used_bytes(B, ctx, mats)
+        layout_bytes = sum(10 * e["m"].blocks for e in mats)
     ncopies = copies_needed(layout_bytes)
     # the oracle checks the first layer (the multi-layer stacks) or the whole step: only those codes are kept
     checked = 7 if n_gemv > 7 else n_gemv
-    copies = make_copies(B, ctx, mats, B.PLANES, ncopies, device, grouped=not args.ungrouped,
+    copies = make_copies(B, ctx, mats, L, ncopies, device, grouped=not args.ungrouped,
                          keep_codes={e["m"].tensor_id for e in mats[:checked]})
     torch.cuda.synchronize()
     launches_per_step = len(copies[0].launches)
@@ -541,16 +609,16 @@ def main():
     # expander throughput (load-time step, outside the timed region)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     big = max(mats[:checked], key=lambda e: e["m"].blocks)
-    B.expand(ctx, B.PLANES, big["codes"], big["m"].rows, big["m"].nb)
+    B.expand(ctx, L, big["codes"], big["m"].rows, big["m"].nb)
     e0.record()
-    B.expand(ctx, B.PLANES, big["codes"], big["m"].rows, big["m"].nb)
+    B.expand(ctx, L, big["codes"], big["m"].rows, big["m"].nb)
     e1.record()
     e1.synchronize()
     expand_rate = big["m"].blocks / (e0.elapsed_time(e1) * 1e-3)
 
     # parity first (every row of the checked launches, copy 0), which also times the oracle on the host cores
     cores = os.cpu_count() or 1
-    run_step(B, ctx, B.PLANES, copies[0])
+    run_step(B, ctx, L, copies[0])
     torch.cuda.synchronize()
     from oracle import oracle as O
 
@@ -565,7 +633,7 @@ def main():
                         "split": "decode_us = the index decode alone timed on one core over 262144 codes a matrix, scaled by blocks and divided by the cores; matvec_us = the rest"}
 
     # warm-up: ramp the clocks, then the protocol
-    step_fn = lambda i: run_step(B, ctx, B.PLANES, copies[i % ncopies])
+    step_fn = lambda i: run_step(B, ctx, L, copies[i % ncopies])
     ramp = capture_graphs(step_fn, max(2, min(64, 4000 // launches_per_step)))
     t_end = time.perf_counter() + 0.4
     while time.perf_counter() < t_end:
@@ -621,7 +689,7 @@ def main():
         def issue(plist=plist):
             dev_x.copy_(host_x, non_blocking=True)
             for probs, xv, kp in plist:
-                B.gemv_grouped(ctx, B.PLANES, probs, xv, kp)
+                B.gemv_grouped(ctx, L, probs, xv, kp)
             host_y.copy_(dev_y, non_blocking=True)
         with torch.cuda.stream(side):
             issue()
@@ -652,7 +720,7 @@ def main():
         e2e_rounds.append((time.perf_counter() - t1) / e2e_steps * 1e6 / n_gemv / world)
     e2e_us, e2e_min, e2e_max, _ = summarise_rounds(e2e_rounds)
     # ... and they are the right results: one matrix of the last step against the untimed path's y (same records, same x)
-    run_step(B, ctx, B.PLANES, copies[(e2e_steps - 1) % ncopies])
+    run_step(B, ctx, L, copies[(e2e_steps - 1) % ncopies])
     torch.cuda.synchronize()
     assert torch.equal(host_y[y_off[0]:y_off[0] + l0[0]["mats"][0].rows], copies[(e2e_steps - 1) % ncopies].launches[0]["ys"][0].cpu())
     del e2e_graphs, e2e_keep
@@ -672,7 +740,8 @@ def main():
             "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
             "dtype": "u8 x s8 -> s32 (tensor cores), f32 block scale, int64 row sums", "data": "synthetic",
             "config": {"workload": f"config {wl.config}: {wl.name}", "gemvs_per_step": n_gemv, "launches_per_step": launches_per_step,
-                       "layout": "Planes14: 14 B per 24 weights - class, gain, 24 four-bit sign+level codes (4.67 b/w payload; the paper's 4.80 b/w label counts its f32 tail and scales)",
+                       "layout": "Planes14: 14 B per 24 weights - class, gain, 24 four-bit sign+level codes (4.67 b/w payload; the paper's 4.80 b/w label counts its f32 tail and scales)"
+                                 if L == B.PLANES else "Planes10x: 10 B per 24 weights - one header byte, 24 three-bit window codes - plus the exact records of the blocks no window holds",
                        "l2": f"records and scales: {ncopies} distinct cop{'y' if ncopies == 1 else 'ies'} ({ncopies * layout_bytes / 1e6:.0f} MB, at least three times L2) so no launch finds its records in L2; x (a few KB a launch) is one buffer, as in a decoder where it is the previous operator's output",
                        "multi_gpu": "replicas only: each rank runs the whole step on its own copy", "seed": wl.seed,
                        "oracle_check": f"every row of the first {ogemvs} GEMVs before timing"},
@@ -681,7 +750,7 @@ def main():
                        "ms_per_round": ms_rounds},
             "gbps": gbps, "hbm_frac": gbps / peak, "bytes_per_step": step_bytes,
             "roofline": {"bound": "hbm", "achieved": gbps, "peak": peak, "unit": "GB/s", "frac": gbps / peak,
-                         "traffic": step_bytes / launches_per_step * NCU_TRAFFIC_PER_ALGORITHMIC_BYTE,
+                         "traffic": step_bytes / launches_per_step * NCU_TRAFFIC_PER_ALGORITHMIC_BYTE if L == B.PLANES else None,
                          "traffic_note": "DRAM bytes per launch (mean over the step's launches): ncu capture of the 8192x8192 launch scaled by bytes",
                          "kernel": "gemv_planes_kernel", "peak_source": peak_src,
                          # the competing ceiling, from the ncu capture in profiles/ (8192 x 8192 launch): instruction issue

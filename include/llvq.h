@@ -5,6 +5,7 @@
  * The path (paper sections in brackets):
  *   llvq_expand      [Sec. 2.2 "Unfolding at load time"]  48-bit block codes -> in-memory records
  *   llvq_gemv        [Sec. 2.3 "The kernel"]               records, row scales, x -> y
+ *   llvq_overlay_count, llvq_overlay_bytes [Sec. 3.3, the sparse overlay] size the exception table of LLVQ_PLANES10X
  *   llvq_gemv_grouped[Sec. 3.4 "Attribution": row-concatenated q/k/v and gate/up launches]
  *   llvq_gemv_batch  [Sec. 5 "Batching"]                  the same for 2..8 activation vectors a pass
  *   llvq_gemv_static                                      llvq_gemv without a context or any allocation
@@ -62,11 +63,8 @@
  *                distinct magnitudes.  Per cell five arrays of 32 words (word t of row l at
  *                128t+4l): V0 = smask | class[7:0]<<24, V1 = mask1 | class[8]<<24 | gain<<25,
  *                V2..V4 = mask2..mask4.  A row group takes 640*nb bytes.
- *   LLVQ_PLANES13 13 bytes a block, exact for every block.  Not the paper's next rate point: its "Planes12x" layout
- *                [Sec. 3.3: 12 bytes for blocks of up to four levels, the five-level blocks kept exactly in a side table
- *                and applied by further thread blocks] is smaller (about 12.1 bytes a block of payload on this library's
- *                synthetic data against 13; 4.342 against about 4.47 bits a weight on the paper's accounting) and is not
- *                built here.
+ *   LLVQ_PLANES13 13 bytes a block, exact for every block.  Not the paper's next rate point (its sparse overlay, for
+ *                which see LLVQ_PLANES10X below): no short record, no exception table.
  *                Here the rate comes from the header instead of the levels: the matvec needs of the
  *                class only what fixes the block's scale and the parity of its coordinates, so the
  *                16-bit header becomes one byte = shell (4 bits, 0 for the empty record) | parity << 4
@@ -113,9 +111,9 @@
  *                  hold every block exactly and never make an exception.  A row group takes
  *                  1280 (nb / 4) + 416 (nb mod 4) bytes.
  *                  After the last row group, at the next multiple of 128 bytes: the index, one uint32 a
- *                  row group and one more - entry g = table entries of the row groups before g.  After
- *                  the index, at the next multiple of 128 bytes: the table, 16 bytes an entry, ordered by
- *                  row group, tile, block, row:  word 0 = shell | parity << 4 | gain << 5 | (row of the
+ *                  tile (row group by row group, nb / 4 tiles each) and one more - entry i = table entries
+ *                  of the tiles before tile i.  After the index, at the next multiple of 128 bytes: the
+ *                  table, 16 bytes an entry, ordered by row group, tile, block, row:  word 0 = shell | parity << 4 | gain << 5 | (row of the
  *                  group) << 8 | (block column) << 13;  words 1..3 = the 24 four-bit codes, coordinate
  *                  8 j + n in nibble n of word 1 + j.  Bytes between the parts are zero.
  *                The table's size depends on the data: llvq_overlay_count counts the exceptions of a matrix,

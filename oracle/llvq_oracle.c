@@ -626,15 +626,16 @@ void llvqo_pack_planes13(const uint64_t *codes, int64_t rows, int64_t nb, uint8_
  * Vk of lane L at 16 L + 4 k (k < 4), 512 + 16 L + 4 (k - 4) (k < 8), 1024 + 4 L (k = 8); header byte of pair P,
  * half-step h, row half e at 1152 + 8 P + 2 h + e.
  * The nb mod 4 last blocks follow in the 13-byte layout's pair and single (four-bit codes, that layout's header byte, exact).
- * After the row groups, at the next multiple of 128: the index (row groups + 1 uint32; entry g = exceptions of the
- * row groups before g, never above the capacity); after it, at the next multiple of 128: the table, 16 bytes an
+ * After the row groups, at the next multiple of 128: the index (one uint32 a tile, row group by row group, and one
+ * more; entry i = exceptions of the tiles before tile i, never above the capacity); after it, at the next multiple
+ * of 128: the table, 16 bytes an
  * entry, in the order row group, tile, block, row: word 0 = shell | parity << 4 | gain << 5 | row of the group << 8 |
  * block column << 13, words 1..3 the four-bit codes (coordinate 8 j + n in nibble n of word 1 + j).
  */
 static size_t up128(size_t v) { return (v + 127u) & ~(size_t)127u; }
 static size_t p10_group_bytes(int64_t nb) { return (size_t)(nb / 4) * 1280u + (size_t)(nb % 4) * 416u; }
 static size_t p10_index_offset(int64_t rows, int64_t nb) { return up128((size_t)((rows + 31) / 32) * p10_group_bytes(nb)); }
-static size_t p10_table_offset(int64_t rows, int64_t nb) { return p10_index_offset(rows, nb) + up128((size_t)((rows + 31) / 32 + 1) * 4u); }
+static size_t p10_table_offset(int64_t rows, int64_t nb) { return p10_index_offset(rows, nb) + up128((size_t)((rows + 31) / 32 * (nb / 4) + 1) * 4u); }
 size_t llvqo_planes10x_bytes(int64_t rows, int64_t nb, uint64_t exceptions) { return p10_table_offset(rows, nb) + (size_t)exceptions * 16u; }
 
 /* window base of a block's codes, 0 if none fits */
@@ -659,7 +660,6 @@ int64_t llvqo_pack_planes10x(const uint64_t *codes, int64_t rows, int64_t nb, ui
     uint8_t *exc = malloc((size_t)32 * nb);
     uint64_t count = 0;
     for (int64_t rg = 0; rg < ngroups; rg++) {
-        index[rg] = (uint32_t)(count < capacity ? count : capacity);
         for (int r = 0; r < 32; r++)
             for (int64_t b = 0; b < nb; b++) {
                 record_t rec;
@@ -679,6 +679,7 @@ int64_t llvqo_pack_planes10x(const uint64_t *codes, int64_t rows, int64_t nb, ui
         uint8_t *grp = out + (size_t)rg * gbytes;
         /* the tiles: three-bit codes */
         for (int64_t T = 0; T < ntiles; T++) {
+            index[rg * ntiles + T] = (uint32_t)(count < capacity ? count : capacity);
             uint8_t *tile = grp + (size_t)T * 1280u;
             for (int g = 0; g < 8; g++)
                 for (int t = 0; t < 4; t++) {
@@ -754,7 +755,7 @@ int64_t llvqo_pack_planes10x(const uint64_t *codes, int64_t rows, int64_t nb, ui
             }
         free(hdr16);
     }
-    index[ngroups] = (uint32_t)(count < capacity ? count : capacity);
+    index[ngroups * ntiles] = (uint32_t)(count < capacity ? count : capacity);
     free(u); free(v); free(hb); free(hs); free(exc);
     return (int64_t)count;
 }

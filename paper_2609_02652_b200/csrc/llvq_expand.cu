@@ -160,9 +160,8 @@ __device__ __forceinline__ uint32_t header_byte(const DeviceTables &T, const Dec
 
 // LAYOUT = LLVQ_PLANES, LLVQ_PLANES13 (the same code words, the header one byte) or LLVQ_PLANES10X (tiles of
 // three-bit window codes, the blocks a window cannot hold listed in the exception table; the leftover blocks as in
-// LLVQ_PLANES13).  For LLVQ_PLANES10X the first word of every tile holds, on entry, the tile's first entry in its row
-// group's part of the table (overlay_offsets_kernel), `index` the row groups' first entries, and `capacity` the
-// entries the table has room for.
+// LLVQ_PLANES13).  For LLVQ_PLANES10X `index` holds, on entry, every tile's first entry in the table, and `capacity`
+// is the number of entries the table has room for.
 template <int LAYOUT>
 __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, const uint64_t *__restrict__ codes, int64_t rows, int64_t nb,
                                                             uint8_t *__restrict__ out, uint32_t *bad_count, uint32_t *ctx_bad,
@@ -186,10 +185,7 @@ __global__ void __launch_bounds__(256) expand_planes_kernel(DeviceTables T, cons
     const int ncell = is_tile ? 4 : (is_pair ? 2 : 1);
     const int64_t b0 = is_tile ? u * kTileCells : (is_pair ? tiles * kTileCells : nb - 1);
     uint32_t next_entry = 0;                               // OVERLAY: where this tile's next exception goes
-    if (OVERLAY && is_tile) {
-        next_entry = index[rg] + *reinterpret_cast<const uint32_t *>(grp + (size_t)u * kTile);
-        __syncwarp();                                      // every lane has read the word before any lane overwrites it
-    }
+    if (OVERLAY && is_tile) next_entry = index[rg * tiles + u];
     int bad = 0;
 #pragma unroll 1
     for (int q = 0; q < ncell; q++) {
@@ -343,11 +339,12 @@ __global__ void __launch_bounds__(256) expand_onehot_kernel(DeviceTables T, cons
 
 
 // ---- the exception table of the 10-byte layout is filled in a fixed order, so its entries' places are known before
-// they are written.  One warp a tile counts the tile's exceptions (lane = row).  WRITE: the count goes to the tile's
-// first word (the tile itself is written later); else the counts are added up in *total.
-template <bool WRITE>
+// they are written.  One warp a tile counts the tile's exceptions (lane = row).  INDEX: the count goes to the index
+// entry after the tile's (the running sum over the index then gives every tile's first entry); else the counts are
+// added up in *total.
+template <bool INDEX>
 __global__ void __launch_bounds__(256) overlay_count_kernel(DeviceTables T, const uint64_t *__restrict__ codes, int64_t rows, int64_t nb,
-                                                            uint8_t *out, unsigned long long *total) {
+                                                            uint32_t *index, unsigned long long *total) {
     const int64_t tiles = nb / kTileCells;
     const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int lane = (int)(gid & 31);
@@ -367,46 +364,21 @@ __global__ void __launch_bounds__(256) overlay_count_kernel(DeviceTables T, cons
         count += __popc(__ballot_sync(0xffffffffu, exception));
     }
     if (lane == 0) {
-        if (WRITE) *reinterpret_cast<uint32_t *>(out + (size_t)rg * overlay_group_bytes(nb) + (size_t)u * kTile10Bytes) = count;
+        if (INDEX) index[tile_id + 1] = count;
         else if (count) atomicAdd(total, (unsigned long long)count);
     }
 }
 
-// One warp a row group: the tiles' counts become their first entries inside the row group's part of the table
-// (an exclusive running sum, left in the same words), and the row group's total goes to index[g + 1].
-__global__ void __launch_bounds__(256) overlay_offsets_kernel(uint8_t *out, int64_t groups, int64_t nb, uint32_t *index) {
-    const int64_t gid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int lane = (int)(gid & 31);
-    const int64_t rg = gid >> 5, tiles = nb / kTileCells;
-    if (rg >= groups) return;
-    uint8_t *grp = out + (size_t)rg * overlay_group_bytes(nb);
-    uint32_t running = 0;
-    for (int64_t base = 0; base < tiles; base += 32) {
-        const int64_t u = base + lane;
-        uint32_t *word = reinterpret_cast<uint32_t *>(grp + (size_t)u * kTile10Bytes);
-        const uint32_t c = u < tiles ? *word : 0u;
-        uint32_t incl = c;
-#pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, off);
-            if (lane >= off) incl += v;
-        }
-        if (u < tiles) *word = running + incl - c;
-        running += __shfl_sync(0xffffffffu, incl, 31);
-    }
-    if (lane == 0) index[rg + 1] = running;
-}
-
-// One CTA: index[g + 1] = totals of the row groups up to g (index[0] = 0), in place.
-__global__ void __launch_bounds__(1024) overlay_index_kernel(uint32_t *index, int64_t groups) {
+// One CTA: index[i + 1] = counts of the tiles up to i (index[0] = 0), in place.
+__global__ void __launch_bounds__(1024) overlay_index_kernel(uint32_t *index, int64_t n) {
     __shared__ uint32_t warp_sum[32];
     __shared__ uint32_t carry_s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid == 0) { carry_s = 0; index[0] = 0; }
     __syncthreads();
-    for (int64_t base = 0; base < groups; base += 1024) {
+    for (int64_t base = 0; base < n; base += 1024) {
         const int64_t g = base + tid;
-        const uint32_t c = g < groups ? index[g + 1] : 0u;
+        const uint32_t c = g < n ? index[g + 1] : 0u;
         uint32_t incl = c;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -417,7 +389,7 @@ __global__ void __launch_bounds__(1024) overlay_index_kernel(uint32_t *index, in
         __syncthreads();
         uint32_t before = carry_s;
         for (int w = 0; w < warp; w++) before += warp_sum[w];
-        if (g < groups) index[g + 1] = before + incl;
+        if (g < n) index[g + 1] = before + incl;
         __syncthreads();
         if (tid == 1023) carry_s = before + incl;
         __syncthreads();
@@ -426,15 +398,15 @@ __global__ void __launch_bounds__(1024) overlay_index_kernel(uint32_t *index, in
 
 // After the table is filled (one CTA): the index stops at the capacity (so that no reader looks past the table), the
 // entries that found no room are counted, and the bytes between the parts of the buffer are zeroed.
-__global__ void __launch_bounds__(256) overlay_finish_kernel(uint8_t *out, size_t records_end, size_t index_offset, size_t table_offset,
-                                                             int64_t groups, uint32_t capacity, uint32_t *overflow) {
+__global__ void __launch_bounds__(1024) overlay_finish_kernel(uint8_t *out, size_t records_end, size_t index_offset, size_t table_offset,
+                                                              int64_t n, uint32_t capacity, uint32_t *overflow) {
     uint32_t *index = reinterpret_cast<uint32_t *>(out + index_offset);
     const int tid = threadIdx.x;
-    if (tid == 0 && index[groups] > capacity) atomicAdd(overflow, index[groups] - capacity);
+    if (tid == 0 && index[n] > capacity) atomicAdd(overflow, index[n] - capacity);
     __syncthreads();                                       // the total is read before it is clamped
-    for (int64_t i = tid; i <= groups; i += blockDim.x) index[i] = min(index[i], capacity);
+    for (int64_t i = tid; i <= n; i += blockDim.x) index[i] = min(index[i], capacity);
     for (size_t i = records_end + tid; i < index_offset; i += blockDim.x) out[i] = 0;
-    for (size_t i = index_offset + (size_t)(groups + 1) * 4 + tid; i < table_offset; i += blockDim.x) out[i] = 0;
+    for (size_t i = index_offset + (size_t)(n + 1) * 4 + tid; i < table_offset; i += blockDim.x) out[i] = 0;
 }
 
 }  // namespace
@@ -463,16 +435,13 @@ cudaError_t launch_expand(const llvq_ctx *ctx, int layout, const uint64_t *codes
             uint4 *table = reinterpret_cast<uint4 *>(o8 + table_offset);
             const size_t room = (out_bytes - table_offset) / 16;
             const uint32_t capacity = room > 0xffffffffull ? 0xffffffffu : (uint32_t)room;
-            if (tiles > 0) {
-                overlay_count_kernel<true><<<(unsigned)((groups * tiles * 32 + 255) / 256), 256, 0, s>>>(ctx->dev, codes, rows, nb, o8, nullptr);
-                overlay_offsets_kernel<<<(unsigned)((groups * 32 + 255) / 256), 256, 0, s>>>(o8, groups, nb, index);
-            } else {
-                cudaMemsetAsync(index, 0, (size_t)(groups + 1) * 4, s);
-            }
-            overlay_index_kernel<<<1, 1024, 0, s>>>(index, groups);
+            // count the tiles' exceptions into the index, turn the counts into first entries, expand, close the index
+            if (tiles > 0)
+                overlay_count_kernel<true><<<(unsigned)((groups * tiles * 32 + 255) / 256), 256, 0, s>>>(ctx->dev, codes, rows, nb, index, nullptr);
+            overlay_index_kernel<<<1, 1024, 0, s>>>(index, groups * tiles);
             expand_planes_kernel<LLVQ_PLANES10X><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, o8, bad_count, ctx->bad_codes, index, table, capacity);
-            overlay_finish_kernel<<<1, 256, 0, s>>>(o8, (size_t)groups * overlay_group_bytes(nb), index_offset, table_offset, groups, capacity,
-                                                    ctx->overflow);
+            overlay_finish_kernel<<<1, 1024, 0, s>>>(o8, (size_t)groups * overlay_group_bytes(nb), index_offset, table_offset, groups * tiles, capacity,
+                                                     ctx->overflow);
         } else if (layout == LLVQ_PLANES13) {
             expand_planes_kernel<LLVQ_PLANES13><<<(unsigned)blocks, 256, 0, s>>>(ctx->dev, codes, rows, nb, (uint8_t *)out, bad_count, ctx->bad_codes, nullptr, nullptr, 0);
         } else {

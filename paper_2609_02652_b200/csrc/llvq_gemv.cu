@@ -360,18 +360,20 @@ __device__ __forceinline__ uint32_t spread_nibbles(uint32_t h) {
 // One entry of the exception table against the x record of its block (`rec`): the block's whole product, in the
 // accumulator's quanta.  The arithmetic of the tile path for one block: integer sums limb pair by limb pair, the
 // block's scale in f32.  `tail_tab` is the table of the four-bit records' headers (the entry's header byte indexes it).
+// Rolled loops: this runs for one block in thousands, and its size in the instruction stream is what every run pays.
 __device__ __forceinline__ long long exception_value(const uint4 &ent, uint32_t rec, uint32_t tail_tab, float inv_q) {
     const float2 k = lds_f2(tail_tab + 8 * (ent.x & 63u));
-    const uint32_t cw[3] = {ent.y, ent.z, ent.w};
     int d[4] = {0, 0, 0, 0};
-#pragma unroll
+    uint32_t cw = ent.y;
+#pragma unroll 1
     for (int j = 0; j < 3; j++) {
-        const uint32_t lo4 = spread_nibbles(cw[j]), hi4 = spread_nibbles(cw[j] >> 16);
+        const uint32_t lo4 = spread_nibbles(cw), hi4 = spread_nibbles(cw >> 16);
 #pragma unroll
         for (int l = 0; l < 4; l++) {
-            d[l] = __dp4a((int)lo4, (int)lds32(rec + 24 * l + 8 * j), d[l]);
-            d[l] = __dp4a((int)hi4, (int)lds32(rec + 24 * l + 8 * j + 4), d[l]);
+            const uint2 x8 = lds64(rec + 24 * l + 8 * j);
+            d[l] = __dp4a((int)hi4, (int)x8.y, __dp4a((int)lo4, (int)x8.x, d[l]));
         }
+        cw = j == 0 ? ent.z : ent.w;
     }
     const int off = __float_as_int(k.y);
     const int e_lo = off * (int)lds32(rec + 100) + (d[0] + 256 * d[1]);
@@ -661,18 +663,22 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
         const int row0 = (cc.group - p0.group_begin) * kRowsPerGroup + my_row;
         if (row0 < p0.rows) asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(first_scale_bits) : "l"(p0.row_scale + row0));
     }
-    // 10-byte layout: the first run's range of the exception table, and the index entry after it (see the run loop)
-    uint32_t exc_first0 = 0, exc_first1 = 0, exc_ahead = 0;
-    int exc_q = 0, exc_lg = 0;
+    // 10-byte layout: a slot a row for the products of exception blocks (this warp's 32, where a rotation would keep its sums)
+    unsigned long long *exc_scratch = reinterpret_cast<unsigned long long *>(rot) + warp * 32;
+    if constexpr (OVERLAY) {
+        exc_scratch[lane] = 0ull;
+        __syncwarp();
+    }
+    // 10-byte layout: the first run's range of the exception table (the caller's constants, like the records)
+    uint32_t exc_first0 = 0, exc_first1 = 0;
     if constexpr (OVERLAY) {
         if (n_units > 0) {
+            // the tiles [col, col + run) of the run's row group: index entries col and col + run of that row group
             const GemvProblemDev &p0 = p.prob[q];
-            exc_lg = cc.group - p0.group_begin;
-            const uint32_t *ix = p0.exc_index + exc_lg;
-            asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_first0) : "l"(ix));
-            asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_first1) : "l"(ix + 1));
-            if (exc_lg + 2 <= ((p0.rows + kRowsPerGroup - 1) >> 5)) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_ahead) : "l"(ix + 2));
-            exc_q = q;
+            const int run0 = min(cc.end - cc.col, n_units);
+            const uint32_t *ix = p0.exc_index + (size_t)(cc.group - p0.group_begin) * h_tiles;
+            asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_first0) : "l"(ix + min(cc.col, h_tiles)));
+            asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_first1) : "l"(ix + min(cc.col + run0, h_tiles)));
         }
     }
     uint32_t warm = 0;
@@ -901,26 +907,16 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
         const uint32_t tq = tab0 + q * 8192;
         const uint32_t tq_tail = OVERLAY ? tq + 2048 : tq;          // the table the four-bit records' header bytes index
         const int run = min(cc.end - cc.col, n_units - n);
-        // 10-byte layout: the row group's range of the exception table, on its way while the run is summed
-        // 10-byte layout: the row group's range [exc_begin, exc_end) of the exception table.  The first run's was loaded
-        // at the start of the CTA; a run on the next row group of the same matrix takes it from what the run before
-        // loaded ahead; and this lane's entry of the range goes out now, to be used when the run's tiles are summed.
+        // 10-byte layout: the run's range [exc_begin, exc_end) of the exception table (the index has an entry a tile, and
+        // the table follows the order of the tiles).  The first run's was loaded at the start of the CTA, a later run's
+        // is read here; this lane's entry of the range goes out now, to be used when the run's tiles are summed.
         uint32_t exc_begin = exc_first0, exc_end = exc_first1;
         uint4 exc_entry = make_uint4(~0u, 0u, 0u, 0u);          // a block column no run contains
         if constexpr (OVERLAY) {
-            const int lg = cc.group - pr.group_begin;
-            const uint32_t *ix = pr.exc_index + lg;
             if (n != 0) {
-                if (q == exc_q && lg == exc_lg + 1) {
-                    exc_begin = exc_first1;
-                    exc_end = exc_ahead;
-                } else {
-                    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_begin) : "l"(ix));
-                    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_end) : "l"(ix + 1));
-                }
-                exc_first0 = exc_begin; exc_first1 = exc_end;
-                exc_q = q; exc_lg = lg;
-                if (lg + 2 <= ((pr.rows + kRowsPerGroup - 1) >> 5)) asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_ahead) : "l"(ix + 2));
+                const uint32_t *ix = pr.exc_index + (size_t)(cc.group - pr.group_begin) * tiles;
+                asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_begin) : "l"(ix + min(cc.col, tiles)));
+                asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_end) : "l"(ix + min(cc.col + run, tiles)));
             }
             if (exc_begin + lane < exc_end) exc_entry = __ldg(pr.exc_table + exc_begin + lane);
         }
@@ -1075,26 +1071,23 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
             if (sbuf == sbuf_end) { sbuf = my_ring; bar = my_bar; parity ^= 1u; }
         }
         if constexpr (OVERLAY) {
-            // The exact records of this run's exception blocks: every lane takes an entry of the row group's range,
-            // keeps those whose tile lies in the run, and hands the product to the lane that owns the entry's row.
-            // Integer additions in a fixed order: the result does not depend on the launch.
+            // The exact records of this run's exception blocks: every lane takes an entry of the run's range and adds
+            // the product to its row's slot of the warp's scratch (integer additions: the order does not matter);
+            // then every lane collects its own row's slot.
+            const bool any = exc_begin < exc_end;
+#pragma unroll 1
             for (uint32_t e0 = exc_begin; e0 < exc_end; e0 += 32) {
                 if (e0 != exc_begin) exc_entry = e0 + lane < exc_end ? __ldg(pr.exc_table + e0 + lane) : make_uint4(~0u, 0u, 0u, 0u);
-                long long v = 0;
-                int r = -1;
-                const int b = (int)(exc_entry.x >> 13), unit = b >> 2;
-                if (unit >= cc.col && unit < cc.col + run) {
-                    r = (int)((exc_entry.x >> 8) & 31u);
-                    v = exception_value(exc_entry, xs0 + (uint32_t)b * kXRecBytes, tq_tail, inv_q);
+                if (exc_entry.x != ~0u) {
+                    const long long v = exception_value(exc_entry, xs0 + (exc_entry.x >> 13) * kXRecBytes, tq_tail, inv_q);
+                    atomicAdd(exc_scratch + ((exc_entry.x >> 8) & 31u), (unsigned long long)v);
                 }
-                uint32_t votes = __ballot_sync(0xffffffffu, r >= 0);
-                while (votes) {
-                    const int src = __ffs(votes) - 1;
-                    votes &= votes - 1;
-                    const int rr = __shfl_sync(0xffffffffu, r, src);
-                    const long long vv = __shfl_sync(0xffffffffu, v, src);
-                    if (rr == my_row) sum[0] += vv;
-                }
+            }
+            if (any) {
+                __syncwarp();
+                sum[0] += (long long)exc_scratch[my_row];
+                __syncwarp();
+                exc_scratch[my_row] = 0ull;
             }
         }
         // with no records read (the control launch) every unit contributes zero
@@ -1292,7 +1285,8 @@ __device__ __forceinline__ void read_overlay_record(const uint8_t *buf, int64_t 
         const uint32_t *index = reinterpret_cast<const uint32_t *>(buf + overlay_index_offset(rows, nb));
         const uint4 *table = reinterpret_cast<const uint4 *>(buf + overlay_table_offset(rows, nb));
         hdr = 0; c[0] = c[1] = c[2] = 0x88888888u;
-        for (uint32_t i = index[rg]; i < index[rg + 1]; i++) {
+        const int64_t tile_id = rg * tiles + b / kTileCells;
+        for (uint32_t i = index[tile_id]; i < index[tile_id + 1]; i++) {
             const uint4 ent = table[i];
             if ((ent.x >> 13) == (uint32_t)b && ((ent.x >> 8) & 31u) == (uint32_t)r) { hdr = ent.x & 63u; c[0] = ent.y; c[1] = ent.z; c[2] = ent.w; }
         }
@@ -1462,6 +1456,7 @@ GemvLaunch gemv_plan(int layout, GemvParams &p, int sm_count) {
     const int vectors = p.batch <= 1 ? 1 : (p.batch == 2 ? 2 : 4);             // the kernel is built for 1, 2 and 4
     const size_t xbytes = ((size_t)p.xblocks * kXRecBytes + 127) / 128 * 128 * vectors;
     g.smem = (size_t)kWarps * kSlots * kTileBytes + 8192 /* alignment of the tables */ + (size_t)p.nprob * 8192 + xbytes + kWarps * kSlots * 8 + kWarps * 4 * vectors + 16 + (size_t)p.rot_span * 8;
+    if (layout == LLVQ_PLANES10X) g.smem += (size_t)kWarps * 32 * 8;        // the warps' slots for the products of exception blocks
     return g;
 }
 

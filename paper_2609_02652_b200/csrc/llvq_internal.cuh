@@ -27,7 +27,8 @@ __host__ __device__ inline size_t overlay_index_offset(int64_t rows, int64_t nb)
     return ((size_t)((rows + kRowsPerGroup - 1) / kRowsPerGroup) * overlay_group_bytes(nb) + 127) / 128 * 128;
 }
 __host__ __device__ inline size_t overlay_table_offset(int64_t rows, int64_t nb) {
-    return overlay_index_offset(rows, nb) + ((size_t)((rows + kRowsPerGroup - 1) / kRowsPerGroup + 1) * 4 + 127) / 128 * 128;
+    // the index: one entry a tile, and one more
+    return overlay_index_offset(rows, nb) + ((size_t)((rows + kRowsPerGroup - 1) / kRowsPerGroup * (nb / kTileCells) + 1) * 4 + 127) / 128 * 128;
 }
 
 struct DeviceTables {
@@ -69,7 +70,7 @@ struct GemvProblemDev {
     int group_begin;   // index of this matrix's first row group in the concatenation
     float gain0, gain1;
     int qexp_base;     // log2 of this matrix's fixed-point quantum, before the exponent of max |x| is added
-    const uint32_t *exc_index;   // 10-byte layout: entry g = exception-table entries of this matrix's row groups before g
+    const uint32_t *exc_index;   // 10-byte layout: entry i = exception-table entries of this matrix's tiles before tile i (row group by row group)
     const uint4 *exc_table;      // 10-byte layout: the exact records the short records leave out
 };
 

@@ -438,7 +438,7 @@ def _p10_offsets(rows, nb):
     groups = (rows + 31) // 32
     gbytes = (nb // 4) * 1280 + (nb % 4) * 416
     idx = -(-groups * gbytes // 128) * 128
-    return groups, gbytes, idx, idx + -(-(groups + 1) * 4 // 128) * 128
+    return groups, gbytes, idx, idx + -(-(groups * (nb // 4) + 1) * 4 // 128) * 128
 
 
 def _unpack_planes10x_cell(buf, rows, nb, row, b):
@@ -518,10 +518,11 @@ def test_planes10x_layout_round_trip(oracle, rows, nb, rate):
     assert buf.size == tab_off + 16 * n == oracle.planes10x_bytes(rows, nb, n)
     xs, cls = oracle.decode_batch(codes)
     want_o = window_base(xs)
-    index = buf[idx_off: idx_off + 4 * (groups + 1)].view(np.uint32)
+    ntiles = nb // 4
+    index = buf[idx_off: idx_off + 4 * (groups * ntiles + 1)].view(np.uint32)
     table = buf[tab_off:].view(np.uint32).reshape(-1, 4)
     assert index[0] == 0 and index[-1] == n and (np.diff(index.astype(np.int64)) >= 0).all()
-    assert not buf[groups * gbytes: idx_off].any() and not buf[idx_off + 4 * (groups + 1): tab_off].any()
+    assert not buf[groups * gbytes: idx_off].any() and not buf[idx_off + 4 * (groups * ntiles + 1): tab_off].any()
     expected_entries = []
     for rg in range(groups):
         per_group = []
@@ -544,7 +545,8 @@ def test_planes10x_layout_round_trip(oracle, rows, nb, rate):
                     assert o == want_o[at] and hb == (((o - 3) | par << 2 | gain << 3) ^ shell) | shell << 4
                     assert [c + o for c in v] == u and [2 * (c + o - 8) + par for c in v] == x.tolist()
         per_group.sort(key=lambda t: t[:3])
-        assert index[rg + 1] - index[rg] == len(per_group)
+        for T in range(ntiles):                      # one index entry a tile: the entries of the tiles before it
+            assert index[rg * ntiles + T] == len(expected_entries) + sum(1 for t in per_group if t[0] < T)
         expected_entries += per_group
     assert len(expected_entries) == n
     for ent, (tile, q, r, hb, u) in zip(table, expected_entries):
@@ -555,7 +557,7 @@ def test_planes10x_layout_round_trip(oracle, rows, nb, rate):
         small, n2 = oracle.pack_planes10x(codes, rows, nb, capacity=n // 2)
         assert n2 == n and small.size == tab_off + 16 * (n // 2)
         assert np.array_equal(small[:idx_off], buf[:idx_off]) and np.array_equal(small[tab_off:], buf[tab_off: tab_off + 16 * (n // 2)])
-        assert np.array_equal(small[idx_off: idx_off + 4 * (groups + 1)].view(np.uint32), np.minimum(index, n // 2))
+        assert np.array_equal(small[idx_off: idx_off + 4 * (groups * ntiles + 1)].view(np.uint32), np.minimum(index, n // 2))
 
 
 def test_planes10x_layout_worked_example_by_hand(oracle):
@@ -579,7 +581,7 @@ def test_planes10x_layout_worked_example_by_hand(oracle):
     assert not words[rest].any()
     hdr = buf[1152:1280]
     assert int(hdr[0]) == (2 << 4 | 2) and int(hdr[4]) == (2 << 4 | (8 ^ 2)) and int(hdr.astype(np.int64).sum()) == 34 + 42
-    assert buf[1280:1288].view(np.uint32).tolist() == [0, 1]
+    assert buf[1280:1288].view(np.uint32).tolist() == [0, 1]           # one tile: nothing before it, one entry in all
     assert buf[1408:1424].view(np.uint32).tolist() == [8 | 0 << 8 | 3 << 13, 0x8888884C, 0x88888888, 0x88888888]
 
 
