@@ -63,6 +63,38 @@ def test_config1_in_full(B, ctx, oracle):
             check_gemv(oracle, case, y, nthreads=16)
 
 
+def test_config1_in_full_in_the_10_byte_layout(B, ctx, oracle):
+    """The same layer in the 10-byte layout with its exception table, as the bench's arm runs it: buffers sized from the
+    count call, every byte (short records, index, table) against the oracle, every row of the grouped launches."""
+    from paper_2609_02652_b200 import datagen
+
+    wl = datagen.workload(1)
+    groups = {}
+    for m in wl.matrices:
+        groups.setdefault(m.group, []).append(m)
+    exceptions = 0
+    for members in groups.values():
+        probs, keep = [], []
+        for m in members:
+            case = make_case(m.rows, m.k, seed=wl.seed, tensor_id=m.tensor_id)
+            n = B.overlay_count(ctx, case.d_codes, m.rows, m.nb)
+            buf = B.expand(ctx, B.PLANES10X, case.d_codes, m.rows, m.nb,
+                           out=torch.empty(B.overlay_bytes(m.rows, m.k_padded, n), dtype=torch.uint8, device="cuda"))
+            want, n_ref = oracle.pack_planes10x(case.codes, m.rows, m.nb)
+            assert n == n_ref and np.array_equal(buf.cpu().numpy(), want), m.name
+            exceptions += n
+            y = torch.full((m.rows,), float("nan"), dtype=torch.float32, device="cuda")
+            probs.append((buf, case.d_scale, GAIN, y, m.rows))
+            keep.append((m, case, y))
+        x = keep[0][1]
+        B.gemv_grouped(ctx, B.PLANES10X, probs, x.d_x, members[0].k_padded)
+        B.status(ctx)
+        for m, case, y in keep:
+            case.x = x.x
+            check_gemv(oracle, case, y, nthreads=16)
+    assert 100 < exceptions < 2000          # about one block in eight thousand of the 4.2 million
+
+
 @pytest.mark.parametrize("config,layers", [(2, (0, 17, 35)), (3, (0, 39))])
 def test_stacks_sampled(B, ctx, oracle, config, layers):
     """Every matrix of the sampled layers runs as the bench runs it (row-concatenated groups); 96 rows
