@@ -37,7 +37,8 @@ def expand_exact(B, ctx, case):
 
 # (rows, k, share of the blocks replaced by exception blocks)
 SHAPES = [(1, 24, 0.0), (3, 96, 0.5), (33, 24 * 33, 0.1), (40, 24 * 7, 0.3), (64, 24 * 9 - 5, 0.0), (32, 96, 1.0), (31, 24 * 13, 0.05),
-          (257, 24 * 21, 0.02), (70, 24 * 30, 0.2), (96, 24 * 406, 0.01), (1024, 2560, 0.0), (3072, 3072, 0.03), (2100, 24 * 130, 0.5)]
+          (257, 24 * 21, 0.02), (70, 24 * 30, 0.2), (96, 24 * 406, 0.01), (1024, 2560, 0.0), (3072, 3072, 0.03), (2100, 24 * 130, 0.5),
+          (64, 98304, 0.01), (1, 98304, 0.2), (5000, 24 * 5, 0.3), (70000, 48, 0.1)]      # the longest rows the GEMV takes; tall and thin; no tile at all
 
 
 @pytest.mark.parametrize("rows,k,rate", SHAPES)
@@ -135,7 +136,7 @@ def test_gemv_every_row(B, ctx, oracle, rows, k, rate):
     # (low and high limb pair) whose split depends on the stored code, each half is rounded to f32, and an exception's
     # product is rounded to the accumulator's quantum by itself.  The two agree to far below f32's step.
     assert float((y - y14).abs().max()) <= 1e-6 * float(y14.abs().max())
-    assert n > 0 or rate == 0.0
+    assert n > 0 or rate == 0.0 or case.nb < 4          # blocks past the tiles are never exceptions
 
 
 def test_gemv_special_cases_and_grouped(B, ctx, oracle):
