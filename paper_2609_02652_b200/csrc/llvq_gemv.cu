@@ -1088,6 +1088,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
                 sum[0] += (long long)exc_scratch[my_row];
                 __syncwarp();
                 exc_scratch[my_row] = 0ull;
+                __syncwarp();                          // the slots are clear before any lane adds to them again
             }
         }
         // with no records read (the control launch) every unit contributes zero
