@@ -360,12 +360,11 @@ __device__ __forceinline__ uint32_t spread_nibbles(uint32_t h) {
 // One entry of the exception table against the x record of its block (`rec`): the block's whole product, in the
 // accumulator's quanta.  The arithmetic of the tile path for one block: integer sums limb pair by limb pair, the
 // block's scale in f32.  `tail_tab` is the table of the four-bit records' headers (the entry's header byte indexes it).
-// Rolled loops: this runs for one block in thousands, and its size in the instruction stream is what every run pays.
 __device__ __forceinline__ long long exception_value(const uint4 &ent, uint32_t rec, uint32_t tail_tab, float inv_q) {
     const float2 k = lds_f2(tail_tab + 8 * (ent.x & 63u));
     int d[4] = {0, 0, 0, 0};
     uint32_t cw = ent.y;
-#pragma unroll 1
+#pragma unroll
     for (int j = 0; j < 3; j++) {
         const uint32_t lo4 = spread_nibbles(cw), hi4 = spread_nibbles(cw >> 16);
 #pragma unroll
@@ -1072,7 +1071,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
         }
         if constexpr (OVERLAY) {
             // The exact records of this run's exception blocks: every lane takes an entry of the run's range and adds
-            // the product to its row's slot of the warp's scratch (integer additions: the order does not matter);
+            // the product to its row's slot of the warp's scratch (integer additions, so the order does not matter);
             // then every lane collects its own row's slot.
             const bool any = exc_begin < exc_end;
 #pragma unroll 1
@@ -1080,12 +1079,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
                 if (e0 != exc_begin) exc_entry = e0 + lane < exc_end ? __ldg(pr.exc_table + e0 + lane) : make_uint4(~0u, 0u, 0u, 0u);
                 if (exc_entry.x != ~0u) {
                     const long long v = exception_value(exc_entry, xs0 + (exc_entry.x >> 13) * kXRecBytes, tq_tail, inv_q);
-                    atomicAdd(exc_scratch + ((exc_entry.x >> 8) & 31u), (unsigned long long)v);
+                    // in two 32-bit halves, v = hi * 2^24 + lo with lo in [0, 2^24): a row meets at most 64 entries
+                    // a run and |v| < 2^40, so neither half overflows its word
+                    uint32_t *half = reinterpret_cast<uint32_t *>(exc_scratch + ((exc_entry.x >> 8) & 31u));
+                    atomicAdd(half, (uint32_t)(v & 0xffffff));
+                    atomicAdd(reinterpret_cast<int *>(half + 1), (int)(v >> 24));
                 }
             }
             if (any) {
                 __syncwarp();
-                sum[0] += (long long)exc_scratch[my_row];
+                const uint2 halves = *reinterpret_cast<const uint2 *>(exc_scratch + my_row);
+                sum[0] += ((long long)(int)halves.y << 24) + (long long)halves.x;
                 __syncwarp();
                 exc_scratch[my_row] = 0ull;
                 __syncwarp();                          // the slots are clear before any lane adds to them again
