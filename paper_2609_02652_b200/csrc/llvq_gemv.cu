@@ -917,7 +917,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
                 asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_begin) : "l"(ix + min(cc.col, tiles)));
                 asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(exc_end) : "l"(ix + min(cc.col + run, tiles)));
             }
-            if (exc_begin + lane < exc_end) exc_entry = __ldg(pr.exc_table + exc_begin + lane);
+            // a run of `run` tiles holds at most 128 * run blocks: whatever the index says, the loop over the range ends
+            exc_end = exc_begin + min(exc_end - exc_begin, (uint32_t)run * 128u);
+            if (lane < exc_end - exc_begin) exc_entry = __ldg(pr.exc_table + exc_begin + lane);
         }
         const int run_tiles = NO_WEIGHTS ? 0 : max(0, min(run, tiles - cc.col));
         // the row's scale is needed only by the arrival that finishes the row, but loading it now
@@ -1073,10 +1075,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemv_planes_kernel(const __grid_c
             // The exact records of this run's exception blocks: every lane takes an entry of the run's range and adds
             // the product to its row's slot of the warp's scratch (integer additions, so the order does not matter);
             // then every lane collects its own row's slot.
-            const bool any = exc_begin < exc_end;
+            const uint32_t exc_count = exc_end - exc_begin;          // at most 2048 (bounded where the range was read)
+            const bool any = exc_count != 0;
 #pragma unroll 1
-            for (uint32_t e0 = exc_begin; e0 < exc_end; e0 += 32) {
-                if (e0 != exc_begin) exc_entry = e0 + lane < exc_end ? __ldg(pr.exc_table + e0 + lane) : make_uint4(~0u, 0u, 0u, 0u);
+            for (uint32_t done = 0; done < exc_count; done += 32) {
+                if (done != 0) exc_entry = done + lane < exc_count ? __ldg(pr.exc_table + exc_begin + done + lane) : make_uint4(~0u, 0u, 0u, 0u);
                 if (exc_entry.x != ~0u) {
                     const long long v = exception_value(exc_entry, xs0 + (exc_entry.x >> 13) * kXRecBytes, tq_tail, inv_q);
                     // in two 32-bit halves, v = hi * 2^24 + lo with lo in [0, 2^24): a row meets at most 64 entries
