@@ -1294,7 +1294,8 @@ __device__ __forceinline__ void read_overlay_record(const uint8_t *buf, int64_t 
         const uint4 *table = reinterpret_cast<const uint4 *>(buf + overlay_table_offset(rows, nb));
         hdr = 0; c[0] = c[1] = c[2] = 0x88888888u;
         const int64_t tile_id = rg * tiles + b / kTileCells;
-        for (uint32_t i = index[tile_id]; i < index[tile_id + 1]; i++) {
+        const uint32_t first = index[tile_id], count = min(index[tile_id + 1] - first, 128u);      // a tile has 128 blocks
+        for (uint32_t i = first; i < first + count; i++) {
             const uint4 ent = table[i];
             if ((ent.x >> 13) == (uint32_t)b && ((ent.x >> 8) & 31u) == (uint32_t)r) { hdr = ent.x & 63u; c[0] = ent.y; c[1] = ent.z; c[2] = ent.w; }
         }
